@@ -1,0 +1,206 @@
+/*
+ * ftp -- fused tile-partitioned CNN training step for NVIDIA B200 (sm_100a).
+ *
+ * C-ABI of the library.  It implements the training cycle of "Distributed
+ * Convolutional Neural Network Training on Mobile and Edge Clusters"
+ * (arXiv 2409.09083): feature maps (forward) and delta maps (backward) are cut
+ * into a grid of tiles, matching tiles of consecutive conv / max-pool layers are
+ * fused into independent stacks, layers are combined into groups that exchange
+ * boundary data only at group inputs (Section 3, Section 4.2), every tile
+ * produces a partial filter-gradient set, and the sets are summed once per
+ * batch and used to update the filters (Section 4.1).  Here a tile stack runs
+ * in a thread block of one GPU instead of on an edge device.
+ *
+ * Conventions
+ *  - Every tensor pointer is CALLER-OWNED DEVICE memory, dense fp32, NCHW.
+ *  - `params` is one flat vector: for each conv layer in order the filter
+ *    [cout][cin][k][k] followed by the bias [cout].
+ *  - `workspace` is caller-allocated device memory of at least the size
+ *    ftp_plan_sizes reports, 256-byte aligned.  It holds the maps at group
+ *    boundaries, the saved layer outputs the backward pass reads, the per-tile
+ *    partial gradient sets and small tables.  Its contents carry state from
+ *    ftp_forward to ftp_backward and are otherwise scratch.
+ *  - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and
+ *    return without synchronising.  The first launch on a plan uploads the
+ *    plan's tables to the device with a blocking copy (a few KB, one
+ *    cudaMalloc); make that first call outside any stream capture.
+ *  - Return value: 0 on success, a negative FTP_ERR_* code otherwise.  Invalid
+ *    arguments are detected on the host before anything is launched.  The
+ *    library never aborts, throws or traps.
+ *  - A plan is immutable after creation; using one plan from several host
+ *    threads at once, or on overlapping streams with the same workspace, races.
+ */
+#ifndef FTP_H
+#define FTP_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    FTP_OK            =  0,
+    FTP_ERR_ARG       = -1,  /* null pointer, non-positive size, bad index        */
+    FTP_ERR_LAYERS    = -2,  /* unsupported layer or channel mismatch             */
+    FTP_ERR_GRID      = -3,  /* more tiles than pixels in a group's output map    */
+    FTP_ERR_GROUPS    = -4,  /* groups not contiguous or not covering 1..L        */
+    FTP_ERR_WORKSPACE = -5,  /* no sub-tile of a group fits in shared memory      */
+    FTP_ERR_CUDA      = -6,  /* a CUDA runtime call failed                        */
+    FTP_ERR_TIMEOUT   = -7,  /* reserved: a bounded device-side wait ran out      */
+    FTP_ERR_PRECISION = -8   /* requested arithmetic is not built                 */
+};
+
+enum { FTP_CONV = 0, FTP_MAXPOOL = 1 };
+enum { FTP_FP32 = 0, FTP_BF16_FP32ACC = 1 };
+
+/* Layer descriptor: kernel K_l x K_l and stride S_l in the paper's notation
+ * (Section 4.2).  Supported: conv with odd k <= 7, stride 1, pad = k / 2,
+ * followed by bias and leaky ReLU with negative slope `leaky` (derivative
+ * `leaky` at exactly 0); max-pool with k = 2, stride 2, pad 0 on even extents
+ * (first maximum in row-major window order receives the gradient). */
+typedef struct {
+    int   kind;          /* FTP_CONV or FTP_MAXPOOL */
+    int   cin, cout;     /* conv only */
+    int   k, stride, pad;
+    float leaky;         /* conv only */
+} ftp_layer;
+
+/* A group as an inclusive 1-based layer range.  The paper's tuple (s, e)
+ * "starting at the input to layer s and ending at the input to layer e"
+ * (Section 4.2) is (first, last + 1).  Boundary data is exchanged only at the
+ * input map of `first`. */
+typedef struct { int first, last; } ftp_group;
+
+typedef struct ftp_plan ftp_plan;   /* opaque, host-owned */
+
+/*
+ * Tile-region planner (Section 4.2).  For every group the group's output map
+ * is partitioned equally among the grid_y x grid_x tiles (tile i of g owns
+ * [floor(i*E/g), floor((i+1)*E/g) - 1] along an axis of extent E), and each
+ * tile's span at every earlier map of the group follows from the receptive
+ * field recursion, Eq. (1), generalised with explicit padding so that it also
+ * covers the 2x2/2 pool (in1 = out1*S - P, in2 = out2*S - P + K - 1), clamped
+ * to the map at every step.  Tiles are further cut into sub-tiles whose whole
+ * layer stack fits the shared memory of one thread block; results do not
+ * depend on that cut.  A requested group whose stack can be held in shared
+ * memory only with sub-tiles so small that halo recomputation explodes (deep
+ * stacks at high resolution, or layers with many channels) is executed as
+ * several consecutive groups, i.e. with the
+ * finer grouping profile ftp_plan_exec_groups reports; the method's result does
+ * not depend on the profile (Section 3), only its cost does.
+ * N, C, H, W: shape of the network input X_1.  `layers`/`groups` are copied.
+ * Errors: FTP_ERR_ARG, _LAYERS, _GRID, _GROUPS, _WORKSPACE, _PRECISION.
+ * Needs no GPU.
+ */
+int ftp_plan_create(const ftp_layer* layers, int n_layers,
+                    int N, int C, int H, int W,
+                    int grid_y, int grid_x,
+                    const ftp_group* groups, int n_groups,
+                    int precision, ftp_plan** out);
+
+/* Planner options; zero-initialise, set struct_size = sizeof(ftp_plan_opts),
+ * and leave a field 0 for its default. */
+typedef struct {
+    int struct_size;
+    int max_redundancy_pct; /* a requested group is cut into shorter groups when the multiply-accumulates
+                           of its sub-tile stacks (halo recomputation included) exceed this percentage of
+                           the untiled ones in either pass (default 150, minimum 100) */
+    int max_subtile;    /* upper bound on the sub-tile extent (default: none) */
+    int smem_bytes;     /* dynamic shared memory a block may use (default and maximum 230400) */
+    int strict_groups;  /* 1: never cut a requested group; FTP_ERR_WORKSPACE if it cannot fit at all */
+} ftp_plan_opts;
+
+/* ftp_plan_create with explicit planner options (NULL = defaults). */
+int ftp_plan_create_opts(const ftp_layer* layers, int n_layers,
+                         int N, int C, int H, int W,
+                         int grid_y, int grid_x,
+                         const ftp_group* groups, int n_groups,
+                         int precision, const ftp_plan_opts* opts, ftp_plan** out);
+
+/* The grouping profile that is executed (see ftp_plan_create): writes up to
+ * `capacity` groups to groups_out (may be NULL) and the count to *n_groups. */
+int ftp_plan_exec_groups(const ftp_plan* plan, int* n_groups, ftp_group* groups_out, int capacity);
+
+void ftp_plan_destroy(ftp_plan* plan);
+
+/*
+ * Span of user tile (ty, tx) at map X_{map_index} (1-based; must lie in
+ * first..last+1 of `group`, 0-based group index): span_out = {x1, y1, x2, y2},
+ * inclusive, the paper's (x1, y1), (x2, y2) (Section 4.2).
+ * pass 0: feature-map span of the forward pass, Eq. (1).
+ * pass 1: delta-map span the tile back-propagates.  The backward pass runs in
+ *   adjoint form: a tile pushes the delta of its owned part of the group's
+ *   output map back through its own forward stack, so these spans equal the
+ *   forward spans, and overlapping contributions are summed at the group
+ *   input.
+ * pass 2: Eq. (2) gather-form span, for reference: the delta span at
+ *   X_{map_index} needed to produce the tile's equal share of the group's
+ *   INPUT delta map.
+ */
+int ftp_plan_region(const ftp_plan* plan, int pass, int group, int map_index,
+                    int ty, int tx, int span_out[4]);
+
+/*
+ * Sizes: number of parameter floats, workspace bytes, floats of the network
+ * output X_{L+1} (N*C*H*W of the last map), and the forward redundancy factor
+ * (multiply-accumulates executed with halo recomputation / untiled ones).
+ * Any out pointer may be NULL.
+ */
+int ftp_plan_sizes(const ftp_plan* plan, size_t* param_floats,
+                   size_t* workspace_bytes, size_t* out_floats,
+                   double* redundancy);
+
+/*
+ * Sub-tiling chosen for an EXECUTED group (0-based index into the profile of
+ * ftp_plan_exec_groups) and pass (0 forward, 1 backward):
+ * number of sub-tile rows and columns over the whole map, dynamic shared
+ * memory per block in bytes, and blocks launched.  Any out pointer may be NULL.
+ */
+int ftp_plan_subtiles(const ftp_plan* plan, int pass, int group,
+                      int* rows, int* cols, size_t* smem_bytes, int* blocks);
+
+/*
+ * Forward pass (Section 3; Section 4.1 forward; Section 4.2 groups): one fused
+ * launch per group, halo exchange through the group's input map in HBM.
+ *   x [N,C,H,W] in, params in, y [N,C_out,H_out,W_out] out (may be NULL).
+ * Layer outputs are kept in `workspace` for ftp_backward.
+ */
+int ftp_forward(ftp_plan* plan, const float* x, const float* params, float* y,
+                void* workspace, void* stream);
+
+/*
+ * Backward pass (Section 4.1 back-propagation and filter gradients; Section
+ * 4.2): needs a preceding ftp_forward with the same plan, x, params and
+ * workspace.  dy = dLoss/dX_{L+1} in.  dx = dLoss/dX_1 out, may be NULL (then
+ * it is not computed).  dparams out, same layout as params: the sum over all
+ * tiles of the partial filter and bias gradients, in a fixed order.
+ */
+int ftp_backward(ftp_plan* plan, const float* x, const float* dy,
+                 const float* params, float* dx, float* dparams,
+                 void* workspace, void* stream);
+
+/*
+ * One training cycle (Section 3: forward, backward, sum of the partial
+ * filter-gradient sets once per batch, update): params <- params - lr * grad
+ * in place (plain SGD).  Give exactly one of
+ *   dy      the loss delta at the last map, or
+ *   target  [same shape as the output] for the mean-squared-error loss
+ *           L = mean((X_{L+1} - target)^2).
+ * loss_out (device, 1 float, may be NULL) receives L when `target` is given.
+ * dx (may be NULL) receives dLoss/dX_1.
+ */
+int ftp_step(ftp_plan* plan, const float* x, const float* dy,
+             const float* target, float* params, float lr, float* loss_out,
+             float* dx, void* workspace, void* stream);
+
+/* Number of kernels the library launched on the calling thread's behalf since
+ * the plan was created (for launch accounting in benchmarks). */
+long long ftp_plan_launch_count(const ftp_plan* plan);
+
+const char* ftp_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FTP_H */

@@ -1,0 +1,190 @@
+"""Thin ctypes binding of the C-ABI in include/ftp.h: argument marshalling only.
+
+Every step of the path runs in the CUDA library.  If `libftp.so` has not been
+built the import fails; there is no CPU fallback.  Tensors are torch CUDA
+tensors (fp32, contiguous); torch is used for device memory and streams only.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libftp.so")
+
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build it with `python -m paper_2409_09083_b200.build` "
+        "(there is no CPU fallback)")
+_lib = ctypes.CDLL(_LIB_PATH)
+
+FTP_CONV, FTP_MAXPOOL = 0, 1
+FTP_FP32, FTP_BF16_FP32ACC = 0, 1
+
+
+class ftp_layer(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int), ("cin", ctypes.c_int), ("cout", ctypes.c_int),
+                ("k", ctypes.c_int), ("stride", ctypes.c_int), ("pad", ctypes.c_int),
+                ("leaky", ctypes.c_float)]
+
+
+class ftp_group(ctypes.Structure):
+    _fields_ = [("first", ctypes.c_int), ("last", ctypes.c_int)]
+
+
+_vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+_lib.ftp_plan_create.argtypes = [ctypes.POINTER(ftp_layer), _i, _i, _i, _i, _i, _i, _i,
+                                 ctypes.POINTER(ftp_group), _i, _i, ctypes.POINTER(_vp)]
+_lib.ftp_plan_create.restype = _i
+
+
+class ftp_plan_opts(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_int), ("max_redundancy_pct", ctypes.c_int), ("max_subtile", ctypes.c_int),
+                ("smem_bytes", ctypes.c_int), ("strict_groups", ctypes.c_int)]
+
+
+_lib.ftp_plan_create_opts.argtypes = [ctypes.POINTER(ftp_layer), _i, _i, _i, _i, _i, _i, _i,
+                                      ctypes.POINTER(ftp_group), _i, _i, ctypes.POINTER(ftp_plan_opts),
+                                      ctypes.POINTER(_vp)]
+_lib.ftp_plan_create_opts.restype = _i
+_lib.ftp_plan_exec_groups.argtypes = [_vp, ctypes.POINTER(_i), ctypes.POINTER(ftp_group), _i]
+_lib.ftp_plan_exec_groups.restype = _i
+_lib.ftp_plan_destroy.argtypes = [_vp]
+_lib.ftp_plan_destroy.restype = None
+_lib.ftp_plan_region.argtypes = [_vp, _i, _i, _i, _i, _i, ctypes.POINTER(_i * 4)]
+_lib.ftp_plan_region.restype = _i
+_lib.ftp_plan_sizes.argtypes = [_vp, ctypes.POINTER(_sz), ctypes.POINTER(_sz), ctypes.POINTER(_sz),
+                                ctypes.POINTER(ctypes.c_double)]
+_lib.ftp_plan_sizes.restype = _i
+_lib.ftp_plan_subtiles.argtypes = [_vp, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i),
+                                   ctypes.POINTER(_sz), ctypes.POINTER(_i)]
+_lib.ftp_plan_subtiles.restype = _i
+_lib.ftp_forward.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
+_lib.ftp_forward.restype = _i
+_lib.ftp_backward.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.ftp_backward.restype = _i
+_lib.ftp_step.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp, _vp, _vp]
+_lib.ftp_step.restype = _i
+_lib.ftp_plan_launch_count.argtypes = [_vp]
+_lib.ftp_plan_launch_count.restype = ctypes.c_longlong
+_lib.ftp_strerror.argtypes = [_i]
+_lib.ftp_strerror.restype = ctypes.c_char_p
+
+
+class FtpError(RuntimeError):
+    def __init__(self, code):
+        self.code = code
+        super().__init__(f"ftp error {code}: {_lib.ftp_strerror(code).decode()}")
+
+
+def ftp_strerror(code: int) -> str:
+    return _lib.ftp_strerror(code).decode()
+
+
+def _check(rc):
+    if rc != 0:
+        raise FtpError(rc)
+
+
+def _ptr(t, name, allow_none=False):
+    if t is None:
+        if allow_none:
+            return None
+        raise ValueError(f"{name} must not be None")
+    if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise ValueError(f"{name} must be a contiguous float32 CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _as_layers(layers):
+    arr = (ftp_layer * len(layers))()
+    for a, l in zip(arr, layers):
+        conv = l.kind in ("conv", FTP_CONV)
+        a.kind = FTP_CONV if conv else FTP_MAXPOOL
+        a.cin, a.cout, a.k, a.stride, a.pad, a.leaky = l.cin, l.cout, l.k, l.stride, l.pad, l.leaky
+    return arr
+
+
+def _as_groups(groups):
+    arr = (ftp_group * len(groups))()
+    for a, g in zip(arr, groups):
+        a.first, a.last = g
+    return arr
+
+
+class Plan:
+    """Owner of an ftp_plan handle (ftp_plan_create / ftp_plan_destroy)."""
+
+    def __init__(self, layers, N, C, H, W, grid, groups, precision=FTP_FP32, max_redundancy_pct=0, max_subtile=0,
+                 smem_bytes=0, strict_groups=False):
+        self._h = _vp()
+        la, ga = _as_layers(layers), _as_groups(groups)
+        opts = ftp_plan_opts(ctypes.sizeof(ftp_plan_opts), max_redundancy_pct, max_subtile, smem_bytes,
+                             1 if strict_groups else 0)
+        _check(_lib.ftp_plan_create_opts(la, len(layers), N, C, H, W, grid[0], grid[1], ga, len(groups),
+                                         precision, ctypes.byref(opts), ctypes.byref(self._h)))
+        self.layers, self.shape, self.grid, self.groups = list(layers), (N, C, H, W), tuple(grid), list(groups)
+        pf, wb, of, red = _sz(), _sz(), _sz(), ctypes.c_double()
+        _check(_lib.ftp_plan_sizes(self._h, ctypes.byref(pf), ctypes.byref(wb), ctypes.byref(of),
+                                   ctypes.byref(red)))
+        self.param_floats, self.workspace_bytes, self.out_floats = pf.value, wb.value, of.value
+        self.redundancy = red.value
+
+    def __del__(self):
+        h = getattr(self, "_h", None)
+        if h and _lib is not None:
+            _lib.ftp_plan_destroy(h)
+            self._h = None
+
+    def exec_groups(self):
+        """The grouping profile that is executed (a requested group may have been cut)."""
+        n = _i()
+        _check(_lib.ftp_plan_exec_groups(self._h, ctypes.byref(n), None, 0))
+        arr = (ftp_group * n.value)()
+        _check(_lib.ftp_plan_exec_groups(self._h, ctypes.byref(n), arr, n.value))
+        return [(g.first, g.last) for g in arr]
+
+    def region(self, pass_, group, map_index, ty, tx):
+        """(x1, y1, x2, y2), inclusive, of user tile (ty, tx) at map X_{map_index}."""
+        out = (_i * 4)()
+        _check(_lib.ftp_plan_region(self._h, pass_, group, map_index, ty, tx, ctypes.byref(out)))
+        return tuple(out)
+
+    def subtiles(self, pass_, group):
+        r, c, s, b = _i(), _i(), _sz(), _i()
+        _check(_lib.ftp_plan_subtiles(self._h, pass_, group, ctypes.byref(r), ctypes.byref(c),
+                                      ctypes.byref(s), ctypes.byref(b)))
+        return dict(rows=r.value, cols=c.value, smem_bytes=s.value, blocks=b.value)
+
+    def launch_count(self):
+        return int(_lib.ftp_plan_launch_count(self._h))
+
+    def new_workspace(self, device="cuda"):
+        return torch.empty(self.workspace_bytes, dtype=torch.uint8, device=device)
+
+
+def ftp_plan(layers, N, C, H, W, tile_grid, groups, precision=FTP_FP32, **opts) -> Plan:
+    return Plan(layers, N, C, H, W, tile_grid, groups, precision, **opts)
+
+
+def ftp_forward(plan, x, params, y, workspace, stream=None):
+    _check(_lib.ftp_forward(plan._h, _ptr(x, "x"), _ptr(params, "params"), _ptr(y, "y", True),
+                            workspace.data_ptr(), _stream(stream)))
+
+
+def ftp_backward(plan, x, dy, params, dx, dparams, workspace, stream=None):
+    _check(_lib.ftp_backward(plan._h, _ptr(x, "x"), _ptr(dy, "dy"), _ptr(params, "params"),
+                             _ptr(dx, "dx", True), _ptr(dparams, "dparams"), workspace.data_ptr(),
+                             _stream(stream)))
+
+
+def ftp_step(plan, x, params, lr, workspace, dy=None, target=None, loss_out=None, dx=None, stream=None):
+    _check(_lib.ftp_step(plan._h, _ptr(x, "x"), _ptr(dy, "dy", True), _ptr(target, "target", True),
+                         _ptr(params, "params"), float(lr), _ptr(loss_out, "loss_out", True),
+                         _ptr(dx, "dx", True), workspace.data_ptr(), _stream(stream)))

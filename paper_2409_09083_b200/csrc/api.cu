@@ -1,0 +1,312 @@
+// C-ABI entry points: argument checks, lazy upload of the plan tables, kernel launches.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstring>
+#include <new>
+
+#include "ftp.h"
+#include "kernels.cuh"
+#include "plan.hpp"
+
+using namespace ftp;
+
+namespace {
+
+inline float* ws_ptr(void* ws, size_t off) { return reinterpret_cast<float*>(static_cast<unsigned char*>(ws) + off); }
+
+int ensure_device(ftp_plan* p)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FTP_ERR_CUDA;
+    if (p->dev_tables && p->dev_id == dev) return FTP_OK;
+    if (p->dev_tables) { cudaFree(p->dev_tables); p->dev_tables = nullptr; }
+    if (cudaFuncSetAttribute(fwd_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(bwd_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess)
+        return FTP_ERR_CUDA;
+    const size_t bytes = p->tables.size() * sizeof(int);
+    if (cudaMalloc(&p->dev_tables, bytes) != cudaSuccess) return FTP_ERR_CUDA;
+    if (cudaMemcpy(p->dev_tables, p->tables.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess) return FTP_ERR_CUDA;
+    p->dev_id = dev;
+    return FTP_OK;
+}
+
+inline bool launched_ok() { return cudaGetLastError() == cudaSuccess; }
+
+const float* map_ptr(const ftp_plan* p, const float* x, void* ws, int l /* X_l, 1-based */)
+{
+    return l == 1 ? x : ws_ptr(ws, p->ws.map_off[l - 1]);
+}
+
+void fill_common(const ftp_plan* p, const GroupPlan& g, bool backward, const float* x, const float* params,
+                 void* ws, GroupArgs& a)
+{
+    const PassPlan& pp = backward ? g.bwd : g.fwd;
+    std::memset(&a, 0, sizeof(a));
+    a.n_ops = g.n_ops; a.R = pp.y.count; a.Q = pp.x.count; a.N = p->N;
+    for (int i = 0; i < g.n_ops; ++i) a.op[i] = backward ? g.bwd_ops[i] : g.fwd_ops[i];
+    a.map[0] = map_ptr(p, x, ws, g.first);
+    for (int i = 0; i < g.n_ops; ++i) {
+        const OpDesc& op = a.op[i];
+        a.map[i + 1] = map_ptr(p, x, ws, op.out_map);
+        a.map_out[i + 1] = const_cast<float*>(a.map[i + 1]);
+        a.arg[i] = op.kind == kOpConvPool
+                       ? static_cast<unsigned char*>(ws) + p->ws.arg_off[op.out_map - 1] : nullptr;
+    }
+    a.yspan = p->dev_tables + pp.dev_yspan; a.xspan = p->dev_tables + pp.dev_xspan;
+    a.ycell = p->dev_tables + pp.dev_ycell; a.xcell = p->dev_tables + pp.dev_xcell;
+    a.yoff = p->dev_tables + pp.dev_yoff;   a.xoff = p->dev_tables + pp.dev_xoff;
+    a.ytile = p->dev_tables + pp.dev_ytile; a.xtile = p->dev_tables + pp.dev_xtile;
+    a.wpk = ws_ptr(ws, backward ? p->ws.wb_off : p->ws.wf_off);
+    a.params = params;
+}
+
+int pack_filters(ftp_plan* p, const float* params, void* ws, cudaStream_t st)
+{
+    PackArgs pa{};
+    for (const GroupPlan& g : p->groups)
+        for (int i = 0; i < g.n_ops; ++i) {
+            const OpDesc& op = g.fwd_ops[i];
+            if (op.kind == kOpPool) continue;
+            if (pa.n == kMaxOps * 2) {   // flush a full batch
+                pack_filters_kernel<<<dim3(64, pa.n), 256, 0, st>>>(pa, params, ws_ptr(ws, p->ws.wf_off), ws_ptr(ws, p->ws.wb_off));
+                ++p->launches;
+                pa.n = 0;
+            }
+            pa.l[pa.n++] = PackLayer{op.p_off, op.wf_off, op.wb_off, op.cin, op.cout, op.k, op.cout_pad, op.cin_pad};
+        }
+    if (pa.n) {
+        pack_filters_kernel<<<dim3(64, pa.n), 256, 0, st>>>(pa, params, ws_ptr(ws, p->ws.wf_off), ws_ptr(ws, p->ws.wb_off));
+        ++p->launches;
+    }
+    return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
+}
+
+int forward_impl(ftp_plan* p, const float* x, const float* params, float* y, void* ws, cudaStream_t st)
+{
+    int rc = pack_filters(p, params, ws, st);
+    if (rc != FTP_OK) return rc;
+    for (const GroupPlan& g : p->groups) {
+        GroupArgs a;
+        fill_common(p, g, false, x, params, ws, a);
+        fwd_group_kernel<<<dim3(a.R * a.Q, p->N), kThreads, g.fwd.smem_bytes, st>>>(a);
+        ++p->launches;
+        if (!launched_ok()) return FTP_ERR_CUDA;
+    }
+    if (y) {
+        const MapShape& s = p->maps.back();
+        const size_t bytes = (size_t)p->N * s.C * s.H * s.W * sizeof(float);
+        if (cudaMemcpyAsync(y, map_ptr(p, x, ws, (int)p->layers.size() + 1), bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+            return FTP_ERR_CUDA;
+    }
+    return FTP_OK;
+}
+
+// Backward of all groups in reverse order, halo sums at the group inputs, then the cross-tile
+// reduction; `sgd_params` non-null applies the update in the same kernel.
+int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* params, float* dx, float* grad_out,
+                  float* sgd_params, float lr, void* ws, cudaStream_t st)
+{
+    const int G = (int)p->groups.size();
+    for (int gi = G - 1; gi >= 0; --gi) {
+        const GroupPlan& g = p->groups[gi];
+        GroupArgs a;
+        fill_common(p, g, true, x, params, ws, a);
+        a.dmap_out = gi == G - 1 ? dy : ws_ptr(ws, p->ws.dmap_off[gi + 1]);
+        a.scratch = ws_ptr(ws, p->ws.scratch_off);
+        a.partial = ws_ptr(ws, g.partial_off);
+        a.param_floats = (long long)g.param_floats;
+        a.splits = g.bwd.splits; a.tiles_x = p->grid_x;
+        a.need_dx = (gi > 0 || dx != nullptr) ? 1 : 0;
+        bwd_group_kernel<<<g.bwd.blocks, kThreads, g.bwd.smem_bytes, st>>>(a);
+        ++p->launches;
+        if (!launched_ok()) return FTP_ERR_CUDA;
+        if (a.need_dx) {
+            const MapShape& s = p->maps[g.first - 1];
+            HaloSumArgs h{};
+            h.scratch = a.scratch;
+            h.out = gi == 0 ? dx : ws_ptr(ws, p->ws.dmap_off[gi]);
+            h.yspan = a.yspan; h.xspan = a.xspan; h.yoff = a.yoff; h.xoff = a.xoff;
+            h.ycover = p->dev_tables + g.bwd.dev_ycover; h.xcover = p->dev_tables + g.bwd.dev_xcover;
+            h.N = p->N; h.C = s.C; h.H = s.H; h.W = s.W; h.R = a.R; h.Q = a.Q;
+            h.Htot = g.bwd.y.scratch_off[a.R]; h.Wtot = g.bwd.x.scratch_off[a.Q];
+            const size_t total = (size_t)p->N * s.C * s.H * s.W;
+            const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16);
+            halo_sum_kernel<<<blocks, 256, 0, st>>>(h);
+            ++p->launches;
+            if (!launched_ok()) return FTP_ERR_CUDA;
+        }
+    }
+    ReduceArgs ra{};
+    for (const GroupPlan& g : p->groups) {
+        if (g.param_floats == 0) continue;
+        ra.g[ra.n++] = ReduceGroup{g.param_begin, (long long)g.param_floats, ws_ptr(ws, g.partial_off), g.bwd.blocks};
+    }
+    if (ra.n) {
+        const long long total = (long long)p->param_floats;
+        const int blocks = (int)std::min<long long>((total + 255) / 256, (long long)kSmCount * 16);
+        reduce_sgd_kernel<<<blocks, 256, 0, st>>>(ra, total, sgd_params, lr, grad_out);
+        ++p->launches;
+        if (!launched_ok()) return FTP_ERR_CUDA;
+    }
+    return FTP_OK;
+}
+
+bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+int ftp_plan_create_opts(const ftp_layer* layers, int n_layers, int N, int C, int H, int W, int grid_y, int grid_x,
+                         const ftp_group* groups, int n_groups, int precision, const ftp_plan_opts* opts,
+                         ftp_plan** out)
+{
+    if (!out) return FTP_ERR_ARG;
+    *out = nullptr;
+    PlanOpts po;
+    if (opts) {
+        if (opts->struct_size != (int)sizeof(ftp_plan_opts)) return FTP_ERR_ARG;
+        if (opts->max_redundancy_pct) po.max_redundancy_pct = opts->max_redundancy_pct;
+        if (opts->max_subtile) po.max_subtile = opts->max_subtile;
+        if (opts->smem_bytes) po.smem_bytes = opts->smem_bytes;
+        po.strict_groups = opts->strict_groups;
+    }
+    ftp_plan* p = new (std::nothrow) ftp_plan();
+    if (!p) return FTP_ERR_ARG;
+    int rc = FTP_ERR_ARG;
+    try {
+        rc = build_plan(*p, layers, n_layers, N, C, H, W, grid_y, grid_x, groups, n_groups, precision, po);
+    } catch (...) {
+        rc = FTP_ERR_ARG;
+    }
+    if (rc != FTP_OK) { delete p; return rc; }
+    *out = p;
+    return FTP_OK;
+}
+
+int ftp_plan_create(const ftp_layer* layers, int n_layers, int N, int C, int H, int W, int grid_y, int grid_x,
+                    const ftp_group* groups, int n_groups, int precision, ftp_plan** out)
+{
+    return ftp_plan_create_opts(layers, n_layers, N, C, H, W, grid_y, grid_x, groups, n_groups, precision, nullptr, out);
+}
+
+int ftp_plan_exec_groups(const ftp_plan* plan, int* n_groups, ftp_group* groups_out, int capacity)
+{
+    if (!plan || !n_groups) return FTP_ERR_ARG;
+    *n_groups = (int)plan->groups.size();
+    if (groups_out)
+        for (int i = 0; i < *n_groups && i < capacity; ++i) groups_out[i] = ftp_group{plan->groups[i].first, plan->groups[i].last};
+    return FTP_OK;
+}
+
+void ftp_plan_destroy(ftp_plan* plan)
+{
+    if (!plan) return;
+    if (plan->dev_tables) cudaFree(plan->dev_tables);
+    delete plan;
+}
+
+int ftp_plan_region(const ftp_plan* plan, int pass, int group, int map_index, int ty, int tx, int span_out[4])
+{
+    if (!plan) return FTP_ERR_ARG;
+    return region(*plan, pass, group, map_index, ty, tx, span_out);
+}
+
+int ftp_plan_sizes(const ftp_plan* plan, size_t* param_floats, size_t* workspace_bytes, size_t* out_floats,
+                   double* redundancy)
+{
+    if (!plan) return FTP_ERR_ARG;
+    if (param_floats) *param_floats = plan->param_floats;
+    if (workspace_bytes) *workspace_bytes = plan->ws.total;
+    if (out_floats) {
+        const MapShape& s = plan->maps.back();
+        *out_floats = (size_t)plan->N * s.C * s.H * s.W;
+    }
+    if (redundancy) {
+        double done = 0, base = 0;
+        for (const GroupPlan& g : plan->groups) { done += g.macs_done; base += g.macs_untiled; }
+        *redundancy = base > 0 ? done / base : 1.0;
+    }
+    return FTP_OK;
+}
+
+int ftp_plan_subtiles(const ftp_plan* plan, int pass, int group, int* rows, int* cols, size_t* smem_bytes, int* blocks)
+{
+    if (!plan || group < 0 || group >= (int)plan->groups.size() || pass < 0 || pass > 1) return FTP_ERR_ARG;
+    const PassPlan& pp = pass ? plan->groups[group].bwd : plan->groups[group].fwd;
+    if (rows) *rows = pp.y.count;
+    if (cols) *cols = pp.x.count;
+    if (smem_bytes) *smem_bytes = pp.smem_bytes;
+    if (blocks) *blocks = pp.blocks;
+    return FTP_OK;
+}
+
+int ftp_forward(ftp_plan* plan, const float* x, const float* params, float* y, void* workspace, void* stream)
+{
+    if (!plan || !x || !params || !workspace || !aligned256(workspace)) return FTP_ERR_ARG;
+    int rc = ensure_device(plan);
+    if (rc != FTP_OK) return rc;
+    return forward_impl(plan, x, params, y, workspace, static_cast<cudaStream_t>(stream));
+}
+
+int ftp_backward(ftp_plan* plan, const float* x, const float* dy, const float* params, float* dx, float* dparams,
+                 void* workspace, void* stream)
+{
+    if (!plan || !x || !dy || !params || !dparams || !workspace || !aligned256(workspace)) return FTP_ERR_ARG;
+    int rc = ensure_device(plan);
+    if (rc != FTP_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = pack_filters(plan, params, workspace, st);
+    if (rc != FTP_OK) return rc;
+    return backward_impl(plan, x, dy, params, dx, dparams, nullptr, 0.f, workspace, st);
+}
+
+int ftp_step(ftp_plan* plan, const float* x, const float* dy, const float* target, float* params, float lr,
+             float* loss_out, float* dx, void* workspace, void* stream)
+{
+    if (!plan || !x || !params || !workspace || !aligned256(workspace)) return FTP_ERR_ARG;
+    if ((dy == nullptr) == (target == nullptr)) return FTP_ERR_ARG;
+    int rc = ensure_device(plan);
+    if (rc != FTP_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = forward_impl(plan, x, params, nullptr, workspace, st);
+    if (rc != FTP_OK) return rc;
+    const float* delta = dy;
+    if (target) {
+        const MapShape& s = plan->maps.back();
+        const size_t M = (size_t)plan->N * s.C * s.H * s.W;
+        float* d = ws_ptr(workspace, plan->ws.dy_off);
+        float* sums = ws_ptr(workspace, plan->ws.loss_off);
+        mse_delta_kernel<<<plan->loss_blocks, 256, 0, st>>>(map_ptr(plan, x, workspace, (int)plan->layers.size() + 1),
+                                                           target, d, M, sums);
+        ++plan->launches;
+        if (loss_out) {
+            mse_finish_kernel<<<1, 32, 0, st>>>(sums, plan->loss_blocks, M, loss_out);
+            ++plan->launches;
+        }
+        if (!launched_ok()) return FTP_ERR_CUDA;
+        delta = d;
+    }
+    return backward_impl(plan, x, delta, params, dx, nullptr, params, lr, workspace, st);
+}
+
+long long ftp_plan_launch_count(const ftp_plan* plan) { return plan ? plan->launches : 0; }
+
+const char* ftp_strerror(int code)
+{
+    switch (code) {
+    case FTP_OK: return "ok";
+    case FTP_ERR_ARG: return "invalid argument (null pointer, bad size or index, unaligned workspace)";
+    case FTP_ERR_LAYERS: return "unsupported layer (conv: odd k<=7, stride 1, pad k/2; maxpool: 2x2/2 on even extents) or channel mismatch";
+    case FTP_ERR_GRID: return "tile grid has more tiles than pixels in a group's output map";
+    case FTP_ERR_GROUPS: return "groups must be contiguous, cover layers 1..L, and hold at most 16 layers each";
+    case FTP_ERR_WORKSPACE: return "no sub-tile of a group fits in shared memory; use smaller groups";
+    case FTP_ERR_CUDA: return "a CUDA runtime call failed";
+    case FTP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case FTP_ERR_PRECISION: return "requested arithmetic is not built into this library";
+    default: return "unknown error";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,464 @@
+// Host-side tile-region planner (Section 4.2 of the paper): validation, map shapes, the
+// equal partition of each group's output map, the receptive-field recursion of Eq. (1)
+// generalised with explicit padding, sub-tiling for shared memory, workspace layout.
+// Pure C++; no CUDA calls.
+#include "plan.hpp"
+
+#include <algorithm>
+#include <cstring>
+
+namespace ftp {
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int round4(int v) { return (v + 3) / 4 * 4; }
+inline int extent(Span s) { return s.b - s.a + 1; }
+
+// Inputs read by outputs o.a..o.b of a window op (kernel K, stride S, padding P), clamped to
+// the input map.  For odd K, S = 1, P = K/2 this is Eq. (1) literally.
+inline Span back_project(Span o, int K, int S, int P, int in_extent)
+{
+    Span s{o.a * S - P, o.b * S - P + K - 1};
+    s.a = std::max(s.a, 0);
+    s.b = std::min(s.b, in_extent - 1);
+    return s;
+}
+
+inline int floor_div(int a, int b) { int q = a / b, r = a % b; return (r != 0 && ((r < 0) != (b < 0))) ? q - 1 : q; }
+inline int ceil_div(int a, int b) { return -floor_div(-a, b); }
+
+// Outputs that touch inputs i.a..i.b.  For odd K, P = K/2 this is Eq. (2) literally.
+inline Span forward_project(Span i, int K, int S, int P, int out_extent)
+{
+    Span s{ceil_div(i.a + P - K + 1, S), floor_div(i.b + P, S)};
+    s.a = std::max(s.a, 0);
+    s.b = std::min(s.b, out_extent - 1);
+    return s;
+}
+
+// "Partitioned ... equally among the tiles": part i of n owns [floor(i*E/n), floor((i+1)*E/n) - 1].
+std::vector<Span> equal_partition(int a0, int len, int parts)
+{
+    std::vector<Span> out;
+    for (int i = 0; i < parts; ++i) {
+        long long lo = (long long)i * len / parts, hi = (long long)(i + 1) * len / parts - 1;
+        out.push_back(Span{a0 + (int)lo, a0 + (int)hi});
+    }
+    return out;
+}
+
+struct AxisInfo {
+    int n_ops;
+    int K[kMaxOps], S[kMaxOps], P[kMaxOps];
+    int ext[kMaxOps + 1];
+};
+
+void build_axis(AxisTables& t, const AxisInfo& ax, const std::vector<Span>& tiles, int split)
+{
+    const int n = ax.n_ops;
+    std::vector<Span> cuts;
+    t.tile_begin.clear();
+    for (const Span& tl : tiles) {
+        t.tile_begin.push_back((int)cuts.size());
+        int len = extent(tl);
+        int k = std::min(split, len);
+        for (const Span& s : equal_partition(tl.a, len, k)) cuts.push_back(s);
+    }
+    t.tile_begin.push_back((int)cuts.size());
+    t.count = (int)cuts.size();
+    const int cnt = t.count;
+    t.span.assign((size_t)(n + 1) * cnt * 2, 0);
+    t.cell.assign((size_t)(n + 1) * cnt * 2, 0);
+    t.maxext.assign(n + 1, 0);
+    for (int r = 0; r < cnt; ++r) {
+        Span s = cuts[r], c = cuts[r];
+        for (int m = n; m >= 0; --m) {
+            if (m < n) {
+                s = back_project(s, ax.K[m], ax.S[m], ax.P[m], ax.ext[m]);
+                c = Span{c.a * ax.S[m], c.b * ax.S[m] + ax.S[m] - 1};
+            }
+            t.span[((size_t)m * cnt + r) * 2 + 0] = s.a;
+            t.span[((size_t)m * cnt + r) * 2 + 1] = s.b;
+            t.cell[((size_t)m * cnt + r) * 2 + 0] = c.a;
+            t.cell[((size_t)m * cnt + r) * 2 + 1] = c.b;
+            t.maxext[m] = std::max(t.maxext[m], extent(s));
+        }
+    }
+    t.scratch_off.assign(cnt + 1, 0);
+    for (int r = 0; r < cnt; ++r)
+        t.scratch_off[r + 1] = t.scratch_off[r] + (t.span[(size_t)r * 2 + 1] - t.span[(size_t)r * 2] + 1);
+    t.cover.assign((size_t)ax.ext[0] * 2, 0);
+    for (int pos = 0; pos < ax.ext[0]; ++pos) {
+        int lo = -1, hi = -1;
+        for (int r = 0; r < cnt; ++r)
+            if (t.span[(size_t)r * 2] <= pos && pos <= t.span[(size_t)r * 2 + 1]) {
+                if (lo < 0) lo = r;
+                hi = r;
+            }
+        t.cover[(size_t)pos * 2] = lo;
+        t.cover[(size_t)pos * 2 + 1] = hi;
+    }
+}
+
+AxisInfo axis_info(const GroupPlan& g, bool y_axis)
+{
+    AxisInfo ax{};
+    ax.n_ops = g.n_ops;
+    for (int i = 0; i < g.n_ops; ++i) {
+        const OpDesc& op = g.fwd_ops[i];
+        ax.K[i] = op.keff; ax.S[i] = op.S; ax.P[i] = op.pad;
+        ax.ext[i] = y_axis ? op.in_H : op.in_W;
+        ax.ext[i + 1] = y_axis ? op.out_H : op.out_W;
+    }
+    return ax;
+}
+
+// Shared-memory geometry of the forward pass.  The input buffers of consecutive ops sit at
+// opposite ends of the dynamic area (even ops at the bottom, odd ops at the top), so the area
+// only has to hold the largest pair of neighbours.  Returns bytes incl. header.
+size_t layout_forward(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
+{
+    int size[kMaxOps + 1] = {0};
+    for (int i = 0; i < g.n_ops; ++i) {
+        OpDesc& op = g.fwd_ops[i];
+        int oh = ty.maxext[i + 1], ow = tx.maxext[i + 1];
+        int bh = (oh - 1) * op.S + op.keff, bw = (ow - 1) * op.S + op.keff;
+        op.in_pitch = bw;
+        op.in_cs = bh * bw;
+        size[i] = round4(op.cin * op.in_cs);
+    }
+    int total = 0;
+    for (int i = 0; i < g.n_ops; ++i) total = std::max(total, size[i] + size[i + 1]);
+    for (int i = 0; i < g.n_ops; ++i) g.fwd_ops[i].in_off = (i % 2 == 0) ? 0 : total - size[i];
+    return (size_t)kSmemHeader + 4 * (size_t)total;
+}
+
+// Backward: while op i runs, the delta at its output (D_i), a copy of its input and the delta it
+// produces (D_{i-1}) are alive.  Successive D buffers alternate between the two ends of the area
+// and the input copy sits next to the bottom one, so the area holds the largest such triple.
+size_t layout_backward(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
+{
+    const int n = g.n_ops;
+    int dsize[kMaxOps], xsize[kMaxOps];
+    for (int i = 0; i < n; ++i) {
+        OpDesc& op = g.bwd_ops[i];
+        int oh = ty.maxext[i + 1], ow = tx.maxext[i + 1];
+        int bh = (oh - 1) * op.S + op.keff, bw = (ow - 1) * op.S + op.keff;
+        op.in_pitch = bw;
+        op.in_cs = bh * bw;
+        xsize[i] = round4(op.cin * op.in_cs);
+        op.d_pitch = ow;
+        op.d_cs = oh * ow;
+        int dfl = round4(op.cout * op.d_cs);
+        op.d_arg_off = dfl * 4;                       // relative to the D buffer, fixed up below
+        dsize[i] = dfl + (op.kind == kOpConvPool ? round4((op.cout * op.d_cs + 3) / 4) : 0);
+    }
+    int total = 0;
+    for (int i = 0; i < n; ++i) total = std::max(total, dsize[i] + xsize[i] + (i > 0 ? dsize[i - 1] : 0));
+    for (int i = 0; i < n; ++i) {
+        OpDesc& op = g.bwd_ops[i];
+        const bool low = ((n - 1 - i) % 2) == 0;
+        op.d_off = low ? 0 : total - dsize[i];
+        op.in_off = low ? dsize[i] : (i > 0 ? dsize[i - 1] : 0);
+        op.d_arg_off += op.d_off * 4;
+    }
+    return (size_t)kSmemHeader + 4 * (size_t)total;
+}
+
+// Smallest split (largest sub-tile) whose buffers fit the shared-memory budget.
+int choose_subtiles(GroupPlan& g, bool backward, const PlanOpts& o)
+{
+    const AxisInfo ay = axis_info(g, true), ax = axis_info(g, false);
+    int max_h = 0, max_w = 0;
+    for (const Span& s : g.tile_y) max_h = std::max(max_h, extent(s));
+    for (const Span& s : g.tile_x) max_w = std::max(max_w, extent(s));
+    PassPlan& pp = backward ? g.bwd : g.fwd;
+    const int kmax = std::max(max_h, max_w);
+    int k0 = 1;
+    if (o.max_subtile > 0) k0 = std::max(1, (kmax + o.max_subtile - 1) / o.max_subtile);
+    for (int k = k0; k <= kmax; ++k) {
+        const int cand[3][2] = {{k, k}, {k + 1, k}, {k, k + 1}};
+        for (const auto& c : cand) {
+            int ky = std::min(c[0], max_h), kx = std::min(c[1], max_w);
+            build_axis(pp.y, ay, g.tile_y, ky);
+            build_axis(pp.x, ax, g.tile_x, kx);
+            size_t bytes = backward ? layout_backward(g, pp.y, pp.x) : layout_forward(g, pp.y, pp.x);
+            if (bytes <= (size_t)o.smem_bytes) {
+                pp.smem_bytes = bytes;
+                return FTP_OK;
+            }
+        }
+    }
+    return FTP_ERR_WORKSPACE;
+}
+
+// Multiply-accumulates of the sub-tile stacks of one pass (halo recomputation included) and of the
+// untiled layers.
+void count_macs(const GroupPlan& g, const PassPlan& pp, double* done, double* untiled)
+{
+    *done = 0; *untiled = 0;
+    for (int i = 0; i < g.n_ops; ++i) {
+        const OpDesc& op = g.fwd_ops[i];
+        if (op.kind == kOpPool) continue;
+        const double f = op.kind == kOpConvPool ? 2.0 : 1.0;     // conv runs at twice the pooled extent
+        const double per_px = (double)op.cin * op.cout * op.k * op.k;
+        const AxisTables& ty = pp.y; const AxisTables& tx = pp.x;
+        double sy = 0, sx = 0;
+        for (int r = 0; r < ty.count; ++r)
+            sy += f * (ty.span[((size_t)(i + 1) * ty.count + r) * 2 + 1] - ty.span[((size_t)(i + 1) * ty.count + r) * 2] + 1);
+        for (int q = 0; q < tx.count; ++q)
+            sx += f * (tx.span[((size_t)(i + 1) * tx.count + q) * 2 + 1] - tx.span[((size_t)(i + 1) * tx.count + q) * 2] + 1);
+        *done += per_px * sy * sx;
+        *untiled += per_px * (f * op.out_H) * (f * op.out_W);
+    }
+}
+
+struct LayerOffsets { std::vector<long long> p_off, wf_off, wb_off; };
+
+// Builds the ops, the sub-tiling and the block counts of one executed group (layers first..last).
+// Returns FTP_ERR_WORKSPACE if nothing fits; *redundancy is the larger of the two passes' ratios of
+// multiply-accumulates executed to untiled ones.
+int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, const PlanOpts& o, GroupPlan& g,
+               double* redundancy)
+{
+    g = GroupPlan{};
+    g.first = first; g.last = last;
+    const int N = p.N, gy = p.grid_y, gx = p.grid_x;
+    const MapShape& out = p.maps[last];
+    g.tile_y = equal_partition(0, out.H, gy);
+    g.tile_x = equal_partition(0, out.W, gx);
+    g.param_begin = -1;
+    long long gp = 0;
+    for (int li = first - 1; li < last; ++li) {
+        const ftp_layer& l = p.layers[li];
+        OpDesc op{};
+        const bool fuse = l.kind == FTP_CONV && li + 1 < last && p.layers[li + 1].kind == FTP_MAXPOOL;
+        const int le = fuse ? li + 1 : li;          // last layer of this op (0-based)
+        op.kind = l.kind == FTP_MAXPOOL ? kOpPool : (fuse ? kOpConvPool : kOpConv);
+        op.cin = p.maps[li].C; op.cout = p.maps[le + 1].C;
+        op.k = l.k; op.pad = l.pad; op.slope = l.leaky;
+        op.S = op.kind == kOpConv ? 1 : 2;
+        op.keff = op.kind == kOpConvPool ? l.k + 1 : l.k;
+        op.prev_has_act = (g.n_ops > 0 && g.fwd_ops[g.n_ops - 1].kind != kOpPool) ? 1 : 0;
+        op.in_map = li + 1; op.out_map = le + 2;
+        op.in_H = p.maps[li].H; op.in_W = p.maps[li].W;
+        op.out_H = p.maps[le + 1].H; op.out_W = p.maps[le + 1].W;
+        if (l.kind == FTP_CONV) {
+            op.cout_pad = (l.cout + kCoutTile - 1) / kCoutTile * kCoutTile;
+            op.cin_pad = (l.cin + kCoutTile - 1) / kCoutTile * kCoutTile;
+            op.wf_off = lo.wf_off[li]; op.wb_off = lo.wb_off[li];
+            op.p_off = lo.p_off[li];
+            if (g.param_begin < 0) g.param_begin = lo.p_off[li];
+            op.gp_off = lo.p_off[li] - g.param_begin;
+            gp = op.gp_off + (long long)l.cout * l.cin * l.k * l.k + l.cout;
+        }
+        g.fwd_ops[g.n_ops] = op;
+        g.bwd_ops[g.n_ops] = op;
+        ++g.n_ops;
+        li = le;
+    }
+    if (g.param_begin < 0) g.param_begin = 0;
+    g.param_floats = (size_t)gp;
+
+    int rc = choose_subtiles(g, false, o);
+    if (rc != FTP_OK) return rc;
+    rc = choose_subtiles(g, true, o);
+    if (rc != FTP_OK) return rc;
+    double bwd_done = 0, bwd_untiled = 0;
+    count_macs(g, g.fwd, &g.macs_done, &g.macs_untiled);
+    count_macs(g, g.bwd, &bwd_done, &bwd_untiled);
+    if (redundancy)
+        *redundancy = g.macs_untiled > 0 ? std::max(g.macs_done, bwd_done) / g.macs_untiled : 1.0;
+
+    g.fwd.blocks = g.fwd.y.count * g.fwd.x.count * N;
+    // backward: `splits` blocks per user tile, each owning one partial gradient set
+    int min_items = 1 << 30;
+    for (int ty = 0; ty < gy; ++ty)
+        for (int tx = 0; tx < gx; ++tx) {
+            int items = N * (g.bwd.y.tile_begin[ty + 1] - g.bwd.y.tile_begin[ty]) *
+                        (g.bwd.x.tile_begin[tx + 1] - g.bwd.x.tile_begin[tx]);
+            min_items = std::min(min_items, items);
+        }
+    g.bwd.splits = std::max(1, std::min(min_items, kSmCount / (gy * gx)));
+    g.bwd.blocks = gy * gx * g.bwd.splits;
+    g.bwd.scratch_floats = (size_t)N * p.maps[first - 1].C * g.bwd.y.scratch_off[g.bwd.y.count] *
+                           g.bwd.x.scratch_off[g.bwd.x.count];
+
+    return FTP_OK;
+}
+
+}  // namespace
+
+int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C, int H, int W,
+               int gy, int gx, const ftp_group* groups, int n_groups, int precision, const PlanOpts& opts)
+{
+    if (!layers || !groups || n_layers <= 0 || n_groups <= 0 || N <= 0 || C <= 0 || H <= 0 || W <= 0 ||
+        gy <= 0 || gx <= 0)
+        return FTP_ERR_ARG;
+    if (opts.max_redundancy_pct < 100 || opts.max_subtile < 0 || opts.smem_bytes < 2 * kSmemHeader || opts.smem_bytes > kSmemBudget)
+        return FTP_ERR_ARG;
+    if (precision != FTP_FP32) return precision == FTP_BF16_FP32ACC ? FTP_ERR_PRECISION : FTP_ERR_ARG;
+    p.layers.assign(layers, layers + n_layers);
+    p.N = N; p.grid_y = gy; p.grid_x = gx; p.precision = precision;
+
+    // layer validation and map shapes X_1 .. X_{L+1}
+    p.maps.clear();
+    p.maps.push_back(MapShape{C, H, W});
+    LayerOffsets lo;
+    lo.p_off.assign(n_layers, 0); lo.wf_off.assign(n_layers, 0); lo.wb_off.assign(n_layers, 0);
+    long long params = 0, wf = 0, wb = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        const ftp_layer& l = p.layers[i];
+        MapShape in = p.maps.back();
+        if (l.kind == FTP_CONV) {
+            if (l.k < 1 || l.k > 7 || l.k % 2 == 0 || l.stride != 1 || l.pad != l.k / 2 || l.cin != in.C ||
+                l.cout <= 0 || !(l.leaky >= 0.0f))
+                return FTP_ERR_LAYERS;
+            p.maps.push_back(MapShape{l.cout, in.H, in.W});
+            lo.p_off[i] = params;
+            params += (long long)l.cout * l.cin * l.k * l.k + l.cout;
+            int cout_pad = (l.cout + kCoutTile - 1) / kCoutTile * kCoutTile;
+            int cin_pad = (l.cin + kCoutTile - 1) / kCoutTile * kCoutTile;
+            lo.wf_off[i] = wf; wf += (long long)l.cin * l.k * l.k * cout_pad;
+            lo.wb_off[i] = wb; wb += (long long)l.cout * l.k * l.k * cin_pad;
+        } else if (l.kind == FTP_MAXPOOL) {
+            if (l.k != 2 || l.stride != 2 || l.pad != 0 || in.H % 2 || in.W % 2) return FTP_ERR_LAYERS;
+            p.maps.push_back(MapShape{in.C, in.H / 2, in.W / 2});
+        } else {
+            return FTP_ERR_LAYERS;
+        }
+    }
+    p.param_floats = (size_t)params;
+    p.wf_floats = (size_t)wf;
+    p.wb_floats = (size_t)wb;
+
+    // groups: contiguous, covering 1..L
+    int expect = 1;
+    for (int g = 0; g < n_groups; ++g) {
+        if (groups[g].first != expect || groups[g].last < groups[g].first || groups[g].last > n_layers)
+            return FTP_ERR_GROUPS;
+        expect = groups[g].last + 1;
+        const MapShape& out = p.maps[groups[g].last];
+        if (gy > out.H || gx > out.W) return FTP_ERR_GRID;
+    }
+    if (expect != n_layers + 1) return FTP_ERR_GROUPS;
+    p.user_groups.assign(groups, groups + n_groups);
+
+    // executed groups: a requested group is kept whole when a sub-tile stack of a useful size fits in
+    // shared memory, otherwise it is cut greedily into the longest runs of layers that do
+    p.groups.clear();
+    for (int gi = 0; gi < n_groups; ++gi) {
+        int start = groups[gi].first;
+        const int last = groups[gi].last;
+        while (start <= last) {
+            GroupPlan g;
+            double red = 1.0;
+            int chosen = -1;
+            const int hi = std::min(last, start + kMaxOps - 1);
+            if (opts.strict_groups) {
+                if (hi != last) return FTP_ERR_GROUPS;
+                int rc = make_group(p, lo, start, last, opts, g, &red);
+                if (rc != FTP_OK) return rc;
+                chosen = last;
+            } else {
+                // longest run of layers whose halo recomputation stays below the cap in both passes;
+                // a conv is not separated from the pool after it unless nothing else works
+                for (int pass = 0; pass < 3 && chosen < 0; ++pass)
+                    for (int end = hi; end >= start; --end) {
+                        const bool splits_pair = end < last && p.layers[end - 1].kind == FTP_CONV &&
+                                                 p.layers[end].kind == FTP_MAXPOOL;
+                        if (pass == 0 && splits_pair) continue;
+                        int rc = make_group(p, lo, start, end, opts, g, &red);
+                        if (rc == FTP_OK && (pass == 2 || red * 100.0 <= opts.max_redundancy_pct)) { chosen = end; break; }
+                    }
+                if (chosen < 0) return FTP_ERR_WORKSPACE;
+            }
+            p.groups.push_back(g);
+            start = chosen + 1;
+        }
+    }
+    if (p.groups.size() > 64) return FTP_ERR_GROUPS;
+    const int n_exec = (int)p.groups.size();
+
+    // device tables
+    p.tables.clear();
+    auto push = [&](const std::vector<int>& v) { int o = (int)p.tables.size(); p.tables.insert(p.tables.end(), v.begin(), v.end()); return o; };
+    for (GroupPlan& g : p.groups)
+        for (PassPlan* pp : {&g.fwd, &g.bwd}) {
+            pp->dev_yspan = push(pp->y.span);   pp->dev_xspan = push(pp->x.span);
+            pp->dev_ycell = push(pp->y.cell);   pp->dev_xcell = push(pp->x.cell);
+            pp->dev_yoff = push(pp->y.scratch_off); pp->dev_xoff = push(pp->x.scratch_off);
+            pp->dev_ycover = push(pp->y.cover); pp->dev_xcover = push(pp->x.cover);
+            pp->dev_ytile = push(pp->y.tile_begin); pp->dev_xtile = push(pp->x.tile_begin);
+        }
+
+    // workspace layout
+    Workspace& ws = p.ws;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    ws.map_off.assign(n_layers + 1, 0);
+    ws.arg_off.assign(n_layers + 1, 0);
+    for (const GroupPlan& g : p.groups)
+        for (int i = 0; i < g.n_ops; ++i) {
+            const OpDesc& op = g.fwd_ops[i];
+            const MapShape& s = p.maps[op.out_map - 1];
+            ws.map_off[op.out_map - 1] = take((size_t)N * s.C * s.H * s.W * 4);
+            if (op.kind == kOpConvPool) ws.arg_off[op.out_map - 1] = take((size_t)N * s.C * s.H * s.W);
+        }
+    ws.dmap_off.assign(n_exec, 0);
+    for (int gi = 1; gi < n_exec; ++gi) {
+        const MapShape& s = p.maps[p.groups[gi].first - 1];
+        ws.dmap_off[gi] = take((size_t)N * s.C * s.H * s.W * 4);
+    }
+    {
+        const MapShape& s = p.maps[n_layers];
+        ws.dy_off = take((size_t)N * s.C * s.H * s.W * 4);
+        size_t total = (size_t)N * s.C * s.H * s.W;
+        p.loss_blocks = (int)std::min<size_t>(1024, (total + 1023) / 1024);
+        ws.loss_off = take((size_t)p.loss_blocks * 4);
+    }
+    size_t scratch = 0;
+    for (const GroupPlan& g : p.groups) scratch = std::max(scratch, g.bwd.scratch_floats);
+    ws.scratch_off = take(scratch * 4);
+    ws.wf_off = take(p.wf_floats * 4);
+    ws.wb_off = take(p.wb_floats * 4);
+    ws.partial_off = off;
+    for (GroupPlan& g : p.groups) g.partial_off = take((size_t)g.bwd.blocks * g.param_floats * 4);
+    ws.grad_off = take(p.param_floats * 4);
+    ws.total = off;
+    return FTP_OK;
+}
+
+int region(const ftp_plan& p, int pass, int group, int map_index, int ty, int tx, int out[4])
+{
+    if (!out || group < 0 || group >= (int)p.user_groups.size() || pass < 0 || pass > 2) return FTP_ERR_ARG;
+    const ftp_group& g = p.user_groups[group];
+    if (map_index < g.first || map_index > g.last + 1 || ty < 0 || ty >= p.grid_y || tx < 0 || tx >= p.grid_x)
+        return FTP_ERR_ARG;
+    const int m = map_index - g.first;      // 0 = group input
+    Span sy, sx;
+    if (pass == 0 || pass == 1) {
+        const MapShape& om = p.maps[g.last];
+        sy = equal_partition(0, om.H, p.grid_y)[ty];
+        sx = equal_partition(0, om.W, p.grid_x)[tx];
+        for (int i = g.last - g.first; i >= m; --i) {
+            const ftp_layer& l = p.layers[g.first - 1 + i];
+            sy = back_project(sy, l.k, l.stride, l.pad, p.maps[g.first - 1 + i].H);
+            sx = back_project(sx, l.k, l.stride, l.pad, p.maps[g.first - 1 + i].W);
+        }
+    } else {
+        const MapShape& in = p.maps[g.first - 1];
+        sy = equal_partition(0, in.H, p.grid_y)[ty];
+        sx = equal_partition(0, in.W, p.grid_x)[tx];
+        for (int i = 0; i < m; ++i) {
+            const ftp_layer& l = p.layers[g.first - 1 + i];
+            sy = forward_project(sy, l.k, l.stride, l.pad, p.maps[g.first + i].H);
+            sx = forward_project(sx, l.k, l.stride, l.pad, p.maps[g.first + i].W);
+        }
+    }
+    out[0] = sx.a; out[1] = sy.a; out[2] = sx.b; out[3] = sy.b;
+    return FTP_OK;
+}
+
+}  // namespace ftp

@@ -1,0 +1,125 @@
+// Internal plan structures shared by the host planner and the kernel launchers.
+// Host-only logic lives in plan.cpp; nothing here depends on the CUDA runtime.
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+#include "ftp.h"
+
+namespace ftp {
+
+constexpr int kMaxOps      = 16;      // layers per group
+constexpr int kThreads     = 512;     // threads per block of the fused kernels
+constexpr int kSmCount     = 148;     // B200
+constexpr int kSmemBudget  = 225 * 1024;  // dynamic shared memory a block may use
+constexpr int kSmemHeader  = 1024;    // bytes reserved at the start for per-block tables
+constexpr int kCoutTile    = 8;       // output channels per thread task (packed weights are padded to it)
+
+struct Span { int a, b; };            // inclusive interval on one axis
+
+// One layer inside a group, as the kernels see it.
+enum { kOpConv = 0, kOpPool = 1, kOpConvPool = 2 };   // an op is one layer, or a conv fused with the pool after it
+
+struct OpDesc {
+    int   kind;                 // kOpConv / kOpPool / kOpConvPool
+    int   cin, cout, k, pad;    // conv part (pool: cin == cout, k = 2, pad = 0)
+    int   S, keff;              // output -> input coordinate scale and effective window (conv K; pool 2; fused K+1)
+    float slope;
+    int   prev_has_act;         // the producer of this op's input, inside the same group, ends in a leaky ReLU
+    int   in_map, out_map;      // 1-based indices l of the maps X_l this op reads / writes
+    int   in_H, in_W;           // extents of the input map
+    int   out_H, out_W;         // extents of the output map
+    // shared-memory geometry (float offsets from the start of the dynamic area after the header)
+    int   in_off, in_pitch, in_cs;     // forward input buffer / backward copy of the op's input
+    int   d_off, d_pitch, d_cs;        // backward: delta at this op's output (no apron)
+    int   d_arg_off;                   // backward, fused op: byte offset of the arg-max copy (same geometry as d)
+    int   cout_pad, cin_pad;           // channel counts padded to kCoutTile in the packed filters
+    long long wf_off, wb_off;          // float offsets into the packed forward / rotated filters
+    long long p_off;                   // float offset of the filter in params (bias follows it)
+    long long gp_off;                  // float offset of the filter inside the group's partial set
+};
+
+// Axis tables of one (group, pass): for sub-tile index r and map m (0 = group input ... n_ops = output)
+//   span[(m * count + r) * 2 + {0,1}]   clamped span the sub-tile touches at map m
+//   cell[(m * count + r) * 2 + {0,1}]   the part of map m this sub-tile owns (disjoint, covering)
+struct AxisTables {
+    int count = 0;                        // sub-tiles along this axis over the whole map
+    std::vector<int> span, cell;
+    std::vector<int> tile_begin;          // per user tile: first sub-tile index; size tiles + 1
+    std::vector<int> scratch_off;         // prefix sum of span extents at map 0; size count + 1
+    std::vector<int> cover;               // per position of map 0: first and last sub-tile covering it
+    std::vector<int> maxext;              // per map m: max span extent
+};
+
+struct PassPlan {
+    AxisTables y, x;
+    size_t smem_bytes = 0;
+    int blocks = 0;                 // forward: R*Q*N ; backward: tiles * splits
+    int splits = 1;                 // backward: blocks per user tile
+    size_t scratch_floats = 0;      // backward: floats of per-sub-tile group-input deltas (all images)
+    // offsets (in ints) of the tables inside the plan's device table blob
+    int dev_yspan = 0, dev_xspan = 0, dev_ycell = 0, dev_xcell = 0;
+    int dev_yoff = 0, dev_xoff = 0, dev_ycover = 0, dev_xcover = 0;
+    int dev_ytile = 0, dev_xtile = 0;
+};
+
+struct GroupPlan {
+    int first = 0, last = 0;        // 1-based layers
+    int n_ops = 0;
+    OpDesc fwd_ops[kMaxOps];
+    OpDesc bwd_ops[kMaxOps];
+    PassPlan fwd, bwd;
+    std::vector<Span> tile_y, tile_x;   // user-tile partition of the group's output map
+    size_t param_floats = 0;            // floats of this group's partial gradient set
+    long long param_begin = 0;          // offset of the group's first parameter in params
+    size_t partial_off = 0;             // float offset of the group's partial sets in the workspace
+    double macs_done = 0, macs_untiled = 0;
+};
+
+struct MapShape { int C, H, W; };
+
+struct Workspace {                 // byte offsets, all 256-aligned
+    std::vector<size_t> map_off;   // X_2 .. X_{L+1}  (index l-1; entry 0 unused; maps inside a fused op have none)
+    std::vector<size_t> arg_off;   // arg-max bytes of the pooled map X_l written by a fused op (index l-1)
+    std::vector<size_t> dmap_off;  // delta maps at group inputs of groups 1.. (index = group), and slot for dY
+    size_t dy_off = 0;             // loss delta at the last map (ftp_step with target)
+    size_t scratch_off = 0;
+    size_t wf_off = 0, wb_off = 0; // packed filters
+    size_t partial_off = 0;
+    size_t grad_off = 0;           // summed gradient (ftp_step keeps it internal)
+    size_t loss_off = 0;           // per-block partial sums of the MSE
+    size_t total = 0;
+};
+
+}  // namespace ftp
+
+struct ftp_plan {
+    std::vector<ftp_layer> layers;
+    std::vector<ftp::MapShape> maps;        // X_1 .. X_{L+1}; index l-1
+    std::vector<ftp_group> user_groups;     // the requested grouping profile
+    std::vector<ftp::GroupPlan> groups;     // the executed groups (a requested group may be cut, see build_plan)
+    int N = 0, grid_y = 0, grid_x = 0, precision = 0;
+    size_t param_floats = 0;
+    size_t wf_floats = 0, wb_floats = 0;
+    ftp::Workspace ws;
+    std::vector<int> tables;                // host copy of all device tables
+    int*  dev_tables = nullptr;             // uploaded lazily by the first launch
+    int   dev_id = -1;
+    long long launches = 0;
+    int loss_blocks = 0;
+};
+
+namespace ftp {
+struct PlanOpts {
+    int max_redundancy_pct = 150;   // a requested group is cut when its halo recomputation exceeds this (percent of untiled MACs)
+    int max_subtile = 0;            // 0 = as large as fits; else an upper bound (tests use it to force sub-tiling)
+    int smem_bytes = kSmemBudget;   // dynamic shared memory a block may use
+    int strict_groups = 0;          // 1 = never cut a requested group
+};
+// Builds everything but the device upload.  Returns FTP_OK or an error code.
+int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C, int H, int W,
+               int gy, int gx, const ftp_group* groups, int n_groups, int precision, const PlanOpts& opts);
+int region(const ftp_plan& p, int pass, int group, int map_index, int ty, int tx, int out[4]);
+}  // namespace ftp

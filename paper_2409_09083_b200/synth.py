@@ -146,3 +146,37 @@ def draw(wl: Workload, bias_std: float = 0.0, N: Optional[int] = None):
     c, h, w = map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
     target = rng.standard_normal((n, c, h, w), dtype=np.float32)
     return x, params, target
+
+
+def with_slope(wl: Workload, slope: float) -> Workload:
+    """Same workload with another leaky-ReLU slope on every conv layer."""
+    layers = tuple(Layer(l.kind, l.cin, l.cout, l.k, l.stride, l.pad, slope if l.kind == "conv" else 0.0)
+                   for l in wl.layers)
+    return wl.with_(layers=layers)
+
+
+def draw_dyadic(wl: Workload, nnz: int = 3, N: Optional[int] = None):
+    """Inputs whose forward pass is exact in fp32 whatever the summation order:
+    integer pixels in [-3, 3], filters with `nnz` non-zero taps of value +-1 per
+    output channel, biases in {-0.5, 0, 0.5}.  With a dyadic leaky slope (use
+    with_slope(wl, 0.5)) every activation is a small multiple of a power of
+    two, so fp32 and fp64 agree bit for bit and every arg-max and sign decision
+    is the same on both sides (exact ties included).  The target is N(0,1)."""
+    rng = np.random.default_rng(wl.seed + 7919)
+    n = wl.N if N is None else N
+    x = rng.integers(-3, 4, size=(n, wl.C, wl.H, wl.W)).astype(np.float32)
+    parts = []
+    for l in wl.layers:
+        if l.kind != "conv":
+            continue
+        fan = l.cin * l.k * l.k
+        F = np.zeros((l.cout, fan), dtype=np.float32)
+        for co in range(l.cout):
+            idx = rng.choice(fan, size=min(nnz, fan), replace=False)
+            F[co, idx] = rng.choice(np.array([-1.0, 1.0], dtype=np.float32), size=idx.size)
+        parts.append(F.ravel())
+        parts.append(rng.integers(-1, 2, size=l.cout).astype(np.float32) * 0.5)
+    params = np.concatenate(parts)
+    c, h, w = map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    target = rng.standard_normal((n, c, h, w), dtype=np.float32)
+    return x, params, target

@@ -1,0 +1,75 @@
+"""Shared helpers of the GPU parity tests: run the CUDA path through the C-ABI
+binding and the fp64 oracle on the same seeded inputs and compare per tensor."""
+import numpy as np
+import torch
+
+import paper_2409_09083_b200 as ftp
+from oracle import reference as orc
+from paper_2409_09083_b200 import synth
+
+# Tolerance of the fp32 path: per tensor, max_i |a_i - o_i| / max_j |o_j| <= 1e-4.
+FP32_TOL = 1e-4
+
+
+def rel_err(a, o):
+    a = np.asarray(a, dtype=np.float64)
+    o = np.asarray(o, dtype=np.float64)
+    scale = np.abs(o).max()
+    if scale == 0.0:
+        return float(np.abs(a).max())
+    return float(np.abs(a - o).max() / scale)
+
+
+def run_gpu(wl, x, params, target=None, dy=None, want_dx=True, **plan_opts):
+    """forward + backward through the library; returns dict of numpy arrays."""
+    dev = "cuda"
+    plan = ftp.ftp_plan(wl.layers, x.shape[0], wl.C, wl.H, wl.W, wl.grid, wl.groups, **plan_opts)
+    ws = plan.new_workspace(dev)
+    xd = torch.from_numpy(x).to(dev)
+    pd = torch.from_numpy(params).to(dev)
+    c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    y = torch.empty((x.shape[0], c, h, w), dtype=torch.float32, device=dev)
+    ftp.ftp_forward(plan, xd, pd, y, ws)
+    torch.cuda.synchronize()
+    yh = y.cpu().numpy()
+    if dy is None:
+        M = yh.size
+        dy = (2.0 * (yh.astype(np.float64) - target.astype(np.float64)) / M).astype(np.float32)
+    dyd = torch.from_numpy(np.ascontiguousarray(dy)).to(dev)
+    dx = torch.empty_like(xd) if want_dx else None
+    dparams = torch.empty_like(pd)
+    ftp.ftp_backward(plan, xd, dyd, pd, dx, dparams, ws)
+    torch.cuda.synchronize()
+    return dict(plan=plan, y=yh, dy=dy, dx=None if dx is None else dx.cpu().numpy(),
+                dparams=dparams.cpu().numpy())
+
+
+def run_gpu_step(wl, x, params, target, lr, want_dx=True, **plan_opts):
+    dev = "cuda"
+    plan = ftp.ftp_plan(wl.layers, x.shape[0], wl.C, wl.H, wl.W, wl.grid, wl.groups, **plan_opts)
+    ws = plan.new_workspace(dev)
+    xd = torch.from_numpy(x).to(dev)
+    pd = torch.from_numpy(params.copy()).to(dev)
+    td = torch.from_numpy(target).to(dev)
+    loss = torch.zeros(1, dtype=torch.float32, device=dev)
+    dx = torch.empty_like(xd) if want_dx else None
+    ftp.ftp_step(plan, xd, pd, lr, ws, target=td, loss_out=loss, dx=dx)
+    torch.cuda.synchronize()
+    return dict(plan=plan, loss=float(loss.item()), new_params=pd.cpu().numpy(),
+                dx=None if dx is None else dx.cpu().numpy())
+
+
+def run_oracle(wl, x, params, target=None, dy=None, lr=0.0):
+    return orc.step(list(wl.layers), x.astype(np.float64), params.astype(np.float64), lr,
+                    target=None if target is None else target.astype(np.float64),
+                    dy=None if dy is None else dy.astype(np.float64))
+
+
+def per_layer_errors(layers, got, ref):
+    """Relative error of each conv layer's filter and bias gradient."""
+    out = []
+    for i, (g, r) in enumerate(zip(orc.unpack_params(layers, got), orc.unpack_params(layers, ref))):
+        if g is None:
+            continue
+        out.append((i + 1, rel_err(g[0], r[0]), rel_err(g[1], r[1])))
+    return out
