@@ -1,0 +1,273 @@
+#!/usr/bin/env python
+"""Benchmark of the fused tile-partitioned training step.
+
+    python bench.py --gpus N --steps K --warmup W [--workload C1] [--impl reference]
+
+A step is one pass of the whole hot path (forward, loss delta, backward with input gradient,
+cross-tile reduction of the partial gradient sets, SGD update) over one batch of synthetic input.
+Rank 0 prints ONE JSON line.  With --gpus N > 1 (launched by torchrun, one rank per GPU) every
+rank runs the one-GPU path on its own batch (weak scaling) and the summed gradients are
+all-reduced over NCCL before the update.  --impl reference times the CPU oracle instead.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2409_09083_b200 import synth  # noqa: E402
+
+METRIC = "train-step images/sec (fwd+bwd+dW reduce+SGD)"
+UNIT = "images/s"
+# fp32 FMA peak of the CUDA cores: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (derived, not measured)
+FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+KIND = {0: "pack_filters", 1: "fwd_group", 2: "loss_delta", 3: "bwd_group", 4: "halo_sum", 5: "reduce_sgd"}
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="C1", choices=["C0", "C1", "C2", "C3"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def config_of(wl, extra=None):
+    cfg = {"workload": f"{wl.name}: {len(wl.layers)}-layer YOLOv2-style stack, batch {wl.N}x{wl.C}x{wl.H}x{wl.W} fp32, "
+                       f"tile grid {wl.grid[0]}x{wl.grid[1]}, groups {list(wl.groups)}, MSE loss, SGD lr {wl.lr}",
+           "global_batch": wl.N, "tile_grid": list(wl.grid), "groups": [list(g) for g in wl.groups]}
+    cfg.update(extra or {})
+    return cfg
+
+
+def time_oracle(wl, images, steps, warmup):
+    """Seconds per oracle training step on `images` images of the workload (as it stands)."""
+    from oracle import reference as orc
+    x, params, target = synth.draw(wl, N=images)
+    layers = list(wl.layers)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        orc.step(layers, x, params, wl.lr, target=target)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    return sum(times) / len(times), orc.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = synth.workload(args.workload)
+    images = 1
+    sec, cores = time_oracle(wl, images, args.steps, args.warmup)
+    value = images / sec
+    sample = f"each step = one full training step of the fp64 oracle on {images} image of {wl.name} at full resolution"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_of(wl, {"sample_images_per_step": images}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for row in open(self.path):
+                f = [c.strip() for c in row.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    sm.append(float(f[0])); mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, v in zip(names, f[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def run_ours(args):
+    import torch
+    import paper_2409_09083_b200 as ftp
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the training step has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    wl = synth.workload(args.workload).with_(seed=rank)       # per-GPU batch is fixed: weak scaling
+    x, params, target = synth.draw(wl)
+    if world > 1:                                             # same initial parameters on every rank
+        params = synth.draw(wl.with_(seed=0))[1]
+    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups)
+    ws = plan.new_workspace()
+    xd, pd, td = (torch.from_numpy(a).cuda() for a in (x, params, target))
+    dx = torch.empty_like(xd)
+    grad = torch.empty_like(pd)
+    loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB L2
+
+    def step():
+        if world == 1:
+            ftp.ftp_step(plan, xd, pd, wl.lr, ws, target=td, loss_out=loss, dx=dx)
+        else:
+            ftp.ftp_step_grad(plan, xd, pd, grad, ws, target=td, loss_out=loss, dx=dx)
+            dist.all_reduce(grad)                             # sum of the per-GPU gradient sums
+            ftp.ftp_sgd(pd, grad, wl.lr / world)              # loss is the mean over the global batch
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    plan.timing(True)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    launches0 = plan.launch_count()
+    per_kind = {}
+    barrier()
+    for a, b in ev:
+        flush.zero_()                                         # evict the previous step from L2 (not timed)
+        a.record()
+        step()
+        b.record()
+        torch.cuda.synchronize()
+        for kind, group, ms in plan.timing_read():
+            per_kind[(kind, group)] = per_kind.get((kind, group), 0.0) + ms
+    barrier()
+    launches = plan.launch_count() - launches0
+    plan.timing(False)
+    total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    clocks = sampler.stop() if sampler else None
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    # end to end: batch and target start in pinned host memory every step, the loss comes back to the host
+    e2e = None
+    if world == 1:
+        xh, th = torch.from_numpy(x).pin_memory(), torch.from_numpy(target).pin_memory()
+        lh = torch.zeros(1, dtype=torch.float32).pin_memory()
+        for _ in range(2):
+            ftp.ftp_step_host(plan, xh, th, pd, wl.lr, lh, ws, dx=dx)
+        torch.cuda.synchronize()
+        ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in ev2:
+            flush.zero_()
+            a.record()
+            ftp.ftp_step_host(plan, xh, th, pd, wl.lr, lh, ws, dx=dx)
+            b.record()
+            torch.cuda.synchronize()
+            _ = float(lh[0])
+        e2e_ms = sum(a.elapsed_time(b) for a, b in ev2)
+        e2e = {"value": wl.N * args.steps / (e2e_ms / 1e3), "unit": UNIT,
+               "h2d_bytes_per_step": int(xh.numel() * 4 + th.numel() * 4), "d2h_bytes_per_step": 4}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    macs = synth.forward_macs_per_image(wl.layers, wl.C, wl.H, wl.W)
+    steps = args.steps
+    ms_step = total_ms / steps
+    breakdown = {}
+    for (kind, group), ms in per_kind.items():
+        breakdown[KIND[kind]] = breakdown.get(KIND[kind], 0.0) + ms / steps
+    # dominant kernel: the fused backward (delta back-propagation + filter gradients = 2 forward-equivalents)
+    bwd_ms = breakdown.get("bwd_group", 0.0)
+    bwd_flops = 4.0 * macs * wl.N
+    n_bwd = sum(1 for (k, g) in per_kind if k == 3)
+    achieved = bwd_flops / (bwd_ms / 1e3) / 1e12 if bwd_ms > 0 else None
+    roofline = {"bound": "alu", "kernel": "bwd_group_kernel", "achieved": achieved, "peak": FP32_PEAK_TFLOPS,
+                "unit": "TFLOP/s", "frac": achieved / FP32_PEAK_TFLOPS if achieved else None, "traffic": None,
+                "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                "launches_per_step": n_bwd, "avg_launch_ms": bwd_ms / n_bwd if n_bwd else None,
+                "algorithmic_flops_per_step": bwd_flops,
+                "step_frac_of_fp32_peak": 6.0 * macs * wl.N / (ms_step / 1e3) / 1e12 / FP32_PEAK_TFLOPS}
+    line = {"metric": METRIC, "value": world * wl.N * steps / (total_ms / 1e3), "unit": UNIT, "n_gpus": world,
+            "steps": steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": config_of(wl, {"global_batch": wl.N * world, "executed_groups": plan.exec_groups(),
+                                     "parallelism": f"dp{world}", "l2": "flushed between timed steps (256 MiB write)",
+                                     "redundancy_fwd": plan.redundancy}),
+            "clocks": clocks, "gpu_launches": int(launches), "breakdown_ms_per_step": breakdown,
+            "roofline": roofline, "loss": float(loss.item())}
+    if e2e is not None:
+        line["e2e"] = e2e
+    if world == 1 and not args.no_cpu_baseline:
+        images = min(wl.N, 2)
+        sec, cores = time_oracle(wl, images, 1, 0)
+        line["cpu_baseline"] = {"value": images / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"one fp64 oracle training step on {images} image(s) of {wl.name} at full resolution"}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

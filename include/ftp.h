@@ -194,6 +194,43 @@ int ftp_step(ftp_plan* plan, const float* x, const float* dy,
              const float* target, float* params, float lr, float* loss_out,
              float* dx, void* workspace, void* stream);
 
+/*
+ * ftp_step for callers whose batch lives in HOST memory: copies x_host and target_host
+ * (pinned memory recommended; shapes as in ftp_step) into staging areas of the workspace,
+ * runs the training cycle with the mean-squared-error loss and copies the loss (1 float) to
+ * loss_host, all enqueued on `stream`; loss_host is valid once the stream is synchronised.
+ * params stays in device memory and is updated in place.  dx (device, may be NULL) receives
+ * dLoss/dX_1 as in ftp_step.
+ */
+int ftp_step_host(ftp_plan* plan, const float* x_host, const float* target_host, float* params,
+                  float lr, float* loss_host, float* dx, void* workspace, void* stream);
+
+/*
+ * The two halves of ftp_step for data-parallel replicas (one process per GPU, the batch split
+ * across them; Section 4.1 sums the partial gradient sets "once per batch", which across GPUs is
+ * an all-reduce the caller runs between these two calls):
+ * ftp_step_grad = ftp_step without the update: forward, loss delta, backward, and the fixed-order
+ *   sum of this GPU's partial sets written to dparams (device, same layout as params).
+ * ftp_sgd = params[i] -= lr * grad[i] for i < count (device pointers).
+ */
+int ftp_step_grad(ftp_plan* plan, const float* x, const float* dy, const float* target,
+                  const float* params, float* dparams, float* loss_out, float* dx,
+                  void* workspace, void* stream);
+int ftp_sgd(float* params, const float* grad, size_t count, float lr, void* stream);
+
+/*
+ * Per-launch device timing for benchmarks.  ftp_plan_timing(plan, 1) makes every later call on
+ * this plan record a CUDA event before and after each kernel it launches, on the stream it
+ * launches on (events are created here, not in the hot path); 0 switches it off and frees them.
+ * After synchronising the stream, ftp_plan_timing_read returns, for the launches of the most
+ * recent ftp_forward / ftp_backward / ftp_step* call(s) since the last read, up to `capacity`
+ * records {kind, group, milliseconds}: kind 0 filter packing, 1 fused forward, 2 loss delta,
+ * 3 fused backward, 4 halo sum, 5 reduction (+SGD); group = executed-group index or -1.
+ */
+typedef struct { int kind; int group; float ms; } ftp_launch_time;
+int ftp_plan_timing(ftp_plan* plan, int enable);
+int ftp_plan_timing_read(ftp_plan* plan, int* n, ftp_launch_time* out, int capacity);
+
 /* Number of kernels the library launched on the calling thread's behalf since
  * the plan was created (for launch accounting in benchmarks). */
 long long ftp_plan_launch_count(const ftp_plan* plan);

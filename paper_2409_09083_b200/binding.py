@@ -65,6 +65,22 @@ _lib.ftp_backward.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.ftp_backward.restype = _i
 _lib.ftp_step.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp, _vp, _vp]
 _lib.ftp_step.restype = _i
+_lib.ftp_step_host.argtypes = [_vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp, _vp, _vp]
+_lib.ftp_step_host.restype = _i
+_lib.ftp_step_grad.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.ftp_step_grad.restype = _i
+_lib.ftp_sgd.argtypes = [_vp, _vp, _sz, ctypes.c_float, _vp]
+_lib.ftp_sgd.restype = _i
+
+
+class ftp_launch_time(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int), ("group", ctypes.c_int), ("ms", ctypes.c_float)]
+
+
+_lib.ftp_plan_timing.argtypes = [_vp, _i]
+_lib.ftp_plan_timing.restype = _i
+_lib.ftp_plan_timing_read.argtypes = [_vp, ctypes.POINTER(_i), ctypes.POINTER(ftp_launch_time), _i]
+_lib.ftp_plan_timing_read.restype = _i
 _lib.ftp_plan_launch_count.argtypes = [_vp]
 _lib.ftp_plan_launch_count.restype = ctypes.c_longlong
 _lib.ftp_strerror.argtypes = [_i]
@@ -165,6 +181,17 @@ class Plan:
     def launch_count(self):
         return int(_lib.ftp_plan_launch_count(self._h))
 
+    def timing(self, enable=True):
+        _check(_lib.ftp_plan_timing(self._h, 1 if enable else 0))
+
+    def timing_read(self):
+        """[(kind, group, ms)] of the launches since the last read; synchronise the stream first."""
+        cap = 512
+        arr = (ftp_launch_time * cap)()
+        n = _i()
+        _check(_lib.ftp_plan_timing_read(self._h, ctypes.byref(n), arr, cap))
+        return [(arr[i].kind, arr[i].group, arr[i].ms) for i in range(min(n.value, cap))]
+
     def new_workspace(self, device="cuda"):
         return torch.empty(self.workspace_bytes, dtype=torch.uint8, device=device)
 
@@ -188,3 +215,23 @@ def ftp_step(plan, x, params, lr, workspace, dy=None, target=None, loss_out=None
     _check(_lib.ftp_step(plan._h, _ptr(x, "x"), _ptr(dy, "dy", True), _ptr(target, "target", True),
                          _ptr(params, "params"), float(lr), _ptr(loss_out, "loss_out", True),
                          _ptr(dx, "dx", True), workspace.data_ptr(), _stream(stream)))
+
+
+def ftp_step_grad(plan, x, params, dparams, workspace, dy=None, target=None, loss_out=None, dx=None, stream=None):
+    _check(_lib.ftp_step_grad(plan._h, _ptr(x, "x"), _ptr(dy, "dy", True), _ptr(target, "target", True),
+                              _ptr(params, "params"), _ptr(dparams, "dparams"), _ptr(loss_out, "loss_out", True),
+                              _ptr(dx, "dx", True), workspace.data_ptr(), _stream(stream)))
+
+
+def ftp_sgd(params, grad, lr, stream=None):
+    _check(_lib.ftp_sgd(_ptr(params, "params"), _ptr(grad, "grad"), params.numel(), float(lr), _stream(stream)))
+
+
+def ftp_step_host(plan, x_host, target_host, params, lr, loss_host, workspace, dx=None, stream=None):
+    """x_host, target_host, loss_host: float32 CPU tensors (pinned memory recommended)."""
+    for name, t in (("x_host", x_host), ("target_host", target_host), ("loss_host", loss_host)):
+        if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous float32 CPU tensor")
+    _check(_lib.ftp_step_host(plan._h, x_host.data_ptr(), target_host.data_ptr(), _ptr(params, "params"),
+                              float(lr), loss_host.data_ptr(), _ptr(dx, "dx", True), workspace.data_ptr(),
+                              _stream(stream)))

@@ -1,6 +1,7 @@
 // C-ABI entry points: argument checks, lazy upload of the plan tables, kernel launches.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdint>
 #include <cstring>
 #include <new>
@@ -32,6 +33,23 @@ int ensure_device(ftp_plan* p)
 }
 
 inline bool launched_ok() { return cudaGetLastError() == cudaSuccess; }
+
+constexpr int kMaxTimed = 512;
+
+// Brackets one kernel launch with events when timing is on, and counts the launch.
+struct Timed {
+    ftp_plan* p; cudaStream_t st; int slot = -1;
+    Timed(ftp_plan* plan, cudaStream_t s, int kind, int group) : p(plan), st(s)
+    {
+        ++p->launches;
+        if (p->timing && p->ev_used < (int)p->ev_begin.size()) {
+            slot = p->ev_used++;
+            p->ev_kind[slot] = kind; p->ev_group[slot] = group;
+            cudaEventRecord(static_cast<cudaEvent_t>(p->ev_begin[slot]), st);
+        }
+    }
+    ~Timed() { if (slot >= 0) cudaEventRecord(static_cast<cudaEvent_t>(p->ev_end[slot]), st); }
+};
 
 const float* map_ptr(const ftp_plan* p, const float* x, void* ws, int l /* X_l, 1-based */)
 {
@@ -69,15 +87,15 @@ int pack_filters(ftp_plan* p, const float* params, void* ws, cudaStream_t st)
             const OpDesc& op = g.fwd_ops[i];
             if (op.kind == kOpPool) continue;
             if (pa.n == kMaxOps * 2) {   // flush a full batch
-                pack_filters_kernel<<<dim3(64, pa.n), 256, 0, st>>>(pa, params, ws_ptr(ws, p->ws.wf_off), ws_ptr(ws, p->ws.wb_off));
-                ++p->launches;
+                { Timed t(p, st, 0, -1);
+                  pack_filters_kernel<<<dim3(64, pa.n), 256, 0, st>>>(pa, params, ws_ptr(ws, p->ws.wf_off), ws_ptr(ws, p->ws.wb_off)); }
                 pa.n = 0;
             }
             pa.l[pa.n++] = PackLayer{op.p_off, op.wf_off, op.wb_off, op.cin, op.cout, op.k, op.cout_pad, op.cin_pad};
         }
     if (pa.n) {
+        Timed t(p, st, 0, -1);
         pack_filters_kernel<<<dim3(64, pa.n), 256, 0, st>>>(pa, params, ws_ptr(ws, p->ws.wf_off), ws_ptr(ws, p->ws.wb_off));
-        ++p->launches;
     }
     return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
 }
@@ -86,11 +104,12 @@ int forward_impl(ftp_plan* p, const float* x, const float* params, float* y, voi
 {
     int rc = pack_filters(p, params, ws, st);
     if (rc != FTP_OK) return rc;
-    for (const GroupPlan& g : p->groups) {
+    for (size_t gi = 0; gi < p->groups.size(); ++gi) {
+        const GroupPlan& g = p->groups[gi];
         GroupArgs a;
         fill_common(p, g, false, x, params, ws, a);
-        fwd_group_kernel<<<dim3(a.R * a.Q, p->N), kThreads, g.fwd.smem_bytes, st>>>(a);
-        ++p->launches;
+        { Timed t(p, st, 1, (int)gi);
+          fwd_group_kernel<<<dim3(a.R * a.Q, p->N), kThreads, g.fwd.smem_bytes, st>>>(a); }
         if (!launched_ok()) return FTP_ERR_CUDA;
     }
     if (y) {
@@ -118,8 +137,8 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
         a.param_floats = (long long)g.param_floats;
         a.splits = g.bwd.splits; a.tiles_x = p->grid_x;
         a.need_dx = (gi > 0 || dx != nullptr) ? 1 : 0;
-        bwd_group_kernel<<<g.bwd.blocks, kThreads, g.bwd.smem_bytes, st>>>(a);
-        ++p->launches;
+        { Timed t(p, st, 3, gi);
+          bwd_group_kernel<<<g.bwd.blocks, kThreads, g.bwd.smem_bytes, st>>>(a); }
         if (!launched_ok()) return FTP_ERR_CUDA;
         if (a.need_dx) {
             const MapShape& s = p->maps[g.first - 1];
@@ -132,8 +151,8 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
             h.Htot = g.bwd.y.scratch_off[a.R]; h.Wtot = g.bwd.x.scratch_off[a.Q];
             const size_t total = (size_t)p->N * s.C * s.H * s.W;
             const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16);
-            halo_sum_kernel<<<blocks, 256, 0, st>>>(h);
-            ++p->launches;
+            { Timed t(p, st, 4, gi);
+              halo_sum_kernel<<<blocks, 256, 0, st>>>(h); }
             if (!launched_ok()) return FTP_ERR_CUDA;
         }
     }
@@ -145,8 +164,8 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
     if (ra.n) {
         const long long total = (long long)p->param_floats;
         const int blocks = (int)std::min<long long>((total + 255) / 256, (long long)kSmCount * 16);
-        reduce_sgd_kernel<<<blocks, 256, 0, st>>>(ra, total, sgd_params, lr, grad_out);
-        ++p->launches;
+        { Timed t(p, st, 5, -1);
+          reduce_sgd_kernel<<<blocks, 256, 0, st>>>(ra, total, sgd_params, lr, grad_out); }
         if (!launched_ok()) return FTP_ERR_CUDA;
     }
     return FTP_OK;
@@ -203,6 +222,7 @@ int ftp_plan_exec_groups(const ftp_plan* plan, int* n_groups, ftp_group* groups_
 void ftp_plan_destroy(ftp_plan* plan)
 {
     if (!plan) return;
+    ftp_plan_timing(plan, 0);
     if (plan->dev_tables) cudaFree(plan->dev_tables);
     delete plan;
 }
@@ -262,8 +282,9 @@ int ftp_backward(ftp_plan* plan, const float* x, const float* dy, const float* p
     return backward_impl(plan, x, dy, params, dx, dparams, nullptr, 0.f, workspace, st);
 }
 
-int ftp_step(ftp_plan* plan, const float* x, const float* dy, const float* target, float* params, float lr,
-             float* loss_out, float* dx, void* workspace, void* stream)
+static int step_impl(ftp_plan* plan, const float* x, const float* dy, const float* target, const float* params,
+                     float* sgd_params, float lr, float* grad_out, float* loss_out, float* dx, void* workspace,
+                     void* stream)
 {
     if (!plan || !x || !params || !workspace || !aligned256(workspace)) return FTP_ERR_ARG;
     if ((dy == nullptr) == (target == nullptr)) return FTP_ERR_ARG;
@@ -278,17 +299,91 @@ int ftp_step(ftp_plan* plan, const float* x, const float* dy, const float* targe
         const size_t M = (size_t)plan->N * s.C * s.H * s.W;
         float* d = ws_ptr(workspace, plan->ws.dy_off);
         float* sums = ws_ptr(workspace, plan->ws.loss_off);
-        mse_delta_kernel<<<plan->loss_blocks, 256, 0, st>>>(map_ptr(plan, x, workspace, (int)plan->layers.size() + 1),
-                                                           target, d, M, sums);
-        ++plan->launches;
+        { Timed t(plan, st, 2, -1);
+          mse_delta_kernel<<<plan->loss_blocks, 256, 0, st>>>(map_ptr(plan, x, workspace, (int)plan->layers.size() + 1),
+                                                             target, d, M, sums); }
         if (loss_out) {
+            Timed t(plan, st, 2, -1);
             mse_finish_kernel<<<1, 32, 0, st>>>(sums, plan->loss_blocks, M, loss_out);
-            ++plan->launches;
         }
         if (!launched_ok()) return FTP_ERR_CUDA;
         delta = d;
     }
-    return backward_impl(plan, x, delta, params, dx, nullptr, params, lr, workspace, st);
+    return backward_impl(plan, x, delta, params, dx, grad_out, sgd_params, lr, workspace, st);
+}
+
+int ftp_step(ftp_plan* plan, const float* x, const float* dy, const float* target, float* params, float lr,
+             float* loss_out, float* dx, void* workspace, void* stream)
+{
+    return step_impl(plan, x, dy, target, params, params, lr, nullptr, loss_out, dx, workspace, stream);
+}
+
+int ftp_step_host(ftp_plan* plan, const float* x_host, const float* target_host, float* params, float lr,
+                  float* loss_host, float* dx, void* workspace, void* stream)
+{
+    if (!plan || !x_host || !target_host || !params || !workspace || !aligned256(workspace)) return FTP_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const MapShape& in = plan->maps.front();
+    const MapShape& out = plan->maps.back();
+    float* xs = ws_ptr(workspace, plan->ws.x_stage_off);
+    float* ts = ws_ptr(workspace, plan->ws.t_stage_off);
+    float* lv = ws_ptr(workspace, plan->ws.loss_val_off);
+    if (cudaMemcpyAsync(xs, x_host, (size_t)plan->N * in.C * in.H * in.W * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ts, target_host, (size_t)plan->N * out.C * out.H * out.W * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return FTP_ERR_CUDA;
+    int rc = step_impl(plan, xs, nullptr, ts, params, params, lr, nullptr, lv, dx, workspace, stream);
+    if (rc != FTP_OK) return rc;
+    if (loss_host && cudaMemcpyAsync(loss_host, lv, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FTP_ERR_CUDA;
+    return FTP_OK;
+}
+
+int ftp_step_grad(ftp_plan* plan, const float* x, const float* dy, const float* target, const float* params,
+                  float* dparams, float* loss_out, float* dx, void* workspace, void* stream)
+{
+    if (!dparams) return FTP_ERR_ARG;
+    return step_impl(plan, x, dy, target, params, nullptr, 0.f, dparams, loss_out, dx, workspace, stream);
+}
+
+int ftp_sgd(float* params, const float* grad, size_t count, float lr, void* stream)
+{
+    if (!params || !grad) return FTP_ERR_ARG;
+    if (count == 0) return FTP_OK;
+    const int blocks = (int)std::min<size_t>((count + 255) / 256, (size_t)kSmCount * 16);
+    sgd_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(params, grad, count, lr);
+    return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
+}
+
+int ftp_plan_timing(ftp_plan* plan, int enable)
+{
+    if (!plan) return FTP_ERR_ARG;
+    for (void* e : plan->ev_begin) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+    for (void* e : plan->ev_end) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+    plan->ev_begin.clear(); plan->ev_end.clear(); plan->ev_kind.clear(); plan->ev_group.clear();
+    plan->ev_used = 0;
+    plan->timing = false;
+    if (!enable) return FTP_OK;
+    for (int i = 0; i < kMaxTimed; ++i) {
+        cudaEvent_t a, b;
+        if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return FTP_ERR_CUDA;
+        plan->ev_begin.push_back(a); plan->ev_end.push_back(b);
+    }
+    plan->ev_kind.assign(kMaxTimed, 0); plan->ev_group.assign(kMaxTimed, -1);
+    plan->timing = true;
+    return FTP_OK;
+}
+
+int ftp_plan_timing_read(ftp_plan* plan, int* n, ftp_launch_time* out, int capacity)
+{
+    if (!plan || !n) return FTP_ERR_ARG;
+    *n = plan->ev_used;
+    for (int i = 0; i < plan->ev_used && i < capacity && out; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, static_cast<cudaEvent_t>(plan->ev_begin[i]), static_cast<cudaEvent_t>(plan->ev_end[i])) != cudaSuccess)
+            return FTP_ERR_CUDA;
+        out[i] = ftp_launch_time{plan->ev_kind[i], plan->ev_group[i], ms};
+    }
+    plan->ev_used = 0;
+    return FTP_OK;
 }
 
 long long ftp_plan_launch_count(const ftp_plan* plan) { return plan ? plan->launches : 0; }

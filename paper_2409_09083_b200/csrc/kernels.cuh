@@ -637,6 +637,12 @@ __global__ void reduce_sgd_kernel(const __grid_constant__ ReduceArgs A, long lon
     }
 }
 
+__global__ void sgd_kernel(float* __restrict__ params, const float* __restrict__ grad, size_t count, float lr)
+{
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < count; e += (size_t)gridDim.x * blockDim.x)
+        params[e] = params[e] - lr * grad[e];
+}
+
 // Mean-squared-error loss delta d = 2 (y - t) / M and per-block partial sums of (y - t)^2.
 __global__ void mse_delta_kernel(const float* __restrict__ y, const float* __restrict__ t, float* __restrict__ d,
                                  size_t M, float* __restrict__ block_sums)

@@ -417,6 +417,9 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         size_t total = (size_t)N * s.C * s.H * s.W;
         p.loss_blocks = (int)std::min<size_t>(1024, (total + 1023) / 1024);
         ws.loss_off = take((size_t)p.loss_blocks * 4);
+        ws.loss_val_off = take(4);
+        ws.t_stage_off = take(total * 4);
+        ws.x_stage_off = take((size_t)N * C * H * W * 4);
     }
     size_t scratch = 0;
     for (const GroupPlan& g : p.groups) scratch = std::max(scratch, g.bwd.scratch_floats);

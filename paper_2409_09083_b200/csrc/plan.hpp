@@ -90,6 +90,8 @@ struct Workspace {                 // byte offsets, all 256-aligned
     size_t partial_off = 0;
     size_t grad_off = 0;           // summed gradient (ftp_step keeps it internal)
     size_t loss_off = 0;           // per-block partial sums of the MSE
+    size_t loss_val_off = 0;       // the loss value (ftp_step_host)
+    size_t x_stage_off = 0, t_stage_off = 0;   // device copies of a host batch (ftp_step_host)
     size_t total = 0;
 };
 
@@ -108,6 +110,11 @@ struct ftp_plan {
     int*  dev_tables = nullptr;             // uploaded lazily by the first launch
     int   dev_id = -1;
     long long launches = 0;
+    // optional per-launch timing (see ftp_plan_timing)
+    bool timing = false;
+    std::vector<void*> ev_begin, ev_end;    // cudaEvent_t, pre-created
+    std::vector<int> ev_kind, ev_group;
+    int ev_used = 0;
     int loss_blocks = 0;
 };
 

@@ -73,3 +73,35 @@ def per_layer_errors(layers, got, ref):
             continue
         out.append((i + 1, rel_err(g[0], r[0]), rel_err(g[1], r[1])))
     return out
+
+
+def decision_margin(layers, ref):
+    """Smallest relative margin of the discrete decisions the oracle took: |Z| of every
+    leaky-ReLU input and the gap between the two largest values of every pooling window, each
+    relative to the largest magnitude of its map.  A case whose margin is far above fp32
+    rounding takes the same decisions in fp32 and fp64."""
+    worst = np.inf
+    maps = ref["maps"]
+    for i, l in enumerate(layers):
+        out = maps[i + 1]
+        if l.kind == "conv":
+            worst = min(worst, np.abs(out).min() / max(np.abs(out).max(), 1e-300))
+        else:
+            X = maps[i]
+            N, C, H, W = X.shape
+            w = X.reshape(N, C, H // 2, 2, W // 2, 2).transpose(0, 1, 2, 4, 3, 5).reshape(N, C, H // 2, W // 2, 4)
+            s = np.sort(w, axis=-1)
+            worst = min(worst, (s[..., 3] - s[..., 2]).min() / max(np.abs(X).max(), 1e-300))
+    return float(worst)
+
+
+def draw_unambiguous(wl, bias_std=0.5, tau=2e-5, tries=200):
+    """First seed >= wl.seed whose oracle decisions all have a margin above tau; returns
+    (workload with that seed, x, params, target, oracle result)."""
+    for s in range(wl.seed, wl.seed + tries):
+        w = wl.with_(seed=s)
+        x, params, target = synth.draw(w, bias_std=bias_std)
+        ref = run_oracle(w, x, params, target=target)
+        if decision_margin(list(w.layers), ref) > tau:
+            return w, x, params, target, ref
+    raise RuntimeError("no seed with unambiguous decisions found")

@@ -1,0 +1,181 @@
+"""Parity of the CUDA path (through the C-ABI binding) with the fp64 oracle, element by element
+on the same seeded inputs.  Tolerance of the fp32 path: per tensor
+max|gpu - oracle| / max|oracle| <= 1e-4 for activations, input gradients and weight gradients.
+
+Max-pool arg-max and leaky-ReLU sign are discrete decisions taken on floating-point values; a
+near-tie decided differently in fp32 and fp64 moves a whole delta to another pixel.  Gradient
+parity is therefore checked on inputs where both precisions decide alike: small cases whose
+oracle-side decision margins are verified to be far above fp32 rounding, and larger cases with
+dyadic data whose forward pass is exact in fp32 (activations then also match bit for bit, exact
+ties included).  Activations are checked on the paper-like inputs at every size."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2409_09083_b200 as ftp
+from paper_2409_09083_b200 import synth
+from _util import (FP32_TOL, draw_unambiguous, rel_err, run_gpu, run_gpu_step, run_oracle)
+
+pytestmark = pytest.mark.gpu
+
+W = synth.Workload
+conv, pool = synth.conv, synth.pool
+
+SMALL = {
+    "C0": (synth.workload("C0"), {}),
+    "C0-1x1grid": (synth.workload("C0").with_(grid=(1, 1)), {}),
+    "C0-per-layer": (synth.workload("C0").with_(groups=((1, 1), (2, 2), (3, 3))), {}),
+    "C0-subtiled": (synth.workload("C0"), dict(max_subtile=3)),
+    "C0-16tiles": (synth.workload("C0").with_(grid=(16, 16)), {}),          # one output pixel per tile
+    "one-conv": (W("a", (conv(3, 8, 3),), 2, 3, 20, 28, (2, 2), ((1, 1),), x_dist="normal"), {}),
+    "conv1x1-odd-channels": (W("b", (conv(5, 13, 1),), 2, 5, 10, 14, (2, 3), ((1, 1),), x_dist="normal"), {}),
+    "conv5-pool-conv": (W("c", (conv(2, 6, 5), pool(), conv(6, 4, 3)), 1, 2, 24, 24, (2, 2), ((1, 3),), x_dist="normal"), {}),
+    "conv7": (W("d", (conv(1, 3, 7),), 1, 1, 18, 22, (2, 2), ((1, 1),), x_dist="normal"), {}),
+    "conv-pool": (W("e", (conv(3, 8, 3), pool()), 1, 3, 16, 24, (2, 2), ((1, 2),), x_dist="normal"), {}),
+    "pool-first": (W("f", (pool(), conv(3, 8, 3), pool(), pool()), 1, 3, 32, 48, (2, 2), ((1, 4),), x_dist="normal"), {}),
+    "pool|conv-split": (W("g", (conv(3, 6, 3), pool(), conv(6, 5, 3)), 3, 3, 12, 20, (3, 2), ((1, 1), (2, 3)), x_dist="normal"), {}),
+}
+
+
+@pytest.mark.parametrize("name", sorted(SMALL))
+def test_small_cases_match_oracle(name):
+    wl, opts = SMALL[name]
+    wl, x, params, target, ref = draw_unambiguous(wl)
+    got = run_gpu(wl, x, params, target=target, **opts)
+    assert rel_err(got["y"], ref["y"]) <= FP32_TOL
+    ref = run_oracle(wl, x, params, dy=got["dy"])     # same loss delta on both sides
+    assert rel_err(got["dx"], ref["dx"]) <= FP32_TOL
+    assert rel_err(got["dparams"], ref["dparams"]) <= FP32_TOL
+
+
+@pytest.mark.parametrize("name", ["C0", "conv5-pool-conv", "pool|conv-split"])
+def test_step_updates_parameters_like_the_oracle(name):
+    wl, opts = SMALL[name]
+    wl, x, params, target, ref = draw_unambiguous(wl)
+    lr = 0.05
+    ref = run_oracle(wl, x, params, target=target, lr=lr)
+    got = run_gpu_step(wl, x, params, target, lr, **opts)
+    assert got["loss"] == pytest.approx(ref["loss"], rel=1e-5)
+    assert rel_err(got["new_params"] - params, ref["new_params"] - params) <= FP32_TOL
+    assert rel_err(got["dx"], ref["dx"]) <= FP32_TOL
+    # without dx the same update must come out
+    got2 = run_gpu_step(wl, x, params, target, lr, want_dx=False, **opts)
+    assert np.array_equal(got2["new_params"], got["new_params"])
+
+
+Y8 = W("y8", tuple(synth.stack_yolo8()), 2, 3, 64, 96, (3, 3), ((1, 8),))
+Y16 = W("y16", tuple(synth.stack_yolo16()), 1, 3, 96, 160, (5, 5), ((1, 4), (5, 8), (9, 16)))
+DYADIC = {
+    "yolo8-one-group": (Y8, 3, {}),
+    "yolo8-strict-one-group": (Y8, 3, dict(strict_groups=True)),
+    "yolo8-two-groups-4x4": (Y8.with_(grid=(4, 4), groups=((1, 4), (5, 8))), 3, {}),
+    "yolo8-per-layer": (Y8.with_(groups=synth.groups_per_layer(Y8.layers)), 3, {}),
+    "yolo8-per-maxpool": (Y8.with_(groups=synth.groups_per_maxpool(Y8.layers)), 3, {}),
+    "yolo8-subtile4": (Y8.with_(grid=(2, 2), groups=((1, 4), (5, 8))), 3, dict(max_subtile=4)),
+    "yolo8-ragged-5x7grid": (Y8.with_(H=88, W=104, grid=(5, 7), groups=((1, 2), (3, 8))), 3, {}),
+    "yolo8-1x1grid": (Y8.with_(grid=(1, 1), N=3), 3, {}),
+    "yolo16-three-groups": (Y16, 2, {}),
+    "yolo16-all-in-one": (Y16.with_(groups=((1, 16),), grid=(2, 3)), 2, {}),
+}
+
+
+@pytest.mark.parametrize("name", sorted(DYADIC))
+def test_mid_size_stacks_match_oracle(name):
+    wl, nnz, opts = DYADIC[name]
+    wl = synth.with_slope(wl, 0.5)
+    x, params, target = synth.draw_dyadic(wl, nnz=nnz)
+    ref = run_oracle(wl, x, params, target=target)
+    got = run_gpu(wl, x, params, target=target, **opts)
+    assert np.array_equal(got["y"].astype(np.float64), ref["y"])       # forward is exact
+    assert rel_err(got["dx"], ref["dx"]) <= FP32_TOL
+    assert rel_err(got["dparams"], ref["dparams"]) <= FP32_TOL
+
+
+def test_result_does_not_depend_on_grid_or_groups_and_is_reproducible():
+    wl = Y8
+    x, params, target = synth.draw(wl, bias_std=0.1)
+    rng = np.random.default_rng(1)
+    dy = rng.standard_normal((wl.N, 128, 8, 12)).astype(np.float32)
+    base = run_gpu(wl.with_(grid=(1, 1)), x, params, dy=dy, strict_groups=True)
+    again = run_gpu(wl.with_(grid=(1, 1)), x, params, dy=dy, strict_groups=True)
+    for k in ("y", "dx", "dparams"):
+        assert np.array_equal(base[k], again[k]), f"{k} differs from run to run"
+    variants = [dict(grid=(3, 3)), dict(grid=(4, 2), groups=((1, 4), (5, 8))),
+                dict(grid=(2, 5), groups=synth.groups_per_layer(wl.layers)), dict(grid=(8, 12))]
+    for v in variants:
+        got = run_gpu(wl.with_(**v), x, params, dy=dy)
+        assert np.array_equal(got["y"], base["y"])                   # same arithmetic per output value
+        assert rel_err(got["dx"], base["dx"]) <= 1e-5                # sums in another order
+        assert rel_err(got["dparams"], base["dparams"]) <= 1e-5
+
+
+def _crop_check(wl, x, params, y_gpu, n, oy, ox, size):
+    """Oracle forward on a crop that contains the receptive field of y[n, :, oy:oy+size, ox:ox+size]."""
+    from oracle import spans
+    layers = list(wl.layers)
+    shapes = synth.map_shapes(layers, wl.C, wl.H, wl.W)
+    scale = wl.H // shapes[-1][1]
+    def crop_axis(o, extent_out, extent_in):
+        a, b = spans.forward_spans(layers, extent_out, (o, o + size - 1))[0]
+        a = (a // scale) * scale
+        b = min(extent_in, -(-(b + 1) // scale) * scale)
+        return a, b
+    y0, y1 = crop_axis(oy, shapes[-1][1], wl.H)
+    x0, x1 = crop_axis(ox, shapes[-1][2], wl.W)
+    sub = wl.with_(H=y1 - y0, W=x1 - x0, N=1)
+    from oracle import reference as orc
+    maps, _ = orc.forward(list(sub.layers), x[n:n + 1, :, y0:y1, x0:x1].astype(np.float64), params.astype(np.float64))
+    ref = maps[-1][0, :, oy - y0 // scale: oy - y0 // scale + size, ox - x0 // scale: ox - x0 // scale + size]
+    got = y_gpu[n, :, oy:oy + size, ox:ox + size]
+    return float(np.abs(got - ref).max()), float(np.abs(ref).max())
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3"])
+def test_full_size_activations_on_sampled_regions(name):
+    """Benchmark launch configuration, paper-like inputs: output regions sampled at the map
+    corners, at tile boundaries and in the interior, each recomputed by the oracle from the
+    crop of the input that contains its receptive field."""
+    wl = synth.workload(name)
+    x, params, target = synth.draw(wl)
+    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups)
+    ws = plan.new_workspace()
+    xd, pd = torch.from_numpy(x).cuda(), torch.from_numpy(params).cuda()
+    c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    y = torch.empty((wl.N, c, h, w), dtype=torch.float32, device="cuda")
+    ftp.ftp_forward(plan, xd, pd, y, ws)
+    torch.cuda.synchronize()
+    yh = y.cpu().numpy()
+    scale = float(np.abs(yh).max())
+    size = 4
+    ty = h // wl.grid[0]
+    spots = [(0, 0, 0), (wl.N - 1, h - size, w - size), (wl.N // 2, ty - 2, ty - 2), (0, h // 2, w // 3),
+             (wl.N - 1, 0, w - size)]
+    for n, oy, ox in spots:
+        err, _ = _crop_check(wl, x, params, yh, n, oy, ox, size)
+        assert err / scale <= FP32_TOL, (n, oy, ox, err / scale)
+
+
+@pytest.mark.parametrize("name,images", [("C1", None), ("C2", None), ("C3", (0, 15))])
+def test_full_size_gradients(name, images):
+    """Benchmark launch configuration with dyadic data (forward exact, so both sides take the
+    same arg-max and sign decisions).  C1 and C2: the whole batch against the oracle.  C3: the
+    loss delta is zero except on two images, so the batch's filter gradient equals the oracle's
+    on those two images alone (the gradient is a sum over images)."""
+    wl = synth.with_slope(synth.workload(name), 0.5)
+    x, params, target = synth.draw_dyadic(wl, nnz=2)
+    c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    rng = np.random.default_rng(3)
+    dy = rng.standard_normal((wl.N, c, h, w)).astype(np.float32)
+    if images is not None:
+        mask = np.zeros(wl.N, dtype=bool)
+        mask[list(images)] = True
+        dy[~mask] = 0.0
+    got = run_gpu(wl, x, params, dy=dy)
+    sel = slice(None) if images is None else list(images)
+    ref = run_oracle(wl.with_(N=len(x[sel])), x[sel], params, dy=dy[sel])
+    assert np.array_equal(got["y"][sel].astype(np.float64), ref["y"])
+    assert rel_err(got["dx"][sel], ref["dx"]) <= FP32_TOL
+    assert rel_err(got["dparams"], ref["dparams"]) <= FP32_TOL
+    if images is not None:
+        rest = [i for i in range(wl.N) if i not in images]
+        assert not got["dx"][rest].any()

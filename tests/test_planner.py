@@ -1,0 +1,150 @@
+"""Host logic: the C-ABI library loads and exports what include/ftp.h declares, the planner
+reproduces Eq. (1)/(2) and the hand-derived spans, and bad arguments turn into error codes.
+No GPU is touched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2409_09083_b200 as ftp
+from oracle import spans
+from paper_2409_09083_b200 import binding, synth
+from test_spans_oracle import STACKS, read_golden
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "ftp.h")).read()
+    names = set(re.findall(r"\b(ftp_[a-z_]+)\s*\(", header))
+    assert {"ftp_plan_create", "ftp_forward", "ftp_backward", "ftp_step"} <= names
+    lib = ctypes.CDLL(os.path.join(ROOT, "paper_2409_09083_b200", "libftp.so"))
+    for n in sorted(names):
+        assert hasattr(lib, n), f"{n} declared in ftp.h but not exported"
+
+
+def test_binding_has_the_same_names():
+    for n in ("ftp_plan", "ftp_forward", "ftp_backward", "ftp_step", "ftp_strerror"):
+        assert callable(getattr(ftp, n))
+
+
+@pytest.mark.parametrize("row", read_golden())
+def test_region_matches_hand_derived_spans(row):
+    stack, first, last, extent, parts, tile, sp = row
+    layers = STACKS[stack]()
+    # put the group under test into a valid profile over the whole stack
+    groups = []
+    if first > 1:
+        groups.append((1, first - 1))
+    groups.append((first, last))
+    if last < len(layers):
+        groups.append((last + 1, len(layers)))
+    size = {"tiny": 32, "yolo8": 416, "yolo16": 608}[stack]
+    plan = ftp.ftp_plan(layers, 1, 3, size, size, (parts, parts), groups)
+    gi = groups.index((first, last))
+    for m, want in zip(range(last + 1, first - 1, -1), sp):
+        x1, y1, x2, y2 = plan.region(0, gi, m, tile, tile)
+        assert (x1, x2) == want and (y1, y2) == want
+        assert plan.region(1, gi, m, tile, tile) == (x1, y1, x2, y2)
+
+
+@pytest.mark.parametrize("name", ["C0", "C1", "C2", "C3"])
+def test_region_equals_span_recursion_on_all_tiles(name):
+    wl = synth.workload(name)
+    plan = ftp.ftp_plan(wl.layers, 1, wl.C, wl.H, wl.W, wl.grid, wl.groups)
+    shapes = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)
+    for gi, (first, last) in enumerate(wl.groups):
+        layers = list(wl.layers[first - 1:last])
+        oh, ow = shapes[last][1], shapes[last][2]
+        ys = [spans.forward_spans(layers, oh, c) for c in spans.equal_partition(oh, wl.grid[0])]
+        xs = [spans.forward_spans(layers, ow, c) for c in spans.equal_partition(ow, wl.grid[1])]
+        for ty in range(wl.grid[0]):
+            for tx in range(wl.grid[1]):
+                for m in range(first, last + 2):
+                    x1, y1, x2, y2 = plan.region(0, gi, m, ty, tx)
+                    assert (y1, y2) == ys[ty][m - first] and (x1, x2) == xs[tx][m - first]
+
+
+def test_gather_form_equals_eq2_for_conv_stack():
+    layers = [synth.conv(3, 4, 3), synth.conv(4, 4, 5), synth.conv(4, 2, 1)]
+    plan = ftp.ftp_plan(layers, 1, 3, 40, 40, (4, 4), [(1, 3)])
+    for t in range(4):
+        a, b = spans.equal_partition(40, 4)[t]
+        for m, l in zip(range(2, 5), layers):
+            a, b = spans.eq2_conv(a, b, l.k, 1)
+            a, b = spans.clamp(a, b, 40)
+            x1, y1, x2, y2 = plan.region(2, 0, m, t, t)
+            assert (x1, x2) == (a, b) and (y1, y2) == (a, b)
+
+
+def test_exec_groups_refine_the_requested_profile():
+    for name in ["C0", "C1", "C2", "C3"]:
+        wl = synth.workload(name)
+        plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups)
+        eg = plan.exec_groups()
+        assert eg[0][0] == 1 and eg[-1][1] == len(wl.layers)
+        for (a, b), (c, d) in zip(eg, eg[1:]):
+            assert c == b + 1
+        starts = {g[0] for g in eg}
+        assert {g[0] for g in wl.groups} <= starts        # every requested boundary is kept
+        assert plan.redundancy >= 1.0
+        assert plan.param_floats == synth.param_count(wl.layers)
+        for gi in range(len(eg)):
+            for pass_ in (0, 1):
+                st = plan.subtiles(pass_, gi)
+                assert st["smem_bytes"] <= 225 * 1024 and st["blocks"] >= 1
+                assert st["rows"] >= wl.grid[0] and st["cols"] >= wl.grid[1]
+    # C2's requested groups fit as they are
+    wl = synth.workload("C2")
+    assert ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups).exec_groups() == list(wl.groups)
+
+
+def test_strict_groups_keeps_or_refuses():
+    wl = synth.workload("C1")
+    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, strict_groups=True)
+    assert plan.exec_groups() == [(1, 8)]
+    wl = synth.workload("C3")
+    with pytest.raises(binding.FtpError) as e:
+        ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, strict_groups=True)
+    assert e.value.code == -5
+
+
+def _code(fn):
+    with pytest.raises(binding.FtpError) as e:
+        fn()
+    return e.value.code
+
+
+def test_argument_errors_are_codes_not_crashes():
+    L = synth.stack_tiny()
+    ok = dict(N=1, C=3, H=32, W=32)
+    mk = lambda layers=L, grid=(2, 2), groups=((1, 3),), **kw: ftp.ftp_plan(
+        layers, kw.get("N", 1), kw.get("C", 3), kw.get("H", 32), kw.get("W", 32), grid, groups,
+        **{k: v for k, v in kw.items() if k not in ok})
+    assert _code(lambda: mk(N=0)) == -1
+    assert _code(lambda: mk(grid=(0, 2))) == -1
+    assert _code(lambda: mk(C=4)) == -2                                   # channel mismatch
+    assert _code(lambda: mk(layers=[synth.Layer("conv", 3, 8, 4, 1, 2, 0.1)], groups=((1, 1),))) == -2   # even kernel
+    assert _code(lambda: mk(layers=[synth.Layer("conv", 3, 8, 3, 2, 1, 0.1)], groups=((1, 1),))) == -2   # stride 2
+    assert _code(lambda: mk(layers=[synth.Layer("conv", 3, 8, 3, 1, 0, 0.1)], groups=((1, 1),))) == -2   # pad != k/2
+    assert _code(lambda: mk(layers=[synth.pool()], groups=((1, 1),), H=31)) == -2                        # odd extent
+    assert _code(lambda: mk(groups=((1, 2),))) == -4                      # not covering
+    assert _code(lambda: mk(groups=((1, 1), (3, 3)))) == -4               # gap
+    assert _code(lambda: mk(groups=((2, 3), (1, 1)))) == -4               # order
+    assert _code(lambda: mk(grid=(17, 2))) == -3                          # more tiles than output rows
+    assert _code(lambda: mk(precision=1)) == -8                           # bf16 path not built
+    assert _code(lambda: mk(precision=5)) == -1
+    assert "shared memory" in ftp.ftp_strerror(-5)
+    assert ftp.ftp_strerror(0) == "ok"
+
+
+def test_null_pointers_are_rejected_on_the_host():
+    wl = synth.workload("C0")
+    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups)
+    lib = binding._lib
+    assert lib.ftp_forward(plan._h, None, None, None, None, None) == -1
+    assert lib.ftp_backward(plan._h, None, None, None, None, None, None, None) == -1
+    assert lib.ftp_step(plan._h, None, None, None, None, 0.0, None, None, None, None) == -1
+    assert lib.ftp_forward(None, None, None, None, None, None) == -1
+    assert plan.launch_count() == 0
