@@ -134,6 +134,7 @@ class ClockSampler:
 def run_ours(args):
     import torch
     import paper_2409_09083_b200 as ftp
+    from paper_2409_09083_b200 import dp
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -163,8 +164,7 @@ def run_ours(args):
             ftp.ftp_step(plan, xd, pd, wl.lr, ws, target=td, loss_out=loss, dx=dx)
         else:
             ftp.ftp_step_grad(plan, xd, pd, grad, ws, target=td, loss_out=loss, dx=dx)
-            dist.all_reduce(grad)                             # sum of the per-GPU gradient sums
-            ftp.ftp_sgd(pd, grad, wl.lr / world)              # loss is the mean over the global batch
+            dp.allreduce_and_update(grad, wl.lr, world, dist.all_reduce, lambda g, lr: ftp.ftp_sgd(pd, g, lr))
 
     def barrier():
         if dist is not None:

@@ -1,0 +1,60 @@
+"""The multi-GPU exchange step on CPU: two gloo ranks, each holding half of the batch, must arrive
+at the update of the whole batch.  The per-rank gradient comes from the oracle here (the CUDA path
+needs a GPU); what is tested is the sharding, the all-reduce and the learning-rate scaling that
+`bench.py --gpus N` uses."""
+import os
+import socket
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from oracle import reference as orc
+from paper_2409_09083_b200 import dp, synth
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _worker(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    wl = synth.workload("C0").with_(N=4)
+    x, params, target = synth.draw(wl, bias_std=0.3)
+    lo, hi = dp.shard_range(wl.N, rank, world)
+    local = orc.step(list(wl.layers), x[lo:hi], params, 0.0, target=target[lo:hi])
+    grad = torch.from_numpy(local["dparams"].copy())
+    new = torch.from_numpy(params.astype(np.float64))
+
+    def sgd(g, lr_eff):
+        new.sub_(lr_eff * g)
+
+    dp.allreduce_and_update(grad, 0.05, world, dist.all_reduce, sgd)
+    np.save(os.path.join(out_dir, f"rank{rank}.npy"), new.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_reproduce_the_full_batch_update(tmp_path):
+    world = 2
+    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    wl = synth.workload("C0").with_(N=4)
+    x, params, target = synth.draw(wl, bias_std=0.3)
+    ref = orc.step(list(wl.layers), x, params, 0.05, target=target)
+    a = np.load(tmp_path / "rank0.npy")
+    b = np.load(tmp_path / "rank1.npy")
+    assert np.array_equal(a, b)
+    assert np.abs(a - ref["new_params"]).max() <= 1e-12 * np.abs(ref["new_params"]).max()
+
+
+def test_shard_ranges_partition_the_batch():
+    for total, world in [(16, 8), (4, 2), (7, 3), (1, 1)]:
+        r = [dp.shard_range(total, k, world) for k in range(world)]
+        assert r[0][0] == 0 and r[-1][1] == total
+        assert all(a[1] == b[0] for a, b in zip(r, r[1:]))
