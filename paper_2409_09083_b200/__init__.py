@@ -11,6 +11,8 @@ _BINDING_NAMES = None
 
 def __getattr__(name):
     import importlib
+    if name in ("build", "binding", "dp"):          # plain submodules: no library needed to import `build`
+        return importlib.import_module("." + name, __name__)
     binding = importlib.import_module(".binding", __name__)
     if hasattr(binding, name):
         return getattr(binding, name)
