@@ -195,6 +195,17 @@ int ftp_step(ftp_plan* plan, const float* x, const float* dy,
              float* dx, void* workspace, void* stream);
 
 /*
+ * The loss-delta injection of the training cycle on its own (Section 3: the initial delta of the
+ * loss enters at the last layer), for callers that drive ftp_forward and ftp_backward themselves:
+ * mean-squared error L = mean((y - target)^2) over the plan's output map X_{L+1}
+ * ([N,C_out,H_out,W_out], y and target), dy = dL/dy = 2 (y - target) / M with M the element count.
+ * dy (device, same shape) and loss_out (device, 1 float) may each be NULL but not both.
+ * Uses a few KB of `workspace` as scratch for per-block partial sums; the sum order is fixed.
+ */
+int ftp_loss_mse(ftp_plan* plan, const float* y, const float* target, float* dy, float* loss_out,
+                 void* workspace, void* stream);
+
+/*
  * ftp_step for callers whose batch lives in HOST memory: copies x_host and target_host
  * (pinned memory recommended; shapes as in ftp_step) into staging areas of the workspace,
  * runs the training cycle with the mean-squared-error loss and copies the loss (1 float) to

@@ -69,6 +69,8 @@ _lib.ftp_step_host.argtypes = [_vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp, _vp
 _lib.ftp_step_host.restype = _i
 _lib.ftp_step_grad.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.ftp_step_grad.restype = _i
+_lib.ftp_loss_mse.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.ftp_loss_mse.restype = _i
 _lib.ftp_sgd.argtypes = [_vp, _vp, _sz, ctypes.c_float, _vp]
 _lib.ftp_sgd.restype = _i
 
@@ -221,6 +223,11 @@ def ftp_step_grad(plan, x, params, dparams, workspace, dy=None, target=None, los
     _check(_lib.ftp_step_grad(plan._h, _ptr(x, "x"), _ptr(dy, "dy", True), _ptr(target, "target", True),
                               _ptr(params, "params"), _ptr(dparams, "dparams"), _ptr(loss_out, "loss_out", True),
                               _ptr(dx, "dx", True), workspace.data_ptr(), _stream(stream)))
+
+
+def ftp_loss_mse(plan, y, target, dy, loss_out, workspace, stream=None):
+    _check(_lib.ftp_loss_mse(plan._h, _ptr(y, "y"), _ptr(target, "target"), _ptr(dy, "dy", True),
+                             _ptr(loss_out, "loss_out", True), workspace.data_ptr(), _stream(stream)))
 
 
 def ftp_sgd(params, grad, lr, stream=None):

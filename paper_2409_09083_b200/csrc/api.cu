@@ -312,6 +312,24 @@ static int step_impl(ftp_plan* plan, const float* x, const float* dy, const floa
     return backward_impl(plan, x, delta, params, dx, grad_out, sgd_params, lr, workspace, st);
 }
 
+int ftp_loss_mse(ftp_plan* plan, const float* y, const float* target, float* dy, float* loss_out, void* workspace,
+                 void* stream)
+{
+    if (!plan || !y || !target || (!dy && !loss_out) || !workspace || !aligned256(workspace)) return FTP_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const MapShape& s = plan->maps.back();
+    const size_t M = (size_t)plan->N * s.C * s.H * s.W;
+    float* d = dy ? dy : ws_ptr(workspace, plan->ws.dy_off);
+    float* sums = ws_ptr(workspace, plan->ws.loss_off);
+    { Timed t(plan, st, 2, -1);
+      mse_delta_kernel<<<plan->loss_blocks, 256, 0, st>>>(y, target, d, M, sums); }
+    if (loss_out) {
+        Timed t(plan, st, 2, -1);
+        mse_finish_kernel<<<1, 32, 0, st>>>(sums, plan->loss_blocks, M, loss_out);
+    }
+    return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
+}
+
 int ftp_step(ftp_plan* plan, const float* x, const float* dy, const float* target, float* params, float lr,
              float* loss_out, float* dx, void* workspace, void* stream)
 {

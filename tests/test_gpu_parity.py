@@ -179,3 +179,24 @@ def test_full_size_gradients(name, images):
     if images is not None:
         rest = [i for i in range(wl.N) if i not in images]
         assert not got["dx"][rest].any()
+
+
+@pytest.mark.parametrize("shape", [(1, 16, 8, 8), (3, 5, 7, 9)])
+def test_loss_mse_matches_oracle(shape):
+    """The loss-delta injection on its own: L = mean((y - t)^2), dy = 2 (y - t) / M."""
+    from oracle import reference as orc
+    N, C, H, Wd = shape
+    wl = W("mse", (conv(2, C, 1),), N, 2, H, Wd, (1, 1), ((1, 1),))
+    plan = ftp.ftp_plan(wl.layers, N, wl.C, H, Wd, wl.grid, wl.groups)
+    ws = plan.new_workspace()
+    rng = np.random.default_rng(5)
+    y = rng.standard_normal(shape).astype(np.float32)
+    t = rng.standard_normal(shape).astype(np.float32)
+    yd, td = torch.from_numpy(y).cuda(), torch.from_numpy(t).cuda()
+    dy = torch.empty_like(yd)
+    loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ftp.ftp_loss_mse(plan, yd, td, dy, loss, ws)
+    torch.cuda.synchronize()
+    ref_loss, ref_dy = orc.mse_loss(y.astype(np.float64), t.astype(np.float64))
+    assert loss.item() == pytest.approx(ref_loss, rel=1e-5)
+    assert rel_err(dy.cpu().numpy(), ref_dy) <= 1e-6
