@@ -48,7 +48,8 @@ enum {
     FTP_ERR_WORKSPACE = -5,  /* no sub-tile of a group fits in shared memory      */
     FTP_ERR_CUDA      = -6,  /* a CUDA runtime call failed                        */
     FTP_ERR_TIMEOUT   = -7,  /* reserved: a bounded device-side wait ran out      */
-    FTP_ERR_PRECISION = -8   /* requested arithmetic is not built                 */
+    FTP_ERR_PRECISION = -8,  /* requested arithmetic is not built                 */
+    FTP_ERR_TOO_LARGE = -9   /* size beyond the fixed capacity of a no-allocation entry point */
 };
 
 enum { FTP_CONV = 0, FTP_MAXPOOL = 1 };
@@ -204,6 +205,40 @@ int ftp_step(ftp_plan* plan, const float* x, const float* dy,
  */
 int ftp_loss_mse(ftp_plan* plan, const float* y, const float* target, float* dy, float* loss_out,
                  void* workspace, void* stream);
+
+/*
+ * ftp_loss_mse for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for the environments named below, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a CUDA stream capture,
+ * under a framework or allocator that owns all device memory and forbids side allocations, in a
+ * real-time loop that must not take the driver's allocation lock, or in a process whose memory
+ * budget is fixed at start-up.  ftp_loss_mse needs a plan (whose first use allocates its tables)
+ * and a workspace; this call needs neither.  It calls no cudaMalloc, no cudaFree and no
+ * allocating library routine.
+ *
+ * Same arithmetic as ftp_loss_mse: L = mean((y - target)^2) over `count` elements,
+ * dy[i] = 2 (y[i] - target[i]) / count.  y, target: device, `count` floats.  dy (device, `count`
+ * floats) and loss_out (device, 1 float) may each be NULL but not both.  The partial sums are
+ * added in a fixed order, which is not ftp_loss_mse's order: the two losses agree to rounding.
+ *
+ * Scratch: the per-block partial sums sit in a fixed 16 KB array inside the library image (every
+ * GPU that loads the library holds it until the process exits).  That fixes the capacity:
+ * count <= FTP_LOSS_STATIC_MAX_COUNT, else FTP_ERR_TOO_LARGE and nothing is launched.
+ *
+ * All calls on one GPU share that array.  Nothing in it has to start at zero (each call overwrites
+ * every slot it later reads), so calls one after the other on a stream need no clearing; two calls
+ * whose kernels overlap on the GPU (different streams, no ordering) race on it and may both return
+ * a wrong loss.  Order them, or use ftp_loss_mse with separate workspaces.
+ *
+ * The first call on each device looks up the array's device address (once, with that device
+ * current, under a host lock); make that first call before any stream capture begins.
+ * Errors: FTP_ERR_ARG (null pointer, count 0, device ordinal >= 64), FTP_ERR_TOO_LARGE,
+ * FTP_ERR_CUDA.
+ */
+#define FTP_LOSS_STATIC_MAX_COUNT (1u << 26)   /* 67 108 864 elements (256 MiB per fp32 tensor) */
+int ftp_loss_mse_static(const float* y, const float* target, float* dy, float* loss_out,
+                        size_t count, void* stream);
 
 /*
  * ftp_step for callers whose batch lives in HOST memory: copies x_host and target_host

@@ -71,6 +71,8 @@ _lib.ftp_step_grad.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.ftp_step_grad.restype = _i
 _lib.ftp_loss_mse.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.ftp_loss_mse.restype = _i
+_lib.ftp_loss_mse_static.argtypes = [_vp, _vp, _vp, _vp, _sz, _vp]
+_lib.ftp_loss_mse_static.restype = _i
 _lib.ftp_sgd.argtypes = [_vp, _vp, _sz, ctypes.c_float, _vp]
 _lib.ftp_sgd.restype = _i
 
@@ -228,6 +230,14 @@ def ftp_step_grad(plan, x, params, dparams, workspace, dy=None, target=None, los
 def ftp_loss_mse(plan, y, target, dy, loss_out, workspace, stream=None):
     _check(_lib.ftp_loss_mse(plan._h, _ptr(y, "y"), _ptr(target, "target"), _ptr(dy, "dy", True),
                              _ptr(loss_out, "loss_out", True), workspace.data_ptr(), _stream(stream)))
+
+
+def ftp_loss_mse_static(y, target, dy, loss_out, stream=None):
+    """MSE loss and delta without a plan, a workspace or any device allocation (see ftp.h)."""
+    if target.numel() != y.numel():
+        raise ValueError("y and target must have the same number of elements")
+    _check(_lib.ftp_loss_mse_static(_ptr(y, "y"), _ptr(target, "target"), _ptr(dy, "dy", True),
+                                    _ptr(loss_out, "loss_out", True), y.numel(), _stream(stream)))
 
 
 def ftp_sgd(params, grad, lr, stream=None):

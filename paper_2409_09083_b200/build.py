@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libftp.so")
-SOURCES = [os.path.join(CSRC, "api.cu"), os.path.join(CSRC, "plan.cpp")]
+SOURCES = [os.path.join(CSRC, "api.cu"), os.path.join(CSRC, "noalloc.cu"), os.path.join(CSRC, "plan.cpp")]
 HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(CSRC, "plan.hpp"),
            os.path.join(ROOT, "include", "ftp.h")]
 

@@ -418,6 +418,7 @@ const char* ftp_strerror(int code)
     case FTP_ERR_CUDA: return "a CUDA runtime call failed";
     case FTP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case FTP_ERR_PRECISION: return "requested arithmetic is not built into this library";
+    case FTP_ERR_TOO_LARGE: return "size exceeds the fixed capacity of this no-allocation entry point";
     default: return "unknown error";
     }
 }
