@@ -47,7 +47,7 @@ enum {
     FTP_ERR_GROUPS    = -4,  /* groups not contiguous or not covering 1..L        */
     FTP_ERR_WORKSPACE = -5,  /* no sub-tile of a group fits in shared memory      */
     FTP_ERR_CUDA      = -6,  /* a CUDA runtime call failed                        */
-    FTP_ERR_TIMEOUT   = -7,  /* reserved: a bounded device-side wait ran out      */
+    FTP_ERR_TIMEOUT   = -7,  /* a bounded device-side wait ran out (ftp_plan_check) */
     FTP_ERR_PRECISION = -8,  /* requested arithmetic is not built                 */
     FTP_ERR_TOO_LARGE = -9   /* size beyond the fixed capacity of a no-allocation entry point */
 };
@@ -280,6 +280,16 @@ int ftp_plan_timing_read(ftp_plan* plan, int* n, ftp_launch_time* out, int capac
 /* Number of kernels the library launched on the calling thread's behalf since
  * the plan was created (for launch accounting in benchmarks). */
 long long ftp_plan_launch_count(const ftp_plan* plan);
+
+/*
+ * Synchronises `stream` and reports whether a kernel of the bf16 tensor-core path gave up on one
+ * of its bounded waits (for a filter stage to arrive or for the tensor core to finish) since the
+ * last ftp_forward / ftp_step* call on this plan and workspace: FTP_ERR_TIMEOUT if so -- the results
+ * of that call are then invalid -- else FTP_OK.  Kernels never wait without a limit; after a
+ * failed wait they skip the remaining waits, release their tensor memory and return.  Always
+ * FTP_OK for the fp32 path, which has no device-side waits.
+ */
+int ftp_plan_check(ftp_plan* plan, void* workspace, void* stream);
 
 const char* ftp_strerror(int code);
 

@@ -123,15 +123,33 @@ def maxpool_backward(dY, arg, in_shape):
     return dX
 
 
-def forward(layers, x, params):
+def round_bf16(a):
+    """Nearest bfloat16 value (8 significant bits, ties to even) of every entry,
+    returned in fp64.  Written from the format's definition: the significand
+    m in [0.5, 1) of a = m * 2^e is rounded to a multiple of 2^-8."""
+    a = np.asarray(a, dtype=np.float64)
+    m, e = np.frexp(a)
+    return np.ldexp(np.rint(m * 256.0) / 256.0, e)
+
+
+def forward(layers, x, params, store=None):
     """Whole-map forward pass. Returns (maps, tape): maps[l-1] = X_l for
-    l = 1..L+1, tape[l-1] = what layer l's backward needs."""
+    l = 1..L+1, tape[l-1] = what layer l's backward needs.
+
+    store="bf16" models a path that keeps its feature maps in bfloat16: the
+    output of every conv layer (after the leaky ReLU) is rounded to bf16 before
+    anything else reads it, so pooling and its arg-max act on the stored
+    values.  Arithmetic inside a layer stays exact.  The paper does not fix a
+    storage precision; None (the default) keeps everything in fp64."""
+    assert store in (None, "bf16")
     per = unpack_params(layers, np.asarray(params, dtype=np.float64))
     maps = [_c(x)]
     tape = []
     for l, fb in zip(layers, per):
         if l.kind == "conv":
             Z, Y = conv_forward(maps[-1], fb[0], fb[1], l.pad, l.leaky)
+            if store:
+                Y = round_bf16(Y)
             tape.append(Z)
             maps.append(Y)
         else:
@@ -149,9 +167,14 @@ def mse_loss(y, target):
     return float(np.sum(diff * diff) / M), 2.0 * diff / M
 
 
-def backward(layers, maps, tape, params, dy):
+def backward(layers, maps, tape, params, dy, store=None):
     """Whole-map backward pass from dL/dX_{L+1} = dy.
-    Returns (dx, dparams flat, deltas) with deltas[l-1] = dL/dX_l."""
+    Returns (dx, dparams flat, deltas) with deltas[l-1] = dL/dX_l.
+
+    store="bf16" models a path that also keeps the delta in front of every
+    conv layer's activation, dL/dZ = dL/dY * leaky'(Z), in bfloat16: it is
+    rounded before the filter, bias and input gradients are formed from it."""
+    assert store in (None, "bf16")
     per = unpack_params(layers, np.asarray(params, dtype=np.float64))
     L = len(layers)
     deltas = [None] * (L + 1)
@@ -159,7 +182,11 @@ def backward(layers, maps, tape, params, dy):
     grads = [None] * L
     for i in range(L - 1, -1, -1):
         l = layers[i]
-        if l.kind == "conv":
+        if l.kind == "conv" and store:
+            dZ = round_bf16(deltas[i + 1] * np.where(tape[i] > 0.0, 1.0, l.leaky))
+            dX, dF, db = conv_backward(maps[i], per[i][0], np.ones_like(dZ), dZ, l.pad, 1.0)
+            grads[i] = (dF, db)
+        elif l.kind == "conv":
             dX, dF, db = conv_backward(maps[i], per[i][0], tape[i], deltas[i + 1],
                                        l.pad, l.leaky)
             grads[i] = (dF, db)
@@ -169,18 +196,19 @@ def backward(layers, maps, tape, params, dy):
     return deltas[0], pack_params(layers, grads), deltas
 
 
-def step(layers, x, params, lr, target=None, dy=None):
+def step(layers, x, params, lr, target=None, dy=None, store=None):
     """One training cycle (forward, back-propagation, filter-gradient sum,
     update; Sections 3 and 4.1): plain SGD, w <- w - lr * dL/dw.
 
     Give either `target` (MSE loss) or `dy` (the loss delta at the last map).
+    `store`: see forward / backward.
     Returns dict(loss, y, dx, dparams, new_params, maps, deltas).
     """
     params = np.asarray(params, dtype=np.float64)
-    maps, tape = forward(layers, x, params)
+    maps, tape = forward(layers, x, params, store)
     loss = None
     if dy is None:
         loss, dy = mse_loss(maps[-1], target)
-    dx, dparams, deltas = backward(layers, maps, tape, params, dy)
+    dx, dparams, deltas = backward(layers, maps, tape, params, dy, store)
     return dict(loss=loss, y=maps[-1], dx=dx, dparams=dparams,
                 new_params=params - lr * dparams, maps=maps, deltas=deltas)

@@ -87,6 +87,8 @@ _lib.ftp_plan_timing_read.argtypes = [_vp, ctypes.POINTER(_i), ctypes.POINTER(ft
 _lib.ftp_plan_timing_read.restype = _i
 _lib.ftp_plan_launch_count.argtypes = [_vp]
 _lib.ftp_plan_launch_count.restype = ctypes.c_longlong
+_lib.ftp_plan_check.argtypes = [_vp, _vp, _vp]
+_lib.ftp_plan_check.restype = _i
 _lib.ftp_strerror.argtypes = [_i]
 _lib.ftp_strerror.restype = ctypes.c_char_p
 
@@ -195,6 +197,10 @@ class Plan:
         n = _i()
         _check(_lib.ftp_plan_timing_read(self._h, ctypes.byref(n), arr, cap))
         return [(arr[i].kind, arr[i].group, arr[i].ms) for i in range(min(n.value, cap))]
+
+    def check(self, workspace, stream=None):
+        """Synchronise and raise FtpError(FTP_ERR_TIMEOUT) if a device-side wait of the bf16 path ran out."""
+        _check(_lib.ftp_plan_check(self._h, workspace.data_ptr(), _stream(stream)))
 
     def new_workspace(self, device="cuda"):
         return torch.empty(self.workspace_bytes, dtype=torch.uint8, device=device)

@@ -8,6 +8,7 @@
 
 #include "ftp.h"
 #include "kernels.cuh"
+#include "kernels_tc.cuh"
 #include "plan.hpp"
 
 using namespace ftp;
@@ -23,7 +24,9 @@ int ensure_device(ftp_plan* p)
     if (p->dev_tables && p->dev_id == dev) return FTP_OK;
     if (p->dev_tables) { cudaFree(p->dev_tables); p->dev_tables = nullptr; }
     if (cudaFuncSetAttribute(fwd_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(bwd_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess)
+        cudaFuncSetAttribute(bwd_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(fwd_group_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(bwd_group_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess)
         return FTP_ERR_CUDA;
     const size_t bytes = p->tables.size() * sizeof(int);
     if (cudaMalloc(&p->dev_tables, bytes) != cudaSuccess) return FTP_ERR_CUDA;
@@ -100,8 +103,90 @@ int pack_filters(ftp_plan* p, const float* params, void* ws, cudaStream_t st)
     return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
 }
 
+inline bool is_tc(const ftp_plan* p) { return p->precision == FTP_BF16_FP32ACC; }
+inline int* err_ptr(void* ws, const ftp_plan* p) { return reinterpret_cast<int*>(static_cast<unsigned char*>(ws) + p->ws.err_off); }
+constexpr size_t kTcMinSmem = 120 * 1024;     // more than half an SM's shared memory: one block per SM, so the
+                                              // block's 512 tensor-memory columns are always available
+
+void fill_common_tc(const ftp_plan* p, const GroupPlan& g, bool backward, const float* x, const float* params,
+                    void* ws, TcGroupArgs& a)
+{
+    const PassPlan& pp = backward ? g.bwd : g.fwd;
+    std::memset(&a, 0, sizeof(a));
+    a.n_ops = g.n_ops; a.R = pp.y.count; a.Q = pp.x.count; a.N = p->N;
+    for (int i = 0; i < g.n_ops; ++i) a.op[i] = backward ? g.bwd_ops[i] : g.fwd_ops[i];
+    a.in_f32 = g.first == 1 ? 1 : 0;
+    a.in_C = p->maps[g.first - 1].C;
+    a.map[0] = map_ptr(p, x, ws, g.first);
+    for (int i = 0; i < g.n_ops; ++i) {
+        const OpDesc& op = a.op[i];
+        a.map[i + 1] = map_ptr(p, x, ws, op.out_map);
+        a.map_out[i + 1] = reinterpret_cast<__nv_bfloat16*>(const_cast<float*>(map_ptr(p, x, ws, op.out_map)));
+        a.arg[i] = op.kind == kOpConvPool
+                       ? static_cast<unsigned char*>(ws) + p->ws.arg_off[op.out_map - 1] : nullptr;
+    }
+    a.yspan = p->dev_tables + pp.dev_yspan; a.xspan = p->dev_tables + pp.dev_xspan;
+    a.ycell = p->dev_tables + pp.dev_ycell; a.xcell = p->dev_tables + pp.dev_xcell;
+    a.yoff = p->dev_tables + pp.dev_yoff;   a.xoff = p->dev_tables + pp.dev_xoff;
+    a.ytile = p->dev_tables + pp.dev_ytile; a.xtile = p->dev_tables + pp.dev_xtile;
+    a.wpk = reinterpret_cast<const __nv_bfloat16*>(ws_ptr(ws, backward ? p->ws.wb_off : p->ws.wf_off));
+    a.params = params;
+    a.error = err_ptr(ws, p);
+}
+
+int pack_filters_tc(ftp_plan* p, const float* params, void* ws, cudaStream_t st)
+{
+    __nv_bfloat16* wf = reinterpret_cast<__nv_bfloat16*>(ws_ptr(ws, p->ws.wf_off));
+    __nv_bfloat16* wb = reinterpret_cast<__nv_bfloat16*>(ws_ptr(ws, p->ws.wb_off));
+    TcPackArgs pa{};
+    auto flush = [&]() {
+        if (!pa.n) return;
+        Timed t(p, st, 0, -1);
+        pack_filters_tc_kernel<<<dim3(64, pa.n), 256, 0, st>>>(pa, params, wf, wb);
+        pa.n = 0;
+    };
+    for (const GroupPlan& g : p->groups)
+        for (int i = 0; i < g.n_ops; ++i) {
+            const OpDesc& op = g.fwd_ops[i];
+            if (op.kind == kOpPool) continue;
+            if (pa.n == kMaxOps * 2) flush();
+            pa.l[pa.n++] = TcPackLayer{op.p_off, op.twf_off, op.cin, op.cout, op.k, op.cin16, op.cout16};
+        }
+    flush();
+    return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
+}
+
+int forward_tc(ftp_plan* p, const float* x, const float* params, float* y, void* ws, cudaStream_t st)
+{
+    if (cudaMemsetAsync(err_ptr(ws, p), 0, 4, st) != cudaSuccess) return FTP_ERR_CUDA;
+    int rc = pack_filters_tc(p, params, ws, st);
+    if (rc != FTP_OK) return rc;
+    for (size_t gi = 0; gi < p->groups.size(); ++gi) {
+        const GroupPlan& g = p->groups[gi];
+        TcGroupArgs a;
+        fill_common_tc(p, g, false, x, params, ws, a);
+        const int items = a.R * a.Q * p->N;
+        { Timed t(p, st, 1, (int)gi);
+          const size_t smem = std::max(g.fwd.smem_bytes, kTcMinSmem);
+          fwd_group_tc_kernel<<<std::min(items, kSmCount), kTcThreads, smem, st>>>(a, (int)(smem - kTcFixedBytes)); }
+        if (!launched_ok()) return FTP_ERR_CUDA;
+    }
+    if (y) {
+        const MapShape& s = p->maps.back();
+        const size_t total = (size_t)p->N * s.C * s.H * s.W;
+        const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16);
+        ++p->launches;
+        planes_to_nchw_kernel<<<blocks, 256, 0, st>>>(
+            reinterpret_cast<const __nv_bfloat16*>(map_ptr(p, x, ws, (int)p->layers.size() + 1)), y, p->N, s.C,
+            (s.C + 15) / 16 * 16, s.H, s.W);
+        if (!launched_ok()) return FTP_ERR_CUDA;
+    }
+    return FTP_OK;
+}
+
 int forward_impl(ftp_plan* p, const float* x, const float* params, float* y, void* ws, cudaStream_t st)
 {
+    if (is_tc(p)) return forward_tc(p, x, params, y, ws, st);
     int rc = pack_filters(p, params, ws, st);
     if (rc != FTP_OK) return rc;
     for (size_t gi = 0; gi < p->groups.size(); ++gi) {
@@ -121,11 +206,65 @@ int forward_impl(ftp_plan* p, const float* x, const float* params, float* y, voi
     return FTP_OK;
 }
 
+int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* params, float* dx, float* grad_out,
+                float* sgd_params, float lr, void* ws, cudaStream_t st)
+{
+    const int G = (int)p->groups.size();
+    for (int gi = G - 1; gi >= 0; --gi) {
+        const GroupPlan& g = p->groups[gi];
+        TcGroupArgs a;
+        fill_common_tc(p, g, true, x, params, ws, a);
+        a.dmap_out = gi == G - 1 ? dy : ws_ptr(ws, p->ws.dmap_off[gi + 1]);
+        a.scratch = ws_ptr(ws, p->ws.scratch_off);
+        a.partial = ws_ptr(ws, g.partial_off);
+        a.set_floats = (long long)g.param_floats;
+        a.splits = g.bwd.splits; a.tiles_x = p->grid_x;
+        a.need_dx = (gi > 0 || dx != nullptr) ? 1 : 0;
+        { Timed t(p, st, 3, gi);
+          const size_t smem = std::max(g.bwd.smem_bytes, kTcMinSmem);
+          bwd_group_tc_kernel<<<g.bwd.blocks, kTcThreads, smem, st>>>(a, (int)(smem - kTcFixedBytes)); }
+        if (!launched_ok()) return FTP_ERR_CUDA;
+        if (a.need_dx) {
+            const MapShape& s = p->maps[g.first - 1];
+            HaloSumArgs h{};
+            h.scratch = a.scratch;
+            h.out = gi == 0 ? dx : ws_ptr(ws, p->ws.dmap_off[gi]);
+            h.yspan = a.yspan; h.xspan = a.xspan; h.yoff = a.yoff; h.xoff = a.xoff;
+            h.ycover = p->dev_tables + g.bwd.dev_ycover; h.xcover = p->dev_tables + g.bwd.dev_xcover;
+            h.N = p->N; h.C = s.C; h.H = s.H; h.W = s.W; h.R = a.R; h.Q = a.Q;
+            h.Htot = g.bwd.y.scratch_off[a.R]; h.Wtot = g.bwd.x.scratch_off[a.Q];
+            const size_t total = (size_t)p->N * s.C * s.H * s.W;
+            const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16);
+            { Timed t(p, st, 4, gi);
+              halo_sum_kernel<<<blocks, 256, 0, st>>>(h); }
+            if (!launched_ok()) return FTP_ERR_CUDA;
+        }
+    }
+    TcReduceArgs ra{};
+    auto flush = [&]() {
+        if (!ra.n) return;
+        Timed t(p, st, 5, -1);
+        reduce_sgd_tc_kernel<<<dim3(64, ra.n), 256, 0, st>>>(ra, sgd_params, lr, grad_out);
+        ra.n = 0;
+    };
+    for (const GroupPlan& g : p->groups)
+        for (int i = 0; i < g.n_ops; ++i) {
+            const OpDesc& op = g.bwd_ops[i];
+            if (op.kind == kOpPool) continue;
+            if (ra.n == kMaxOps * 2) flush();
+            ra.l[ra.n++] = TcReduceLayer{op.p_off, ws_ptr(ws, g.partial_off), (long long)g.param_floats, op.tgp_off,
+                                         g.bwd.blocks, op.cin, op.cout, op.k, op.cin16, op.cout16};
+        }
+    flush();
+    return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
+}
+
 // Backward of all groups in reverse order, halo sums at the group inputs, then the cross-tile
 // reduction; `sgd_params` non-null applies the update in the same kernel.
 int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* params, float* dx, float* grad_out,
                   float* sgd_params, float lr, void* ws, cudaStream_t st)
 {
+    if (is_tc(p)) return backward_tc(p, x, dy, params, dx, grad_out, sgd_params, lr, ws, st);
     const int G = (int)p->groups.size();
     for (int gi = G - 1; gi >= 0; --gi) {
         const GroupPlan& g = p->groups[gi];
@@ -277,7 +416,7 @@ int ftp_backward(ftp_plan* plan, const float* x, const float* dy, const float* p
     int rc = ensure_device(plan);
     if (rc != FTP_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = pack_filters(plan, params, workspace, st);
+    rc = is_tc(plan) ? pack_filters_tc(plan, params, workspace, st) : pack_filters(plan, params, workspace, st);
     if (rc != FTP_OK) return rc;
     return backward_impl(plan, x, dy, params, dx, dparams, nullptr, 0.f, workspace, st);
 }
@@ -291,7 +430,8 @@ static int step_impl(ftp_plan* plan, const float* x, const float* dy, const floa
     int rc = ensure_device(plan);
     if (rc != FTP_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = forward_impl(plan, x, params, nullptr, workspace, st);
+    float* y32 = (is_tc(plan) && target) ? ws_ptr(workspace, plan->ws.y32_off) : nullptr;
+    rc = forward_impl(plan, x, params, y32, workspace, st);
     if (rc != FTP_OK) return rc;
     const float* delta = dy;
     if (target) {
@@ -300,7 +440,7 @@ static int step_impl(ftp_plan* plan, const float* x, const float* dy, const floa
         float* d = ws_ptr(workspace, plan->ws.dy_off);
         float* sums = ws_ptr(workspace, plan->ws.loss_off);
         { Timed t(plan, st, 2, -1);
-          mse_delta_kernel<<<plan->loss_blocks, 256, 0, st>>>(map_ptr(plan, x, workspace, (int)plan->layers.size() + 1),
+          mse_delta_kernel<<<plan->loss_blocks, 256, 0, st>>>(y32 ? y32 : map_ptr(plan, x, workspace, (int)plan->layers.size() + 1),
                                                              target, d, M, sums); }
         if (loss_out) {
             Timed t(plan, st, 2, -1);
@@ -405,6 +545,16 @@ int ftp_plan_timing_read(ftp_plan* plan, int* n, ftp_launch_time* out, int capac
 }
 
 long long ftp_plan_launch_count(const ftp_plan* plan) { return plan ? plan->launches : 0; }
+
+int ftp_plan_check(ftp_plan* plan, void* workspace, void* stream)
+{
+    if (!plan || !workspace) return FTP_ERR_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return FTP_ERR_CUDA;
+    if (!is_tc(plan)) return FTP_OK;
+    int word = 0;
+    if (cudaMemcpy(&word, err_ptr(workspace, plan), 4, cudaMemcpyDeviceToHost) != cudaSuccess) return FTP_ERR_CUDA;
+    return word ? FTP_ERR_TIMEOUT : FTP_OK;
+}
 
 const char* ftp_strerror(int code)
 {

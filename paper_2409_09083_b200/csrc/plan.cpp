@@ -166,6 +166,75 @@ size_t layout_backward(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
     return (size_t)kSmemHeader + 4 * (size_t)total;
 }
 
+inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+// Tensor-core path.  A tile is [planes][Hp][Wp] entries of 16 bytes plus a tail of kTcTailEntries
+// entries per plane.  The MMA operands address 16-row x 8-column pixel blocks (or runs of 16
+// pixels) that may run past the rows and columns a tile really holds: such reads land in the
+// following plane or tile and only reach accumulator rows that are discarded, so tiles carry no
+// per-row padding; the activation area as a whole ends with a slack that keeps the furthest such
+// read inside the block's shared memory.  Ping-pong placement as in layout_forward.  Bytes.
+size_t tc_slack(int Wp, int planes_beyond, size_t plane_bytes)
+{
+    return ((size_t)16 * Wp + 32) * 16 + (size_t)planes_beyond * plane_bytes;
+}
+
+size_t layout_forward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
+{
+    size_t size[kMaxOps + 1] = {0}, slack = 0;
+    for (int i = 0; i < g.n_ops; ++i) {
+        OpDesc& op = g.fwd_ops[i];
+        const int oh = ty.maxext[i + 1], ow = tx.maxext[i + 1];
+        op.t_in_Hp = (oh - 1) * op.S + op.keff;
+        op.t_in_Wp = (ow - 1) * op.S + op.keff;
+        const size_t plane = ((size_t)op.t_in_Hp * op.t_in_Wp + kTcTailEntries) * 16;
+        size[i] = (size_t)(op.cin16 / 8) * plane;
+        slack = std::max(slack, tc_slack(op.t_in_Wp, 0, plane));
+    }
+    size_t total = 0;
+    for (int i = 0; i < g.n_ops; ++i) total = std::max(total, size[i] + size[i + 1]);
+    for (int i = 0; i < g.n_ops; ++i) g.fwd_ops[i].t_in_off = (i % 2 == 0) ? 0 : (int)(total - size[i]);
+    return (size_t)kTcFixedBytes + total + slack;
+}
+
+// Tensor-core path, backward.  While op i runs, three tiles are alive: dz_i (delta at the conv output,
+// before the pool, inside a zero apron of k-1), a copy of the op's input with the same pitch (the
+// filter gradient contracts over runs of 16 pixels of both), and dz_{i-1} which the op produces.
+// The filter-gradient operand spans 64 or 128 channels; channels beyond the real ones are reserved
+// in the tile so that the operand stays inside it.
+size_t layout_backward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
+{
+    const int n = g.n_ops;
+    size_t dsize[kMaxOps], xsize[kMaxOps], slack = 0;
+    for (int i = 0; i < n; ++i) {
+        OpDesc& op = g.bwd_ops[i];
+        const int oh = ty.maxext[i + 1], ow = tx.maxext[i + 1];
+        if (op.kind == kOpPool) {
+            op.t_dz_Hp = oh; op.t_dz_Wp = ow; op.t_dz_planes = op.cout16 / 8;
+            op.t_x_Hp = 2 * oh; op.t_x_Wp = 2 * ow;
+        } else {
+            const int coh = op.S * oh, cow = op.S * ow, a = op.k - 1;
+            op.t_dz_Hp = coh + 2 * a; op.t_dz_Wp = cow + 2 * a;
+            op.t_dz_planes = op.cout16 <= 64 ? 8 : round_up(op.cout16, 128) / 8;
+            op.t_x_Hp = coh + a; op.t_x_Wp = op.t_dz_Wp;
+        }
+        const size_t dplane = ((size_t)op.t_dz_Hp * op.t_dz_Wp + kTcTailEntries) * 16;
+        const size_t xplane = ((size_t)op.t_x_Hp * op.t_x_Wp + kTcTailEntries) * 16;
+        dsize[i] = (size_t)op.t_dz_planes * dplane;
+        xsize[i] = (size_t)(op.cin16 / 8) * xplane;
+        slack = std::max(slack, std::max(tc_slack(op.t_dz_Wp, 0, dplane), tc_slack(op.t_x_Wp, 0, xplane)));
+    }
+    size_t total = 0;
+    for (int i = 0; i < n; ++i) total = std::max(total, dsize[i] + xsize[i] + (i > 0 ? dsize[i - 1] : 0));
+    for (int i = 0; i < n; ++i) {
+        OpDesc& op = g.bwd_ops[i];
+        const bool low = ((n - 1 - i) % 2) == 0;
+        op.t_dz_off = low ? 0 : (int)(total - dsize[i]);
+        op.t_x_off = low ? (int)dsize[i] : (int)(i > 0 ? dsize[i - 1] : 0);
+    }
+    return (size_t)kTcFixedBytes + total + slack;
+}
+
 // Smallest split (largest sub-tile) whose buffers fit the shared-memory budget.
 int choose_subtiles(GroupPlan& g, bool backward, const PlanOpts& o)
 {
@@ -183,8 +252,10 @@ int choose_subtiles(GroupPlan& g, bool backward, const PlanOpts& o)
             int ky = std::min(c[0], max_h), kx = std::min(c[1], max_w);
             build_axis(pp.y, ay, g.tile_y, ky);
             build_axis(pp.x, ax, g.tile_x, kx);
-            size_t bytes = backward ? layout_backward(g, pp.y, pp.x) : layout_forward(g, pp.y, pp.x);
-            if (bytes <= (size_t)o.smem_bytes) {
+            size_t bytes;
+            if (o.tensor_cores) bytes = backward ? layout_backward_tc(g, pp.y, pp.x) : layout_forward_tc(g, pp.y, pp.x);
+            else bytes = backward ? layout_backward(g, pp.y, pp.x) : layout_forward(g, pp.y, pp.x);
+            if (bytes <= (size_t)(o.tensor_cores ? std::min(kTcSmemBudget, o.smem_bytes + 2048) : o.smem_bytes)) {
                 pp.smem_bytes = bytes;
                 return FTP_OK;
             }
@@ -214,7 +285,7 @@ void count_macs(const GroupPlan& g, const PassPlan& pp, double* done, double* un
     }
 }
 
-struct LayerOffsets { std::vector<long long> p_off, wf_off, wb_off; };
+struct LayerOffsets { std::vector<long long> p_off, wf_off, wb_off, twf_off, twb_off; };
 
 // Builds the ops, the sub-tiling and the block counts of one executed group (layers first..last).
 // Returns FTP_ERR_WORKSPACE if nothing fits; *redundancy is the larger of the two passes' ratios of
@@ -229,7 +300,8 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
     g.tile_y = equal_partition(0, out.H, gy);
     g.tile_x = equal_partition(0, out.W, gx);
     g.param_begin = -1;
-    long long gp = 0;
+    long long gp = 0, tgp = 0;
+    const bool tcp = p.precision == FTP_BF16_FP32ACC;
     for (int li = first - 1; li < last; ++li) {
         const ftp_layer& l = p.layers[li];
         OpDesc op{};
@@ -244,7 +316,11 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
         op.in_map = li + 1; op.out_map = le + 2;
         op.in_H = p.maps[li].H; op.in_W = p.maps[li].W;
         op.out_H = p.maps[le + 1].H; op.out_W = p.maps[le + 1].W;
+        op.cin16 = round_up(op.cin, 16); op.cout16 = round_up(op.cout, 16);
         if (l.kind == FTP_CONV) {
+            op.twf_off = lo.twf_off[li]; op.twb_off = lo.twb_off[li];
+            op.tgp_off = tgp;
+            tgp += (long long)l.k * l.k * op.cout16 * op.cin16 + op.cout16;
             op.cout_pad = (l.cout + kCoutTile - 1) / kCoutTile * kCoutTile;
             op.cin_pad = (l.cin + kCoutTile - 1) / kCoutTile * kCoutTile;
             op.wf_off = lo.wf_off[li]; op.wb_off = lo.wb_off[li];
@@ -259,7 +335,7 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
         li = le;
     }
     if (g.param_begin < 0) g.param_begin = 0;
-    g.param_floats = (size_t)gp;
+    g.param_floats = (size_t)(tcp ? tgp : gp);
 
     int rc = choose_subtiles(g, false, o);
     if (rc != FTP_OK) return rc;
@@ -298,7 +374,10 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         return FTP_ERR_ARG;
     if (opts.max_redundancy_pct < 100 || opts.max_subtile < 0 || opts.smem_bytes < 2 * kSmemHeader || opts.smem_bytes > kSmemBudget)
         return FTP_ERR_ARG;
-    if (precision != FTP_FP32) return precision == FTP_BF16_FP32ACC ? FTP_ERR_PRECISION : FTP_ERR_ARG;
+    if (precision != FTP_FP32 && precision != FTP_BF16_FP32ACC) return FTP_ERR_ARG;
+    const bool tcp = precision == FTP_BF16_FP32ACC;
+    PlanOpts popts = opts;
+    popts.tensor_cores = tcp ? 1 : 0;
     p.layers.assign(layers, layers + n_layers);
     p.N = N; p.grid_y = gy; p.grid_x = gx; p.precision = precision;
 
@@ -307,7 +386,8 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     p.maps.push_back(MapShape{C, H, W});
     LayerOffsets lo;
     lo.p_off.assign(n_layers, 0); lo.wf_off.assign(n_layers, 0); lo.wb_off.assign(n_layers, 0);
-    long long params = 0, wf = 0, wb = 0;
+    lo.twf_off.assign(n_layers, 0); lo.twb_off.assign(n_layers, 0);
+    long long params = 0, wf = 0, wb = 0, twf = 0;
     for (int i = 0; i < n_layers; ++i) {
         const ftp_layer& l = p.layers[i];
         MapShape in = p.maps.back();
@@ -322,6 +402,9 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
             int cin_pad = (l.cin + kCoutTile - 1) / kCoutTile * kCoutTile;
             lo.wf_off[i] = wf; wf += (long long)l.cin * l.k * l.k * cout_pad;
             lo.wb_off[i] = wb; wb += (long long)l.cout * l.k * l.k * cin_pad;
+            if (tcp && (l.cin > kTcTmemCols || l.cout > kTcTmemCols)) return FTP_ERR_LAYERS;
+            lo.twf_off[i] = lo.twb_off[i] = twf;        // both packed layouts hold k*k*cin16*cout16 elements
+            twf += (long long)l.k * l.k * round_up(l.cin, 16) * round_up(l.cout, 16);
         } else if (l.kind == FTP_MAXPOOL) {
             if (l.k != 2 || l.stride != 2 || l.pad != 0 || in.H % 2 || in.W % 2) return FTP_ERR_LAYERS;
             p.maps.push_back(MapShape{in.C, in.H / 2, in.W / 2});
@@ -330,8 +413,8 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         }
     }
     p.param_floats = (size_t)params;
-    p.wf_floats = (size_t)wf;
-    p.wb_floats = (size_t)wb;
+    p.wf_floats = (size_t)(tcp ? twf : wf);
+    p.wb_floats = (size_t)(tcp ? twf : wb);
 
     // groups: contiguous, covering 1..L
     int expect = 1;
@@ -358,7 +441,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
             const int hi = std::min(last, start + kMaxOps - 1);
             if (opts.strict_groups) {
                 if (hi != last) return FTP_ERR_GROUPS;
-                int rc = make_group(p, lo, start, last, opts, g, &red);
+                int rc = make_group(p, lo, start, last, popts, g, &red);
                 if (rc != FTP_OK) return rc;
                 chosen = last;
             } else {
@@ -369,7 +452,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
                         const bool splits_pair = end < last && p.layers[end - 1].kind == FTP_CONV &&
                                                  p.layers[end].kind == FTP_MAXPOOL;
                         if (pass == 0 && splits_pair) continue;
-                        int rc = make_group(p, lo, start, end, opts, g, &red);
+                        int rc = make_group(p, lo, start, end, popts, g, &red);
                         if (rc == FTP_OK && (pass == 2 || red * 100.0 <= opts.max_redundancy_pct)) { chosen = end; break; }
                     }
                 if (chosen < 0) return FTP_ERR_WORKSPACE;
@@ -403,6 +486,12 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         for (int i = 0; i < g.n_ops; ++i) {
             const OpDesc& op = g.fwd_ops[i];
             const MapShape& s = p.maps[op.out_map - 1];
+            if (tcp) {      // bf16 planes [n][C16/8][H][W][8]; arg-max bytes in the same arrangement
+                const size_t c16 = (size_t)round_up(s.C, 16);
+                ws.map_off[op.out_map - 1] = take((size_t)N * c16 * s.H * s.W * 2);
+                if (op.kind == kOpConvPool) ws.arg_off[op.out_map - 1] = take((size_t)N * c16 * s.H * s.W);
+                continue;
+            }
             ws.map_off[op.out_map - 1] = take((size_t)N * s.C * s.H * s.W * 4);
             if (op.kind == kOpConvPool) ws.arg_off[op.out_map - 1] = take((size_t)N * s.C * s.H * s.W);
         }
@@ -414,6 +503,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     {
         const MapShape& s = p.maps[n_layers];
         ws.dy_off = take((size_t)N * s.C * s.H * s.W * 4);
+        if (tcp) ws.y32_off = take((size_t)N * s.C * s.H * s.W * 4);
         size_t total = (size_t)N * s.C * s.H * s.W;
         p.loss_blocks = (int)std::min<size_t>(1024, (total + 1023) / 1024);
         ws.loss_off = take((size_t)p.loss_blocks * 4);
@@ -424,8 +514,9 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     size_t scratch = 0;
     for (const GroupPlan& g : p.groups) scratch = std::max(scratch, g.bwd.scratch_floats);
     ws.scratch_off = take(scratch * 4);
-    ws.wf_off = take(p.wf_floats * 4);
-    ws.wb_off = take(p.wb_floats * 4);
+    ws.wf_off = take(p.wf_floats * (tcp ? 2 : 4));
+    ws.wb_off = take(p.wb_floats * (tcp ? 2 : 4));
+    ws.err_off = take(256);
     ws.partial_off = off;
     for (GroupPlan& g : p.groups) g.partial_off = take((size_t)g.bwd.blocks * g.param_floats * 4);
     ws.grad_off = take(p.param_floats * 4);

@@ -17,6 +17,16 @@ constexpr int kSmemBudget  = 225 * 1024;  // dynamic shared memory a block may u
 constexpr int kSmemHeader  = 1024;    // bytes reserved at the start for per-block tables
 constexpr int kCoutTile    = 8;       // output channels per thread task (packed weights are padded to it)
 
+// Tensor-core (bf16) tile kernels: one block per SM, all 512 tensor-memory columns.
+constexpr int kTcThreads    = 256;
+constexpr int kTcStages     = 2;          // weight ring: stages of kTcStageBytes
+constexpr int kTcStageBytes = 16384;
+constexpr int kTcTmemCols   = 512;
+constexpr int kTcHeader     = 4096;       // per-block tables, barriers, bias staging
+constexpr int kTcFixedBytes = kTcHeader + kTcStages * kTcStageBytes;   // shared memory before the activation area
+constexpr int kTcSmemBudget = 227 * 1024; // dynamic shared memory a tensor-core block may use
+constexpr int kTcTailEntries = 16;        // 16-byte entries appended to every tile plane
+
 struct Span { int a, b; };            // inclusive interval on one axis
 
 // One layer inside a group, as the kernels see it.
@@ -39,6 +49,14 @@ struct OpDesc {
     long long wf_off, wb_off;          // float offsets into the packed forward / rotated filters
     long long p_off;                   // float offset of the filter in params (bias follows it)
     long long gp_off;                  // float offset of the filter inside the group's partial set
+    // --- bf16 tensor-core path: shared-memory tiles are [channel/8][row][col][8] bf16 planes ---
+    int   cin16, cout16;               // channel counts padded to 16 (pool: both = padded channels of the map)
+    int   t_in_off, t_in_Hp, t_in_Wp;  // forward input tile: byte offset in the activation area, padded rows / cols
+    int   t_x_off, t_x_Hp, t_x_Wp;     // backward: copy of the op's input
+    int   t_dz_off, t_dz_Hp, t_dz_Wp;  // backward: delta at the conv output (before the pool), zero apron of k-1 around it
+    int   t_dz_planes;                 // planes reserved for it (8, or a multiple of 16: the M = 64 / 128 operand stays inside)
+    long long twf_off, twb_off;        // bf16 element offsets of the packed forward / rotated filters
+    long long tgp_off;                 // float offset inside the group's partial set in the tensor-core layout
 };
 
 // Axis tables of one (group, pass): for sub-tile index r and map m (0 = group input ... n_ops = output)
@@ -72,7 +90,7 @@ struct GroupPlan {
     OpDesc bwd_ops[kMaxOps];
     PassPlan fwd, bwd;
     std::vector<Span> tile_y, tile_x;   // user-tile partition of the group's output map
-    size_t param_floats = 0;            // floats of this group's partial gradient set
+    size_t param_floats = 0;            // floats of this group's partial gradient set (tensor-core path: padded layout)
     long long param_begin = 0;          // offset of the group's first parameter in params
     size_t partial_off = 0;             // float offset of the group's partial sets in the workspace
     double macs_done = 0, macs_untiled = 0;
@@ -92,6 +110,8 @@ struct Workspace {                 // byte offsets, all 256-aligned
     size_t loss_off = 0;           // per-block partial sums of the MSE
     size_t loss_val_off = 0;       // the loss value (ftp_step_host)
     size_t x_stage_off = 0, t_stage_off = 0;   // device copies of a host batch (ftp_step_host)
+    size_t y32_off = 0;            // tensor-core path: fp32 NCHW copy of the last map for the loss (ftp_step with target)
+    size_t err_off = 0;            // device error word of the tensor-core kernels (a bounded wait ran out)
     size_t total = 0;
 };
 
@@ -104,7 +124,7 @@ struct ftp_plan {
     std::vector<ftp::GroupPlan> groups;     // the executed groups (a requested group may be cut, see build_plan)
     int N = 0, grid_y = 0, grid_x = 0, precision = 0;
     size_t param_floats = 0;
-    size_t wf_floats = 0, wb_floats = 0;
+    size_t wf_floats = 0, wb_floats = 0;    // packed filters (tensor-core path: counted in bf16 elements)
     ftp::Workspace ws;
     std::vector<int> tables;                // host copy of all device tables
     int*  dev_tables = nullptr;             // uploaded lazily by the first launch
@@ -124,6 +144,7 @@ struct PlanOpts {
     int max_subtile = 0;            // 0 = as large as fits; else an upper bound (tests use it to force sub-tiling)
     int smem_bytes = kSmemBudget;   // dynamic shared memory a block may use
     int strict_groups = 0;          // 1 = never cut a requested group
+    int tensor_cores = 0;           // set by build_plan from the precision: shared-memory layouts of the bf16 path
 };
 // Builds everything but the device upload.  Returns FTP_OK or an error code.
 int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C, int H, int W,

@@ -59,10 +59,16 @@ def run_gpu_step(wl, x, params, target, lr, want_dx=True, **plan_opts):
                 dx=None if dx is None else dx.cpu().numpy())
 
 
-def run_oracle(wl, x, params, target=None, dy=None, lr=0.0):
+def run_oracle(wl, x, params, target=None, dy=None, lr=0.0, store=None):
     return orc.step(list(wl.layers), x.astype(np.float64), params.astype(np.float64), lr,
                     target=None if target is None else target.astype(np.float64),
-                    dy=None if dy is None else dy.astype(np.float64))
+                    dy=None if dy is None else dy.astype(np.float64), store=store)
+
+
+def bf16_grid(a):
+    """The same array with every value moved to the nearest bfloat16 (still float32): inputs that a
+    bf16 path and the oracle can both take without an input-rounding difference."""
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(torch.bfloat16).to(torch.float32).numpy()
 
 
 def per_layer_errors(layers, got, ref):
@@ -95,13 +101,16 @@ def decision_margin(layers, ref):
     return float(worst)
 
 
-def draw_unambiguous(wl, bias_std=0.5, tau=2e-5, tries=200):
+def draw_unambiguous(wl, bias_std=0.5, tau=2e-5, tries=200, store=None):
     """First seed >= wl.seed whose oracle decisions all have a margin above tau; returns
-    (workload with that seed, x, params, target, oracle result)."""
+    (workload with that seed, x, params, target, oracle result).  store="bf16": inputs on the
+    bf16 grid, oracle with bf16 feature-map storage."""
     for s in range(wl.seed, wl.seed + tries):
         w = wl.with_(seed=s)
         x, params, target = synth.draw(w, bias_std=bias_std)
-        ref = run_oracle(w, x, params, target=target)
+        if store:
+            x, params = bf16_grid(x), bf16_grid(params)
+        ref = run_oracle(w, x, params, target=target, store=store)
         if decision_margin(list(w.layers), ref) > tau:
             return w, x, params, target, ref
     raise RuntimeError("no seed with unambiguous decisions found")

@@ -208,3 +208,32 @@ def test_result_independent_of_thread_count(monkeypatch):
     b = orc.step(layers, x, params, lr=0.1, target=target)
     assert np.array_equal(a["new_params"], b["new_params"])
     assert np.array_equal(a["dx"], b["dx"])
+
+
+def test_round_bf16_matches_library_conversion_and_ties_go_to_even():
+    rng = np.random.default_rng(9)
+    a = np.concatenate([rng.standard_normal(5000) * 10.0 ** rng.integers(-6, 6, 5000), [0.0, 1.0, -1.0, 255.0, 256.0]])
+    a = a.astype(np.float32).astype(np.float64)          # fp32-representable, as the library routine expects
+    want = torch.from_numpy(a.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(orc.round_bf16(a), want)
+    # 1 + 2^-8 lies half way between 1 and 1 + 2^-7: ties to even keeps 1; 1 + 3*2^-8 goes up to 1 + 2^-6
+    assert orc.round_bf16(np.array([1.0 + 2.0 ** -8]))[0] == 1.0
+    assert orc.round_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+
+
+def test_bf16_storage_only_rounds_stored_maps():
+    layers = _tiny_net()
+    x, params, target = _draw(layers, 1, 2, 8, 8, 4)
+    maps64, _ = orc.forward(layers, x, params)
+    maps16, tape = orc.forward(layers, x, params, store="bf16")
+    assert np.array_equal(maps16[1], orc.round_bf16(maps64[1]))           # first conv output: rounded once
+    for m, l in zip(maps16[1:], layers):
+        if l.kind == "conv":
+            assert np.array_equal(m, orc.round_bf16(m))                   # every stored conv output is a bf16 value
+    # without discrete decisions (slope 1, no pool) storage rounding only perturbs the gradients
+    lin = [synth.conv(2, 3, 3, leaky=1.0), synth.conv(3, 2, 3, leaky=1.0)]
+    x, params, target = _draw(lin, 1, 2, 8, 8, 4)
+    r = orc.step(lin, x, params, 0.0, target=target, store="bf16")
+    r64 = orc.step(lin, x, params, 0.0, target=target)
+    err = np.abs(r["dparams"] - r64["dparams"]).max() / np.abs(r64["dparams"]).max()
+    assert 0.0 < err <= 2e-2

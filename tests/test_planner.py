@@ -133,7 +133,6 @@ def test_argument_errors_are_codes_not_crashes():
     assert _code(lambda: mk(groups=((1, 1), (3, 3)))) == -4               # gap
     assert _code(lambda: mk(groups=((2, 3), (1, 1)))) == -4               # order
     assert _code(lambda: mk(grid=(17, 2))) == -3                          # more tiles than output rows
-    assert _code(lambda: mk(precision=1)) == -8                           # bf16 path not built
     assert _code(lambda: mk(precision=5)) == -1
     assert "shared memory" in ftp.ftp_strerror(-5)
     assert ftp.ftp_strerror(0) == "ok"
