@@ -32,6 +32,15 @@ FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 KIND = {0: "pack_filters", 1: "fwd_group", 2: "loss_delta", 3: "bwd_group", 4: "halo_sum", 5: "reduce_sgd"}
 
 
+def measured_bf16_peak():
+    """Sustained dense bf16 TFLOP/s measured on this machine's B200s (generated file), else the fallback."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "of measured (MEASURED_PEAKS.json, sustained cuBLAS bf16)"
+    except (OSError, KeyError, ValueError):
+        return 1400.0, "of fallback (1.4 PFLOP/s sustained)"
+
+
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -39,6 +48,8 @@ def parse():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="C1", choices=["C0", "C1", "C2", "C3"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--precision", default="fp32", choices=["fp32", "bf16"],
+                    help="fp32: CUDA-core path (tolerance 1e-4); bf16: tcgen05 tensor-core path, bf16 maps, fp32 accumulation (2e-2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -151,7 +162,8 @@ def run_ours(args):
     x, params, target = synth.draw(wl)
     if world > 1:                                             # same initial parameters on every rank
         params = synth.draw(wl.with_(seed=0))[1]
-    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups)
+    tcp = args.precision == "bf16"
+    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=1 if tcp else 0)
     ws = plan.new_workspace()
     xd, pd, td = (torch.from_numpy(a).cuda() for a in (x, params, target))
     dx = torch.empty_like(xd)
@@ -174,6 +186,7 @@ def run_ours(args):
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
+    plan.check(ws)          # a bounded device-side wait that ran out would invalidate everything below
 
     sampler = ClockSampler(local) if rank == 0 else None
     plan.timing(True)
@@ -228,26 +241,35 @@ def run_ours(args):
     steps = args.steps
     ms_step = total_ms / steps
     breakdown = {}
+    per_group = {}
     for (kind, group), ms in per_kind.items():
         breakdown[KIND[kind]] = breakdown.get(KIND[kind], 0.0) + ms / steps
+        if group >= 0:
+            per_group[f"{KIND[kind]}[{group}]"] = per_group.get(f"{KIND[kind]}[{group}]", 0.0) + ms / steps
     # dominant kernel: the fused backward (delta back-propagation + filter gradients = 2 forward-equivalents)
     bwd_ms = breakdown.get("bwd_group", 0.0)
     bwd_flops = 4.0 * macs * wl.N
     n_bwd = sum(1 for (k, g) in per_kind if k == 3)
     achieved = bwd_flops / (bwd_ms / 1e3) / 1e12 if bwd_ms > 0 else None
-    roofline = {"bound": "alu", "kernel": "bwd_group_kernel", "achieved": achieved, "peak": FP32_PEAK_TFLOPS,
-                "unit": "TFLOP/s", "frac": achieved / FP32_PEAK_TFLOPS if achieved else None, "traffic": None,
-                "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+    if tcp:
+        peak, src = measured_bf16_peak()
+        bound, kernel = "tensor", "bwd_group_tc_kernel"
+    else:
+        peak, src = FP32_PEAK_TFLOPS, "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz"
+        bound, kernel = "alu", "bwd_group_kernel"
+    roofline = {"bound": bound, "kernel": kernel, "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": achieved / peak if achieved else None, "traffic": None,
+                "peak_source": src,
                 "launches_per_step": n_bwd, "avg_launch_ms": bwd_ms / n_bwd if n_bwd else None,
                 "algorithmic_flops_per_step": bwd_flops,
-                "step_frac_of_fp32_peak": 6.0 * macs * wl.N / (ms_step / 1e3) / 1e12 / FP32_PEAK_TFLOPS}
+                "step_frac_of_peak": 6.0 * macs * wl.N / (ms_step / 1e3) / 1e12 / peak}
     line = {"metric": METRIC, "value": world * wl.N * steps / (total_ms / 1e3), "unit": UNIT, "n_gpus": world,
             "steps": steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": config_of(wl, {"global_batch": wl.N * world, "executed_groups": plan.exec_groups(),
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if tcp else "f32", "data": "synthetic",
+            "config": config_of(wl, {"global_batch": wl.N * world, "precision": args.precision, "executed_groups": plan.exec_groups(),
                                      "parallelism": f"dp{world}", "l2": "flushed between timed steps (256 MiB write)",
                                      "redundancy_fwd": plan.redundancy}),
-            "clocks": clocks, "gpu_launches": int(launches), "breakdown_ms_per_step": breakdown,
+            "clocks": clocks, "gpu_launches": int(launches), "breakdown_ms_per_step": breakdown, "per_group_ms_per_step": per_group,
             "roofline": roofline, "loss": float(loss.item())}
     if e2e is not None:
         line["e2e"] = e2e

@@ -10,7 +10,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libftp.so")
+_LIB_PATH = os.environ.get("FTP_LIBRARY") or os.path.join(_HERE, "libftp.so")   # FTP_LIBRARY: another build of the same library
 
 if not os.path.exists(_LIB_PATH):
     raise ImportError(

@@ -128,29 +128,47 @@ __device__ __forceinline__ void conv_mma(Pipe& p, uint32_t a_base, int a_Wp, uin
                 bulk_g2s(p.ring + slot * kTcStageBytes, w + (size_t)s * spp * N * 8, bytes, smem_u32(&p.h->full[slot]));
             }
         } else if (warp == 0 && lane == 0) {
-            // MMA issue
+            // MMA issue.  Descriptor halves are advanced with adds only (no division or multiplication
+            // inside the loops): the tensor core idles while this thread computes.
+            const uint32_t a_hi = desc_hi((uint32_t)a_Wp * 16), b_hi = desc_hi(128);
+            const uint32_t plane16 = a_plane >> 4, bplane16 = plane_bytes >> 4;
+            const uint32_t idesc_full = make_idesc(128, min(N, 256), false, false);
+            const uint32_t idesc_rest = N > 256 ? make_idesc(128, N - 256, false, false) : 0u;
+            int gp0 = 0;                                            // first plane of the stage
             for (int s = 0; s < nstages; ++s) {
                 const uint32_t q = p.stages_done + s, slot = q % kTcStages, par = (q / kTcStages) & 1;
                 if (!wait_or_fail(p, &p.h->full[slot], par)) break;
                 fence_after_sync();
-                const int pl = min(spp, planes - s * spp);
-                const uint32_t bstage = p.ring + slot * kTcStageBytes;
+                const int pl = min(spp, planes - gp0);
+                const uint32_t b_lo0 = desc_lo(p.ring + slot * kTcStageBytes, plane_bytes);
+                // window position and channel plane at which the stage starts (once per stage)
+                const int tap0 = gp0 / kplanes, kc0 = gp0 - tap0 * kplanes, ky0 = tap0 / K, kx0 = tap0 - ky0 * K;
+                const uint32_t off0 = (uint32_t)kc0 * plane16 + (uint32_t)(ky0 * a_Wp + kx0);
+                int by = b0 / nbx, bx = b0 - by * nbx;
+                uint32_t tcol = tmem;
                 for (int bi = 0; bi < nb; ++bi) {
-                    const int b = b0 + bi, by = b / nbx, bx = b % nbx;
-                    const uint32_t a_blk = a_base + (uint32_t)((by * 16) * a_Wp + bx * 8) * 16;
+                    const uint32_t a_lo0 = desc_lo(a_base + (uint32_t)((by * 16) * a_Wp + bx * 8) * 16, a_plane);
+                    uint32_t off = off0, b_lo = b_lo0;
+                    int kc = kc0, kx = kx0;
+                    bool acc = gp0 > 0;
                     for (int pp = 0; pp < pl; pp += 2) {
-                        const int gp = s * spp + pp, tap = gp / kplanes, kc = gp - tap * kplanes;
-                        const int ky = tap / K, kx = tap - ky * K;
-                        const uint64_t ad = make_desc(a_blk + (uint32_t)kc * a_plane + (uint32_t)(ky * a_Wp + kx) * 16,
-                                                      a_plane, (uint32_t)a_Wp * 16);
-                        for (int n0 = 0; n0 < N; n0 += 256) {
-                            const int nn = min(256, N - n0);
-                            const uint64_t bd = make_desc(bstage + (uint32_t)pp * plane_bytes + (uint32_t)n0 * 16, plane_bytes, 128);
-                            mma_bf16(tmem + (uint32_t)(bi * N + n0), ad, bd, make_idesc(128, nn, false, false), gp > 0);
+                        const uint64_t ad = desc64(a_hi, a_lo0 + off);
+                        mma_bf16(tcol, ad, desc64(b_hi, b_lo), idesc_full, acc);
+                        if (N > 256) mma_bf16(tcol + 256, ad, desc64(b_hi, b_lo + 256), idesc_rest, acc);
+                        acc = true;
+                        b_lo += 2 * bplane16;
+                        kc += 2; off += 2 * plane16;
+                        if (kc == kplanes) {                        // next window position
+                            kc = 0; off -= (uint32_t)kplanes * plane16;
+                            ++kx; ++off;
+                            if (kx == K) { kx = 0; off += (uint32_t)(a_Wp - K); }
                         }
                     }
+                    tcol += (uint32_t)N;
+                    if (++bx == nbx) { bx = 0; ++by; }
                 }
                 mma_commit(smem_u32(&p.h->empty[slot]));
+                gp0 += pl;
             }
             mma_commit(smem_u32(&p.h->done));
         }
@@ -312,20 +330,31 @@ __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*addre
             cols += c; ++u1;
         }
         if (warp == 0 && lane == 0) {
+            // adds only between two MMAs (see conv_mma)
+            const uint32_t a_hi = desc_hi(dz_plane), x_hi = desc_hi(x_plane);
+            const uint32_t a_lo0 = desc_lo(dz_run, 128), x_lo0 = desc_lo(x_base, 128);
+            const uint64_t ones_d = make_desc(ones, 0, 0);
+            const uint32_t slice16 = 16u * (dz_plane >> 4), xhalf16 = 32u * (x_plane >> 4);
+            const int s0 = u0 / (KK + 1), t0 = u0 - s0 * (KK + 1), ky0 = t0 / K, kx0 = t0 - ky0 * K;
             for (int ks = 0; ks < nk; ++ks) {
-                int col = 0;
+                const bool acc = ks > 0;
+                const uint32_t kso = (uint32_t)ks * 16u;
+                uint32_t a_lo = a_lo0 + (uint32_t)s0 * slice16 + kso;
+                uint32_t x_lo = x_lo0 + (uint32_t)(ky0 * Wp + kx0) + kso;
+                uint32_t tcol = tmem;
+                int t = t0, kx = kx0;
                 for (int u = u0; u < u1; ++u) {
-                    const int slice = u / (KK + 1), t = u % (KK + 1);
-                    const uint64_t ad = make_desc(dz_run + (uint32_t)slice * 16u * dz_plane + (uint32_t)ks * 256u, 128, dz_plane);
+                    const uint64_t ad = desc64(a_hi, a_lo);
                     if (t == KK) {
-                        mma_bf16(tmem + col, ad, make_desc(ones, 0, 0), idesc_bias, ks > 0);
-                        col += 16;
+                        mma_bf16(tcol, ad, ones_d, idesc_bias, acc);
+                        tcol += 16;
+                        t = 0; kx = 0; a_lo += slice16; x_lo = x_lo0 + kso;      // next slice of output channels
                     } else {
-                        const int ky = t / K, kx = t - ky * K;
-                        const uint32_t xa = x_base + (uint32_t)(ky * Wp + kx) * 16u + (uint32_t)ks * 256u;
-                        mma_bf16(tmem + col, ad, make_desc(xa, 128, x_plane), idesc_tap0, ks > 0);
-                        if (cin16 > 256) mma_bf16(tmem + col + 256, ad, make_desc(xa + 32u * x_plane, 128, x_plane), idesc_tap1, ks > 0);
-                        col += cin16;
+                        mma_bf16(tcol, ad, desc64(x_hi, x_lo), idesc_tap0, acc);
+                        if (cin16 > 256) mma_bf16(tcol + 256, ad, desc64(x_hi, x_lo + xhalf16), idesc_tap1, acc);
+                        tcol += (uint32_t)cin16;
+                        ++t; ++kx; ++x_lo;
+                        if (kx == K) { kx = 0; x_lo += (uint32_t)(Wp - K); }
                     }
                 }
             }
@@ -350,14 +379,13 @@ __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*addre
                 if (row_ok && co < cout16) {
                     if (t == KK) {
                         float* g = gset + (size_t)KK * cout16 * cin16 + co;
-                        *g = first ? v[0] : *g + v[0];
+                        if (first) *g = v[0]; else atomicAdd(g, v[0]);
                     } else {
-                        float4* g = reinterpret_cast<float4*>(gset + ((size_t)t * cout16 + co) * cin16 + c0);
+                        float* g = gset + ((size_t)t * cout16 + co) * cin16 + c0;
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            float4 o = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                            if (!first) { const float4 old = g[j]; o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w; }
-                            g[j] = o;
+                            if (first) *reinterpret_cast<float4*>(g + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                            else red_add_v4(g + 4 * j, v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
                         }
                     }
                 }

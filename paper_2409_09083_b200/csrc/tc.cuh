@@ -30,6 +30,21 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
 }
 
+// The two 32-bit halves of that descriptor.  The issuing thread keeps the high half fixed and moves
+// the start address by adding 16-byte units to the low half: a single thread feeds the tensor core,
+// so every instruction between two MMAs costs tensor-core time.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes)
+{
+    return ((saddr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ uint32_t desc_hi(uint32_t sbo_bytes) { return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14); }
+__device__ __forceinline__ uint64_t desc64(uint32_t hi, uint32_t lo)
+{
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
+
 // Instruction descriptor of kind::f16 with bf16 operands and fp32 accumulation.
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool a_mn_major, bool b_mn_major)
 {
@@ -66,6 +81,13 @@ __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols)
 __device__ __forceinline__ void tmem_dealloc(uint32_t base, uint32_t cols)
 {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(base), "r"(cols) : "memory");
+}
+
+// 16-byte vector add to global memory without a return value.  Every address of a partial gradient
+// set is only ever updated by one thread, in program order, so the sums keep a fixed order.
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" :: "l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
 // 32 lanes x 16 consecutive fp32 columns: thread i of the warp gets row (lane base + i).
