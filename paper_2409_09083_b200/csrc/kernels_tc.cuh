@@ -52,6 +52,8 @@ struct Header {
     volatile int failed;                         // a wait ran out: skip every later wait
     int pad_[2];
     __align__(16) __nv_bfloat16 ones[64];        // one core matrix of 1.0: operand of the bias-gradient contraction
+    __align__(16) uint4 dw_unit[2 * kTcMaxUnits]; // filter gradient: MMAs of the current pass {a_lo, x_lo, idesc, column}
+    uint2 dw_bias[kTcMaxUnits];                  //                  bias MMAs {a_lo, column}
     float bias[kTcTmemCols];
 };
 static_assert(sizeof(Header) <= kTcHeader, "header does not fit");
@@ -299,63 +301,80 @@ __device__ __forceinline__ void teardown(Header* h)
 // 16 consecutive tile entries is one K step for both operands (MN-major: 8 pixels x 8 channels per
 // core matrix); the zero apron and tail of dz make the entries between the rows of the region and
 // after its end contribute nothing.  The bias gradient is the same contraction against a tile of
-// ones.  Accumulators: one unit of N = cin16 columns per (64- or 128-channel slice of cout, window
-// position), 16 columns per slice for the bias; as many units as fit in tensor memory per pass.
+// ones.  Accumulators ("units"): per 64- or 128-channel slice of cout one unit of N = cin16 columns
+// per window position and 16 columns for the bias; as many units as fit in tensor memory per pass.
+// With at most 8 input channels (the first layer) the K window positions of one filter row share a
+// unit instead: N-chunk j of the x operand is the same plane moved by j pixels (stride 16 bytes),
+// so one MMA yields G for kx = 0..K-1 and the layer needs K + 1 MMAs per K step instead of K*K + 1
+// (an MMA costs the tensor core about 45 cycles however narrow it is).
 // The result is added to (first: stored into) this block's partial set, arranged per layer as
 // [t][cout16][cin16] followed by [cout16] bias entries.
 __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*address of the region's first pixel*/,
                                                 uint32_t dz_plane, uint32_t x_base, uint32_t x_plane, int Wp, int K,
-                                                int cout16, int cin16, int run /*entries from first to last pixel*/,
+                                                int cout16, int cin16, int cin, int run /*entries from first to last pixel*/,
                                                 float* __restrict__ gset, bool first)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KK = K * K;
     const int Ms = cout16 <= 64 ? 64 : 128;
     const int nslices = cout16 <= 64 ? 1 : (cout16 + 127) / 128;
-    const int nunits = nslices * (KK + 1);
+    const bool folded = cin <= 8;
+    const int T = folded ? K : KK;                       // window units per slice
+    const int ucols = folded ? (8 * K + 15) / 16 * 16 : cin16;
+    const int nunits = nslices * (T + 1);
     const int nk = (run + 15) >> 4;
     const uint32_t tmem = p.h->tmem_base;
-    const uint32_t ones = smem_u32(p.h->ones);
-    const uint32_t idesc_tap0 = make_idesc(Ms, min(cin16, 256), true, true);
-    const uint32_t idesc_tap1 = cin16 > 256 ? make_idesc(Ms, cin16 - 256, true, true) : 0u;
-    const uint32_t idesc_bias = make_idesc(Ms, 16, true, true);
+    Header* H = p.h;
 
     int u0 = 0;
     while (u0 < nunits) {
         // units of this pass: as many as fit in the tensor-memory columns
         int u1 = u0, cols = 0;
-        while (u1 < nunits) {
-            const int c = (u1 % (KK + 1)) == KK ? 16 : cin16;
+        while (u1 < nunits && u1 - u0 < kTcMaxUnits) {
+            const int c = (u1 % (T + 1)) == T ? 16 : ucols;
             if (cols + c > kTcTmemCols) break;
             cols += c; ++u1;
         }
         if (warp == 0 && lane == 0) {
-            // adds only between two MMAs (see conv_mma)
-            const uint32_t a_hi = desc_hi(dz_plane), x_hi = desc_hi(x_plane);
+            // Table of this pass's MMAs (operand descriptor halves, instruction descriptor, accumulator
+            // column), built once; the K loop below then only adds the step to the descriptors.
+            const uint32_t a_hi = desc_hi(dz_plane);
+            const uint32_t x_hi = desc_hi(folded ? 16u : x_plane);
             const uint32_t a_lo0 = desc_lo(dz_run, 128), x_lo0 = desc_lo(x_base, 128);
-            const uint64_t ones_d = make_desc(ones, 0, 0);
             const uint32_t slice16 = 16u * (dz_plane >> 4), xhalf16 = 32u * (x_plane >> 4);
-            const int s0 = u0 / (KK + 1), t0 = u0 - s0 * (KK + 1), ky0 = t0 / K, kx0 = t0 - ky0 * K;
+            const uint32_t id0 = make_idesc(Ms, min(ucols, 256), true, true);
+            const uint32_t id1 = ucols > 256 ? make_idesc(Ms, ucols - 256, true, true) : 0u;
+            const uint32_t idb = make_idesc(Ms, 16, true, true);
+            int nw = 0, nbias = 0;
+            {
+                const int s0 = u0 / (T + 1);
+                int t = u0 - s0 * (T + 1), ky = folded ? t : t / K, kx = folded ? 0 : t - ky * K;
+                uint32_t a_lo = a_lo0 + (uint32_t)s0 * slice16, col = tmem;
+                for (int u = u0; u < u1; ++u) {
+                    if (t == T) {
+                        H->dw_bias[nbias++] = make_uint2(a_lo, col);
+                        col += 16; t = 0; ky = 0; kx = 0; a_lo += slice16;
+                    } else {
+                        const uint32_t x_lo = x_lo0 + (uint32_t)(ky * Wp + kx);
+                        H->dw_unit[nw] = make_uint4(a_lo, x_lo, id0, col); ++nw;
+                        if (ucols > 256) { H->dw_unit[nw] = make_uint4(a_lo, x_lo + xhalf16, id1, col + 256); ++nw; }
+                        col += (uint32_t)ucols; ++t;
+                        if (folded) ++ky; else if (++kx == K) { kx = 0; ++ky; }
+                    }
+                }
+            }
+            const uint64_t ones_d = make_desc(smem_u32(H->ones), 0, 0);
             for (int ks = 0; ks < nk; ++ks) {
                 const bool acc = ks > 0;
                 const uint32_t kso = (uint32_t)ks * 16u;
-                uint32_t a_lo = a_lo0 + (uint32_t)s0 * slice16 + kso;
-                uint32_t x_lo = x_lo0 + (uint32_t)(ky0 * Wp + kx0) + kso;
-                uint32_t tcol = tmem;
-                int t = t0, kx = kx0;
-                for (int u = u0; u < u1; ++u) {
-                    const uint64_t ad = desc64(a_hi, a_lo);
-                    if (t == KK) {
-                        mma_bf16(tcol, ad, ones_d, idesc_bias, acc);
-                        tcol += 16;
-                        t = 0; kx = 0; a_lo += slice16; x_lo = x_lo0 + kso;      // next slice of output channels
-                    } else {
-                        mma_bf16(tcol, ad, desc64(x_hi, x_lo), idesc_tap0, acc);
-                        if (cin16 > 256) mma_bf16(tcol + 256, ad, desc64(x_hi, x_lo + xhalf16), idesc_tap1, acc);
-                        tcol += (uint32_t)cin16;
-                        ++t; ++kx; ++x_lo;
-                        if (kx == K) { kx = 0; x_lo += (uint32_t)(Wp - K); }
-                    }
+#pragma unroll 4
+                for (int e = 0; e < nw; ++e) {
+                    const uint4 d = H->dw_unit[e];
+                    mma_bf16(d.w, desc64(a_hi, d.x + kso), desc64(x_hi, d.y + kso), d.z, acc);
+                }
+                for (int e = 0; e < nbias; ++e) {
+                    const uint2 d = H->dw_bias[e];
+                    mma_bf16(d.y, desc64(a_hi, d.x + kso), ones_d, idb, acc);
                 }
             }
             mma_commit(smem_u32(&p.h->done));
@@ -370,16 +389,31 @@ __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*addre
         const bool row_ok = Ms == 128 || lane < 16;
         int col = 0;
         for (int u = u0; u < u1; ++u) {
-            const int slice = u / (KK + 1), t = u % (KK + 1);
+            const int slice = u / (T + 1), t = u % (T + 1);
             const int co = slice * 128 + row;
-            const int ncols = t == KK ? 16 : cin16;
+            const int ncols = t == T ? 16 : ucols;
             for (int c0 = (warp >> 2) * 16; c0 < ncols; c0 += 32) {
                 float v[16];
                 tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(col + c0), v);
                 if (row_ok && co < cout16) {
-                    if (t == KK) {
+                    if (t == T) {
                         float* g = gset + (size_t)KK * cout16 * cin16 + co;
                         if (first) *g = v[0]; else atomicAdd(g, v[0]);
+                    } else if (folded) {
+                        // columns c0 .. c0+15 of filter row t: window columns kx = c0/8 and c0/8 + 1, channels 0..7
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const int kx = (c0 >> 3) + h;
+                            if (kx < K) {
+                                float* g = gset + ((size_t)(t * K + kx) * cout16 + co) * cin16;
+#pragma unroll
+                                for (int j = 0; j < 2; ++j) {
+                                    const float* w4 = v + 8 * h + 4 * j;
+                                    if (first) *reinterpret_cast<float4*>(g + 4 * j) = make_float4(w4[0], w4[1], w4[2], w4[3]);
+                                    else red_add_v4(g + 4 * j, w4[0], w4[1], w4[2], w4[3]);
+                                }
+                            }
+                        }
                     } else {
                         float* g = gset + ((size_t)t * cout16 + co) * cin16 + c0;
 #pragma unroll
@@ -684,7 +718,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) bwd_group_tc_kernel(const __gri
             } else {
                 const int a = op.k - 1, coh = op.S * oh, cow = op.S * ow;
                 filter_grad_mma(pipe, tc::smem_u32(DZ.at(0, a, a)), DZ.plane, tc::smem_u32(X.base), X.plane, DZ.Wp, op.k,
-                                op.cout16, op.cin16, (coh - 1) * DZ.Wp + cow, myset + op.tgp_off, first);
+                                op.cout16, op.cin16, op.cin, (coh - 1) * DZ.Wp + cow, myset + op.tgp_off, first);
                 if (need_in_delta)
                     conv_mma(pipe, tc::smem_u32(DZ.at(0, vy0, vx0)), DZ.Wp, DZ.plane, op.cout16 / 8, op.k, op.cin16,
                              A.wpk + op.twb_off, ih, iw,

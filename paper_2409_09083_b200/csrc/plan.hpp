@@ -25,6 +25,7 @@ constexpr int kTcTmemCols   = 512;
 constexpr int kTcHeader     = 4096;       // per-block tables, barriers, bias staging
 constexpr int kTcFixedBytes = kTcHeader + kTcStages * kTcStageBytes;   // shared memory before the activation area
 constexpr int kTcSmemBudget = 227 * 1024; // dynamic shared memory a tensor-core block may use
+constexpr int kTcMaxUnits = 32;           // filter-gradient accumulators per pass (at least 16 columns each)
 constexpr int kTcTailEntries = 16;        // 16-byte entries appended to every tile plane
 
 struct Span { int a, b; };            // inclusive interval on one axis

