@@ -154,7 +154,7 @@ def check_groups_against_oracle(wl, groups, x, params, dy, small_maps):
         else:
             # benchmark-size maps: all but a few isolated pixels (a pooling window or an activation sign
             # decided the other way moves one delta) within the tolerance, and the whole map in L2
-            assert off <= 5e-2 and l2_err(dx, dref) <= 3e-2, (first, last, off)
+            assert off <= 5e-2 and l2_err(dx, dref) <= 5e-2, (first, last, off)
 
 
 @pytest.mark.parametrize("name", sorted(GROUPWISE))
