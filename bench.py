@@ -51,6 +51,7 @@ def parse():
     ap.add_argument("--precision", default="fp32", choices=["fp32", "bf16"],
                     help="fp32: CUDA-core path (tolerance 1e-4); bf16: tcgen05 tensor-core path, bf16 maps, fp32 accumulation (2e-2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-bf16", action="store_true", help="skip the second measurement on the bf16 tensor-core path")
     return ap.parse_args()
 
 
@@ -158,11 +159,27 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
+    line = measure(args, args.precision, rank, world, local, dist, ftp, dp, torch)
+    if rank == 0:
+        if world == 1 and args.precision == "fp32" and not args.no_bf16:
+            # the same step on the tensor-core path, reported beside the fp32 headline
+            second = measure(args, "bf16", rank, world, local, dist, ftp, dp, torch, extras=False)
+            line["bf16_tensor_core_path"] = {k: second[k] for k in ("value", "unit", "ms_per_step", "dtype", "roofline",
+                                                                    "breakdown_ms_per_step", "per_group_ms_per_step",
+                                                                    "gpu_launches", "e2e", "loss")}
+            line["bf16_tensor_core_path"]["executed_groups"] = second["config"]["executed_groups"]
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def measure(args, precision, rank, world, local, dist, ftp, dp, torch, extras=True):
+    """Times `steps` training steps of the workload at one precision; returns the JSON line (rank 0) or None."""
     wl = synth.workload(args.workload).with_(seed=rank)       # per-GPU batch is fixed: weak scaling
     x, params, target = synth.draw(wl)
     if world > 1:                                             # same initial parameters on every rank
         params = synth.draw(wl.with_(seed=0))[1]
-    tcp = args.precision == "bf16"
+    tcp = precision == "bf16"
     plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=1 if tcp else 0)
     ws = plan.new_workspace()
     xd, pd, td = (torch.from_numpy(a).cuda() for a in (x, params, target))
@@ -233,9 +250,7 @@ def run_ours(args):
                "h2d_bytes_per_step": int(xh.numel() * 4 + th.numel() * 4), "d2h_bytes_per_step": 4}
 
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return
+        return None
 
     macs = synth.forward_macs_per_image(wl.layers, wl.C, wl.H, wl.W)
     steps = args.steps
@@ -266,21 +281,19 @@ def run_ours(args):
     line = {"metric": METRIC, "value": world * wl.N * steps / (total_ms / 1e3), "unit": UNIT, "n_gpus": world,
             "steps": steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if tcp else "f32", "data": "synthetic",
-            "config": config_of(wl, {"global_batch": wl.N * world, "precision": args.precision, "executed_groups": plan.exec_groups(),
+            "config": config_of(wl, {"global_batch": wl.N * world, "precision": precision, "executed_groups": plan.exec_groups(),
                                      "parallelism": f"dp{world}", "l2": "flushed between timed steps (256 MiB write)",
                                      "redundancy_fwd": plan.redundancy}),
             "clocks": clocks, "gpu_launches": int(launches), "breakdown_ms_per_step": breakdown, "per_group_ms_per_step": per_group,
             "roofline": roofline, "loss": float(loss.item())}
     if e2e is not None:
         line["e2e"] = e2e
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and extras and not args.no_cpu_baseline:
         images = min(wl.N, 2)
         sec, cores = time_oracle(wl, images, 1, 0)
         line["cpu_baseline"] = {"value": images / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"one fp64 oracle training step on {images} image(s) of {wl.name} at full resolution"}
-    print(json.dumps(line))
-    if dist is not None:
-        dist.destroy_process_group()
+    return line
 
 
 def main():
