@@ -51,6 +51,8 @@ def parse():
     ap.add_argument("--precision", default="fp32", choices=["fp32", "bf16"],
                     help="fp32: CUDA-core path (tolerance 1e-4); bf16: tcgen05 tensor-core path, bf16 maps, fp32 accumulation (2e-2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tc-blocks", type=int, default=0, choices=[0, 1, 2],
+                    help="bf16 path: thread blocks per SM (0 = planner default)")
     ap.add_argument("--no-bf16", action="store_true", help="skip the second measurement on the bf16 tensor-core path")
     return ap.parse_args()
 
@@ -180,7 +182,8 @@ def measure(args, precision, rank, world, local, dist, ftp, dp, torch, extras=Tr
     if world > 1:                                             # same initial parameters on every rank
         params = synth.draw(wl.with_(seed=0))[1]
     tcp = precision == "bf16"
-    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=1 if tcp else 0)
+    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=1 if tcp else 0,
+                        tc_blocks_per_sm=args.tc_blocks if tcp else 0)
     ws = plan.new_workspace()
     xd, pd, td = (torch.from_numpy(a).cuda() for a in (x, params, target))
     dx = torch.empty_like(xd)

@@ -110,6 +110,10 @@ typedef struct {
     int max_subtile;    /* upper bound on the sub-tile extent (default: none) */
     int smem_bytes;     /* dynamic shared memory a block may use (default and maximum 230400) */
     int strict_groups;  /* 1: never cut a requested group; FTP_ERR_WORKSPACE if it cannot fit at all */
+    int tc_blocks_per_sm; /* bf16 path: thread blocks per SM, 1 or 2, for both passes of every group whose layers have at
+                           most 256 channels (two blocks hide each other's latencies but each gets half of the shared
+                           and tensor memory, i.e. smaller sub-tiles).  Default: 2 only in the forward pass of groups
+                           with at most 64 channels */
 } ftp_plan_opts;
 
 /* ftp_plan_create with explicit planner options (NULL = defaults). */

@@ -105,8 +105,10 @@ int pack_filters(ftp_plan* p, const float* params, void* ws, cudaStream_t st)
 
 inline bool is_tc(const ftp_plan* p) { return p->precision == FTP_BF16_FP32ACC; }
 inline int* err_ptr(void* ws, const ftp_plan* p) { return reinterpret_cast<int*>(static_cast<unsigned char*>(ws) + p->ws.err_off); }
-constexpr size_t kTcMinSmem = 120 * 1024;     // more than half an SM's shared memory: one block per SM, so the
-                                              // block's 512 tensor-memory columns are always available
+// Shared memory requested per block, so that exactly `ctas` blocks share an SM and the tensor memory
+// they allocate (512 / ctas columns each) is always available: more than half of the SM's 228 KB for
+// one block, more than a third for two.
+inline size_t tc_smem(size_t need, int ctas) { return std::max(need, (size_t)(ctas == 2 ? 77 : 120) * 1024); }
 
 void fill_common_tc(const ftp_plan* p, const GroupPlan& g, bool backward, const float* x, const float* params,
                     void* ws, TcGroupArgs& a)
@@ -167,8 +169,9 @@ int forward_tc(ftp_plan* p, const float* x, const float* params, float* y, void*
         fill_common_tc(p, g, false, x, params, ws, a);
         const int items = a.R * a.Q * p->N;
         { Timed t(p, st, 1, (int)gi);
-          const size_t smem = std::max(g.fwd.smem_bytes, kTcMinSmem);
-          fwd_group_tc_kernel<<<std::min(items, kSmCount), kTcThreads, smem, st>>>(a, (int)(smem - kTcFixedBytes)); }
+          const size_t smem = tc_smem(g.fwd.smem_bytes, g.fwd.ctas);
+          fwd_group_tc_kernel<<<std::min(items, kSmCount * g.fwd.ctas), kTcThreads, smem, st>>>(
+              a, (int)(smem - kTcFixedBytes), kTcTmemCols / g.fwd.ctas); }
         if (!launched_ok()) return FTP_ERR_CUDA;
     }
     if (y) {
@@ -221,8 +224,8 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
         a.splits = g.bwd.splits; a.tiles_x = p->grid_x;
         a.need_dx = (gi > 0 || dx != nullptr) ? 1 : 0;
         { Timed t(p, st, 3, gi);
-          const size_t smem = std::max(g.bwd.smem_bytes, kTcMinSmem);
-          bwd_group_tc_kernel<<<g.bwd.blocks, kTcThreads, smem, st>>>(a, (int)(smem - kTcFixedBytes)); }
+          const size_t smem = tc_smem(g.bwd.smem_bytes, g.bwd.ctas);
+          bwd_group_tc_kernel<<<g.bwd.blocks, kTcThreads, smem, st>>>(a, (int)(smem - kTcFixedBytes), kTcTmemCols / g.bwd.ctas); }
         if (!launched_ok()) return FTP_ERR_CUDA;
         if (a.need_dx) {
             const MapShape& s = p->maps[g.first - 1];
@@ -329,6 +332,8 @@ int ftp_plan_create_opts(const ftp_layer* layers, int n_layers, int N, int C, in
         if (opts->max_subtile) po.max_subtile = opts->max_subtile;
         if (opts->smem_bytes) po.smem_bytes = opts->smem_bytes;
         po.strict_groups = opts->strict_groups;
+        if (opts->tc_blocks_per_sm < 0 || opts->tc_blocks_per_sm > 2) return FTP_ERR_ARG;
+        po.tc_ctas = opts->tc_blocks_per_sm;
     }
     ftp_plan* p = new (std::nothrow) ftp_plan();
     if (!p) return FTP_ERR_ARG;

@@ -49,8 +49,9 @@ struct Header {
     unsigned long long empty[kTcStages];         // weight stage consumed (tcgen05.commit)
     unsigned long long done;                     // all MMAs of a pass completed
     uint32_t tmem_base;
+    int tmem_cols;                               // columns this block allocated (512, or 256 with two blocks per SM)
     volatile int failed;                         // a wait ran out: skip every later wait
-    int pad_[2];
+    int pad_[1];
     __align__(16) __nv_bfloat16 ones[64];        // one core matrix of 1.0: operand of the bias-gradient contraction
     __align__(16) uint4 dw_unit[2 * kTcMaxUnits]; // filter gradient: MMAs of the current pass {a_lo, x_lo, idesc, column}
     uint2 dw_bias[kTcMaxUnits];                  //                  bias MMAs {a_lo, column}
@@ -109,7 +110,7 @@ __device__ __forceinline__ void conv_mma(Pipe& p, uint32_t a_base, int a_Wp, uin
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nby = (rows + 15) >> 4, nbx = (cols + 7) >> 3, nblocks = nby * nbx;
-    const int in_flight = kTcTmemCols / N;
+    const int in_flight = p.h->tmem_cols / N;
     const int planes = K * K * kplanes;                               // even
     int spp = (kTcStageBytes / (N * 16)) & ~1;                        // planes per stage, even, >= 2
     if (spp > planes) spp = planes;
@@ -269,15 +270,16 @@ __device__ __forceinline__ void zero_bytes(unsigned char* p, size_t bytes)
         *reinterpret_cast<uint4*>(p + e) = make_uint4(0, 0, 0, 0);
 }
 
-__device__ __forceinline__ void setup(Header* h, Pipe& p, unsigned char* smem, int* error, size_t tile_bytes)
+__device__ __forceinline__ void setup(Header* h, Pipe& p, unsigned char* smem, int* error, size_t tile_bytes, int tmem_cols)
 {
     if (threadIdx.x == 0) {
+        h->tmem_cols = tmem_cols;
         for (int s = 0; s < kTcStages; ++s) { mbar_init(smem_u32(&h->full[s]), 1); mbar_init(smem_u32(&h->empty[s]), 1); }
         mbar_init(smem_u32(&h->done), 1);
         h->failed = 0;
         fence_mbar_init();
     }
-    if (threadIdx.x < 32) { __syncwarp(); tmem_alloc(smem_u32(&h->tmem_base), kTcTmemCols); }
+    if (threadIdx.x < 32) { __syncwarp(); tmem_alloc(smem_u32(&h->tmem_base), (uint32_t)tmem_cols); }
     // every byte the tensor core may ever read is a finite bf16 from here on
     zero_bytes(smem + kTcFixedBytes, tile_bytes);
     for (int i = threadIdx.x; i < 64; i += blockDim.x) h->ones[i] = __float2bfloat16(1.0f);
@@ -291,7 +293,7 @@ __device__ __forceinline__ void teardown(Header* h)
 {
     fence_before_sync();
     __syncthreads();
-    if (threadIdx.x < 32) tmem_dealloc(h->tmem_base, kTcTmemCols);
+    if (threadIdx.x < 32) tmem_dealloc(h->tmem_base, (uint32_t)h->tmem_cols);
 }
 
 // Partial filter gradient of one sub-tile on the tensor core (Section 4.1: the feature-map tile
@@ -332,7 +334,7 @@ __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*addre
         int u1 = u0, cols = 0;
         while (u1 < nunits && u1 - u0 < kTcMaxUnits) {
             const int c = (u1 % (T + 1)) == T ? 16 : ucols;
-            if (cols + c > kTcTmemCols) break;
+            if (cols + c > H->tmem_cols) break;
             cols += c; ++u1;
         }
         if (warp == 0 && lane == 0) {
@@ -438,14 +440,14 @@ __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*addre
 // ---------------------------------------------------------------------------------------------
 // Fused forward of one group, bf16: persistent blocks walk over the (image, sub-tile) stacks.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kTcThreads, 1) fwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes)
+__global__ void __launch_bounds__(kTcThreads, 2) fwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes, int tmem_cols)
 {
     using namespace tcd;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Header* H = reinterpret_cast<Header*>(smem_raw);
     unsigned char* tiles = smem_raw + kTcFixedBytes;
     Pipe pipe;
-    setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes);
+    setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes, tmem_cols);
     int* hdr = H->hdr;
     const int items = A.N * A.R * A.Q;
 
@@ -563,14 +565,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) fwd_group_tc_kernel(const __gri
 // Fused backward of one group, bf16 (adjoint form): each block owns one partial gradient set and
 // walks through its share of the (image, sub-tile) stacks of one user tile in a fixed order.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kTcThreads, 1) bwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes)
+__global__ void __launch_bounds__(kTcThreads, 2) bwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes, int tmem_cols)
 {
     using namespace tcd;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Header* H = reinterpret_cast<Header*>(smem_raw);
     unsigned char* tiles = smem_raw + kTcFixedBytes;
     Pipe pipe;
-    setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes);
+    setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes, tmem_cols);
     int* hdr = H->hdr;
 
     const int slot = blockIdx.x, tile = slot / A.splits, split = slot % A.splits;

@@ -255,7 +255,9 @@ int choose_subtiles(GroupPlan& g, bool backward, const PlanOpts& o)
             size_t bytes;
             if (o.tensor_cores) bytes = backward ? layout_backward_tc(g, pp.y, pp.x) : layout_forward_tc(g, pp.y, pp.x);
             else bytes = backward ? layout_backward(g, pp.y, pp.x) : layout_forward(g, pp.y, pp.x);
-            if (bytes <= (size_t)(o.tensor_cores ? std::min(kTcSmemBudget, o.smem_bytes + 2048) : o.smem_bytes)) {
+            size_t budget = (size_t)o.smem_bytes;
+            if (o.tensor_cores) budget = std::min<size_t>(pp.ctas == 2 ? kTcSmemBudget2 : kTcSmemBudget, (size_t)o.smem_bytes + 2048);
+            if (bytes <= budget) {
                 pp.smem_bytes = bytes;
                 return FTP_OK;
             }
@@ -337,10 +339,23 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
     if (g.param_begin < 0) g.param_begin = 0;
     g.param_floats = (size_t)(tcp ? tgp : gp);
 
-    int rc = choose_subtiles(g, false, o);
-    if (rc != FTP_OK) return rc;
-    rc = choose_subtiles(g, true, o);
-    if (rc != FTP_OK) return rc;
+    // Tensor-core path: two blocks per SM hide the latencies of a block's serial phases behind the
+    // other block; each then has half of the shared and tensor memory, so no operand of the group may
+    // span more than 256 accumulator columns.  Left to the planner, only the forward pass of groups
+    // with at most 64 channels runs that way: measured on B200, wider layers and the backward pass
+    // (three live tiles) lose more from the smaller sub-tiles than they gain.
+    int max_ch = 0;
+    for (int i = 0; i < g.n_ops; ++i)
+        if (g.fwd_ops[i].kind != kOpPool) max_ch = std::max(max_ch, std::max(g.fwd_ops[i].cin16, g.fwd_ops[i].cout16));
+    const int want_fwd = !tcp ? 1 : o.tc_ctas == 0 ? (max_ch <= 64 ? 2 : 1) : (o.tc_ctas == 2 && max_ch <= 256 ? 2 : 1);
+    const int want_bwd = tcp && o.tc_ctas == 2 && max_ch <= 256 ? 2 : 1;
+    for (int pass = 0; pass < 2; ++pass) {
+        PassPlan& pp = pass ? g.bwd : g.fwd;
+        pp.ctas = pass ? want_bwd : want_fwd;
+        int rc = choose_subtiles(g, pass == 1, o);
+        if (rc != FTP_OK && pp.ctas == 2) { pp.ctas = 1; rc = choose_subtiles(g, pass == 1, o); }
+        if (rc != FTP_OK) return rc;
+    }
     double bwd_done = 0, bwd_untiled = 0;
     count_macs(g, g.fwd, &g.macs_done, &g.macs_untiled);
     count_macs(g, g.bwd, &bwd_done, &bwd_untiled);
@@ -356,7 +371,7 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
                         (g.bwd.x.tile_begin[tx + 1] - g.bwd.x.tile_begin[tx]);
             min_items = std::min(min_items, items);
         }
-    g.bwd.splits = std::max(1, std::min(min_items, kSmCount / (gy * gx)));
+    g.bwd.splits = std::max(1, std::min(min_items, kSmCount * g.bwd.ctas / (gy * gx)));
     g.bwd.blocks = gy * gx * g.bwd.splits;
     g.bwd.scratch_floats = (size_t)N * p.maps[first - 1].C * g.bwd.y.scratch_off[g.bwd.y.count] *
                            g.bwd.x.scratch_off[g.bwd.x.count];

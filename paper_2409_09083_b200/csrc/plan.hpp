@@ -21,10 +21,11 @@ constexpr int kCoutTile    = 8;       // output channels per thread task (packed
 constexpr int kTcThreads    = 256;
 constexpr int kTcStages     = 2;          // weight ring: stages of kTcStageBytes
 constexpr int kTcStageBytes = 16384;
-constexpr int kTcTmemCols   = 512;
+constexpr int kTcTmemCols   = 512;        // tensor-memory columns of an SM; a block takes all of them, or half with two blocks per SM
 constexpr int kTcHeader     = 4096;       // per-block tables, barriers, bias staging
 constexpr int kTcFixedBytes = kTcHeader + kTcStages * kTcStageBytes;   // shared memory before the activation area
-constexpr int kTcSmemBudget = 227 * 1024; // dynamic shared memory a tensor-core block may use
+constexpr int kTcSmemBudget = 227 * 1024; // dynamic shared memory a tensor-core block may use (one block per SM)
+constexpr int kTcSmemBudget2 = 113 * 1024;// ... with two blocks per SM
 constexpr int kTcMaxUnits = 32;           // filter-gradient accumulators per pass (at least 16 columns each)
 constexpr int kTcTailEntries = 16;        // 16-byte entries appended to every tile plane
 
@@ -77,6 +78,7 @@ struct PassPlan {
     size_t smem_bytes = 0;
     int blocks = 0;                 // forward: R*Q*N ; backward: tiles * splits
     int splits = 1;                 // backward: blocks per user tile
+    int ctas = 1;                   // tensor-core path: blocks per SM (2 = each block takes half of the tensor memory)
     size_t scratch_floats = 0;      // backward: floats of per-sub-tile group-input deltas (all images)
     // offsets (in ints) of the tables inside the plan's device table blob
     int dev_yspan = 0, dev_xspan = 0, dev_ycell = 0, dev_xcell = 0;
@@ -145,6 +147,7 @@ struct PlanOpts {
     int max_subtile = 0;            // 0 = as large as fits; else an upper bound (tests use it to force sub-tiling)
     int smem_bytes = kSmemBudget;   // dynamic shared memory a block may use
     int strict_groups = 0;          // 1 = never cut a requested group
+    int tc_ctas = 0;                // tensor-core path: blocks per SM, 1 or 2 (0 = two where every layer of the group allows it)
     int tensor_cores = 0;           // set by build_plan from the precision: shared-memory layouts of the bf16 path
 };
 // Builds everything but the device upload.  Returns FTP_OK or an error code.
