@@ -51,7 +51,7 @@ struct Header {
     uint32_t tmem_base;
     int tmem_cols;                               // columns this block allocated (512, or 256 with two blocks per SM)
     volatile int failed;                         // a wait ran out: skip every later wait
-    int pad_[1];
+    int dw_nw, dw_nbias;                         // entries of dw_unit / dw_bias in the current pass
     __align__(16) __nv_bfloat16 ones[64];        // one core matrix of 1.0: operand of the bias-gradient contraction
     __align__(16) uint4 dw_unit[2 * kTcMaxUnits]; // filter gradient: MMAs of the current pass {a_lo, x_lo, idesc, column}
     uint2 dw_bias[kTcMaxUnits];                  //                  bias MMAs {a_lo, column}
@@ -120,7 +120,7 @@ __device__ __forceinline__ void conv_mma(Pipe& p, uint32_t a_base, int a_Wp, uin
 
     for (int b0 = 0; b0 < nblocks; b0 += in_flight) {
         const int nb = min(in_flight, nblocks - b0);
-        if (warp == 1 && lane == 0) {
+        if (warp == kTcIssuers && lane == 0) {
             // producer: one bulk copy per stage
             for (int s = 0; s < nstages; ++s) {
                 const uint32_t q = p.stages_done + s, slot = q % kTcStages, par = (q / kTcStages) & 1;
@@ -130,9 +130,12 @@ __device__ __forceinline__ void conv_mma(Pipe& p, uint32_t a_base, int a_Wp, uin
                 mbar_expect_tx(smem_u32(&p.h->full[slot]), bytes);
                 bulk_g2s(p.ring + slot * kTcStageBytes, w + (size_t)s * spp * N * 8, bytes, smem_u32(&p.h->full[slot]));
             }
-        } else if (warp == 0 && lane == 0) {
-            // MMA issue.  Descriptor halves are advanced with adds only (no division or multiplication
-            // inside the loops): the tensor core idles while this thread computes.
+        } else if (warp < kTcIssuers && lane == 0) {
+            // MMA issue.  A single thread cannot keep the tensor core busy (an MMA of this size takes it
+            // about 45 cycles, the thread needs well over 100 to prepare the next one), so lane 0 of the
+            // first kTcIssuers warps each issue the MMAs of every kTcIssuers-th pixel block; their
+            // accumulators are disjoint, so no order between the issuers is needed.  Descriptor halves
+            // are advanced with adds only.
             const uint32_t a_hi = desc_hi((uint32_t)a_Wp * 16), b_hi = desc_hi(128);
             const uint32_t plane16 = a_plane >> 4, bplane16 = plane_bytes >> 4;
             const uint32_t idesc_full = make_idesc(128, min(N, 256), false, false);
@@ -147,9 +150,9 @@ __device__ __forceinline__ void conv_mma(Pipe& p, uint32_t a_base, int a_Wp, uin
                 // window position and channel plane at which the stage starts (once per stage)
                 const int tap0 = gp0 / kplanes, kc0 = gp0 - tap0 * kplanes, ky0 = tap0 / K, kx0 = tap0 - ky0 * K;
                 const uint32_t off0 = (uint32_t)kc0 * plane16 + (uint32_t)(ky0 * a_Wp + kx0);
-                int by = b0 / nbx, bx = b0 - by * nbx;
-                uint32_t tcol = tmem;
-                for (int bi = 0; bi < nb; ++bi) {
+                for (int bi = warp; bi < nb; bi += kTcIssuers) {
+                    const int b = b0 + bi, by = b / nbx, bx = b - by * nbx;
+                    const uint32_t tcol = tmem + (uint32_t)(bi * N);
                     const uint32_t a_lo0 = desc_lo(a_base + (uint32_t)((by * 16) * a_Wp + bx * 8) * 16, a_plane);
                     uint32_t off = off0, b_lo = b_lo0;
                     int kc = kc0, kx = kx0;
@@ -167,8 +170,6 @@ __device__ __forceinline__ void conv_mma(Pipe& p, uint32_t a_base, int a_Wp, uin
                             if (kx == K) { kx = 0; off += (uint32_t)(a_Wp - K); }
                         }
                     }
-                    tcol += (uint32_t)N;
-                    if (++bx == nbx) { bx = 0; ++by; }
                 }
                 mma_commit(smem_u32(&p.h->empty[slot]));
                 gp0 += pl;
@@ -274,8 +275,8 @@ __device__ __forceinline__ void setup(Header* h, Pipe& p, unsigned char* smem, i
 {
     if (threadIdx.x == 0) {
         h->tmem_cols = tmem_cols;
-        for (int s = 0; s < kTcStages; ++s) { mbar_init(smem_u32(&h->full[s]), 1); mbar_init(smem_u32(&h->empty[s]), 1); }
-        mbar_init(smem_u32(&h->done), 1);
+        for (int s = 0; s < kTcStages; ++s) { mbar_init(smem_u32(&h->full[s]), 1); mbar_init(smem_u32(&h->empty[s]), kTcIssuers); }
+        mbar_init(smem_u32(&h->done), kTcIssuers);
         h->failed = 0;
         fence_mbar_init();
     }
@@ -337,47 +338,51 @@ __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*addre
             if (cols + c > H->tmem_cols) break;
             cols += c; ++u1;
         }
+        const uint32_t a_hi = desc_hi(dz_plane);
+        const uint32_t x_hi = desc_hi(folded ? 16u : x_plane);
         if (warp == 0 && lane == 0) {
             // Table of this pass's MMAs (operand descriptor halves, instruction descriptor, accumulator
-            // column), built once; the K loop below then only adds the step to the descriptors.
-            const uint32_t a_hi = desc_hi(dz_plane);
-            const uint32_t x_hi = desc_hi(folded ? 16u : x_plane);
+            // column), built once; the K loops below then only add the step to the descriptors.
             const uint32_t a_lo0 = desc_lo(dz_run, 128), x_lo0 = desc_lo(x_base, 128);
             const uint32_t slice16 = 16u * (dz_plane >> 4), xhalf16 = 32u * (x_plane >> 4);
             const uint32_t id0 = make_idesc(Ms, min(ucols, 256), true, true);
             const uint32_t id1 = ucols > 256 ? make_idesc(Ms, ucols - 256, true, true) : 0u;
-            const uint32_t idb = make_idesc(Ms, 16, true, true);
             int nw = 0, nbias = 0;
-            {
-                const int s0 = u0 / (T + 1);
-                int t = u0 - s0 * (T + 1), ky = folded ? t : t / K, kx = folded ? 0 : t - ky * K;
-                uint32_t a_lo = a_lo0 + (uint32_t)s0 * slice16, col = tmem;
-                for (int u = u0; u < u1; ++u) {
-                    if (t == T) {
-                        H->dw_bias[nbias++] = make_uint2(a_lo, col);
-                        col += 16; t = 0; ky = 0; kx = 0; a_lo += slice16;
-                    } else {
-                        const uint32_t x_lo = x_lo0 + (uint32_t)(ky * Wp + kx);
-                        H->dw_unit[nw] = make_uint4(a_lo, x_lo, id0, col); ++nw;
-                        if (ucols > 256) { H->dw_unit[nw] = make_uint4(a_lo, x_lo + xhalf16, id1, col + 256); ++nw; }
-                        col += (uint32_t)ucols; ++t;
-                        if (folded) ++ky; else if (++kx == K) { kx = 0; ++ky; }
-                    }
+            const int s0 = u0 / (T + 1);
+            int t = u0 - s0 * (T + 1), ky = folded ? t : t / K, kx = folded ? 0 : t - ky * K;
+            uint32_t a_lo = a_lo0 + (uint32_t)s0 * slice16, col = tmem;
+            for (int u = u0; u < u1; ++u) {
+                if (t == T) {
+                    H->dw_bias[nbias++] = make_uint2(a_lo, col);
+                    col += 16; t = 0; ky = 0; kx = 0; a_lo += slice16;
+                } else {
+                    const uint32_t x_lo = x_lo0 + (uint32_t)(ky * Wp + kx);
+                    H->dw_unit[nw] = make_uint4(a_lo, x_lo, id0, col); ++nw;
+                    if (ucols > 256) { H->dw_unit[nw] = make_uint4(a_lo, x_lo + xhalf16, id1, col + 256); ++nw; }
+                    col += (uint32_t)ucols; ++t;
+                    if (folded) ++ky; else if (++kx == K) { kx = 0; ++ky; }
                 }
             }
+            H->dw_nw = nw; H->dw_nbias = nbias;
+        }
+        __syncthreads();
+        if (warp < kTcIssuers && lane == 0) {
+            // every issuer takes every kTcIssuers-th accumulator of the pass (see conv_mma)
+            const int nw = H->dw_nw, nbias = H->dw_nbias;
+            const uint32_t idb = make_idesc(Ms, 16, true, true);
             const uint64_t ones_d = make_desc(smem_u32(H->ones), 0, 0);
-            for (int ks = 0; ks < nk; ++ks) {
-                const bool acc = ks > 0;
-                const uint32_t kso = (uint32_t)ks * 16u;
-#pragma unroll 4
-                for (int e = 0; e < nw; ++e) {
-                    const uint4 d = H->dw_unit[e];
-                    mma_bf16(d.w, desc64(a_hi, d.x + kso), desc64(x_hi, d.y + kso), d.z, acc);
+            for (int e = warp; e < nw; e += kTcIssuers) {
+                const uint4 d = H->dw_unit[e];
+                uint32_t a_lo = d.x, x_lo = d.y;
+                for (int ks = 0; ks < nk; ++ks) {
+                    mma_bf16(d.w, desc64(a_hi, a_lo), desc64(x_hi, x_lo), d.z, ks > 0);
+                    a_lo += 16; x_lo += 16;
                 }
-                for (int e = 0; e < nbias; ++e) {
-                    const uint2 d = H->dw_bias[e];
-                    mma_bf16(d.y, desc64(a_hi, d.x + kso), ones_d, idb, acc);
-                }
+            }
+            for (int e = warp; e < nbias; e += kTcIssuers) {
+                const uint2 d = H->dw_bias[e];
+                uint32_t a_lo = d.x;
+                for (int ks = 0; ks < nk; ++ks) { mma_bf16(d.y, desc64(a_hi, a_lo), ones_d, idb, ks > 0); a_lo += 16; }
             }
             mma_commit(smem_u32(&p.h->done));
         }

@@ -26,6 +26,7 @@ constexpr int kTcHeader     = 4096;       // per-block tables, barriers, bias st
 constexpr int kTcFixedBytes = kTcHeader + kTcStages * kTcStageBytes;   // shared memory before the activation area
 constexpr int kTcSmemBudget = 227 * 1024; // dynamic shared memory a tensor-core block may use (one block per SM)
 constexpr int kTcSmemBudget2 = 113 * 1024;// ... with two blocks per SM
+constexpr int kTcIssuers = 4;             // threads (lane 0 of warps 0..3) that issue MMAs, each for its own accumulators
 constexpr int kTcMaxUnits = 32;           // filter-gradient accumulators per pass (at least 16 columns each)
 constexpr int kTcTailEntries = 16;        // 16-byte entries appended to every tile plane
 

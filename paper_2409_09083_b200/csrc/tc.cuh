@@ -52,13 +52,15 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool a_mn_major,
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// D[tmem] (+)= A[smem] * B[smem]; one thread issues for the whole CTA.
+// D[tmem] (+)= A[smem] * B[smem]; one thread issues for the whole CTA.  (No memory clobber: the
+// statement is volatile, so it keeps its order among the fences, barriers and other MMAs, while the
+// compiler may still move ordinary loads of the issuing thread across it.)
 __device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
-        :: "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+        :: "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate));
 }
 
 // Makes `mbar` receive one arrival once every MMA issued so far by this thread has completed.
