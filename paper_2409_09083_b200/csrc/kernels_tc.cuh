@@ -751,22 +751,28 @@ struct TcReduceArgs { int n; TcReduceLayer l[kMaxOps * 2]; };
 __global__ void reduce_sgd_tc_kernel(const __grid_constant__ TcReduceArgs A, float* __restrict__ params, float lr,
                                      float* __restrict__ grad_out)
 {
+    // Threads walk the set's own arrangement, so the reads of every set are coalesced (the sets are the
+    // bulk of the traffic); the one write per parameter goes to its place in the caller's arrangement.
     const TcReduceLayer L = A.l[blockIdx.y];
     const int KK = L.k * L.k;
-    const long long nf = (long long)L.cout * L.cin * KK, total = nf + L.cout;
+    const long long nf = (long long)KK * L.cout16 * L.cin16, total = nf + L.cout16;
     for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
-        long long src;
+        long long dst;
         if (e < nf) {
-            const int tap = (int)(e % KK); long long t = e / KK;
-            const int ci = (int)(t % L.cin); const int co = (int)(t / L.cin);
-            src = L.tgp_off + ((long long)tap * L.cout16 + co) * L.cin16 + ci;
+            const int ci = (int)(e % L.cin16); long long t = e / L.cin16;
+            const int co = (int)(t % L.cout16); const int tap = (int)(t / L.cout16);
+            if (ci >= L.cin || co >= L.cout) continue;
+            dst = L.p_off + ((long long)co * L.cin + ci) * KK + tap;
         } else {
-            src = L.tgp_off + (long long)KK * L.cout16 * L.cin16 + (e - nf);
+            const int co = (int)(e - nf);
+            if (co >= L.cout) continue;
+            dst = L.p_off + (long long)L.cout * L.cin * KK + co;
         }
+        const float* src = L.partial + L.tgp_off + e;
         float s = 0.f;
-        for (int k = 0; k < L.sets; ++k) s += L.partial[(size_t)k * L.set_floats + src];
-        if (grad_out) grad_out[L.p_off + e] = s;
-        if (params) params[L.p_off + e] = params[L.p_off + e] - lr * s;
+        for (int k = 0; k < L.sets; ++k) s += src[(size_t)k * L.set_floats];
+        if (grad_out) grad_out[dst] = s;
+        if (params) params[dst] = params[dst] - lr * s;
     }
 }
 
