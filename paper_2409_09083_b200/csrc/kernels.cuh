@@ -330,11 +330,119 @@ __device__ __forceinline__ void filter_grad_tile(const float* __restrict__ d, co
     }
 }
 
+// Partial filter gradient, one thread per (block of TCO output channels, input channel): the thread
+// keeps TCO x K x K sums in registers and walks over all delta pixels itself, so no cross-lane
+// reduction is needed and the sum order is fixed.  Lanes of a warp hold consecutive input channels:
+// the delta (and arg-max) reads are broadcasts, the input reads hit distinct banks because the
+// channel stride of the input copy is odd.  Used when there are enough (channel block, channel)
+// pairs to occupy the block; small layers take filter_grad_tile.
+//   !POOLED: the K x K window of the input slides along the row in registers (K new values per pixel).
+//   POOLED:  d is the delta of the pooled map; the arg-max of each 2x2 window (the same for all lanes)
+//            picks which K x K part of the (K+1) x (K+1) input window the delta meets.
+template <int K, int TCO, bool POOLED>
+__device__ __forceinline__ void filter_grad_thread(const float* __restrict__ d, const unsigned char* __restrict__ arg,
+                                                   int d_cs, int d_pitch, const float* __restrict__ xin, int in_cs,
+                                                   int in_pitch, int cin, int cout, int oh, int ow,
+                                                   float* __restrict__ g, bool first)
+{
+    constexpr int KK = K * K, WN = POOLED ? K + 1 : K;
+    const int ncob = (cout + TCO - 1) / TCO;
+    for (int task = threadIdx.x; task < ncob * cin; task += blockDim.x) {
+        const int cob = task / cin, ci = task - cob * cin, co0 = cob * TCO;
+        const float* xp = xin + ci * in_cs;
+        int doff[TCO];
+#pragma unroll
+        for (int a = 0; a < TCO; ++a) doff[a] = min(co0 + a, cout - 1) * d_cs;
+        float acc[TCO][KK];
+#pragma unroll
+        for (int a = 0; a < TCO; ++a)
+#pragma unroll
+            for (int e = 0; e < KK; ++e) acc[a][e] = 0.f;
+        for (int y = 0; y < oh; ++y) {
+            const float* xr = xp + (POOLED ? 2 * y : y) * in_pitch;
+            float w[WN][WN];
+#pragma unroll
+            for (int r = 0; r < WN; ++r)
+#pragma unroll
+                for (int c = POOLED ? 2 : 1; c < WN; ++c) w[r][c] = xr[r * in_pitch + c - (POOLED ? 2 : 1)];
+            for (int x = 0; x < ow; ++x) {
+                // shift the window by one pixel (two input columns when pooled) and load the new columns
+#pragma unroll
+                for (int r = 0; r < WN; ++r) {
+#pragma unroll
+                    for (int c = 0; c + (POOLED ? 2 : 1) < WN; ++c) w[r][c] = w[r][c + (POOLED ? 2 : 1)];
+                    if (POOLED) {
+                        w[r][WN - 2] = xr[r * in_pitch + 2 * x + WN - 2];
+                        w[r][WN - 1] = xr[r * in_pitch + 2 * x + WN - 1];
+                    } else {
+                        w[r][WN - 1] = xr[r * in_pitch + x + WN - 1];
+                    }
+                }
+                const int dp = y * d_pitch + x;
+#pragma unroll
+                for (int a = 0; a < TCO; ++a) {
+                    const float dv = d[doff[a] + dp];
+                    if (POOLED) {
+                        const int am = arg[doff[a] + dp];        // same for every lane: no divergence
+                        if (am == 0) {
+#pragma unroll
+                            for (int ky = 0; ky < K; ++ky)
+#pragma unroll
+                                for (int kx = 0; kx < K; ++kx) acc[a][ky * K + kx] = fmaf(dv, w[ky][kx], acc[a][ky * K + kx]);
+                        } else if (am == 1) {
+#pragma unroll
+                            for (int ky = 0; ky < K; ++ky)
+#pragma unroll
+                                for (int kx = 0; kx < K; ++kx) acc[a][ky * K + kx] = fmaf(dv, w[ky][kx + (POOLED ? 1 : 0)], acc[a][ky * K + kx]);
+                        } else if (am == 2) {
+#pragma unroll
+                            for (int ky = 0; ky < K; ++ky)
+#pragma unroll
+                                for (int kx = 0; kx < K; ++kx) acc[a][ky * K + kx] = fmaf(dv, w[ky + (POOLED ? 1 : 0)][kx], acc[a][ky * K + kx]);
+                        } else {
+#pragma unroll
+                            for (int ky = 0; ky < K; ++ky)
+#pragma unroll
+                                for (int kx = 0; kx < K; ++kx)
+                                    acc[a][ky * K + kx] = fmaf(dv, w[ky + (POOLED ? 1 : 0)][kx + (POOLED ? 1 : 0)], acc[a][ky * K + kx]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int ky = 0; ky < K; ++ky)
+#pragma unroll
+                            for (int kx = 0; kx < K; ++kx) acc[a][ky * K + kx] = fmaf(dv, w[ky][kx], acc[a][ky * K + kx]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int a = 0; a < TCO; ++a)
+            if (co0 + a < cout) {
+                float* dst = g + ((size_t)(co0 + a) * cin + ci) * KK;
+#pragma unroll
+                for (int e = 0; e < KK; ++e) dst[e] = first ? acc[a][e] : dst[e] + acc[a][e];
+            }
+    }
+}
+
 template <bool POOLED>
 __device__ __forceinline__ void filter_grad_k(int K, const float* d, const unsigned char* arg, int d_cs, int d_pitch,
                                               const float* xin, int in_cs, int in_pitch, int cin, int cout, int oh,
                                               int ow, float* g, bool first)
 {
+    // one thread per (channel block, channel) when that occupies at least half of the block's threads;
+    // blocks of 8 output channels if that still fills the block, else blocks of 4
+    if (K == 3) {
+        const int t8 = ((cout + 7) / 8) * cin, t4 = ((cout + 3) / 4) * cin, nt = (int)blockDim.x;
+        if (t8 >= nt || (t8 >= nt / 2 && t4 > 2 * nt)) {
+            filter_grad_thread<3, 8, POOLED>(d, arg, d_cs, d_pitch, xin, in_cs, in_pitch, cin, cout, oh, ow, g, first);
+            return;
+        }
+        if (t4 >= nt / 2) {
+            filter_grad_thread<3, 4, POOLED>(d, arg, d_cs, d_pitch, xin, in_cs, in_pitch, cin, cout, oh, ow, g, first);
+            return;
+        }
+    }
     switch (K) {
     case 1: filter_grad_tile<1, 4, 8, POOLED>(d, arg, d_cs, d_pitch, xin, in_cs, in_pitch, cin, cout, oh, ow, g, first); break;
     case 3: filter_grad_tile<3, 4, 2, POOLED>(d, arg, d_cs, d_pitch, xin, in_cs, in_pitch, cin, cout, oh, ow, g, first); break;

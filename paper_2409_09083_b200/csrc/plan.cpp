@@ -146,7 +146,7 @@ size_t layout_backward(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
         int oh = ty.maxext[i + 1], ow = tx.maxext[i + 1];
         int bh = (oh - 1) * op.S + op.keff, bw = (ow - 1) * op.S + op.keff;
         op.in_pitch = bw;
-        op.in_cs = bh * bw;
+        op.in_cs = (bh * bw) | 1;       // odd channel stride: lanes that read consecutive channels hit distinct banks
         xsize[i] = round4(op.cin * op.in_cs);
         op.d_pitch = ow;
         op.d_cs = oh * ow;
