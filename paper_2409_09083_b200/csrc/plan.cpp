@@ -5,6 +5,7 @@
 #include "plan.hpp"
 
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 
 namespace ftp {
@@ -235,8 +236,13 @@ size_t layout_backward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& 
     return (size_t)kTcFixedBytes + total + slack;
 }
 
-// Smallest split (largest sub-tile) whose buffers fit the shared-memory budget.
-int choose_subtiles(GroupPlan& g, bool backward, const PlanOpts& o)
+void count_macs(const GroupPlan& g, const PassPlan& pp, double* done, double* untiled);
+
+// Sub-tiling of one pass: the smallest split (largest sub-tile) whose buffers fit the shared-memory
+// budget; for the forward pass, whose sub-tile stacks are spread over all SMs, a slightly finer
+// split is taken instead when it fills the last round of blocks better (estimated time = rounds of
+// blocks x multiply-accumulates of one stack, halo recomputation included).
+int choose_subtiles(GroupPlan& g, bool backward, const PlanOpts& o, int N)
 {
     const AxisInfo ay = axis_info(g, true), ax = axis_info(g, false);
     int max_h = 0, max_w = 0;
@@ -246,21 +252,41 @@ int choose_subtiles(GroupPlan& g, bool backward, const PlanOpts& o)
     const int kmax = std::max(max_h, max_w);
     int k0 = 1;
     if (o.max_subtile > 0) k0 = std::max(1, (kmax + o.max_subtile - 1) / o.max_subtile);
+    auto try_split = [&](int ky, int kx) -> size_t {       // bytes if it fits, else 0
+        build_axis(pp.y, ay, g.tile_y, ky);
+        build_axis(pp.x, ax, g.tile_x, kx);
+        size_t bytes;
+        if (o.tensor_cores) bytes = backward ? layout_backward_tc(g, pp.y, pp.x) : layout_forward_tc(g, pp.y, pp.x);
+        else bytes = backward ? layout_backward(g, pp.y, pp.x) : layout_forward(g, pp.y, pp.x);
+        size_t budget = (size_t)o.smem_bytes;
+        if (o.tensor_cores) budget = std::min<size_t>(pp.ctas == 2 ? kTcSmemBudget2 : kTcSmemBudget, (size_t)o.smem_bytes + 2048);
+        return bytes <= budget ? bytes : 0;
+    };
     for (int k = k0; k <= kmax; ++k) {
         const int cand[3][2] = {{k, k}, {k + 1, k}, {k, k + 1}};
         for (const auto& c : cand) {
-            int ky = std::min(c[0], max_h), kx = std::min(c[1], max_w);
-            build_axis(pp.y, ay, g.tile_y, ky);
-            build_axis(pp.x, ax, g.tile_x, kx);
-            size_t bytes;
-            if (o.tensor_cores) bytes = backward ? layout_backward_tc(g, pp.y, pp.x) : layout_forward_tc(g, pp.y, pp.x);
-            else bytes = backward ? layout_backward(g, pp.y, pp.x) : layout_forward(g, pp.y, pp.x);
-            size_t budget = (size_t)o.smem_bytes;
-            if (o.tensor_cores) budget = std::min<size_t>(pp.ctas == 2 ? kTcSmemBudget2 : kTcSmemBudget, (size_t)o.smem_bytes + 2048);
-            if (bytes <= budget) {
-                pp.smem_bytes = bytes;
-                return FTP_OK;
-            }
+            const int ky = std::min(c[0], max_h), kx = std::min(c[1], max_w);
+            size_t bytes = try_split(ky, kx);
+            if (!bytes) continue;
+            if (backward || o.max_subtile > 0 || o.tensor_cores) { pp.smem_bytes = bytes; return FTP_OK; }   // (tensor-core stacks: per-stack overheads outweigh a fuller last round)
+            // forward: look a little further for a split that wastes less of the last round
+            int best_ky = ky, best_kx = kx;
+            double best = -1, fixed = 0;     // fixed: per-stack cost that does not shrink with the tile (loads, syncs)
+            for (int dy = 0; dy <= 3; ++dy)
+                for (int dx = 0; dx <= 3; ++dx) {
+                    const int yy = std::min(ky + dy, max_h), xx = std::min(kx + dx, max_w);
+                    if (!try_split(yy, xx)) continue;
+                    double done = 0, untiled = 0;
+                    count_macs(g, pp, &done, &untiled);
+                    const double items = (double)N * pp.y.count * pp.x.count;
+                    const double slots = (double)kSmCount * pp.ctas;
+                    const double rounds = std::ceil(items / slots);
+                    if (dy == 0 && dx == 0) fixed = 0.3 * done * N / items;
+                    const double est = rounds * (done * N / items + fixed);
+                    if (best < 0 || est < best * 0.97) { best = est; best_ky = yy; best_kx = xx; }
+                }
+            pp.smem_bytes = try_split(best_ky, best_kx);
+            return FTP_OK;
         }
     }
     return FTP_ERR_WORKSPACE;
@@ -352,8 +378,8 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
     for (int pass = 0; pass < 2; ++pass) {
         PassPlan& pp = pass ? g.bwd : g.fwd;
         pp.ctas = pass ? want_bwd : want_fwd;
-        int rc = choose_subtiles(g, pass == 1, o);
-        if (rc != FTP_OK && pp.ctas == 2) { pp.ctas = 1; rc = choose_subtiles(g, pass == 1, o); }
+        int rc = choose_subtiles(g, pass == 1, o, N);
+        if (rc != FTP_OK && pp.ctas == 2) { pp.ctas = 1; rc = choose_subtiles(g, pass == 1, o, N); }
         if (rc != FTP_OK) return rc;
     }
     double bwd_done = 0, bwd_untiled = 0;
