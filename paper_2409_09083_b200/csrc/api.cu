@@ -236,10 +236,10 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
             h.ycover = p->dev_tables + g.bwd.dev_ycover; h.xcover = p->dev_tables + g.bwd.dev_xcover;
             h.N = p->N; h.C = s.C; h.H = s.H; h.W = s.W; h.R = a.R; h.Q = a.Q;
             h.Htot = g.bwd.y.scratch_off[a.R]; h.Wtot = g.bwd.x.scratch_off[a.Q];
-            const size_t total = (size_t)p->N * s.C * s.H * s.W;
-            const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16);
+            const size_t rows = (size_t)p->N * s.C * s.H;
+            const int blocks = (int)std::min<size_t>((rows + 7) / 8, (size_t)kSmCount * 16);
             { Timed t(p, st, 4, gi);
-              halo_sum_kernel<<<blocks, 256, 0, st>>>(h); }
+              halo_sum_kernel<<<blocks, 256, (size_t)(2 * h.W + 2 * h.H + 3 * h.Q + 3 * h.R + 2) * sizeof(int), st>>>(h); }
             if (!launched_ok()) return FTP_ERR_CUDA;
         }
     }
@@ -291,10 +291,10 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
             h.ycover = p->dev_tables + g.bwd.dev_ycover; h.xcover = p->dev_tables + g.bwd.dev_xcover;
             h.N = p->N; h.C = s.C; h.H = s.H; h.W = s.W; h.R = a.R; h.Q = a.Q;
             h.Htot = g.bwd.y.scratch_off[a.R]; h.Wtot = g.bwd.x.scratch_off[a.Q];
-            const size_t total = (size_t)p->N * s.C * s.H * s.W;
-            const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16);
+            const size_t rows = (size_t)p->N * s.C * s.H;
+            const int blocks = (int)std::min<size_t>((rows + 7) / 8, (size_t)kSmCount * 16);
             { Timed t(p, st, 4, gi);
-              halo_sum_kernel<<<blocks, 256, 0, st>>>(h); }
+              halo_sum_kernel<<<blocks, 256, (size_t)(2 * h.W + 2 * h.H + 3 * h.Q + 3 * h.R + 2) * sizeof(int), st>>>(h); }
             if (!launched_ok()) return FTP_ERR_CUDA;
         }
     }
@@ -449,7 +449,7 @@ static int step_impl(ftp_plan* plan, const float* x, const float* dy, const floa
                                                              target, d, M, sums); }
         if (loss_out) {
             Timed t(plan, st, 2, -1);
-            mse_finish_kernel<<<1, 32, 0, st>>>(sums, plan->loss_blocks, M, loss_out);
+            mse_finish_kernel<<<1, 256, 0, st>>>(sums, plan->loss_blocks, M, loss_out);
         }
         if (!launched_ok()) return FTP_ERR_CUDA;
         delta = d;
@@ -470,7 +470,7 @@ int ftp_loss_mse(ftp_plan* plan, const float* y, const float* target, float* dy,
       mse_delta_kernel<<<plan->loss_blocks, 256, 0, st>>>(y, target, d, M, sums); }
     if (loss_out) {
         Timed t(plan, st, 2, -1);
-        mse_finish_kernel<<<1, 32, 0, st>>>(sums, plan->loss_blocks, M, loss_out);
+        mse_finish_kernel<<<1, 256, 0, st>>>(sums, plan->loss_blocks, M, loss_out);
     }
     return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
 }

@@ -685,24 +685,39 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_group_kernel(const __grid_con
 // (row, column) order: the backward boundary exchange at a group input.
 __global__ void halo_sum_kernel(const __grid_constant__ HaloSumArgs A)
 {
-    const size_t total = (size_t)A.N * A.C * A.H * A.W;
-    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
-        const int x = (int)(e % A.W); size_t t = e / A.W;
-        const int y = (int)(t % A.H); t /= A.H;
+    // The cover / span / offset tables go to shared memory first: every output value walks through
+    // three of them in a row, which from global memory is three dependent round trips.
+    extern __shared__ int halo_tab[];
+    int* xcover = halo_tab;              int* xspan = xcover + 2 * A.W;   int* xoff = xspan + 2 * A.Q;
+    int* ycover = xoff + A.Q + 1;        int* yspan = ycover + 2 * A.H;   int* yoff = yspan + 2 * A.R;
+    for (int i = threadIdx.x; i < 2 * A.W; i += blockDim.x) xcover[i] = A.xcover[i];
+    for (int i = threadIdx.x; i < 2 * A.H; i += blockDim.x) ycover[i] = A.ycover[i];
+    for (int i = threadIdx.x; i < 2 * A.Q; i += blockDim.x) xspan[i] = A.xspan[i];
+    for (int i = threadIdx.x; i < 2 * A.R; i += blockDim.x) yspan[i] = A.yspan[i];
+    for (int i = threadIdx.x; i <= A.Q; i += blockDim.x) xoff[i] = A.xoff[i];
+    for (int i = threadIdx.x; i <= A.R; i += blockDim.x) yoff[i] = A.yoff[i];
+    __syncthreads();
+    // one warp per map row (n, c, y): the covering sub-tile rows are looked up once, lanes walk along x
+    const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
+    const long long rows = (long long)A.N * A.C * A.H;
+    for (long long row = (long long)blockIdx.x * wpb + (threadIdx.x >> 5); row < rows; row += (long long)gridDim.x * wpb) {
+        const int y = (int)(row % A.H); long long t = row / A.H;
         const int c = (int)(t % A.C); const int n = (int)(t / A.C);
-        const int r0 = A.ycover[2 * y], r1 = A.ycover[2 * y + 1];
-        const int q0 = A.xcover[2 * x], q1 = A.xcover[2 * x + 1];
-        float s = 0.f;
-        for (int r = r0; r <= r1; ++r) {
-            const int y1 = A.yspan[2 * r], h = A.yspan[2 * r + 1] - y1 + 1;
-            for (int q = q0; q <= q1; ++q) {
-                const int x1 = A.xspan[2 * q], w = A.xspan[2 * q + 1] - x1 + 1;
-                const float* blk = A.scratch + (size_t)n * A.C * A.Htot * A.Wtot +
-                                   (size_t)A.C * ((size_t)A.yoff[r] * A.Wtot + (size_t)h * A.xoff[q]);
-                s += blk[((size_t)c * h + (y - y1)) * w + (x - x1)];
+        const int r0 = ycover[2 * y], r1 = ycover[2 * y + 1];
+        const float* img = A.scratch + (size_t)n * A.C * A.Htot * A.Wtot;
+        for (int x = lane; x < A.W; x += 32) {
+            const int q0 = xcover[2 * x], q1 = xcover[2 * x + 1];
+            float s = 0.f;
+            for (int r = r0; r <= r1; ++r) {
+                const int y1 = yspan[2 * r], h = yspan[2 * r + 1] - y1 + 1;
+                for (int q = q0; q <= q1; ++q) {
+                    const int x1 = xspan[2 * q], w = xspan[2 * q + 1] - x1 + 1;
+                    const float* blk = img + (size_t)A.C * ((size_t)yoff[r] * A.Wtot + (size_t)h * xoff[q]);
+                    s += blk[((size_t)c * h + (y - y1)) * w + (x - x1)];
+                }
             }
+            A.out[row * A.W + x] = s;
         }
-        A.out[e] = s;
     }
 }
 
@@ -772,13 +787,19 @@ __global__ void mse_delta_kernel(const float* __restrict__ y, const float* __res
     if (threadIdx.x == 0) block_sums[blockIdx.x] = red[0];
 }
 
+// Sums the per-block partial sums in a fixed order (strided per thread, then a tree) and writes the mean.
 __global__ void mse_finish_kernel(const float* __restrict__ block_sums, int n, size_t M, float* __restrict__ loss)
 {
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        float s = 0.f;
-        for (int i = 0; i < n; ++i) s += block_sums[i];
-        *loss = s / (float)M;
+    __shared__ float red[256];
+    float s = 0.f;
+    for (int i = threadIdx.x; i < n; i += 256) s += block_sums[i];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int k = 128; k >= 1; k >>= 1) {
+        if ((int)threadIdx.x < k) red[threadIdx.x] += red[threadIdx.x + k];
+        __syncthreads();
     }
+    if (threadIdx.x == 0) *loss = red[0] / (float)M;
 }
 
 }  // namespace ftp
