@@ -697,26 +697,34 @@ __global__ void halo_sum_kernel(const __grid_constant__ HaloSumArgs A)
     for (int i = threadIdx.x; i <= A.Q; i += blockDim.x) xoff[i] = A.xoff[i];
     for (int i = threadIdx.x; i <= A.R; i += blockDim.x) yoff[i] = A.yoff[i];
     __syncthreads();
-    // one warp per map row (n, c, y): the covering sub-tile rows are looked up once, lanes walk along x
+    // one warp per map row (n, c, y): what depends on the covering sub-tile rows only is computed once
+    // per row (32-bit offsets inside an image's scratch area), lanes walk along x
     const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
     const long long rows = (long long)A.N * A.C * A.H;
     for (long long row = (long long)blockIdx.x * wpb + (threadIdx.x >> 5); row < rows; row += (long long)gridDim.x * wpb) {
         const int y = (int)(row % A.H); long long t = row / A.H;
         const int c = (int)(t % A.C); const int n = (int)(t / A.C);
-        const int r0 = ycover[2 * y], r1 = ycover[2 * y + 1];
+        const int r0 = ycover[2 * y], nr = min(ycover[2 * y + 1] - r0 + 1, 4);
+        int base[4], ch[4], dr[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int r = min(r0 + k, A.R - 1);
+            const int y1 = yspan[2 * r], h = yspan[2 * r + 1] - y1 + 1;
+            base[k] = A.C * yoff[r] * A.Wtot; ch[k] = A.C * h; dr[k] = c * h + (y - y1);
+        }
         const float* img = A.scratch + (size_t)n * A.C * A.Htot * A.Wtot;
+        float* orow = A.out + row * A.W;
         for (int x = lane; x < A.W; x += 32) {
             const int q0 = xcover[2 * x], q1 = xcover[2 * x + 1];
             float s = 0.f;
-            for (int r = r0; r <= r1; ++r) {
-                const int y1 = yspan[2 * r], h = yspan[2 * r + 1] - y1 + 1;
-                for (int q = q0; q <= q1; ++q) {
-                    const int x1 = xspan[2 * q], w = xspan[2 * q + 1] - x1 + 1;
-                    const float* blk = img + (size_t)A.C * ((size_t)yoff[r] * A.Wtot + (size_t)h * xoff[q]);
-                    s += blk[((size_t)c * h + (y - y1)) * w + (x - x1)];
-                }
-            }
-            A.out[row * A.W + x] = s;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (k < nr)
+                    for (int q = q0; q <= q1; ++q) {
+                        const int x1 = xspan[2 * q], w = xspan[2 * q + 1] - x1 + 1;
+                        s += img[base[k] + xoff[q] * ch[k] + dr[k] * w + (x - x1)];
+                    }
+            orow[x] = s;
         }
     }
 }
