@@ -114,6 +114,11 @@ typedef struct {
                            most 256 channels (two blocks hide each other's latencies but each gets half of the shared
                            and tensor memory, i.e. smaller sub-tiles).  Default: 2 only in the forward pass of groups
                            with at most 64 channels */
+    int max_group_convs;  /* executed groups hold at most this many conv layers, with the pools that follow them
+                           (default 2; -1: no limit).  A requested group with more is executed as consecutive
+                           shorter groups: measured on B200, on the 8- and 16-layer stacks and both precisions,
+                           conv(+pool) pairs beat longer fused runs (halo recomputation and small sub-tiles cost
+                           more than the extra boundary traffic) and single layers (launches, boundary traffic) */
 } ftp_plan_opts;
 
 /* ftp_plan_create with explicit planner options (NULL = defaults). */

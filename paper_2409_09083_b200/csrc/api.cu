@@ -334,6 +334,8 @@ int ftp_plan_create_opts(const ftp_layer* layers, int n_layers, int N, int C, in
         po.strict_groups = opts->strict_groups;
         if (opts->tc_blocks_per_sm < 0 || opts->tc_blocks_per_sm > 2) return FTP_ERR_ARG;
         po.tc_ctas = opts->tc_blocks_per_sm;
+        if (opts->max_group_convs < -1) return FTP_ERR_ARG;
+        if (opts->max_group_convs) po.max_group_convs = opts->max_group_convs < 0 ? 0 : opts->max_group_convs;
     }
     ftp_plan* p = new (std::nothrow) ftp_plan();
     if (!p) return FTP_ERR_ARG;

@@ -479,7 +479,20 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
             GroupPlan g;
             double red = 1.0;
             int chosen = -1;
-            const int hi = std::min(last, start + kMaxOps - 1);
+            int hi = std::min(last, start + kMaxOps - 1);
+            if (!opts.strict_groups && opts.max_group_convs > 0) {
+                // executed groups hold at most max_group_convs conv layers and end with the pool(s) that
+                // follow a conv
+                int convs = 0, end = start - 1;
+                while (end + 1 <= hi) {
+                    const bool is_conv = p.layers[end].kind == FTP_CONV;
+                    if (is_conv && convs == opts.max_group_convs) break;
+                    if (is_conv && convs > 0 && p.layers[end - 1].kind == FTP_MAXPOOL) break;
+                    if (is_conv) ++convs;
+                    ++end;
+                }
+                hi = std::max(end, start);
+            }
             if (opts.strict_groups) {
                 if (hi != last) return FTP_ERR_GROUPS;
                 int rc = make_group(p, lo, start, last, popts, g, &red);

@@ -148,6 +148,7 @@ struct PlanOpts {
     int max_subtile = 0;            // 0 = as large as fits; else an upper bound (tests use it to force sub-tiling)
     int smem_bytes = kSmemBudget;   // dynamic shared memory a block may use
     int strict_groups = 0;          // 1 = never cut a requested group
+    int max_group_convs = 2;        // executed groups hold at most this many conv layers (0 = no limit)
     int tc_ctas = 0;                // tensor-core path: blocks per SM, 1 or 2 (0 = two where every layer of the group allows it)
     int tensor_cores = 0;           // set by build_plan from the precision: shared-memory layouts of the bf16 path
 };

@@ -95,9 +95,12 @@ def test_exec_groups_refine_the_requested_profile():
                 st = plan.subtiles(pass_, gi)
                 assert st["smem_bytes"] <= 225 * 1024 and st["blocks"] >= 1
                 assert st["rows"] >= wl.grid[0] and st["cols"] >= wl.grid[1]
-    # C2's requested groups fit as they are
+    # C2's requested groups fit as they are; by default they are executed as conv(+pool) pairs
     wl = synth.workload("C2")
-    assert ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups).exec_groups() == list(wl.groups)
+    mk = lambda **kw: ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, **kw).exec_groups()
+    assert mk(max_group_convs=-1) == list(wl.groups)
+    assert mk() == [(1, 2), (3, 4), (5, 6), (7, 8)]
+    assert mk(max_group_convs=1) == [(1, 2), (3, 4), (5, 5), (6, 6), (7, 8)]
 
 
 def test_strict_groups_keeps_or_refuses():
