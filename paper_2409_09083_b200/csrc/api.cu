@@ -217,7 +217,8 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
         const GroupPlan& g = p->groups[gi];
         TcGroupArgs a;
         fill_common_tc(p, g, true, x, params, ws, a);
-        a.dmap_out = gi == G - 1 ? dy : ws_ptr(ws, p->ws.dmap_off[gi + 1]);
+        a.dmap_out = gi == G - 1 ? static_cast<const void*>(dy) : static_cast<const void*>(ws_ptr(ws, p->ws.dmap_off[gi + 1]));
+        a.dmap_planes = gi == G - 1 ? 0 : 1;
         a.scratch = ws_ptr(ws, p->ws.scratch_off);
         a.partial = ws_ptr(ws, g.partial_off);
         a.set_floats = (long long)g.param_floats;
@@ -229,17 +230,20 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
         if (!launched_ok()) return FTP_ERR_CUDA;
         if (a.need_dx) {
             const MapShape& s = p->maps[g.first - 1];
+            const bool planes = g.first > 1;          // group input is a saved bf16 map: deltas travel as planes too
             HaloSumArgs h{};
             h.scratch = a.scratch;
             h.out = gi == 0 ? dx : ws_ptr(ws, p->ws.dmap_off[gi]);
             h.yspan = a.yspan; h.xspan = a.xspan; h.yoff = a.yoff; h.xoff = a.xoff;
             h.ycover = p->dev_tables + g.bwd.dev_ycover; h.xcover = p->dev_tables + g.bwd.dev_xcover;
-            h.N = p->N; h.C = s.C; h.H = s.H; h.W = s.W; h.R = a.R; h.Q = a.Q;
+            h.N = p->N; h.C = planes ? (s.C + 15) / 16 * 16 : s.C; h.H = s.H; h.W = s.W; h.R = a.R; h.Q = a.Q;
             h.Htot = g.bwd.y.scratch_off[a.R]; h.Wtot = g.bwd.x.scratch_off[a.Q];
-            const size_t rows = (size_t)p->N * s.C * s.H;
+            const size_t rows = (size_t)p->N * (planes ? h.C / 8 : h.C) * s.H;
             const int blocks = (int)std::min<size_t>((rows + 7) / 8, (size_t)kSmCount * 16);
+            const size_t tab = (size_t)(2 * h.W + 2 * h.H + 3 * h.Q + 3 * h.R + 2) * sizeof(int);
             { Timed t(p, st, 4, gi);
-              halo_sum_kernel<<<blocks, 256, (size_t)(2 * h.W + 2 * h.H + 3 * h.Q + 3 * h.R + 2) * sizeof(int), st>>>(h); }
+              if (planes) halo_sum_planes_kernel<<<blocks, 256, tab, st>>>(h);
+              else halo_sum_kernel<<<blocks, 256, tab, st>>>(h); }
             if (!launched_ok()) return FTP_ERR_CUDA;
         }
     }

@@ -30,8 +30,10 @@ struct TcGroupArgs {
     const float* params;
     int* error;                          // set to 1 when a bounded wait ran out
     // backward only
-    const float* dmap_out;               // delta at the group's output map (fp32 NCHW)
-    float*       scratch;
+    const void*  dmap_out;               // delta at the group's output map: fp32 NCHW (from the caller / the loss), or
+    int          dmap_planes;            //   bf16 planes written by halo_sum_planes_kernel (dmap_planes = 1)
+    float*       scratch;                // per-sub-tile deltas at the group input: fp32 [c][h][w] blocks for the first
+                                         //   group (network input), else fp32 [c/8][h][w][8] blocks of the padded channels
     const int *yoff, *xoff, *ytile, *xtile;
     float*       partial;
     long long    set_floats;
@@ -630,12 +632,17 @@ __global__ void __launch_bounds__(kTcThreads, 2) bwd_group_tc_kernel(const __gri
                 const int lx = e % ow, t = e / ow, ly = t % oh, pl = t / oh;
                 const int y = ho[0] + ly, x = ho[2] + lx;
                 float v[8];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const int ch = pl * 8 + c;
-                    v[c] = ch < op.cout ? __ldg(A.dmap_out + (((size_t)n * op.cout + ch) * op.out_H + y) * op.out_W + x) : 0.f;
-                }
                 const size_t gi = (((size_t)n * oplanes + pl) * op.out_H + y) * op.out_W + x;
+                if (A.dmap_planes) {
+                    unpack8(__ldg(static_cast<const uint4*>(A.dmap_out) + gi), v);
+                } else {
+                    const float* dsrc = static_cast<const float*>(A.dmap_out);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const int ch = pl * 8 + c;
+                        v[c] = ch < op.cout ? __ldg(dsrc + (((size_t)n * op.cout + ch) * op.out_H + y) * op.out_W + x) : 0.f;
+                    }
+                }
                 if (act) {
                     float yv[8];
                     unpack8(__ldg(ysrc + gi), yv);
@@ -666,9 +673,11 @@ __global__ void __launch_bounds__(kTcThreads, 2) bwd_group_tc_kernel(const __gri
                 zero_bytes(PD.base, (size_t)PD.planes * PD.plane);
             }
             float* sdst = nullptr;
+            const bool scratch_planes = !A.in_f32;
             if (to_scratch) {
                 const int Wtot = A.xoff[A.Q], Htot = A.yoff[A.R];
-                sdst = A.scratch + (size_t)n * op.cin * Htot * Wtot + (size_t)op.cin * ((size_t)A.yoff[r] * Wtot + (size_t)ih * A.xoff[q]);
+                const int sc = scratch_planes ? op.cin16 : op.cin;
+                sdst = A.scratch + (size_t)n * sc * Htot * Wtot + (size_t)sc * ((size_t)A.yoff[r] * Wtot + (size_t)ih * A.xoff[q]);
             }
             const unsigned long long* parg = (!to_scratch && pv.kind == kOpConvPool)
                                                  ? reinterpret_cast<const unsigned long long*>(A.arg[i - 1]) : nullptr;
@@ -688,7 +697,11 @@ __global__ void __launch_bounds__(kTcThreads, 2) bwd_group_tc_kernel(const __gri
 #pragma unroll
                     for (int c = 0; c < 8; ++c) v[c] *= xv[c] > 0.f ? 1.f : pslope;
                 }
-                if (to_scratch) {
+                if (to_scratch && scratch_planes) {
+                    float4* o = reinterpret_cast<float4*>(sdst + (((size_t)pl * ih + uy) * iw + ux) * 8);
+                    o[0] = make_float4(v[0], v[1], v[2], v[3]);
+                    o[1] = make_float4(v[4], v[5], v[6], v[7]);
+                } else if (to_scratch) {
 #pragma unroll
                     for (int c = 0; c < 8; ++c)
                         if (pl * 8 + c < op.cin) sdst[((size_t)(pl * 8 + c) * ih + uy) * iw + ux] = v[c];
@@ -741,6 +754,54 @@ __global__ void __launch_bounds__(kTcThreads, 2) bwd_group_tc_kernel(const __gri
         }
     }
     teardown(H);
+}
+
+// Backward boundary exchange of the tensor-core path for every group but the first: sum of the
+// overlapping per-sub-tile deltas (fp32 [c/8][h][w][8] blocks) in a fixed (row, column) order, written
+// as the bf16 planes the previous group's backward reads.  One warp per row (n, plane, y).
+__global__ void halo_sum_planes_kernel(const __grid_constant__ HaloSumArgs A)
+{
+    extern __shared__ int halo_tab[];
+    int* xcover = halo_tab;              int* xspan = xcover + 2 * A.W;   int* xoff = xspan + 2 * A.Q;
+    int* ycover = xoff + A.Q + 1;        int* yspan = ycover + 2 * A.H;   int* yoff = yspan + 2 * A.R;
+    for (int i = threadIdx.x; i < 2 * A.W; i += blockDim.x) xcover[i] = A.xcover[i];
+    for (int i = threadIdx.x; i < 2 * A.H; i += blockDim.x) ycover[i] = A.ycover[i];
+    for (int i = threadIdx.x; i < 2 * A.Q; i += blockDim.x) xspan[i] = A.xspan[i];
+    for (int i = threadIdx.x; i < 2 * A.R; i += blockDim.x) yspan[i] = A.yspan[i];
+    for (int i = threadIdx.x; i <= A.Q; i += blockDim.x) xoff[i] = A.xoff[i];
+    for (int i = threadIdx.x; i <= A.R; i += blockDim.x) yoff[i] = A.yoff[i];
+    __syncthreads();
+    const int lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
+    const int planes = A.C / 8;                                   // A.C = padded channel count
+    const long long rows = (long long)A.N * planes * A.H;
+    uint4* out = reinterpret_cast<uint4*>(A.out);
+    for (long long row = (long long)blockIdx.x * wpb + (threadIdx.x >> 5); row < rows; row += (long long)gridDim.x * wpb) {
+        const int y = (int)(row % A.H); long long t = row / A.H;
+        const int pl = (int)(t % planes); const int n = (int)(t / planes);
+        const int r0 = ycover[2 * y], nr = min(ycover[2 * y + 1] - r0 + 1, 4);
+        int base[4], ch[4], dr[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int r = min(r0 + k, A.R - 1);
+            const int y1 = yspan[2 * r], h = yspan[2 * r + 1] - y1 + 1;
+            base[k] = A.C * yoff[r] * A.Wtot; ch[k] = A.C * h; dr[k] = pl * h + (y - y1);
+        }
+        const float* img = A.scratch + (size_t)n * A.C * A.Htot * A.Wtot;
+        for (int x = lane; x < A.W; x += 32) {
+            const int q0 = xcover[2 * x], q1 = xcover[2 * x + 1];
+            float s[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (k < nr)
+                    for (int q = q0; q <= q1; ++q) {
+                        const int x1 = xspan[2 * q], w = xspan[2 * q + 1] - x1 + 1;
+                        const float4* e = reinterpret_cast<const float4*>(img + base[k] + xoff[q] * ch[k] + (dr[k] * w + (x - x1)) * 8);
+                        const float4 a = e[0], b = e[1];
+                        s[0] += a.x; s[1] += a.y; s[2] += a.z; s[3] += a.w; s[4] += b.x; s[5] += b.y; s[6] += b.z; s[7] += b.w;
+                    }
+            out[row * A.W + x] = tcd::pack8(s);
+        }
+    }
 }
 
 // Cross-tile reduction of the partial gradient sets of the tensor-core path in a fixed order, fused

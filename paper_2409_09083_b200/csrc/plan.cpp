@@ -399,7 +399,9 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
         }
     g.bwd.splits = std::max(1, std::min(min_items, kSmCount * g.bwd.ctas / (gy * gx)));
     g.bwd.blocks = gy * gx * g.bwd.splits;
-    g.bwd.scratch_floats = (size_t)N * p.maps[first - 1].C * g.bwd.y.scratch_off[g.bwd.y.count] *
+    // (tensor-core path, groups after the first: the blocks hold 8-channel planes of the padded channel count)
+    g.bwd.scratch_floats = (size_t)N * (tcp && first > 1 ? round_up(p.maps[first - 1].C, 16) : p.maps[first - 1].C) *
+                           g.bwd.y.scratch_off[g.bwd.y.count] *
                            g.bwd.x.scratch_off[g.bwd.x.count];
 
     return FTP_OK;
@@ -552,7 +554,8 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     ws.dmap_off.assign(n_exec, 0);
     for (int gi = 1; gi < n_exec; ++gi) {
         const MapShape& s = p.maps[p.groups[gi].first - 1];
-        ws.dmap_off[gi] = take((size_t)N * s.C * s.H * s.W * 4);
+        ws.dmap_off[gi] = tcp ? take((size_t)N * round_up(s.C, 16) * s.H * s.W * 2)     // bf16 planes
+                              : take((size_t)N * s.C * s.H * s.W * 4);
     }
     {
         const MapShape& s = p.maps[n_layers];
