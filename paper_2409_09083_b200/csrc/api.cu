@@ -171,7 +171,7 @@ int forward_tc(ftp_plan* p, const float* x, const float* params, float* y, void*
         { Timed t(p, st, 1, (int)gi);
           const size_t smem = tc_smem(g.fwd.smem_bytes, g.fwd.ctas);
           fwd_group_tc_kernel<<<std::min(items, kSmCount * g.fwd.ctas), kTcThreads, smem, st>>>(
-              a, (int)(smem - kTcFixedBytes), kTcTmemCols / g.fwd.ctas); }
+              a, (int)(smem - tc_fixed_bytes(g.fwd.stages)), kTcTmemCols / g.fwd.ctas, g.fwd.stages); }
         if (!launched_ok()) return FTP_ERR_CUDA;
     }
     if (y) {
@@ -226,7 +226,7 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
         a.need_dx = (gi > 0 || dx != nullptr) ? 1 : 0;
         { Timed t(p, st, 3, gi);
           const size_t smem = tc_smem(g.bwd.smem_bytes, g.bwd.ctas);
-          bwd_group_tc_kernel<<<g.bwd.blocks, kTcThreads, smem, st>>>(a, (int)(smem - kTcFixedBytes), kTcTmemCols / g.bwd.ctas); }
+          bwd_group_tc_kernel<<<g.bwd.blocks, kTcThreads, smem, st>>>(a, (int)(smem - tc_fixed_bytes(g.bwd.stages)), kTcTmemCols / g.bwd.ctas, g.bwd.stages); }
         if (!launched_ok()) return FTP_ERR_CUDA;
         if (a.need_dx) {
             const MapShape& s = p->maps[g.first - 1];

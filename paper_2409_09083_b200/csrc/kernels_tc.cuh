@@ -47,15 +47,16 @@ using namespace tc;
 // Fixed part of the dynamic shared memory (kTcHeader bytes), then the weight ring, then the tiles.
 struct Header {
     int hdr[(kMaxOps + 1) * 8];                  // spans / cells of the current sub-tile
-    unsigned long long full[kTcStages];          // weight stage filled (transaction bytes)
-    unsigned long long empty[kTcStages];         // weight stage consumed (tcgen05.commit)
+    unsigned long long full[kTcMaxStages];          // weight stage filled (transaction bytes)
+    unsigned long long empty[kTcMaxStages];         // weight stage consumed (tcgen05.commit)
     unsigned long long done;                     // all MMAs of a pass completed
     uint32_t tmem_base;
+    int stage_mask, stage_shift;                 // filter ring: stages - 1 and log2(stages)
     int tmem_cols;                               // columns this block allocated (512, or 256 with two blocks per SM)
     volatile int failed;                         // a wait ran out: skip every later wait
     int dw_nw, dw_nbias;                         // entries of dw_unit / dw_bias in the current pass
     __align__(16) __nv_bfloat16 ones[64];        // one core matrix of 1.0: operand of the bias-gradient contraction
-    __align__(16) uint4 dw_unit[2 * kTcMaxUnits]; // filter gradient: MMAs of the current pass {a_lo, x_lo, idesc, column}
+    __align__(16) uint4 dw_unit[kTcMaxUnits + 4];  // filter gradient: MMAs of the current pass {a_lo, x_lo, idesc, column}
     uint2 dw_bias[kTcMaxUnits];                  //                  bias MMAs {a_lo, column}
     float bias[kTcTmemCols];
 };
@@ -125,7 +126,7 @@ __device__ __forceinline__ void conv_mma(Pipe& p, uint32_t a_base, int a_Wp, uin
         if (warp == kTcIssuers && lane == 0) {
             // producer: one bulk copy per stage
             for (int s = 0; s < nstages; ++s) {
-                const uint32_t q = p.stages_done + s, slot = q % kTcStages, par = (q / kTcStages) & 1;
+                const uint32_t q = p.stages_done + s, slot = q & (uint32_t)p.h->stage_mask, par = (q >> p.h->stage_shift) & 1;
                 if (!wait_or_fail(p, &p.h->empty[slot], par ^ 1)) break;
                 const int pl = min(spp, planes - s * spp);
                 const uint32_t bytes = (uint32_t)pl * plane_bytes;
@@ -144,7 +145,7 @@ __device__ __forceinline__ void conv_mma(Pipe& p, uint32_t a_base, int a_Wp, uin
             const uint32_t idesc_rest = N > 256 ? make_idesc(128, N - 256, false, false) : 0u;
             int gp0 = 0;                                            // first plane of the stage
             for (int s = 0; s < nstages; ++s) {
-                const uint32_t q = p.stages_done + s, slot = q % kTcStages, par = (q / kTcStages) & 1;
+                const uint32_t q = p.stages_done + s, slot = q & (uint32_t)p.h->stage_mask, par = (q >> p.h->stage_shift) & 1;
                 if (!wait_or_fail(p, &p.h->full[slot], par)) break;
                 fence_after_sync();
                 const int pl = min(spp, planes - gp0);
@@ -273,18 +274,20 @@ __device__ __forceinline__ void zero_bytes(unsigned char* p, size_t bytes)
         *reinterpret_cast<uint4*>(p + e) = make_uint4(0, 0, 0, 0);
 }
 
-__device__ __forceinline__ void setup(Header* h, Pipe& p, unsigned char* smem, int* error, size_t tile_bytes, int tmem_cols)
+__device__ __forceinline__ void setup(Header* h, Pipe& p, unsigned char* smem, int* error, size_t tile_bytes, int tmem_cols,
+                                      int stages)
 {
     if (threadIdx.x == 0) {
         h->tmem_cols = tmem_cols;
-        for (int s = 0; s < kTcStages; ++s) { mbar_init(smem_u32(&h->full[s]), 1); mbar_init(smem_u32(&h->empty[s]), kTcIssuers); }
+        h->stage_mask = stages - 1; h->stage_shift = stages == 4 ? 2 : 1;
+        for (int s = 0; s < kTcMaxStages; ++s) { mbar_init(smem_u32(&h->full[s]), 1); mbar_init(smem_u32(&h->empty[s]), kTcIssuers); }
         mbar_init(smem_u32(&h->done), kTcIssuers);
         h->failed = 0;
         fence_mbar_init();
     }
     if (threadIdx.x < 32) { __syncwarp(); tmem_alloc(smem_u32(&h->tmem_base), (uint32_t)tmem_cols); }
     // every byte the tensor core may ever read is a finite bf16 from here on
-    zero_bytes(smem + kTcFixedBytes, tile_bytes);
+    zero_bytes(smem + (kTcHeader + stages * kTcStageBytes), tile_bytes);
     for (int i = threadIdx.x; i < 64; i += blockDim.x) h->ones[i] = __float2bfloat16(1.0f);
     fence_before_sync();
     __syncthreads();
@@ -447,14 +450,14 @@ __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*addre
 // ---------------------------------------------------------------------------------------------
 // Fused forward of one group, bf16: persistent blocks walk over the (image, sub-tile) stacks.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kTcThreads, 2) fwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes, int tmem_cols)
+__global__ void __launch_bounds__(kTcThreads, 2) fwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes, int tmem_cols, int stages)
 {
     using namespace tcd;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Header* H = reinterpret_cast<Header*>(smem_raw);
-    unsigned char* tiles = smem_raw + kTcFixedBytes;
+    unsigned char* tiles = smem_raw + (kTcHeader + stages * kTcStageBytes);
     Pipe pipe;
-    setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes, tmem_cols);
+    setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes, tmem_cols, stages);
     int* hdr = H->hdr;
     const int items = A.N * A.R * A.Q;
 
@@ -572,14 +575,14 @@ __global__ void __launch_bounds__(kTcThreads, 2) fwd_group_tc_kernel(const __gri
 // Fused backward of one group, bf16 (adjoint form): each block owns one partial gradient set and
 // walks through its share of the (image, sub-tile) stacks of one user tile in a fixed order.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kTcThreads, 2) bwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes, int tmem_cols)
+__global__ void __launch_bounds__(kTcThreads, 2) bwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes, int tmem_cols, int stages)
 {
     using namespace tcd;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     Header* H = reinterpret_cast<Header*>(smem_raw);
-    unsigned char* tiles = smem_raw + kTcFixedBytes;
+    unsigned char* tiles = smem_raw + (kTcHeader + stages * kTcStageBytes);
     Pipe pipe;
-    setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes, tmem_cols);
+    setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes, tmem_cols, stages);
     int* hdr = H->hdr;
 
     const int slot = blockIdx.x, tile = slot / A.splits, split = slot % A.splits;

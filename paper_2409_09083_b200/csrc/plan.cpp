@@ -180,7 +180,7 @@ size_t tc_slack(int Wp, int planes_beyond, size_t plane_bytes)
     return ((size_t)16 * Wp + 32) * 16 + (size_t)planes_beyond * plane_bytes;
 }
 
-size_t layout_forward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
+size_t layout_forward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& tx, int stages)
 {
     size_t size[kMaxOps + 1] = {0}, slack = 0;
     for (int i = 0; i < g.n_ops; ++i) {
@@ -195,7 +195,7 @@ size_t layout_forward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& t
     size_t total = 0;
     for (int i = 0; i < g.n_ops; ++i) total = std::max(total, size[i] + size[i + 1]);
     for (int i = 0; i < g.n_ops; ++i) g.fwd_ops[i].t_in_off = (i % 2 == 0) ? 0 : (int)(total - size[i]);
-    return (size_t)kTcFixedBytes + total + slack;
+    return (size_t)tc_fixed_bytes(stages) + total + slack;
 }
 
 // Tensor-core path, backward.  While op i runs, three tiles are alive: dz_i (delta at the conv output,
@@ -203,7 +203,7 @@ size_t layout_forward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& t
 // filter gradient contracts over runs of 16 pixels of both), and dz_{i-1} which the op produces.
 // The filter-gradient operand spans 64 or 128 channels; channels beyond the real ones are reserved
 // in the tile so that the operand stays inside it.
-size_t layout_backward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
+size_t layout_backward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& tx, int stages)
 {
     const int n = g.n_ops;
     size_t dsize[kMaxOps], xsize[kMaxOps], slack = 0;
@@ -233,7 +233,7 @@ size_t layout_backward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& 
         op.t_dz_off = low ? 0 : (int)(total - dsize[i]);
         op.t_x_off = low ? (int)dsize[i] : (int)(i > 0 ? dsize[i - 1] : 0);
     }
-    return (size_t)kTcFixedBytes + total + slack;
+    return (size_t)tc_fixed_bytes(stages) + total + slack;
 }
 
 void count_macs(const GroupPlan& g, const PassPlan& pp, double* done, double* untiled);
@@ -256,7 +256,7 @@ int choose_subtiles(GroupPlan& g, bool backward, const PlanOpts& o, int N)
         build_axis(pp.y, ay, g.tile_y, ky);
         build_axis(pp.x, ax, g.tile_x, kx);
         size_t bytes;
-        if (o.tensor_cores) bytes = backward ? layout_backward_tc(g, pp.y, pp.x) : layout_forward_tc(g, pp.y, pp.x);
+        if (o.tensor_cores) bytes = backward ? layout_backward_tc(g, pp.y, pp.x, pp.stages) : layout_forward_tc(g, pp.y, pp.x, pp.stages);
         else bytes = backward ? layout_backward(g, pp.y, pp.x) : layout_forward(g, pp.y, pp.x);
         size_t budget = (size_t)o.smem_bytes;
         if (o.tensor_cores) budget = std::min<size_t>(pp.ctas == 2 ? kTcSmemBudget2 : kTcSmemBudget, (size_t)o.smem_bytes + 2048);
@@ -378,6 +378,7 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
     for (int pass = 0; pass < 2; ++pass) {
         PassPlan& pp = pass ? g.bwd : g.fwd;
         pp.ctas = pass ? want_bwd : want_fwd;
+        pp.stages = 2;      // (four stages were measured on the 256/512-channel groups: the smaller tiles cost more than the deeper ring gains)
         int rc = choose_subtiles(g, pass == 1, o, N);
         if (rc != FTP_OK && pp.ctas == 2) { pp.ctas = 1; rc = choose_subtiles(g, pass == 1, o, N); }
         if (rc != FTP_OK) return rc;

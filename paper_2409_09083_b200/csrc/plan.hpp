@@ -19,11 +19,11 @@ constexpr int kCoutTile    = 8;       // output channels per thread task (packed
 
 // Tensor-core (bf16) tile kernels: one block per SM, all 512 tensor-memory columns.
 constexpr int kTcThreads    = 256;
-constexpr int kTcStages     = 2;          // weight ring: stages of kTcStageBytes
+constexpr int kTcMaxStages  = 4;          // weight ring: 2 or 4 stages of kTcStageBytes (4 for groups with large filters)
 constexpr int kTcStageBytes = 16384;
 constexpr int kTcTmemCols   = 512;        // tensor-memory columns of an SM; a block takes all of them, or half with two blocks per SM
 constexpr int kTcHeader     = 4096;       // per-block tables, barriers, bias staging
-constexpr int kTcFixedBytes = kTcHeader + kTcStages * kTcStageBytes;   // shared memory before the activation area
+constexpr int tc_fixed_bytes(int stages) { return kTcHeader + stages * kTcStageBytes; }   // shared memory before the activation area
 constexpr int kTcSmemBudget = 227 * 1024; // dynamic shared memory a tensor-core block may use (one block per SM)
 constexpr int kTcSmemBudget2 = 113 * 1024;// ... with two blocks per SM
 constexpr int kTcIssuers = 4;             // threads (lane 0 of warps 0..3) that issue MMAs, each for its own accumulators
@@ -79,6 +79,7 @@ struct PassPlan {
     size_t smem_bytes = 0;
     int blocks = 0;                 // forward: R*Q*N ; backward: tiles * splits
     int splits = 1;                 // backward: blocks per user tile
+    int stages = 2;                 // tensor-core path: stages of the filter ring
     int ctas = 1;                   // tensor-core path: blocks per SM (2 = each block takes half of the tensor memory)
     size_t scratch_floats = 0;      // backward: floats of per-sub-tile group-input deltas (all images)
     // offsets (in ints) of the tables inside the plan's device table blob
