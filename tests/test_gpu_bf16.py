@@ -176,9 +176,13 @@ def test_result_does_not_depend_on_grid_or_groups_and_is_reproducible():
     for a, b in zip(base[:3], again[:3]):
         assert np.array_equal(a, b)                                   # run to run: bit for bit
     variants = [dict(grid=(3, 3)), dict(grid=(4, 2), groups=((1, 4), (5, 8))),
-                dict(grid=(2, 5), groups=synth.groups_per_layer(wl.layers)), dict(grid=(8, 12))]
+                dict(grid=(2, 5), groups=synth.groups_per_layer(wl.layers)), dict(grid=(8, 12)),
+                # planner options: whole requested groups fused, one conv per group, two blocks per SM, forced sub-tiling
+                dict(grid=(2, 2), opts=dict(max_group_convs=-1)), dict(grid=(3, 2), opts=dict(max_group_convs=1)),
+                dict(grid=(2, 3), opts=dict(tc_blocks_per_sm=2)), dict(grid=(2, 3), opts=dict(tc_blocks_per_sm=1, max_subtile=3))]
     for v in variants:
-        y, dx, dparams, plan = backward_bf16(wl.with_(**v), x, params, dy)
+        opts = v.pop("opts", {})
+        y, dx, dparams, plan = backward_bf16(wl.with_(**v), x, params, dy, **opts)
         assert np.array_equal(y, base[0])                             # same arithmetic per output value
         # deltas inside a group are rounded to bf16 per sub-tile before overlapping parts are summed
         assert rel_err(dx, base[1]) <= BF16_TOL, v

@@ -101,9 +101,11 @@ def test_result_does_not_depend_on_grid_or_groups_and_is_reproducible():
     for k in ("y", "dx", "dparams"):
         assert np.array_equal(base[k], again[k]), f"{k} differs from run to run"
     variants = [dict(grid=(3, 3)), dict(grid=(4, 2), groups=((1, 4), (5, 8))),
-                dict(grid=(2, 5), groups=synth.groups_per_layer(wl.layers)), dict(grid=(8, 12))]
+                dict(grid=(2, 5), groups=synth.groups_per_layer(wl.layers)), dict(grid=(8, 12)),
+                dict(grid=(2, 2), opts=dict(max_group_convs=-1)), dict(grid=(3, 2), opts=dict(max_group_convs=1))]
     for v in variants:
-        got = run_gpu(wl.with_(**v), x, params, dy=dy)
+        opts = v.pop("opts", {})
+        got = run_gpu(wl.with_(**v), x, params, dy=dy, **opts)
         assert np.array_equal(got["y"], base["y"])                   # same arithmetic per output value
         assert rel_err(got["dx"], base["dx"]) <= 1e-5                # sums in another order
         assert rel_err(got["dparams"], base["dparams"]) <= 1e-5
