@@ -25,8 +25,10 @@ int ensure_device(ftp_plan* p)
     if (p->dev_tables) { cudaFree(p->dev_tables); p->dev_tables = nullptr; }
     if (cudaFuncSetAttribute(fwd_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(fwd_group_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(bwd_group_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess)
+        cudaFuncSetAttribute(fwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(fwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(bwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(bwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess)
         return FTP_ERR_CUDA;
     const size_t bytes = p->tables.size() * sizeof(int);
     if (cudaMalloc(&p->dev_tables, bytes) != cudaSuccess) return FTP_ERR_CUDA;
@@ -170,8 +172,10 @@ int forward_tc(ftp_plan* p, const float* x, const float* params, float* y, void*
         const int items = a.R * a.Q * p->N;
         { Timed t(p, st, 1, (int)gi);
           const size_t smem = tc_smem(g.fwd.smem_bytes, g.fwd.ctas);
-          fwd_group_tc_kernel<<<std::min(items, kSmCount * g.fwd.ctas), kTcThreads, smem, st>>>(
-              a, (int)(smem - tc_fixed_bytes(g.fwd.stages)), kTcTmemCols / g.fwd.ctas, g.fwd.stages); }
+          const int blocks = std::min(items, kSmCount * g.fwd.ctas), tile_bytes = (int)(smem - tc_fixed_bytes(g.fwd.stages));
+          // two blocks of 256 threads per SM, or one of 512: the phases around the MMAs want all the warps they can get
+          if (g.fwd.ctas == 2) fwd_group_tc_kernel<256><<<blocks, 256, smem, st>>>(a, tile_bytes, kTcTmemCols / 2, g.fwd.stages);
+          else fwd_group_tc_kernel<512><<<blocks, 512, smem, st>>>(a, tile_bytes, kTcTmemCols, g.fwd.stages); }
         if (!launched_ok()) return FTP_ERR_CUDA;
     }
     if (y) {
@@ -226,7 +230,9 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
         a.need_dx = (gi > 0 || dx != nullptr) ? 1 : 0;
         { Timed t(p, st, 3, gi);
           const size_t smem = tc_smem(g.bwd.smem_bytes, g.bwd.ctas);
-          bwd_group_tc_kernel<<<g.bwd.blocks, kTcThreads, smem, st>>>(a, (int)(smem - tc_fixed_bytes(g.bwd.stages)), kTcTmemCols / g.bwd.ctas, g.bwd.stages); }
+          const int tile_bytes = (int)(smem - tc_fixed_bytes(g.bwd.stages));
+          if (g.bwd.ctas == 2) bwd_group_tc_kernel<256><<<g.bwd.blocks, 256, smem, st>>>(a, tile_bytes, kTcTmemCols / 2, g.bwd.stages);
+          else bwd_group_tc_kernel<512><<<g.bwd.blocks, 512, smem, st>>>(a, tile_bytes, kTcTmemCols, g.bwd.stages); }
         if (!launched_ok()) return FTP_ERR_CUDA;
         if (a.need_dx) {
             const MapShape& s = p->maps[g.first - 1];

@@ -187,7 +187,7 @@ __device__ __forceinline__ void conv_mma(Pipe& p, uint32_t a_base, int a_Wp, uin
         const int q = warp & 3;
         for (int bi = 0; bi < nb; ++bi) {
             const int b = b0 + bi, by = b / nbx, bx = b % nbx;
-            for (int c0 = (warp >> 2) * 16; c0 < N; c0 += 32) {
+            for (int c0 = (warp >> 2) * 16; c0 < N; c0 += (int)(blockDim.x >> 7) * 16) {
                 float v[16];
                 tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(bi * N + c0), v);
                 epi(by, bx, q, lane, c0, v);
@@ -404,7 +404,7 @@ __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*addre
             const int slice = u / (T + 1), t = u % (T + 1);
             const int co = slice * 128 + row;
             const int ncols = t == T ? 16 : ucols;
-            for (int c0 = (warp >> 2) * 16; c0 < ncols; c0 += 32) {
+            for (int c0 = (warp >> 2) * 16; c0 < ncols; c0 += (int)(blockDim.x >> 7) * 16) {
                 float v[16];
                 tmem_ld16(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(col + c0), v);
                 if (row_ok && co < cout16) {
@@ -450,7 +450,8 @@ __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*addre
 // ---------------------------------------------------------------------------------------------
 // Fused forward of one group, bf16: persistent blocks walk over the (image, sub-tile) stacks.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kTcThreads, 2) fwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes, int tmem_cols, int stages)
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 2 : 1) fwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes, int tmem_cols, int stages)
 {
     using namespace tcd;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -575,7 +576,8 @@ __global__ void __launch_bounds__(kTcThreads, 2) fwd_group_tc_kernel(const __gri
 // Fused backward of one group, bf16 (adjoint form): each block owns one partial gradient set and
 // walks through its share of the (image, sub-tile) stacks of one user tile in a fixed order.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kTcThreads, 2) bwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes, int tmem_cols, int stages)
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 2 : 1) bwd_group_tc_kernel(const __grid_constant__ TcGroupArgs A, int tile_bytes, int tmem_cols, int stages)
 {
     using namespace tcd;
     extern __shared__ __align__(16) unsigned char smem_raw[];
