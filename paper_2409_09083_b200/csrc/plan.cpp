@@ -378,10 +378,17 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
     for (int pass = 0; pass < 2; ++pass) {
         PassPlan& pp = pass ? g.bwd : g.fwd;
         pp.ctas = pass ? want_bwd : want_fwd;
-        pp.stages = 2;      // (four stages were measured on the 256/512-channel groups: the smaller tiles cost more than the deeper ring gains)
+        pp.stages = 2;
         int rc = choose_subtiles(g, pass == 1, o, N);
         if (rc != FTP_OK && pp.ctas == 2) { pp.ctas = 1; rc = choose_subtiles(g, pass == 1, o, N); }
         if (rc != FTP_OK) return rc;
+        if (tcp) {
+            // a four-stage filter ring where it costs no sub-tile size (measured: paying for it with smaller
+            // tiles loses more than the deeper ring gains)
+            const size_t budget = std::min<size_t>(pp.ctas == 2 ? kTcSmemBudget2 : kTcSmemBudget, (size_t)o.smem_bytes + 2048);
+            const size_t bytes4 = pass ? layout_backward_tc(g, pp.y, pp.x, kTcMaxStages) : layout_forward_tc(g, pp.y, pp.x, kTcMaxStages);
+            if (bytes4 <= budget) { pp.stages = kTcMaxStages; pp.smem_bytes = bytes4; }
+        }
     }
     double bwd_done = 0, bwd_untiled = 0;
     count_macs(g, g.fwd, &g.macs_done, &g.macs_untiled);
