@@ -29,6 +29,9 @@ METRIC = "train-step images/sec (fwd+bwd+dW reduce+SGD)"
 UNIT = "images/s"
 # fp32 FMA peak of the CUDA cores: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (derived, not measured)
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+# dram__bytes_read.sum + dram__bytes_write.sum of the fused backward kernel per launch (average over the launches of
+# a step), from the ncu captures summarised under profiles/ (workload C1 only; null for anything else)
+NCU_TRAFFIC = {("C1", "fp32"): 78.0e6, ("C1", "bf16"): 29.7e6}
 KIND = {0: "pack_filters", 1: "fwd_group", 2: "loss_delta", 3: "bwd_group", 4: "halo_sum", 5: "reduce_sgd"}
 
 
@@ -276,7 +279,8 @@ def measure(args, precision, rank, world, local, dist, ftp, dp, torch, extras=Tr
         peak, src = FP32_PEAK_TFLOPS, "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz"
         bound, kernel = "alu", "bwd_group_kernel"
     roofline = {"bound": bound, "kernel": kernel, "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": achieved / peak if achieved else None, "traffic": None,
+                "unit": "TFLOP/s", "frac": achieved / peak if achieved else None,
+                "traffic": NCU_TRAFFIC.get((wl.name, precision)), "traffic_unit": "bytes per launch (ncu, profiles/)",
                 "peak_source": src,
                 "launches_per_step": n_bwd, "avg_launch_ms": bwd_ms / n_bwd if n_bwd else None,
                 "algorithmic_flops_per_step": bwd_flops,
