@@ -253,7 +253,8 @@ int ftp_loss_mse_static(const float* y, const float* target, float* dy, float* l
  * ftp_step for callers whose batch lives in HOST memory: copies x_host and target_host
  * (pinned memory recommended; shapes as in ftp_step) into staging areas of the workspace,
  * runs the training cycle with the mean-squared-error loss and copies the loss (1 float) to
- * loss_host, all enqueued on `stream`; loss_host is valid once the stream is synchronised.
+ * loss_host, all ordered on `stream` (the target's copy runs on a side stream of the plan, created on
+ * the first call, and joins before the loss); loss_host is valid once the stream is synchronised.
  * params stays in device memory and is updated in place.  dx (device, may be NULL) receives
  * dLoss/dX_1 as in ftp_step.
  */

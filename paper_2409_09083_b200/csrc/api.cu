@@ -380,6 +380,11 @@ void ftp_plan_destroy(ftp_plan* plan)
     if (!plan) return;
     ftp_plan_timing(plan, 0);
     if (plan->dev_tables) cudaFree(plan->dev_tables);
+    if (plan->copy_stream) {
+        cudaStreamDestroy(static_cast<cudaStream_t>(plan->copy_stream));
+        cudaEventDestroy(static_cast<cudaEvent_t>(plan->ev_fork));
+        cudaEventDestroy(static_cast<cudaEvent_t>(plan->ev_join));
+    }
     delete plan;
 }
 
@@ -440,7 +445,7 @@ int ftp_backward(ftp_plan* plan, const float* x, const float* dy, const float* p
 
 static int step_impl(ftp_plan* plan, const float* x, const float* dy, const float* target, const float* params,
                      float* sgd_params, float lr, float* grad_out, float* loss_out, float* dx, void* workspace,
-                     void* stream)
+                     void* stream, cudaEvent_t target_ready = nullptr)
 {
     if (!plan || !x || !params || !workspace || !aligned256(workspace)) return FTP_ERR_ARG;
     if ((dy == nullptr) == (target == nullptr)) return FTP_ERR_ARG;
@@ -451,6 +456,7 @@ static int step_impl(ftp_plan* plan, const float* x, const float* dy, const floa
     rc = forward_impl(plan, x, params, y32, workspace, st);
     if (rc != FTP_OK) return rc;
     const float* delta = dy;
+    if (target_ready && cudaStreamWaitEvent(st, target_ready, 0) != cudaSuccess) return FTP_ERR_CUDA;
     if (target) {
         const MapShape& s = plan->maps.back();
         const size_t M = (size_t)plan->N * s.C * s.H * s.W;
@@ -503,10 +509,24 @@ int ftp_step_host(ftp_plan* plan, const float* x_host, const float* target_host,
     float* xs = ws_ptr(workspace, plan->ws.x_stage_off);
     float* ts = ws_ptr(workspace, plan->ws.t_stage_off);
     float* lv = ws_ptr(workspace, plan->ws.loss_val_off);
-    if (cudaMemcpyAsync(xs, x_host, (size_t)plan->N * in.C * in.H * in.W * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(ts, target_host, (size_t)plan->N * out.C * out.H * out.W * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    // The input goes first on the caller's stream; the target is only needed at the loss, so its copy
+    // runs on a side stream (created on first use) while the forward pass computes.
+    if (!plan->copy_stream) {
+        cudaStream_t cs; cudaEvent_t e0, e1;
+        if (cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) != cudaSuccess)
+            return FTP_ERR_CUDA;
+        plan->copy_stream = cs; plan->ev_fork = e0; plan->ev_join = e1;
+    }
+    cudaStream_t cs = static_cast<cudaStream_t>(plan->copy_stream);
+    cudaEvent_t fork = static_cast<cudaEvent_t>(plan->ev_fork), join = static_cast<cudaEvent_t>(plan->ev_join);
+    if (cudaEventRecord(fork, st) != cudaSuccess || cudaStreamWaitEvent(cs, fork, 0) != cudaSuccess ||      // after earlier work on `stream`
+        cudaMemcpyAsync(ts, target_host, (size_t)plan->N * out.C * out.H * out.W * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaEventRecord(join, cs) != cudaSuccess ||
+        cudaMemcpyAsync(xs, x_host, (size_t)plan->N * in.C * in.H * in.W * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return FTP_ERR_CUDA;
-    int rc = step_impl(plan, xs, nullptr, ts, params, params, lr, nullptr, lv, dx, workspace, stream);
+    int rc = step_impl(plan, xs, nullptr, ts, params, params, lr, nullptr, lv, dx, workspace, stream, join);
     if (rc != FTP_OK) return rc;
     if (loss_host && cudaMemcpyAsync(loss_host, lv, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FTP_ERR_CUDA;
     return FTP_OK;

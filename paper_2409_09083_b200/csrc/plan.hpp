@@ -141,6 +141,8 @@ struct ftp_plan {
     std::vector<int> ev_kind, ev_group;
     int ev_used = 0;
     int loss_blocks = 0;
+    // ftp_step_host: side stream and events that let the target's host-to-device copy overlap the forward pass
+    void* copy_stream = nullptr; void* ev_fork = nullptr; void* ev_join = nullptr;
 };
 
 namespace ftp {
