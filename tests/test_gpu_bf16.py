@@ -270,3 +270,32 @@ def test_full_size_groups(name):
     c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
     dy = np.random.default_rng(3).standard_normal((2, c, h, w)).astype(np.float32)
     check_groups_against_oracle(wl, plan.exec_groups(), x, params, dy, small_maps=False)
+
+
+@pytest.mark.parametrize("name", ["C0", "conv5-pool-conv", "one-conv1"])
+def test_step_updates_parameters_like_the_oracle(name):
+    """ftp_step on the bf16 path: loss, update and input gradient of one training cycle; the host-batch
+    variant must give the same update."""
+    wl = FWD[name]
+    x, params, target = synth.draw(wl, bias_std=0.3)
+    x, params = bf16_grid(x), bf16_grid(params)
+    lr = 0.05
+    ref = run_oracle(wl, x, params, target=target, lr=lr, store="bf16")
+    plan = ftp.ftp_plan(wl.layers, x.shape[0], wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=BF16)
+    ws = plan.new_workspace()
+    xd, td = torch.from_numpy(x).cuda(), torch.from_numpy(target).cuda()
+    pd = torch.from_numpy(params.copy()).cuda()
+    loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+    dx = torch.empty_like(xd)
+    ftp.ftp_step(plan, xd, pd, lr, ws, target=td, loss_out=loss, dx=dx)
+    plan.check(ws)
+    assert loss.item() == pytest.approx(ref["loss"], rel=1e-3)
+    new = pd.cpu().numpy()
+    assert rel_err(new - params, ref["new_params"] - params) <= BF16_TOL
+    assert rel_err(dx.cpu().numpy(), ref["dx"]) <= BF16_TOL
+    pd2 = torch.from_numpy(params.copy()).cuda()
+    lh = torch.zeros(1, dtype=torch.float32).pin_memory()
+    ftp.ftp_step_host(plan, torch.from_numpy(x).pin_memory(), torch.from_numpy(target).pin_memory(), pd2, lr, lh, ws)
+    plan.check(ws)
+    assert np.array_equal(pd2.cpu().numpy(), new)
+    assert float(lh[0]) == loss.item()
