@@ -268,7 +268,23 @@ int choose_subtiles(GroupPlan& g, bool backward, const PlanOpts& o, int N)
             const int ky = std::min(c[0], max_h), kx = std::min(c[1], max_w);
             size_t bytes = try_split(ky, kx);
             if (!bytes) continue;
-            if (backward || o.max_subtile > 0 || o.tensor_cores) { pp.smem_bytes = bytes; return FTP_OK; }   // (tensor-core stacks: per-stack overheads outweigh a fuller last round)
+            if (backward || o.max_subtile > 0) { pp.smem_bytes = bytes; return FTP_OK; }
+            if (o.tensor_cores) {
+                // tensor-core stacks: per-stack overheads outweigh a fuller last round, but with fewer stacks
+                // than blocks that can run at once a finer split puts the idle SMs to work
+                const int slots = kSmCount * pp.ctas;
+                int best_ky = ky, best_kx = kx, best_items = N * pp.y.count * pp.x.count;
+                if (best_items < slots)
+                    for (int dy = 0; dy <= 3; ++dy)
+                        for (int dx = 0; dx <= 3; ++dx) {
+                            const int yy = std::min(ky + dy, max_h), xx = std::min(kx + dx, max_w);
+                            if (!try_split(yy, xx)) continue;
+                            const int items = N * pp.y.count * pp.x.count;
+                            if (items <= slots && items > best_items) { best_items = items; best_ky = yy; best_kx = xx; }
+                        }
+                pp.smem_bytes = try_split(best_ky, best_kx);
+                return FTP_OK;
+            }
             // forward: look a little further for a split that wastes less of the last round
             int best_ky = ky, best_kx = kx;
             double best = -1, fixed = 0;     // fixed: per-stack cost that does not shrink with the tile (loads, syncs)
