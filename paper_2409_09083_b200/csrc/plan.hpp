@@ -17,9 +17,9 @@ constexpr int kSmemBudget  = 225 * 1024;  // dynamic shared memory a block may u
 constexpr int kSmemHeader  = 1024;    // bytes reserved at the start for per-block tables
 constexpr int kCoutTile    = 8;       // output channels per thread task (packed weights are padded to it)
 
-// Tensor-core (bf16) tile kernels: one block per SM, all 512 tensor-memory columns.
-constexpr int kTcThreads    = 256;
-constexpr int kTcMaxStages  = 4;          // weight ring: 2 or 4 stages of kTcStageBytes (4 for groups with large filters)
+// Tensor-core (bf16) tile kernels: one block of 512 threads per SM with all 512 tensor-memory columns, or two
+// blocks of 256 threads with 256 columns each.
+constexpr int kTcMaxStages  = 4;          // weight ring: 2 stages of kTcStageBytes, 4 where that costs no sub-tile size
 constexpr int kTcStageBytes = 16384;
 constexpr int kTcTmemCols   = 512;        // tensor-memory columns of an SM; a block takes all of them, or half with two blocks per SM
 constexpr int kTcHeader     = 4096;       // per-block tables, barriers, bias staging

@@ -52,7 +52,7 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool a_mn_major,
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// D[tmem] (+)= A[smem] * B[smem]; one thread issues for the whole CTA.  (No memory clobber: the
+// D[tmem] (+)= A[smem] * B[smem], issued by a single thread (its MMAs execute in issue order).  (No memory clobber: the
 // statement is volatile, so it keeps its order among the fences, barriers and other MMAs, while the
 // compiler may still move ordinary loads of the issuing thread across it.)
 __device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate)
