@@ -56,6 +56,8 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tc-blocks", type=int, default=0, choices=[0, 1, 2],
                     help="bf16 path: thread blocks per SM (0 = planner default)")
+    ap.add_argument("--cost-model", type=int, default=0, choices=[-1, 0, 1],
+                    help="planner's time model for cutting the requested groups: 0 planner default, 1 on, -1 off (fixed rule)")
     ap.add_argument("--no-bf16", action="store_true", help="skip the second measurement on the bf16 tensor-core path")
     return ap.parse_args()
 
@@ -186,7 +188,7 @@ def measure(args, precision, rank, world, local, dist, ftp, dp, torch, extras=Tr
         params = synth.draw(wl.with_(seed=0))[1]
     tcp = precision == "bf16"
     plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=1 if tcp else 0,
-                        tc_blocks_per_sm=args.tc_blocks if tcp else 0)
+                        tc_blocks_per_sm=args.tc_blocks if tcp else 0, cost_model=args.cost_model)
     ws = plan.new_workspace()
     xd, pd, td = (torch.from_numpy(a).cuda() for a in (x, params, target))
     dx = torch.empty_like(xd)

@@ -119,6 +119,10 @@ typedef struct {
                            shorter groups: measured on B200, on the 8- and 16-layer stacks and both precisions,
                            conv(+pool) pairs beat longer fused runs (halo recomputation and small sub-tiles cost
                            more than the extra boundary traffic) and single layers (launches, boundary traffic) */
+    int cost_model;       /* 1: compare all cuts of each requested group into executed groups of one to three conv
+                           layers by the planner's time model (ftp_plan_cost) and take the best one instead of the
+                           max_group_convs rule's cuts when the model puts it at least 3 % ahead; -1: never.
+                           Default: 1, unless max_group_convs is given (then only that rule applies) */
 } ftp_plan_opts;
 
 /* ftp_plan_create with explicit planner options (NULL = defaults). */
@@ -169,6 +173,24 @@ int ftp_plan_sizes(const ftp_plan* plan, size_t* param_floats,
  */
 int ftp_plan_subtiles(const ftp_plan* plan, int pass, int group,
                       int* rows, int* cols, size_t* smem_bytes, int* blocks);
+
+/*
+ * The planner's time model of one pass (0 forward, 1 backward) of an EXECUTED
+ * group.  The paper chooses its grouping profile by weighing halo
+ * recomputation against boundary exchanges (Sections 4.2 and 5.3) but does not
+ * print the procedure; this library estimates the time of a pass as a
+ * weighted sum of FTP_COST_TERMS work terms taken on the pass's critical path
+ * (multiply-accumulates or tensor-core cycles incl. halo recomputation, filter
+ * bytes streamed, partial-set bytes updated, map bytes moved, per-layer
+ * synchronisations, one launch), with weights fitted to measurements on B200.
+ * need_dx: whether the delta at the group's input is produced (it is for every
+ * group but the first of a training step).  terms (host, FTP_COST_TERMS
+ * doubles, may be NULL) receives the terms, estimate_us (host, may be NULL)
+ * the estimate in microseconds.  FTP_ERR_ARG on a bad index.
+ */
+#define FTP_COST_TERMS 8
+int ftp_plan_cost(const ftp_plan* plan, int pass, int group, int need_dx,
+                  double* terms, double* estimate_us);
 
 /*
  * Forward pass (Section 3; Section 4.1 forward; Section 4.2 groups): one fused

@@ -40,7 +40,7 @@ _lib.ftp_plan_create.restype = _i
 
 class ftp_plan_opts(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_int), ("max_redundancy_pct", ctypes.c_int), ("max_subtile", ctypes.c_int),
-                ("smem_bytes", ctypes.c_int), ("strict_groups", ctypes.c_int), ("tc_blocks_per_sm", ctypes.c_int), ("max_group_convs", ctypes.c_int)]
+                ("smem_bytes", ctypes.c_int), ("strict_groups", ctypes.c_int), ("tc_blocks_per_sm", ctypes.c_int), ("max_group_convs", ctypes.c_int), ("cost_model", ctypes.c_int)]
 
 
 _lib.ftp_plan_create_opts.argtypes = [ctypes.POINTER(ftp_layer), _i, _i, _i, _i, _i, _i, _i,
@@ -59,6 +59,8 @@ _lib.ftp_plan_sizes.restype = _i
 _lib.ftp_plan_subtiles.argtypes = [_vp, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i),
                                    ctypes.POINTER(_sz), ctypes.POINTER(_i)]
 _lib.ftp_plan_subtiles.restype = _i
+_lib.ftp_plan_cost.argtypes = [_vp, _i, _i, _i, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
+_lib.ftp_plan_cost.restype = _i
 _lib.ftp_forward.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
 _lib.ftp_forward.restype = _i
 _lib.ftp_backward.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -144,11 +146,11 @@ class Plan:
     """Owner of an ftp_plan handle (ftp_plan_create / ftp_plan_destroy)."""
 
     def __init__(self, layers, N, C, H, W, grid, groups, precision=FTP_FP32, max_redundancy_pct=0, max_subtile=0,
-                 smem_bytes=0, strict_groups=False, tc_blocks_per_sm=0, max_group_convs=0):
+                 smem_bytes=0, strict_groups=False, tc_blocks_per_sm=0, max_group_convs=0, cost_model=0):
         self._h = _vp()
         la, ga = _as_layers(layers), _as_groups(groups)
         opts = ftp_plan_opts(ctypes.sizeof(ftp_plan_opts), max_redundancy_pct, max_subtile, smem_bytes,
-                             1 if strict_groups else 0, tc_blocks_per_sm, max_group_convs)
+                             1 if strict_groups else 0, tc_blocks_per_sm, max_group_convs, int(cost_model))
         _check(_lib.ftp_plan_create_opts(la, len(layers), N, C, H, W, grid[0], grid[1], ga, len(groups),
                                          precision, ctypes.byref(opts), ctypes.byref(self._h)))
         self.layers, self.shape, self.grid, self.groups = list(layers), (N, C, H, W), tuple(grid), list(groups)
@@ -183,6 +185,13 @@ class Plan:
         _check(_lib.ftp_plan_subtiles(self._h, pass_, group, ctypes.byref(r), ctypes.byref(c),
                                       ctypes.byref(s), ctypes.byref(b)))
         return dict(rows=r.value, cols=c.value, smem_bytes=s.value, blocks=b.value)
+
+    def cost(self, pass_, group, need_dx=True):
+        """(terms, estimate in microseconds) of the planner's time model for one pass of an executed group."""
+        terms = (ctypes.c_double * 8)()
+        est = ctypes.c_double()
+        _check(_lib.ftp_plan_cost(self._h, pass_, group, 1 if need_dx else 0, terms, ctypes.byref(est)))
+        return list(terms), est.value
 
     def launch_count(self):
         return int(_lib.ftp_plan_launch_count(self._h))

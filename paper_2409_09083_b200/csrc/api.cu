@@ -346,6 +346,8 @@ int ftp_plan_create_opts(const ftp_layer* layers, int n_layers, int N, int C, in
         po.tc_ctas = opts->tc_blocks_per_sm;
         if (opts->max_group_convs < -1) return FTP_ERR_ARG;
         if (opts->max_group_convs) po.max_group_convs = opts->max_group_convs < 0 ? 0 : opts->max_group_convs;
+        if (opts->cost_model < -1 || opts->cost_model > 1) return FTP_ERR_ARG;
+        po.cost_model = opts->cost_model ? (opts->cost_model > 0 ? 1 : 0) : (opts->max_group_convs ? 0 : 1);
     }
     ftp_plan* p = new (std::nothrow) ftp_plan();
     if (!p) return FTP_ERR_ARG;
@@ -421,6 +423,15 @@ int ftp_plan_subtiles(const ftp_plan* plan, int pass, int group, int* rows, int*
     if (smem_bytes) *smem_bytes = pp.smem_bytes;
     if (blocks) *blocks = pp.blocks;
     return FTP_OK;
+}
+
+int ftp_plan_cost(const ftp_plan* plan, int pass, int group, int need_dx, double* terms, double* estimate_us)
+{
+    if (!plan) return FTP_ERR_ARG;
+    double t[kCostTerms];
+    const int rc = cost_terms(*plan, pass, group, need_dx, t, estimate_us);
+    if (rc == FTP_OK && terms) for (int k = 0; k < kCostTerms; ++k) terms[k] = t[k];
+    return rc;
 }
 
 int ftp_forward(ftp_plan* plan, const float* x, const float* params, float* y, void* workspace, void* stream)

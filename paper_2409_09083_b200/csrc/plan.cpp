@@ -329,6 +329,152 @@ void count_macs(const GroupPlan& g, const PassPlan& pp, double* done, double* un
     }
 }
 
+// ---- cost terms of one pass of an executed group ----
+// Work on the critical path of one pass: every term is the total over all sub-tile stacks of the
+// pass divided by the number of stacks that run side by side (blocks in flight; in the backward
+// pass the blocks of the busiest user tile decide).  The planner's estimate of the pass time is a
+// weighted sum of the terms (see kCostWeights).  Terms, fp32 path (multiply-accumulates in units of
+// 1e6, bytes in MB, elements in units of 1e6):
+//   forward : 0 conv MACs, 1 conv+pool MACs, 2 filter MB read, 3 map MB read + written, 4 ops, 5 outputs, 7 one launch
+//   backward: 0 filter-gradient MACs, 1 input-delta MACs of convs, 2 of conv+pool ops, 3 filter MB read,
+//             4 partial-set MB updated, 5 map MB, 6 ops, 7 one launch
+// bf16 path (tensor-core time in units of 1e3 cycles, taking an MMA with N accumulator columns as max(45, N/2)):
+//   forward : 0 MMA cycles, 1 elements of the fp32 network input, 2 filter MB streamed (once per round of accumulators),
+//             3 map MB, 4 ops, 5 accumulator elements read back, 6 of these, the ones that go through a fused pool
+//   backward: 0 filter-gradient MMA cycles, 1 input-delta MMA cycles, 3 filter MB, 4 partial-set MB, 5 map MB, 6 ops
+constexpr int kCostMaxConvs = 3;   // conv layers per executed group the cost model considers (what the weights were fitted on)
+inline double mma_cycles(int n) { return n <= 0 ? 0.0 : std::max(45.0, n / 2.0); }
+
+void pass_cost_terms(const ftp_plan& p, const GroupPlan& g, bool backward, bool need_dx, double f[kCostTerms])
+{
+    for (int k = 0; k < kCostTerms; ++k) f[k] = 0;
+    const bool tcp = p.precision == FTP_BF16_FP32ACC;
+    const PassPlan& pp = backward ? g.bwd : g.fwd;
+    const AxisTables& ty = pp.y; const AxisTables& tx = pp.x;
+    const int N = p.N, n = g.n_ops;
+    const int tmem_cols = kTcTmemCols / std::max(1, pp.ctas);
+    auto ext = [](const AxisTables& t, int m, int r) { return t.span[((size_t)m * t.count + r) * 2 + 1] - t.span[((size_t)m * t.count + r) * 2] + 1; };
+    auto own = [](const AxisTables& t, int m, int r) { return t.cell[((size_t)m * t.count + r) * 2 + 1] - t.cell[((size_t)m * t.count + r) * 2] + 1; };
+    const double param_mb = g.param_floats * 4.0 / 1e6;
+    const int in_bytes = tcp && g.first > 1 ? 2 : 4, out_bytes = tcp ? 2 : 4;
+    for (int r = 0; r < ty.count; ++r)
+        for (int q = 0; q < tx.count; ++q) {
+            // one sub-tile stack (one image); all terms are multiplied by N at the end
+            for (int i = 0; i < n; ++i) {
+                const OpDesc& op = g.fwd_ops[i];
+                const int oh = ext(ty, i + 1, r), ow = ext(tx, i + 1, q);       // output span of the op
+                const int ih = ext(ty, i, r), iw = ext(tx, i, q);               // input span
+                const int cin_b = tcp ? op.cin16 : op.cin, cout_b = tcp ? op.cout16 : op.cout;
+                if (backward) f[5] += (double)cin_b * ih * iw * (tcp ? 2 : 4) / 1e6;   // copy of the op's input
+                if (backward) f[6] += 1; else f[4] += 1;
+                if (op.kind == kOpPool) continue;
+                const int coh = op.S * oh, cow = op.S * ow;                     // conv output span
+                const double macs = (double)coh * cow * op.cin * op.cout * op.k * op.k / 1e6;
+                const double w_mb = tcp ? (double)op.k * op.k * op.cin16 * op.cout16 * 2 / 1e6
+                                        : (double)op.k * op.k * op.cin * op.cout * 4 / 1e6;
+                const bool dx = backward && (need_dx || i > 0);
+                if (!tcp) {
+                    // the direct convolutions give every thread 4 rows x 8 channels of one output column and
+                    // run in rounds of kThreads such tasks: count the multiply-accumulates of full rounds
+                    auto conv_macs = [&](int rows, int cols, int co_pad, int ci) {
+                        const long long tasks = (long long)(co_pad / kCoutTile) * ((rows + 3) / 4) * cols;
+                        return (double)((tasks + kThreads - 1) / kThreads) * kThreads * 4 * kCoutTile * ci * op.k * op.k / 1e6;
+                    };
+                    if (!backward) {
+                        f[op.kind == kOpConvPool ? 1 : 0] += conv_macs(coh, cow, op.cout_pad, op.cin);
+                        f[2] += w_mb;
+                        f[5] += (double)coh * cow * op.cout / 1e6;
+                    } else {
+                        f[0] += macs;
+                        if (dx) {
+                            f[op.kind == kOpConvPool ? 2 : 1] += conv_macs(ih, iw, op.cin_pad, op.cout);
+                            f[3] += w_mb;
+                        }
+                    }
+                } else if (!backward) {
+                    const int nblocks = ((coh + 15) / 16) * ((cow + 7) / 8);
+                    const int rounds = (nblocks + tmem_cols / op.cout16 - 1) / (tmem_cols / op.cout16);
+                    const double per_block = (double)op.k * op.k * (op.cin16 / 16) *
+                                             (mma_cycles(std::min(op.cout16, 256)) + mma_cycles(op.cout16 - 256));
+                    f[0] += nblocks * per_block / 1e3;
+                    f[2] += rounds * w_mb;
+                    f[5] += (double)nblocks * 128 * op.cout16 / 1e6;
+                    if (op.kind == kOpConvPool) f[6] += (double)coh * cow * op.cout16 / 1e6;
+                } else {
+                    const int Wp = cow + 2 * (op.k - 1);
+                    const int nk = ((coh - 1) * Wp + cow + 15) / 16;
+                    const int slices = op.cout16 <= 64 ? 1 : (op.cout16 + 127) / 128;
+                    const bool folded = op.cin <= 8;
+                    const int units = folded ? op.k : op.k * op.k;
+                    const int ucols = folded ? (8 * op.k + 15) / 16 * 16 : op.cin16;
+                    f[0] += (double)slices * nk * (units * (mma_cycles(std::min(ucols, 256)) + mma_cycles(ucols - 256)) + 45.0) / 1e3;
+                    if (dx) {
+                        const int nblocks = ((ih + 15) / 16) * ((iw + 7) / 8);
+                        const int rounds = (nblocks + tmem_cols / op.cin16 - 1) / (tmem_cols / op.cin16);
+                        f[1] += (double)nblocks * op.k * op.k * (op.cout16 / 16) *
+                                (mma_cycles(std::min(op.cin16, 256)) + mma_cycles(op.cin16 - 256)) / 1e3;
+                        f[3] += rounds * w_mb;
+                    }
+                }
+                (void)cin_b; (void)cout_b;
+            }
+            // maps read and written in global memory by the stack
+            const OpDesc& o0 = g.fwd_ops[0]; const OpDesc& ol = g.fwd_ops[n - 1];
+            const double in_mb = (double)(tcp ? o0.cin16 : o0.cin) * ext(ty, 0, r) * ext(tx, 0, q) / 1e6;
+            const double out_mb = (double)(tcp ? ol.cout16 : ol.cout) * own(ty, n, r) * own(tx, n, q) / 1e6;
+            if (!backward) {
+                f[3] += in_mb * in_bytes;
+                if (tcp && g.first == 1) f[1] += (double)o0.cin * ext(ty, 0, r) * ext(tx, 0, q) / 1e6;
+                for (int i = 0; i < n; ++i) {                                  // every op's output map is kept for the backward pass
+                    const OpDesc& op = g.fwd_ops[i];
+                    f[3] += (double)(tcp ? op.cout16 : op.cout) * own(ty, i + 1, r) * own(tx, i + 1, q) * out_bytes / 1e6;
+                }
+            } else {
+                f[5] += out_mb * out_bytes;                                    // delta at the group's output
+                if (need_dx) f[5] += in_mb * 4 * 2;                            // per-stack input delta, written then summed
+                f[4] += param_mb;
+            }
+        }
+    // stacks that run side by side
+    double parallel;
+    const double items = (double)N * ty.count * tx.count;
+    if (!backward) {
+        const double slots = (double)kSmCount * pp.ctas;
+        parallel = items / std::ceil(items / slots);
+    } else {
+        int busiest = 1;
+        for (size_t a = 0; a + 1 < ty.tile_begin.size(); ++a)
+            for (size_t b = 0; b + 1 < tx.tile_begin.size(); ++b) {
+                const int it = N * (ty.tile_begin[a + 1] - ty.tile_begin[a]) * (tx.tile_begin[b + 1] - tx.tile_begin[b]);
+                busiest = std::max(busiest, (it + pp.splits - 1) / pp.splits);
+            }
+        parallel = items / busiest;
+    }
+    for (int k = 0; k < kCostTerms - 1; ++k) f[k] = f[k] * N / parallel;
+    f[kCostTerms - 1] = 1.0;
+}
+
+// Microseconds per unit of each term, fitted (non-negative least squares on relative errors) to the
+// measured pass times of single executed groups of the 8- and 16-layer stacks on one B200.
+const double kCostWeights[2][2][kCostTerms] = {
+    {   // fp32: forward, backward
+        {7.336, 7.264, 18.73, 167.9, 4.648, 0.1864, 0, 24.84},
+        {5.954, 5.355, 11.66, 266.3, 0, 228.4, 46.65, 34.55},
+    },
+    {   // bf16
+        {0, 1359, 33.91, 33.92, 3.3, 84.78, 224.9, 8.343},
+        {0.4407, 1.217, 0, 0, 71.85, 55.48, 6.834, 12.31},
+    },
+};
+
+double pass_estimate_us(int precision, bool backward, const double f[kCostTerms])
+{
+    const double* w = kCostWeights[precision == FTP_BF16_FP32ACC ? 1 : 0][backward ? 1 : 0];
+    double t = 0;
+    for (int k = 0; k < kCostTerms; ++k) t += w[k] * f[k];
+    return t;
+}
+
 struct LayerOffsets { std::vector<long long> p_off, wf_off, wb_off, twf_off, twb_off; };
 
 // Builds the ops, the sub-tiling and the block counts of one executed group (layers first..last).
@@ -495,20 +641,32 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     if (expect != n_layers + 1) return FTP_ERR_GROUPS;
     p.user_groups.assign(groups, groups + n_groups);
 
-    // executed groups: a requested group is kept whole when a sub-tile stack of a useful size fits in
-    // shared memory, otherwise it is cut greedily into the longest runs of layers that do
+    // Executed groups.  A requested group is first cut by the fixed rule: runs of at most
+    // max_group_convs conv layers that end with the pool after a conv, shortened further while the halo
+    // recomputation exceeds the cap or no sub-tile fits in shared memory.  With the cost model on, all
+    // ways to cut the requested group into executed groups of one to kCostMaxConvs conv layers (a conv
+    // stays with the pool after it) are then compared by the sum of their estimated pass times (found
+    // from the last layer backwards), and the best one replaces the fixed rule's cuts when the model
+    // puts it at least 3 % ahead; the margin keeps the model's error (about 10 % per group) from
+    // trading a measured-good default for a predicted tie.
+    auto estimate = [&](const GroupPlan& g) {
+        double f[kCostTerms];
+        pass_cost_terms(p, g, false, false, f);
+        double t = pass_estimate_us(precision, false, f);
+        pass_cost_terms(p, g, true, g.first > 1, f);
+        return t + pass_estimate_us(precision, true, f);
+    };
     p.groups.clear();
     for (int gi = 0; gi < n_groups; ++gi) {
         int start = groups[gi].first;
-        const int last = groups[gi].last;
+        const int first = start, last = groups[gi].last;
+        std::vector<GroupPlan> cut;                        // the fixed rule's executed groups of this requested group
         while (start <= last) {
             GroupPlan g;
             double red = 1.0;
             int chosen = -1;
             int hi = std::min(last, start + kMaxOps - 1);
             if (!opts.strict_groups && opts.max_group_convs > 0) {
-                // executed groups hold at most max_group_convs conv layers and end with the pool(s) that
-                // follow a conv
                 int convs = 0, end = start - 1;
                 while (end + 1 <= hi) {
                     const bool is_conv = p.layers[end].kind == FTP_CONV;
@@ -537,9 +695,40 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
                     }
                 if (chosen < 0) return FTP_ERR_WORKSPACE;
             }
-            p.groups.push_back(g);
+            cut.push_back(g);
             start = chosen + 1;
         }
+        if (opts.cost_model && !opts.strict_groups) {
+            const double inf = 1e300;
+            std::vector<double> best(last + 2, inf);
+            std::vector<int> end_of(last + 2, -1);         // end_of[s]: last layer of the best executed group that starts at s
+            best[last + 1] = 0;
+            for (int s = last; s >= first; --s) {
+                if (s > first && p.layers[s - 2].kind == FTP_CONV && p.layers[s - 1].kind == FTP_MAXPOOL) continue;
+                int convs = 0;
+                for (int e = s; e <= std::min(last, s + kMaxOps - 1); ++e) {
+                    if (p.layers[e - 1].kind == FTP_CONV && ++convs > kCostMaxConvs) break;
+                    if (e < last && p.layers[e - 1].kind == FTP_CONV && p.layers[e].kind == FTP_MAXPOOL) continue;
+                    if (best[e + 1] >= inf) continue;
+                    GroupPlan g;
+                    double red = 1.0;
+                    if (make_group(p, lo, s, e, popts, g, &red) != FTP_OK || red * 100.0 > opts.max_redundancy_pct) continue;
+                    const double cost = estimate(g) + best[e + 1];
+                    if (cost < best[s]) { best[s] = cost; end_of[s] = e; }
+                }
+            }
+            double fixed_cost = 0;
+            for (const GroupPlan& g : cut) fixed_cost += estimate(g);
+            if (best[first] < 0.97 * fixed_cost) {
+                cut.clear();
+                for (int s = first; s <= last; s = end_of[s] + 1) {
+                    GroupPlan g;
+                    if (end_of[s] < s || make_group(p, lo, s, end_of[s], popts, g, nullptr) != FTP_OK) return FTP_ERR_WORKSPACE;
+                    cut.push_back(g);
+                }
+            }
+        }
+        for (const GroupPlan& g : cut) p.groups.push_back(g);
     }
     if (p.groups.size() > 64) return FTP_ERR_GROUPS;
     const int n_exec = (int)p.groups.size();
@@ -602,6 +791,14 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     for (GroupPlan& g : p.groups) g.partial_off = take((size_t)g.bwd.blocks * g.param_floats * 4);
     ws.grad_off = take(p.param_floats * 4);
     ws.total = off;
+    return FTP_OK;
+}
+
+int cost_terms(const ftp_plan& p, int pass, int group, int need_dx, double terms[kCostTerms], double* est_us)
+{
+    if (group < 0 || group >= (int)p.groups.size() || pass < 0 || pass > 1 || !terms) return FTP_ERR_ARG;
+    pass_cost_terms(p, p.groups[group], pass == 1, need_dx != 0, terms);
+    if (est_us) *est_us = pass_estimate_us(p.precision, pass == 1, terms);
     return FTP_OK;
 }
 

@@ -29,6 +29,7 @@ constexpr int kTcSmemBudget2 = 113 * 1024;// ... with two blocks per SM
 constexpr int kTcIssuers = 4;             // threads (lane 0 of warps 0..3) that issue MMAs, each for its own accumulators
 constexpr int kTcMaxUnits = 32;           // filter-gradient accumulators per pass (at least 16 columns each)
 constexpr int kTcTailEntries = 16;        // 16-byte entries appended to every tile plane
+constexpr int kCostTerms = 8;             // terms of the planner's time estimate of one pass of a group
 
 struct Span { int a, b; };            // inclusive interval on one axis
 
@@ -152,6 +153,7 @@ struct PlanOpts {
     int smem_bytes = kSmemBudget;   // dynamic shared memory a block may use
     int strict_groups = 0;          // 1 = never cut a requested group
     int max_group_convs = 2;        // executed groups hold at most this many conv layers (0 = no limit)
+    int cost_model = 1;             // 1 = the time model (pass_cost_terms) may replace the fixed rule's cuts, see build_plan
     int tc_ctas = 0;                // tensor-core path: blocks per SM, 1 or 2 (0 = two where every layer of the group allows it)
     int tensor_cores = 0;           // set by build_plan from the precision: shared-memory layouts of the bf16 path
 };
@@ -159,4 +161,6 @@ struct PlanOpts {
 int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C, int H, int W,
                int gy, int gx, const ftp_group* groups, int n_groups, int precision, const PlanOpts& opts);
 int region(const ftp_plan& p, int pass, int group, int map_index, int ty, int tx, int out[4]);
+// Cost terms of one pass of executed group `group` (see plan.cpp) and the estimate in microseconds built from them.
+int cost_terms(const ftp_plan& p, int pass, int group, int need_dx, double terms[kCostTerms], double* est_us);
 }  // namespace ftp

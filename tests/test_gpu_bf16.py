@@ -179,6 +179,7 @@ def test_result_does_not_depend_on_grid_or_groups_and_is_reproducible():
                 dict(grid=(2, 5), groups=synth.groups_per_layer(wl.layers)), dict(grid=(8, 12)),
                 # planner options: whole requested groups fused, one conv per group, two blocks per SM, forced sub-tiling
                 dict(grid=(2, 2), opts=dict(max_group_convs=-1)), dict(grid=(3, 2), opts=dict(max_group_convs=1)),
+                dict(grid=(3, 3), opts=dict(cost_model=1)), dict(grid=(3, 3), opts=dict(cost_model=-1)),
                 dict(grid=(2, 3), opts=dict(tc_blocks_per_sm=2)), dict(grid=(2, 3), opts=dict(tc_blocks_per_sm=1, max_subtile=3))]
     for v in variants:
         opts = v.pop("opts", {})

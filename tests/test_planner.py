@@ -101,6 +101,69 @@ def test_exec_groups_refine_the_requested_profile():
     assert mk(max_group_convs=-1) == list(wl.groups)
     assert mk() == [(1, 2), (3, 4), (5, 6), (7, 8)]
     assert mk(max_group_convs=1) == [(1, 2), (3, 4), (5, 5), (6, 6), (7, 8)]
+    assert mk(cost_model=-1) == [(1, 2), (3, 4), (5, 6), (7, 8)]
+
+
+def _conv_counts(layers, groups):
+    return [sum(1 for l in layers[a - 1:b] if l.kind == "conv") for a, b in groups]
+
+
+def test_cost_model_cuts_are_valid_profiles():
+    """The model only moves cuts inside requested groups: executed groups stay contiguous, keep every
+    requested boundary, hold one to three convs and never part a conv from the pool after it; an
+    explicit max_group_convs or cost_model=-1 leaves the fixed rule alone."""
+    for name in ["C1", "C2", "C3"]:
+        wl = synth.workload(name)
+        for prec in (0, 1):
+            mk = lambda **kw: ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=prec, **kw)
+            fixed = mk(cost_model=-1).exec_groups()
+            assert mk(max_group_convs=2).exec_groups() == fixed
+            for plan in (mk(), mk(cost_model=1)):
+                eg = plan.exec_groups()
+                assert eg[0][0] == 1 and eg[-1][1] == len(wl.layers)
+                assert all(c == b + 1 for (a, b), (c, d) in zip(eg, eg[1:]))
+                assert {g[0] for g in wl.groups} <= {g[0] for g in eg}
+                assert all(1 <= n <= 3 for n in _conv_counts(wl.layers, eg))
+                for a, b in eg[:-1]:
+                    assert not (wl.layers[b - 1].kind == "conv" and wl.layers[b].kind == "pool")
+                # the model's own estimate of what it chose is never worse than that of the fixed rule's cuts
+                est = lambda pl: sum(pl.cost(ps, g, a > 1)[1] for g, (a, b) in enumerate(pl.exec_groups()) for ps in (0, 1))
+                assert est(plan) <= est(mk(cost_model=-1)) * (1 + 1e-9)
+
+
+def test_cost_terms_of_a_single_conv_by_hand():
+    """One 3x3 conv 8 -> 16 on a 16 x 16 map, one image, one tile, fp32.  The forward pass cuts the
+    map into R x Q stacks that all run side by side, so each term is that of one average stack: at
+    most 2 x 4 x 16 = 128 thread tasks of 4 rows x 8 channels, i.e. one round of 512, which counts
+    512 x 32 x 8 x 9 multiply-accumulates; the filters, 9 x 8 x 16 floats; the map term, the input
+    spans (own rows and columns plus a halo of 1 where the map goes on) plus the 16 x 16 x 16 output."""
+    layers = [synth.conv(8, 16, 3)]
+    plan = ftp.ftp_plan(layers, 1, 8, 16, 16, (1, 1), ((1, 1),))
+    st = plan.subtiles(0, 0)
+    R, Q = st["rows"], st["cols"]
+    assert 16 % R == 0 and 16 % Q == 0 and R * Q <= 148
+    t, est = plan.cost(0, 0, True)
+    assert t[0] == pytest.approx(512 * 32 * 8 * 9 / 1e6) and t[1] == 0
+    assert t[2] == pytest.approx(9 * 8 * 16 * 4 / 1e6)
+    in_floats = 8 * (16 + 2 * (R - 1)) * (16 + 2 * (Q - 1))
+    assert t[3] == pytest.approx((in_floats + 16 * 256) * 4 / 1e6 / (R * Q))
+    assert t[4] == 1 and t[5] == pytest.approx(16 * 256 / 1e6 / (R * Q)) and t[7] == 1
+    assert est > 0
+    sb = plan.subtiles(1, 0)
+    assert sb["rows"] == 1 and sb["cols"] == 1                      # backward: the largest stack that fits
+    tb, estb = plan.cost(1, 0, True)
+    assert tb[0] == pytest.approx(256 * 8 * 16 * 9 / 1e6)            # filter gradient: plain count
+    assert tb[1] == pytest.approx(512 * 32 * 16 * 9 / 1e6)           # input delta: 1 x 4 x 16 = 64 tasks, one round, 16 input channels each
+    assert tb[4] == pytest.approx((9 * 8 * 16 + 16) * 4 / 1e6)       # the stack's partial set
+    assert plan.cost(1, 0, False)[0][1] == 0                         # no input delta asked for
+    # twice the batch: twice the stacks on as many blocks, so every term but the launch doubles at most
+    plan2 = ftp.ftp_plan(layers, 2, 8, 16, 16, (1, 1), ((1, 1),))
+    t2, est2 = plan2.cost(0, 0, True)
+    assert est2 >= est and all(b <= 2 * a + 1e-12 for a, b in zip(t[:7], t2[:7]))
+    for bad in (dict(pass_=2, group=0), dict(pass_=0, group=1), dict(pass_=0, group=-1)):
+        with pytest.raises(binding.FtpError) as e:
+            plan.cost(bad["pass_"], bad["group"])
+        assert e.value.code == -1
 
 
 def test_strict_groups_keeps_or_refuses():
