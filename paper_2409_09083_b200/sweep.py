@@ -2,6 +2,7 @@
 stack (the axes of the paper's grouping / batch-size experiments, Section 5, on synthetic data).
 
     python -m paper_2409_09083_b200.sweep [--stack yolo16] [--batches 1,4,16] [--grids 1,3,5] [--size 608] [--steps 5]
+                                         [--profiles pairs,planner]
 
 Prints one JSON line per point: images/s, ms per step, executed groups, redundancy, workspace.
 Needs a CUDA device; every step runs in the library.
@@ -14,10 +15,13 @@ from . import synth
 
 def profiles(layers):
     """name -> (requested groups, max_group_convs).  The first three are executed as requested as far as
-    they fit in shared memory; "planner" lets the planner cut one all-in-one group its default way."""
+    they fit in shared memory; "pairs" is one all-in-one group cut by the fixed rule (two convs per
+    executed group, ending at a pool); "planner" lets the planner cut it its default way, i.e. where
+    its time model puts the minimum."""
     return {"all-in-one": (((1, len(layers)),), -1),
             "per-maxpool": (synth.groups_per_maxpool(layers), -1),
             "per-layer": (synth.groups_per_layer(layers), -1),
+            "pairs": (((1, len(layers)),), 2),
             "planner": (((1, len(layers)),), 0)}
 
 
@@ -56,6 +60,7 @@ def main():
     ap.add_argument("--size", type=int, default=608)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--precisions", default="fp32,bf16")
+    ap.add_argument("--profiles", default="", help="comma-separated subset of the profile names (default: all)")
     args = ap.parse_args()
     import torch
     import paper_2409_09083_b200 as ftp
@@ -64,6 +69,8 @@ def main():
         for N in (int(v) for v in args.batches.split(",")):
             for grid in (int(v) for v in args.grids.split(",")):
                 for name, (groups, mgc) in profiles(layers).items():
+                    if args.profiles and name not in args.profiles.split(","):
+                        continue
                     try:
                         r = time_point(ftp, torch, layers, N, args.size, grid, groups, 1 if prec == "bf16" else 0, args.steps,
                                        max_group_convs=mgc)
