@@ -175,6 +175,16 @@ int ftp_plan_subtiles(const ftp_plan* plan, int pass, int group,
                       int* rows, int* cols, size_t* smem_bytes, int* blocks);
 
 /*
+ * fp32 path, backward pass of an EXECUTED group: channels of the shared-memory staging area in
+ * which the delta at the output of a fused conv+pool layer is laid out, routed through the
+ * arg-max and zero-extended, for the input-delta convolution (the back-propagation of Section 3
+ * through a max-pool and a conv in one go).  The planner grants the area where it costs no
+ * sub-tile size; 0 means the convolution expands the pooled delta on the fly instead.  Both forms
+ * compute the same sums in the same order.  FTP_ERR_ARG on a bad index.
+ */
+int ftp_plan_delta_staging(const ftp_plan* plan, int group, int* channels);
+
+/*
  * The planner's time model of one pass (0 forward, 1 backward) of an EXECUTED
  * group.  The paper chooses its grouping profile by weighing halo
  * recomputation against boundary exchanges (Sections 4.2 and 5.3) but does not

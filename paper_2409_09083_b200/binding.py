@@ -59,6 +59,8 @@ _lib.ftp_plan_sizes.restype = _i
 _lib.ftp_plan_subtiles.argtypes = [_vp, _i, _i, ctypes.POINTER(_i), ctypes.POINTER(_i),
                                    ctypes.POINTER(_sz), ctypes.POINTER(_i)]
 _lib.ftp_plan_subtiles.restype = _i
+_lib.ftp_plan_delta_staging.argtypes = [_vp, _i, ctypes.POINTER(_i)]
+_lib.ftp_plan_delta_staging.restype = _i
 _lib.ftp_plan_cost.argtypes = [_vp, _i, _i, _i, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
 _lib.ftp_plan_cost.restype = _i
 _lib.ftp_forward.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
@@ -185,6 +187,12 @@ class Plan:
         _check(_lib.ftp_plan_subtiles(self._h, pass_, group, ctypes.byref(r), ctypes.byref(c),
                                       ctypes.byref(s), ctypes.byref(b)))
         return dict(rows=r.value, cols=c.value, smem_bytes=s.value, blocks=b.value)
+
+    def delta_staging(self, group):
+        """Channels of the backward pass's delta staging area of an executed group (fp32 path; 0 = none)."""
+        ch = _i()
+        _check(_lib.ftp_plan_delta_staging(self._h, group, ctypes.byref(ch)))
+        return ch.value
 
     def cost(self, pass_, group, need_dx=True):
         """(terms, estimate in microseconds) of the planner's time model for one pass of an executed group."""

@@ -425,6 +425,13 @@ int ftp_plan_subtiles(const ftp_plan* plan, int pass, int group, int* rows, int*
     return FTP_OK;
 }
 
+int ftp_plan_delta_staging(const ftp_plan* plan, int group, int* channels)
+{
+    if (!plan || !channels || group < 0 || group >= (int)plan->groups.size()) return FTP_ERR_ARG;
+    *channels = plan->groups[group].bwd.dz_ch;
+    return FTP_OK;
+}
+
 int ftp_plan_cost(const ftp_plan* plan, int pass, int group, int need_dx, double* terms, double* estimate_us)
 {
     if (!plan) return FTP_ERR_ARG;

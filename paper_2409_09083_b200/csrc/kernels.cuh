@@ -228,6 +228,117 @@ __device__ __forceinline__ void conv_tile(const float* __restrict__ in, const un
     }
 }
 
+// Input delta of a conv (or fused conv+pool) op with the output delta staged in shared memory:
+// out[c][u] = sum_{d, ky, kx} w[d][ky][kx][c] * Z[d][vy0 + uy + ky - (K-1)][vx0 + ux + kx - (K-1)]
+// for the ih x iw positions u of the op's input span, where Z is the zh x zw delta at the conv
+// output (zero outside) and w the rotated filter.  Same thread tasks as conv_tile (4 rows x 8
+// channels of one column).  The delta channels are taken `CH` at a time: all threads first write
+// the window of Z the span needs, (ih + K - 1) x (iw + K - 1) values per channel, to `stage`, with
+// the zeros of the border in place and, if `Darg` is given, the pooled delta D routed to the
+// arg-max position of each 2 x 2 window (Z[zy][zx] = D[zy/2][zx/2] if arg = (zy%2)*2 + zx%2, else
+// 0); the inner loop then reads it without any test, like the forward convolution.
+template <int K, class Epilogue>
+__device__ __forceinline__ void delta_conv_staged(const float* __restrict__ D, const unsigned char* __restrict__ Darg,
+                                                  int d_cs, int d_pitch, int zh, int zw, int vy0, int vx0,
+                                                  float* __restrict__ stage, int CH, const float* __restrict__ w,
+                                                  int nd /*delta channels*/, int cin_pad, int cin, int ih, int iw, Epilogue epi)
+{
+    constexpr int TP = 4, TC = kCoutTile;
+    const int rows = ih + K - 1, pitch = iw + K - 1, cs = rows * pitch;
+    const int ncob = cin_pad / TC, nyb = (ih + TP - 1) / TP;
+    const int ntasks = ncob * nyb * iw;
+    for (int t0 = 0; t0 < ntasks; t0 += blockDim.x) {
+        const bool active = t0 + (int)threadIdx.x < ntasks;
+        const int t = active ? t0 + (int)threadIdx.x : ntasks - 1;
+        const int x = t % iw, rem = t / iw, yb = rem % nyb, cob = rem / nyb;
+        const int y0 = yb * TP, c0 = cob * TC;
+        float acc[TP][TC];
+#pragma unroll
+        for (int p = 0; p < TP; ++p)
+#pragma unroll
+            for (int c = 0; c < TC; ++c) acc[p][c] = 0.f;
+        int rowoff[TP + K - 1];
+#pragma unroll
+        for (int r = 0; r < TP + K - 1; ++r) rowoff[r] = min(y0 + r, rows - 1) * pitch + x;
+        for (int d0 = 0; d0 < nd; d0 += CH) {
+            const int nch = min(CH, nd - d0);
+            __syncthreads();                                   // the previous channels have been consumed
+            for (int ch = 0; ch < nch; ++ch) {
+                const float* dp = D + (d0 + ch) * d_cs;
+                const unsigned char* ap = Darg ? Darg + (d0 + ch) * d_cs : nullptr;
+                float* sp = stage + ch * cs;
+                for (int e = threadIdx.x; e < cs; e += blockDim.x) {
+                    const int a = e / pitch, b = e - a * pitch;
+                    const int zy = vy0 + a - (K - 1), zx = vx0 + b - (K - 1);
+                    float v = 0.f;
+                    if (zy >= 0 && zy < zh && zx >= 0 && zx < zw) {
+                        if (ap) {
+                            const int idx = (zy >> 1) * d_pitch + (zx >> 1);
+                            v = (int)ap[idx] == (((zy & 1) << 1) | (zx & 1)) ? dp[idx] : 0.f;
+                        } else {
+                            v = dp[zy * d_pitch + zx];
+                        }
+                    }
+                    sp[e] = v;
+                }
+            }
+            __syncthreads();
+            if (active) {
+                const float* wp = w + c0 + (size_t)d0 * (K * K) * cin_pad;
+                for (int ci = 0; ci < nch; ++ci) {
+                    const float* ip = stage + ci * cs;
+                    const float* wc = wp + (size_t)ci * (K * K) * cin_pad;
+#pragma unroll
+                    for (int kx = 0; kx < K; ++kx) {
+                        float wr[K][TC];
+#pragma unroll
+                        for (int ky = 0; ky < K; ++ky) {
+                            const float4 a = __ldg(reinterpret_cast<const float4*>(wc + (ky * K + kx) * cin_pad));
+                            const float4 b = __ldg(reinterpret_cast<const float4*>(wc + (ky * K + kx) * cin_pad + 4));
+                            wr[ky][0] = a.x; wr[ky][1] = a.y; wr[ky][2] = a.z; wr[ky][3] = a.w;
+                            wr[ky][4] = b.x; wr[ky][5] = b.y; wr[ky][6] = b.z; wr[ky][7] = b.w;
+                        }
+#pragma unroll
+                        for (int r = 0; r < TP + K - 1; ++r) {
+                            const float v = ip[rowoff[r] + kx];
+#pragma unroll
+                            for (int ky = 0; ky < K; ++ky) {
+                                const int p = r - ky;
+                                if (p >= 0 && p < TP) {
+#pragma unroll
+                                    for (int c = 0; c < TC; ++c) acc[p][c] = fmaf(v, wr[ky][c], acc[p][c]);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        if (active) {
+#pragma unroll
+            for (int p = 0; p < TP; ++p)
+                if (y0 + p < ih) {
+#pragma unroll
+                    for (int c = 0; c < TC; ++c)
+                        if (c0 + c < cin) epi(c0 + c, y0 + p, x, acc[p][c], 0);
+                }
+        }
+    }
+}
+
+template <class Epilogue>
+__device__ __forceinline__ void delta_conv_staged_k(int K, const float* D, const unsigned char* Darg, int d_cs, int d_pitch,
+                                                    int zh, int zw, int vy0, int vx0, float* stage, int CH, const float* w,
+                                                    int nd, int cin_pad, int cin, int ih, int iw, Epilogue epi)
+{
+    switch (K) {
+    case 1: delta_conv_staged<1>(D, Darg, d_cs, d_pitch, zh, zw, vy0, vx0, stage, CH, w, nd, cin_pad, cin, ih, iw, epi); break;
+    case 3: delta_conv_staged<3>(D, Darg, d_cs, d_pitch, zh, zw, vy0, vx0, stage, CH, w, nd, cin_pad, cin, ih, iw, epi); break;
+    case 5: delta_conv_staged<5>(D, Darg, d_cs, d_pitch, zh, zw, vy0, vx0, stage, CH, w, nd, cin_pad, cin, ih, iw, epi); break;
+    default: delta_conv_staged<7>(D, Darg, d_cs, d_pitch, zh, zw, vy0, vx0, stage, CH, w, nd, cin_pad, cin, ih, iw, epi); break;
+    }
+}
+
 template <bool POOL_OUT, int MODE, class Epilogue>
 __device__ __forceinline__ void conv_tile_k(int K, const float* in, const unsigned char* arg, int in_cs, int in_pitch,
                                             int in_rows, int in_cols, int y_base, int x_base, const float* w, int cin,
@@ -652,7 +763,10 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_group_kernel(const __grid_con
                     filter_grad_k<true>(op.k, D, Darg, op.d_cs, op.d_pitch, X, op.in_cs, op.in_pitch, op.cin, op.cout,
                                         oh, ow, gw, first);
                     bias_grad_tile(D, op.d_cs, op.d_pitch, op.cout, oh, ow, gw + (size_t)op.cout * op.cin * op.k * op.k, first);
-                    if (need_in_delta)   // the pooled delta is expanded through the arg-max on the fly
+                    if (need_in_delta && op.dz_ch > 0)
+                        delta_conv_staged_k(op.k, D, Darg, op.d_cs, op.d_pitch, 2 * oh, 2 * ow, vy0, vx0, sm + op.dz_off, op.dz_ch,
+                                            A.wpk + op.wb_off, op.cout, op.cin_pad, op.cin, ih, iw, put);
+                    else if (need_in_delta)   // the pooled delta is expanded through the arg-max on the fly
                         conv_tile_k<false, kInExpand>(op.k, D, Darg, op.d_cs, op.d_pitch, 2 * oh, 2 * ow, vy0 - (op.k - 1),
                                                       vx0 - (op.k - 1), A.wpk + op.wb_off, op.cout, op.cin_pad, nullptr,
                                                       op.cin, 0.f, ih, iw, put);

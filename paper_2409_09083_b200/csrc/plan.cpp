@@ -138,10 +138,15 @@ size_t layout_forward(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
 // Backward: while op i runs, the delta at its output (D_i), a copy of its input and the delta it
 // produces (D_{i-1}) are alive.  Successive D buffers alternate between the two ends of the area
 // and the input copy sits next to the bottom one, so the area holds the largest such triple.
-size_t layout_backward(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
+// With dz_ch > 0 every fused conv+pool op also gets a staging area behind its input copy: the
+// input-delta convolution then reads the delta at the conv output from there, dz_ch channels at a
+// time, already routed through the arg-max and zero-extended by K - 1 on every side, instead of
+// testing every value it reads (measured on B200: 29 % off the backward pass of such a group; for
+// a plain conv, whose reads need one range test only, the staging costs more than it saves).
+size_t layout_backward(GroupPlan& g, const AxisTables& ty, const AxisTables& tx, int dz_ch)
 {
     const int n = g.n_ops;
-    int dsize[kMaxOps], xsize[kMaxOps];
+    int dsize[kMaxOps], xsize[kMaxOps], zsize[kMaxOps];
     for (int i = 0; i < n; ++i) {
         OpDesc& op = g.bwd_ops[i];
         int oh = ty.maxext[i + 1], ow = tx.maxext[i + 1];
@@ -154,14 +159,18 @@ size_t layout_backward(GroupPlan& g, const AxisTables& ty, const AxisTables& tx)
         int dfl = round4(op.cout * op.d_cs);
         op.d_arg_off = dfl * 4;                       // relative to the D buffer, fixed up below
         dsize[i] = dfl + (op.kind == kOpConvPool ? round4((op.cout * op.d_cs + 3) / 4) : 0);
+        // the input span is at most the input copy, and the staged delta K - 1 larger than the span
+        op.dz_ch = op.kind == kOpConvPool ? std::min(dz_ch, op.cout) : 0;
+        zsize[i] = round4(op.dz_ch * (bh + op.k - 1) * (bw + op.k - 1));
     }
     int total = 0;
-    for (int i = 0; i < n; ++i) total = std::max(total, dsize[i] + xsize[i] + (i > 0 ? dsize[i - 1] : 0));
+    for (int i = 0; i < n; ++i) total = std::max(total, dsize[i] + xsize[i] + zsize[i] + (i > 0 ? dsize[i - 1] : 0));
     for (int i = 0; i < n; ++i) {
         OpDesc& op = g.bwd_ops[i];
         const bool low = ((n - 1 - i) % 2) == 0;
         op.d_off = low ? 0 : total - dsize[i];
         op.in_off = low ? dsize[i] : (i > 0 ? dsize[i - 1] : 0);
+        op.dz_off = op.in_off + xsize[i];
         op.d_arg_off += op.d_off * 4;
     }
     return (size_t)kSmemHeader + 4 * (size_t)total;
@@ -257,7 +266,7 @@ int choose_subtiles(GroupPlan& g, bool backward, const PlanOpts& o, int N)
         build_axis(pp.x, ax, g.tile_x, kx);
         size_t bytes;
         if (o.tensor_cores) bytes = backward ? layout_backward_tc(g, pp.y, pp.x, pp.stages) : layout_forward_tc(g, pp.y, pp.x, pp.stages);
-        else bytes = backward ? layout_backward(g, pp.y, pp.x) : layout_forward(g, pp.y, pp.x);
+        else bytes = backward ? layout_backward(g, pp.y, pp.x, pp.dz_ch) : layout_forward(g, pp.y, pp.x);
         size_t budget = (size_t)o.smem_bytes;
         if (o.tensor_cores) budget = std::min<size_t>(pp.ctas == 2 ? kTcSmemBudget2 : kTcSmemBudget, (size_t)o.smem_bytes + 2048);
         return bytes <= budget ? bytes : 0;
@@ -461,12 +470,12 @@ void pass_cost_terms(const ftp_plan& p, const GroupPlan& g, bool backward, bool 
 // 0.13-0.21 over the four (precision, pass) fits.
 const double kCostWeights[2][2][kCostTerms] = {
     {   // fp32: forward, backward
-        {7.336, 7.264, 18.73, 167.9, 4.648, 0.1864, 0, 24.84},
-        {5.954, 5.355, 11.66, 266.3, 0, 228.4, 46.65, 34.55},
+        {7.375, 7.318, 17.18, 165.2, 4.796, 8.104, 0, 24.36},
+        {9.669, 5.017, 5.017, 257.6, 0, 242.5, 38.25, 27.79},
     },
     {   // bf16
-        {0, 1359, 33.91, 33.92, 3.3, 84.78, 224.9, 8.343},
-        {0.4407, 1.217, 0, 0, 71.85, 55.48, 6.834, 12.31},
+        {0, 1337, 34.7, 33.13, 3.084, 89.27, 231.8, 8.588},
+        {0.4358, 1.22, 0, 0, 71.85, 54.46, 6.794, 12.65},
     },
 };
 
@@ -547,6 +556,16 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
         int rc = choose_subtiles(g, pass == 1, o, N);
         if (rc != FTP_OK && pp.ctas == 2) { pp.ctas = 1; rc = choose_subtiles(g, pass == 1, o, N); }
         if (rc != FTP_OK) return rc;
+        if (pass == 1 && !tcp) {
+            // delta staging areas (see layout_backward) where they cost no sub-tile size
+            for (int ch : {kDeltaStageChannels, kDeltaStageChannels / 2, 0}) {
+                pp.dz_ch = ch;
+                const size_t bytes = layout_backward(g, pp.y, pp.x, ch);
+                if (bytes <= (size_t)o.smem_bytes) { pp.smem_bytes = bytes; break; }
+            }
+            pp.dz_ch = 0;                                   // report what the ops got
+            for (int i = 0; i < g.n_ops; ++i) pp.dz_ch = std::max(pp.dz_ch, g.bwd_ops[i].dz_ch);
+        }
         if (tcp) {
             // a four-stage filter ring where it costs no sub-tile size (measured: paying for it with smaller
             // tiles loses more than the deeper ring gains)

@@ -16,6 +16,7 @@ constexpr int kSmCount     = 148;     // B200
 constexpr int kSmemBudget  = 225 * 1024;  // dynamic shared memory a block may use
 constexpr int kSmemHeader  = 1024;    // bytes reserved at the start for per-block tables
 constexpr int kCoutTile    = 8;       // output channels per thread task (packed weights are padded to it)
+constexpr int kDeltaStageChannels = 8; // fp32 backward: channels of the output delta staged at a time for the input-delta convolution
 
 // Tensor-core (bf16) tile kernels: one block of 512 threads per SM with all 512 tensor-memory columns, or two
 // blocks of 256 threads with 256 columns each.
@@ -49,6 +50,7 @@ struct OpDesc {
     int   in_off, in_pitch, in_cs;     // forward input buffer / backward copy of the op's input
     int   d_off, d_pitch, d_cs;        // backward: delta at this op's output (no apron)
     int   d_arg_off;                   // backward, fused op: byte offset of the arg-max copy (same geometry as d)
+    int   dz_off, dz_ch;               // backward: staging area of the zero-extended output delta, dz_ch channels at a time (0: none)
     int   cout_pad, cin_pad;           // channel counts padded to kCoutTile in the packed filters
     long long wf_off, wb_off;          // float offsets into the packed forward / rotated filters
     long long p_off;                   // float offset of the filter in params (bias follows it)
@@ -80,6 +82,7 @@ struct PassPlan {
     size_t smem_bytes = 0;
     int blocks = 0;                 // forward: R*Q*N ; backward: tiles * splits
     int splits = 1;                 // backward: blocks per user tile
+    int dz_ch = 0;                  // backward, fp32 path: channels of the delta staging area (see layout_backward)
     int stages = 2;                 // tensor-core path: stages of the filter ring
     int ctas = 1;                   // tensor-core path: blocks per SM (2 = each block takes half of the tensor memory)
     size_t scratch_floats = 0;      // backward: floats of per-sub-tile group-input deltas (all images)

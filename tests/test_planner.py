@@ -213,3 +213,23 @@ def test_null_pointers_are_rejected_on_the_host():
     assert lib.ftp_step(plan._h, None, None, None, None, 0.0, None, None, None, None) == -1
     assert lib.ftp_forward(None, None, None, None, None, None) == -1
     assert plan.launch_count() == 0
+
+
+def test_delta_staging_is_granted_only_where_it_fits():
+    """fp32 backward: a group with a fused conv+pool gets the 8-channel staging area when the
+    sub-tile split leaves room, half of it or none otherwise; groups without such a layer report 0.
+    (The GPU invariance test runs the two reduced settings.)"""
+    wl = synth.Workload("y8", tuple(synth.stack_yolo8()), 2, 3, 64, 96, (2, 2), ((1, 8),))
+    mk = lambda **kw: ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, **kw)
+    full, none, half = mk(), mk(smem_bytes=160000), mk(smem_bytes=100000)
+    assert full.exec_groups()[0] == none.exec_groups()[0] == half.exec_groups()[0] == (1, 4)
+    assert (full.delta_staging(0), none.delta_staging(0), half.delta_staging(0)) == (8, 0, 4)
+    assert none.subtiles(1, 0)["rows"] == full.subtiles(1, 0)["rows"]      # refused rather than paid for with smaller sub-tiles
+    for plan in (full, none, half):
+        for gi, (a, b) in enumerate(plan.exec_groups()):
+            has_pair = any(wl.layers[i].kind == "conv" and wl.layers[i + 1].kind == "pool" for i in range(a - 1, b - 1))
+            assert (plan.delta_staging(gi) > 0) <= has_pair
+            assert plan.subtiles(1, gi)["smem_bytes"] <= 225 * 1024
+    assert mk(precision=1).delta_staging(0) == 0                            # the bf16 path has no such area
+    with pytest.raises(binding.FtpError):
+        full.delta_staging(99)
