@@ -558,7 +558,7 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
         if (rc != FTP_OK) return rc;
         if (pass == 1 && !tcp) {
             // delta staging areas (see layout_backward) where they cost no sub-tile size
-            for (int ch : {kDeltaStageChannels, kDeltaStageChannels / 2, 0}) {
+            for (int ch : {kDeltaStageChannels, kDeltaStageChannels / 2, kDeltaStageChannels / 4, 0}) {
                 pp.dz_ch = ch;
                 const size_t bytes = layout_backward(g, pp.y, pp.x, ch);
                 if (bytes <= (size_t)o.smem_bytes) { pp.smem_bytes = bytes; break; }

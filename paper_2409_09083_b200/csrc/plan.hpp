@@ -16,7 +16,7 @@ constexpr int kSmCount     = 148;     // B200
 constexpr int kSmemBudget  = 225 * 1024;  // dynamic shared memory a block may use
 constexpr int kSmemHeader  = 1024;    // bytes reserved at the start for per-block tables
 constexpr int kCoutTile    = 8;       // output channels per thread task (packed weights are padded to it)
-constexpr int kDeltaStageChannels = 8; // fp32 backward: channels of the output delta staged at a time for the input-delta convolution
+constexpr int kDeltaStageChannels = 16; // fp32 backward: channels of the output delta staged at a time for the input-delta convolution
 
 // Tensor-core (bf16) tile kernels: one block of 512 threads per SM with all 512 tensor-memory columns, or two
 // blocks of 256 threads with 256 columns each.

@@ -104,8 +104,9 @@ def test_result_does_not_depend_on_grid_or_groups_and_is_reproducible():
                 dict(grid=(2, 5), groups=synth.groups_per_layer(wl.layers)), dict(grid=(8, 12)),
                 dict(grid=(2, 2), opts=dict(max_group_convs=-1)), dict(grid=(3, 2), opts=dict(max_group_convs=1)),
                 dict(grid=(3, 3), opts=dict(cost_model=1)), dict(grid=(3, 3), opts=dict(cost_model=-1)),
-                # less shared memory: the conv+pool input delta without its staging area, and with half of it
-                dict(grid=(2, 2), opts=dict(smem_bytes=160000)), dict(grid=(2, 2), opts=dict(smem_bytes=100000))]
+                # less shared memory: the conv+pool input delta without its staging area, and with smaller ones
+                dict(grid=(2, 2), opts=dict(smem_bytes=160000)), dict(grid=(2, 2), opts=dict(smem_bytes=180000)),
+                dict(grid=(2, 2), opts=dict(smem_bytes=100000))]
     for v in variants:
         opts = v.pop("opts", {})
         got = run_gpu(wl.with_(**v), x, params, dy=dy, **opts)

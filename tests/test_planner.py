@@ -216,14 +216,14 @@ def test_null_pointers_are_rejected_on_the_host():
 
 
 def test_delta_staging_is_granted_only_where_it_fits():
-    """fp32 backward: a group with a fused conv+pool gets the 8-channel staging area when the
-    sub-tile split leaves room, half of it or none otherwise; groups without such a layer report 0.
+    """fp32 backward: a group with a fused conv+pool gets the 16-channel staging area when the
+    sub-tile split leaves room, a half or a quarter of it or none otherwise; groups without such a layer report 0.
     (The GPU invariance test runs the two reduced settings.)"""
     wl = synth.Workload("y8", tuple(synth.stack_yolo8()), 2, 3, 64, 96, (2, 2), ((1, 8),))
     mk = lambda **kw: ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, **kw)
     full, none, half = mk(), mk(smem_bytes=160000), mk(smem_bytes=100000)
     assert full.exec_groups()[0] == none.exec_groups()[0] == half.exec_groups()[0] == (1, 4)
-    assert (full.delta_staging(0), none.delta_staging(0), half.delta_staging(0)) == (8, 0, 4)
+    assert (full.delta_staging(0), mk(smem_bytes=180000).delta_staging(0), none.delta_staging(0), half.delta_staging(0)) == (16, 8, 0, 4)
     assert none.subtiles(1, 0)["rows"] == full.subtiles(1, 0)["rows"]      # refused rather than paid for with smaller sub-tiles
     for plan in (full, none, half):
         for gi, (a, b) in enumerate(plan.exec_groups()):
