@@ -91,6 +91,15 @@ __device__ __forceinline__ void zero_apron(float* buf, int cs, int pitch, int bh
     }
 }
 
+// 16-byte asynchronous copy from global to shared memory (both 16-byte aligned), and its group bookkeeping.
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem)
+{
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
+
 // Direct convolution on a shared-memory tile: out(c, y, x) = init(c) + sum_{ci,ky,kx}
 // w[ci][ky*K+kx][c] * in[ci][y+ky][x+kx] for y < oh, x < ow, c < cout.  A thread task is 8
 // output channels x 4 rows at one column; lanes walk along x, so shared-memory reads are
@@ -107,14 +116,19 @@ __device__ __forceinline__ void zero_apron(float* buf, int cs, int pitch, int bh
 //   MODE kInExpand:  as kInChecked, but the rectangle is virtual: `in` is the delta of a pooled map
 //     with its arg-max bytes, and the un-pooled delta at (vy, vx) is in[vy/2][vx/2] if the arg-max
 //     of that window is (vy%2, vx%2), else 0.  in_rows/in_cols count un-pooled positions.
+//   STAGED: the filter words come from shared memory instead of global memory.  The input
+//     channels are taken w_ch at a time; the block copies the filters of the next w_ch channels
+//     (contiguous in both filter layouts) into one half of `wst` with cp.async while it computes on
+//     the other half, so the inner loop waits on shared-memory latency only.  All threads of the
+//     block must make the call (it synchronises).
 enum { kInPlain = 0, kInChecked = 1, kInExpand = 2 };
 
-template <int K, bool POOL_OUT, int MODE, class Epilogue>
+template <int K, bool POOL_OUT, int MODE, bool STAGED, class Epilogue>
 __device__ __forceinline__ void conv_tile(const float* __restrict__ in, const unsigned char* __restrict__ arg,
                                           int in_cs, int in_pitch, int in_rows, int in_cols, int y_base, int x_base,
                                           const float* __restrict__ w, int cin, int cout_pad,
                                           const float* __restrict__ bias, int cout, float slope,
-                                          int oh, int ow, Epilogue epi)
+                                          int oh, int ow, float* __restrict__ wst, int w_ch, Epilogue epi)
 {
     constexpr int TP = 4, TC = kCoutTile;
     const int ncob = cout_pad / TC, nyb = (oh + TP - 1) / TP;
@@ -157,18 +171,38 @@ __device__ __forceinline__ void conv_tile(const float* __restrict__ in, const un
                 else coloff[kx] = cx;
             }
         }
-        const float* wp = w + c0;
-        for (int ci = 0; ci < cin; ++ci) {
+        const int per_ci = K * K * cout_pad;                  // filter words of one input channel
+        const int step = STAGED ? w_ch : cin;
+        auto stage = [&](int ci0) {                            // copy of the filters of channels ci0 .. ci0 + w_ch - 1
+            const int n4 = min(w_ch, cin - ci0) * per_ci / 4;
+            const float4* src = reinterpret_cast<const float4*>(w + (size_t)ci0 * per_ci);
+            float4* dst = reinterpret_cast<float4*>(wst + ((ci0 / w_ch) & 1) * w_ch * per_ci);
+            for (int i = threadIdx.x; i < n4; i += blockDim.x) cp_async16(dst + i, src + i);
+            cp_async_commit();
+        };
+        if (STAGED) stage(0);
+        for (int cb = 0; cb < cin; cb += step) {
+        const int ce = min(cin, cb + step);
+        const float* wp;
+        if (STAGED) {
+            if (ce < cin) { stage(ce); cp_async_wait<1>(); } else cp_async_wait<0>();
+            __syncthreads();
+            wp = wst + ((cb / w_ch) & 1) * w_ch * per_ci + c0 - (size_t)cb * per_ci;
+        } else {
+            wp = w + c0;
+        }
+        for (int ci = cb; ci < ce; ++ci) {
             const float* ip = in + ci * in_cs;
             const unsigned char* ap = MODE == kInExpand ? arg + ci * in_cs : nullptr;
-            const float* wc = wp + (size_t)ci * (K * K) * cout_pad;
+            const float* wc = wp + (size_t)ci * per_ci;
 #pragma unroll
             for (int kx = 0; kx < K; ++kx) {
                 float wr[K][TC];
 #pragma unroll
                 for (int ky = 0; ky < K; ++ky) {
-                    const float4 a = __ldg(reinterpret_cast<const float4*>(wc + (ky * K + kx) * cout_pad));
-                    const float4 b = __ldg(reinterpret_cast<const float4*>(wc + (ky * K + kx) * cout_pad + 4));
+                    const float4* wq = reinterpret_cast<const float4*>(wc + (ky * K + kx) * cout_pad);
+                    const float4 a = STAGED ? wq[0] : __ldg(wq);
+                    const float4 b = STAGED ? wq[1] : __ldg(wq + 1);
                     wr[ky][0] = a.x; wr[ky][1] = a.y; wr[ky][2] = a.z; wr[ky][3] = a.w;
                     wr[ky][4] = b.x; wr[ky][5] = b.y; wr[ky][6] = b.z; wr[ky][7] = b.w;
                 }
@@ -198,6 +232,8 @@ __device__ __forceinline__ void conv_tile(const float* __restrict__ in, const un
                     }
                 }
             }
+        }
+        if (STAGED) __syncthreads();                           // this half of wst may be overwritten now
         }
         if (POOL_OUT) {
 #pragma unroll
@@ -237,11 +273,14 @@ __device__ __forceinline__ void conv_tile(const float* __restrict__ in, const un
 // the zeros of the border in place and, if `Darg` is given, the pooled delta D routed to the
 // arg-max position of each 2 x 2 window (Z[zy][zx] = D[zy/2][zx/2] if arg = (zy%2)*2 + zx%2, else
 // 0); the inner loop then reads it without any test, like the forward convolution.
-template <int K, class Epilogue>
+// WST: the rotated filters of the CH channels are copied to `wst` (cp.async, overlapping the
+// staging of the delta) and read from there.
+template <int K, bool WST, class Epilogue>
 __device__ __forceinline__ void delta_conv_staged(const float* __restrict__ D, const unsigned char* __restrict__ Darg,
                                                   int d_cs, int d_pitch, int zh, int zw, int vy0, int vx0,
                                                   float* __restrict__ stage, int CH, const float* __restrict__ w,
-                                                  int nd /*delta channels*/, int cin_pad, int cin, int ih, int iw, Epilogue epi)
+                                                  int nd /*delta channels*/, int cin_pad, int cin, int ih, int iw,
+                                                  float* __restrict__ wst, Epilogue epi)
 {
     constexpr int TP = 4, TC = kCoutTile;
     const int rows = ih + K - 1, pitch = iw + K - 1, cs = rows * pitch;
@@ -263,6 +302,13 @@ __device__ __forceinline__ void delta_conv_staged(const float* __restrict__ D, c
         for (int d0 = 0; d0 < nd; d0 += CH) {
             const int nch = min(CH, nd - d0);
             __syncthreads();                                   // the previous channels have been consumed
+            if (WST) {
+                const int n4 = nch * (K * K) * cin_pad / 4;
+                const float4* src = reinterpret_cast<const float4*>(w + (size_t)d0 * (K * K) * cin_pad);
+                float4* dst = reinterpret_cast<float4*>(wst);
+                for (int i = threadIdx.x; i < n4; i += blockDim.x) cp_async16(dst + i, src + i);
+                cp_async_commit();
+            }
             for (int ch = 0; ch < nch; ++ch) {
                 const float* dp = D + (d0 + ch) * d_cs;
                 const unsigned char* ap = Darg ? Darg + (d0 + ch) * d_cs : nullptr;
@@ -282,9 +328,10 @@ __device__ __forceinline__ void delta_conv_staged(const float* __restrict__ D, c
                     sp[e] = v;
                 }
             }
+            if (WST) cp_async_wait<0>();
             __syncthreads();
             if (active) {
-                const float* wp = w + c0 + (size_t)d0 * (K * K) * cin_pad;
+                const float* wp = (WST ? wst : w + (size_t)d0 * (K * K) * cin_pad) + c0;
                 for (int ci = 0; ci < nch; ++ci) {
                     const float* ip = stage + ci * cs;
                     const float* wc = wp + (size_t)ci * (K * K) * cin_pad;
@@ -293,8 +340,9 @@ __device__ __forceinline__ void delta_conv_staged(const float* __restrict__ D, c
                         float wr[K][TC];
 #pragma unroll
                         for (int ky = 0; ky < K; ++ky) {
-                            const float4 a = __ldg(reinterpret_cast<const float4*>(wc + (ky * K + kx) * cin_pad));
-                            const float4 b = __ldg(reinterpret_cast<const float4*>(wc + (ky * K + kx) * cin_pad + 4));
+                            const float4* wq = reinterpret_cast<const float4*>(wc + (ky * K + kx) * cin_pad);
+                            const float4 a = WST ? wq[0] : __ldg(wq);
+                            const float4 b = WST ? wq[1] : __ldg(wq + 1);
                             wr[ky][0] = a.x; wr[ky][1] = a.y; wr[ky][2] = a.z; wr[ky][3] = a.w;
                             wr[ky][4] = b.x; wr[ky][5] = b.y; wr[ky][6] = b.z; wr[ky][7] = b.w;
                         }
@@ -329,28 +377,52 @@ __device__ __forceinline__ void delta_conv_staged(const float* __restrict__ D, c
 template <class Epilogue>
 __device__ __forceinline__ void delta_conv_staged_k(int K, const float* D, const unsigned char* Darg, int d_cs, int d_pitch,
                                                     int zh, int zw, int vy0, int vx0, float* stage, int CH, const float* w,
-                                                    int nd, int cin_pad, int cin, int ih, int iw, Epilogue epi)
+                                                    int nd, int cin_pad, int cin, int ih, int iw, float* wst, Epilogue epi)
 {
-    switch (K) {
-    case 1: delta_conv_staged<1>(D, Darg, d_cs, d_pitch, zh, zw, vy0, vx0, stage, CH, w, nd, cin_pad, cin, ih, iw, epi); break;
-    case 3: delta_conv_staged<3>(D, Darg, d_cs, d_pitch, zh, zw, vy0, vx0, stage, CH, w, nd, cin_pad, cin, ih, iw, epi); break;
-    case 5: delta_conv_staged<5>(D, Darg, d_cs, d_pitch, zh, zw, vy0, vx0, stage, CH, w, nd, cin_pad, cin, ih, iw, epi); break;
-    default: delta_conv_staged<7>(D, Darg, d_cs, d_pitch, zh, zw, vy0, vx0, stage, CH, w, nd, cin_pad, cin, ih, iw, epi); break;
+#define FTP_DELTA_CONV(KK, WS) delta_conv_staged<KK, WS>(D, Darg, d_cs, d_pitch, zh, zw, vy0, vx0, stage, CH, w, nd, cin_pad, cin, \
+                                                         ih, iw, wst, epi)
+    if (wst) {
+        switch (K) {
+        case 1: FTP_DELTA_CONV(1, true); break;
+        case 3: FTP_DELTA_CONV(3, true); break;
+        case 5: FTP_DELTA_CONV(5, true); break;
+        default: FTP_DELTA_CONV(7, true); break;
+        }
+    } else {
+        switch (K) {
+        case 1: FTP_DELTA_CONV(1, false); break;
+        case 3: FTP_DELTA_CONV(3, false); break;
+        case 5: FTP_DELTA_CONV(5, false); break;
+        default: FTP_DELTA_CONV(7, false); break;
+        }
     }
+#undef FTP_DELTA_CONV
 }
 
 template <bool POOL_OUT, int MODE, class Epilogue>
 __device__ __forceinline__ void conv_tile_k(int K, const float* in, const unsigned char* arg, int in_cs, int in_pitch,
                                             int in_rows, int in_cols, int y_base, int x_base, const float* w, int cin,
                                             int cout_pad, const float* bias, int cout, float slope, int oh, int ow,
-                                            Epilogue epi)
+                                            float* wst, int w_ch, Epilogue epi)
 {
-    switch (K) {
-    case 1: conv_tile<1, POOL_OUT, MODE>(in, arg, in_cs, in_pitch, in_rows, in_cols, y_base, x_base, w, cin, cout_pad, bias, cout, slope, oh, ow, epi); break;
-    case 3: conv_tile<3, POOL_OUT, MODE>(in, arg, in_cs, in_pitch, in_rows, in_cols, y_base, x_base, w, cin, cout_pad, bias, cout, slope, oh, ow, epi); break;
-    case 5: conv_tile<5, POOL_OUT, MODE>(in, arg, in_cs, in_pitch, in_rows, in_cols, y_base, x_base, w, cin, cout_pad, bias, cout, slope, oh, ow, epi); break;
-    default: conv_tile<7, POOL_OUT, MODE>(in, arg, in_cs, in_pitch, in_rows, in_cols, y_base, x_base, w, cin, cout_pad, bias, cout, slope, oh, ow, epi); break;
+#define FTP_CONV_TILE(KK, ST) conv_tile<KK, POOL_OUT, MODE, ST>(in, arg, in_cs, in_pitch, in_rows, in_cols, y_base, x_base, w, cin, \
+                                                                cout_pad, bias, cout, slope, oh, ow, wst, w_ch, epi)
+    if (w_ch > 0) {
+        switch (K) {
+        case 1: FTP_CONV_TILE(1, true); break;
+        case 3: FTP_CONV_TILE(3, true); break;
+        case 5: FTP_CONV_TILE(5, true); break;
+        default: FTP_CONV_TILE(7, true); break;
+        }
+    } else {
+        switch (K) {
+        case 1: FTP_CONV_TILE(1, false); break;
+        case 3: FTP_CONV_TILE(3, false); break;
+        case 5: FTP_CONV_TILE(5, false); break;
+        default: FTP_CONV_TILE(7, false); break;
+        }
     }
+#undef FTP_CONV_TILE
 }
 
 // Partial filter gradient of one sub-tile (Section 4.1: feature-map tile convolved with the
@@ -645,10 +717,12 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_group_kernel(const __grid_con
             if (op.kind == kOpConv)
                 conv_tile_k<false, kInPlain>(op.k, ib, nullptr, op.in_cs, op.in_pitch, oh + op.k - 1, 0, 0, 0,
                                              A.wpk + op.wf_off, op.cin, op.cout_pad, bias, op.cout, slope, oh, ow,
+                                             sm + op.w_off, op.w_ch,
                                              [&](int c, int ly, int lx, float z, int) { emit(c, ly, lx, leaky(z, slope), 0); });
             else
                 conv_tile_k<true, kInPlain>(op.k, ib, nullptr, op.in_cs, op.in_pitch, 2 * oh + op.k - 1, 0, 0, 0,
-                                            A.wpk + op.wf_off, op.cin, op.cout_pad, bias, op.cout, slope, 2 * oh, 2 * ow, emit);
+                                            A.wpk + op.wf_off, op.cin, op.cout_pad, bias, op.cout, slope, 2 * oh, 2 * ow,
+                                            sm + op.w_off, op.w_ch, emit);
         }
         __syncthreads();
     }
@@ -758,18 +832,19 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_group_kernel(const __grid_con
                     if (need_in_delta)
                         conv_tile_k<false, kInChecked>(op.k, D, nullptr, op.d_cs, op.d_pitch, oh, ow, vy0 - (op.k - 1),
                                                        vx0 - (op.k - 1), A.wpk + op.wb_off, op.cout, op.cin_pad, nullptr,
-                                                       op.cin, 0.f, ih, iw, put);
+                                                       op.cin, 0.f, ih, iw, sm + op.w_off, op.w_ch, put);
                 } else {
                     filter_grad_k<true>(op.k, D, Darg, op.d_cs, op.d_pitch, X, op.in_cs, op.in_pitch, op.cin, op.cout,
                                         oh, ow, gw, first);
                     bias_grad_tile(D, op.d_cs, op.d_pitch, op.cout, oh, ow, gw + (size_t)op.cout * op.cin * op.k * op.k, first);
                     if (need_in_delta && op.dz_ch > 0)
                         delta_conv_staged_k(op.k, D, Darg, op.d_cs, op.d_pitch, 2 * oh, 2 * ow, vy0, vx0, sm + op.dz_off, op.dz_ch,
-                                            A.wpk + op.wb_off, op.cout, op.cin_pad, op.cin, ih, iw, put);
+                                            A.wpk + op.wb_off, op.cout, op.cin_pad, op.cin, ih, iw,
+                                            op.w_ch > 0 ? sm + op.w_off : nullptr, put);
                     else if (need_in_delta)   // the pooled delta is expanded through the arg-max on the fly
                         conv_tile_k<false, kInExpand>(op.k, D, Darg, op.d_cs, op.d_pitch, 2 * oh, 2 * ow, vy0 - (op.k - 1),
                                                       vx0 - (op.k - 1), A.wpk + op.wb_off, op.cout, op.cin_pad, nullptr,
-                                                      op.cin, 0.f, ih, iw, put);
+                                                      op.cin, 0.f, ih, iw, nullptr, 0, put);
                 }
             } else if (need_in_delta) {
                 const int total = op.cout * oh * ow;

@@ -467,15 +467,15 @@ void pass_cost_terms(const ftp_plan& p, const GroupPlan& g, bool backward, bool 
 // kernel times of 168 candidate groups per precision, each measured inside whole training steps of
 // the 8- and 16-layer stacks on one B200 (calibrate.py of the Python package measures them and prints
 // this table).  Error of the fit, |log(estimate / measured)|: median 0.04-0.06, 90th percentile
-// 0.13-0.21 over the four (precision, pass) fits.
+// 0.13-0.22 over the four (precision, pass) fits.
 const double kCostWeights[2][2][kCostTerms] = {
     {   // fp32: forward, backward
-        {7.375, 7.318, 17.18, 165.2, 4.796, 8.104, 0, 24.36},
-        {9.669, 5.017, 5.017, 257.6, 0, 242.5, 38.25, 27.79},
+        {6.501, 7.123, 18.68, 162.4, 3.692, 74.99, 0, 9.23},
+        {10.09, 4.561, 3.758, 281.3, 0, 238, 37.45, 28.97},
     },
     {   // bf16
-        {0, 1337, 34.7, 33.13, 3.084, 89.27, 231.8, 8.588},
-        {0.4358, 1.22, 0, 0, 71.85, 54.46, 6.794, 12.65},
+        {0, 1349, 34.71, 33.52, 3.048, 90.11, 231.7, 8.51},
+        {0.4481, 1.205, 0, 0, 72.01, 54.47, 6.755, 12.4},
     },
 };
 
@@ -556,6 +556,24 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
         int rc = choose_subtiles(g, pass == 1, o, N);
         if (rc != FTP_OK && pp.ctas == 2) { pp.ctas = 1; rc = choose_subtiles(g, pass == 1, o, N); }
         if (rc != FTP_OK) return rc;
+        if (pass == 0 && !tcp) {
+            // Filter staging: what the chosen sub-tiles leave of the shared memory holds, behind the
+            // activation area, two halves of w_ch input channels' filters each (about 32 KB a half at
+            // most).  Ops that would get less than kMinFilterStage words per half, unless that is all
+            // their filters, read global memory: two barriers per half cost more than short halves save.
+            const long long room = ((long long)o.smem_bytes - (long long)pp.smem_bytes) / 4;      // floats
+            const int base = (int)((pp.smem_bytes - kSmemHeader) / 4);
+            long long used = 0;
+            for (int i = 0; i < g.n_ops; ++i) {
+                OpDesc& op = g.fwd_ops[i];
+                op.w_off = base; op.w_ch = 0;
+                if (op.kind == kOpPool) continue;
+                const long long per_ci = (long long)op.k * op.k * op.cout_pad;
+                long long ch = std::min<long long>(op.cin, std::min<long long>(room / (2 * per_ci), std::max<long long>(2, 8192 / per_ci)));
+                if (ch >= 1 && (ch == op.cin || ch * per_ci >= kMinFilterStage)) { op.w_ch = (int)ch; used = std::max(used, 2 * ch * per_ci); }
+            }
+            pp.smem_bytes += (size_t)used * 4;
+        }
         if (pass == 1 && !tcp) {
             // delta staging areas (see layout_backward) where they cost no sub-tile size
             for (int ch : {kDeltaStageChannels, kDeltaStageChannels / 2, kDeltaStageChannels / 4, 0}) {
@@ -565,6 +583,25 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
             }
             pp.dz_ch = 0;                                   // report what the ops got
             for (int i = 0; i < g.n_ops; ++i) pp.dz_ch = std::max(pp.dz_ch, g.bwd_ops[i].dz_ch);
+            // Staging of the rotated filters for the input-delta convolutions, in what is left: two
+            // halves as in the forward pass for a plain conv; for a fused conv+pool with a delta
+            // staging area, the filters of its dz_ch channels (all of them or none).
+            const long long room = ((long long)o.smem_bytes - (long long)pp.smem_bytes) / 4;
+            const int base = (int)((pp.smem_bytes - kSmemHeader) / 4);
+            long long used = 0;
+            for (int i = 0; i < g.n_ops; ++i) {
+                OpDesc& op = g.bwd_ops[i];
+                op.w_off = base; op.w_ch = 0;
+                if (op.kind == kOpPool) continue;
+                const long long per_co = (long long)op.k * op.k * op.cin_pad;
+                if (op.kind == kOpConvPool) {
+                    if (op.dz_ch > 0 && op.dz_ch * per_co <= room) { op.w_ch = op.dz_ch; used = std::max(used, op.dz_ch * per_co); }
+                    continue;
+                }
+                long long ch = std::min<long long>(op.cout, std::min<long long>(room / (2 * per_co), std::max<long long>(2, 8192 / per_co)));
+                if (ch >= 1 && (ch == op.cout || ch * per_co >= kMinFilterStage)) { op.w_ch = (int)ch; used = std::max(used, 2 * ch * per_co); }
+            }
+            pp.smem_bytes += (size_t)used * 4;
         }
         if (tcp) {
             // a four-stage filter ring where it costs no sub-tile size (measured: paying for it with smaller

@@ -16,6 +16,7 @@ constexpr int kSmCount     = 148;     // B200
 constexpr int kSmemBudget  = 225 * 1024;  // dynamic shared memory a block may use
 constexpr int kSmemHeader  = 1024;    // bytes reserved at the start for per-block tables
 constexpr int kCoutTile    = 8;       // output channels per thread task (packed weights are padded to it)
+constexpr int kMinFilterStage = 2048;   // fp32 path: smallest half (floats) of a filter staging area worth its barriers
 constexpr int kDeltaStageChannels = 16; // fp32 backward: channels of the output delta staged at a time for the input-delta convolution
 
 // Tensor-core (bf16) tile kernels: one block of 512 threads per SM with all 512 tensor-memory columns, or two
@@ -51,6 +52,7 @@ struct OpDesc {
     int   d_off, d_pitch, d_cs;        // backward: delta at this op's output (no apron)
     int   d_arg_off;                   // backward, fused op: byte offset of the arg-max copy (same geometry as d)
     int   dz_off, dz_ch;               // backward: staging area of the zero-extended output delta, dz_ch channels at a time (0: none)
+    int   w_off, w_ch;                 // filter staging area (two halves of w_ch input channels each; 0: filters are read from global memory)
     int   cout_pad, cin_pad;           // channel counts padded to kCoutTile in the packed filters
     long long wf_off, wb_off;          // float offsets into the packed forward / rotated filters
     long long p_off;                   // float offset of the filter in params (bias follows it)
