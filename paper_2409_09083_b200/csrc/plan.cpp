@@ -467,15 +467,15 @@ void pass_cost_terms(const ftp_plan& p, const GroupPlan& g, bool backward, bool 
 // kernel times of 168 candidate groups per precision, each measured inside whole training steps of
 // the 8- and 16-layer stacks on one B200 (calibrate.py of the Python package measures them and prints
 // this table).  Error of the fit, |log(estimate / measured)|: median 0.04-0.06, 90th percentile
-// 0.13-0.22 over the four (precision, pass) fits.
+// 0.13-0.23 over the four (precision, pass) fits.
 const double kCostWeights[2][2][kCostTerms] = {
     {   // fp32: forward, backward
-        {6.501, 7.123, 18.68, 162.4, 3.692, 74.99, 0, 9.23},
-        {10.09, 4.561, 3.758, 281.3, 0, 238, 37.45, 28.97},
+        {6.542, 7.174, 18.76, 163.5, 3.134, 72.57, 0, 9.153},
+        {12.11, 2.713, 1.779, 288.3, 0, 258.7, 37.3, 11.19},
     },
     {   // bf16
-        {0, 1349, 34.71, 33.52, 3.048, 90.11, 231.7, 8.51},
-        {0.4481, 1.205, 0, 0, 72.01, 54.47, 6.755, 12.4},
+        {0, 1297, 34.79, 32.73, 3.082, 91.97, 235.4, 8.515},
+        {0.5158, 1.074, 0, 103.9, 22.5, 52.28, 6.621, 17.48},
     },
 };
 
@@ -485,6 +485,63 @@ double pass_estimate_us(int precision, bool backward, const double f[kCostTerms]
     double t = 0;
     for (int k = 0; k < kCostTerms; ++k) t += w[k] * f[k];
     return t;
+}
+
+// Backward launch shape: `splits` blocks per user tile, each owning one partial gradient set.
+void set_backward_blocks(GroupPlan& g, int N, int gy, int gx)
+{
+    int min_items = 1 << 30;
+    for (int ty = 0; ty < gy; ++ty)
+        for (int tx = 0; tx < gx; ++tx) {
+            int items = N * (g.bwd.y.tile_begin[ty + 1] - g.bwd.y.tile_begin[ty]) *
+                        (g.bwd.x.tile_begin[tx + 1] - g.bwd.x.tile_begin[tx]);
+            min_items = std::min(min_items, items);
+        }
+    g.bwd.splits = std::max(1, std::min(min_items, kSmCount * g.bwd.ctas / (gy * gx)));
+    g.bwd.blocks = gy * gx * g.bwd.splits;
+}
+
+// Backward sub-tiling, second step.  choose_subtiles takes the largest sub-tiles that fit; the
+// blocks of a user tile then share its N x (sub-tiles per tile) stacks, and when that number does
+// not divide by the blocks the slowest block runs one stack more than the average.  A somewhat
+// finer split can even that out (8 stacks of 1/8 tile on 4 blocks beat 6 stacks of 1/6).  The
+// candidates up to three cuts finer per axis are compared by the time model's estimate of the
+// pass, which counts the stacks of the busiest block; the first split stays unless another is
+// estimated at least 3 % faster.
+void refine_backward_split(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
+{
+    PassPlan& pp = g.bwd;
+    const AxisInfo ay = axis_info(g, true), ax = axis_info(g, false);
+    int max_h = 0, max_w = 0, ky0 = 1, kx0 = 1;
+    for (const Span& s : g.tile_y) max_h = std::max(max_h, extent(s));
+    for (const Span& s : g.tile_x) max_w = std::max(max_w, extent(s));
+    for (size_t t = 0; t + 1 < pp.y.tile_begin.size(); ++t) ky0 = std::max(ky0, pp.y.tile_begin[t + 1] - pp.y.tile_begin[t]);
+    for (size_t t = 0; t + 1 < pp.x.tile_begin.size(); ++t) kx0 = std::max(kx0, pp.x.tile_begin[t + 1] - pp.x.tile_begin[t]);
+    size_t budget = (size_t)o.smem_bytes;
+    if (o.tensor_cores) budget = std::min<size_t>(pp.ctas == 2 ? kTcSmemBudget2 : kTcSmemBudget, (size_t)o.smem_bytes + 2048);
+    auto eval = [&](int ky, int kx) -> double {               // estimate in microseconds, negative if it does not fit
+        build_axis(pp.y, ay, g.tile_y, ky);
+        build_axis(pp.x, ax, g.tile_x, kx);
+        const size_t bytes = o.tensor_cores ? layout_backward_tc(g, pp.y, pp.x, pp.stages) : layout_backward(g, pp.y, pp.x, 0);
+        if (bytes > budget) return -1.0;
+        pp.smem_bytes = bytes;
+        set_backward_blocks(g, p.N, p.grid_y, p.grid_x);
+        double f[kCostTerms];
+        pass_cost_terms(p, g, true, g.first > 1, f);
+        return pass_estimate_us(p.precision, true, f);
+    };
+    const double first = eval(ky0, kx0);
+    double best = first;
+    int best_ky = ky0, best_kx = kx0;
+    if (first > 0)
+        for (int dy = 0; dy <= 3; ++dy)
+            for (int dx = 0; dx <= 3; ++dx) {
+                if (!dy && !dx) continue;
+                const int ky = std::min(ky0 + dy, max_h), kx = std::min(kx0 + dx, max_w);
+                const double est = eval(ky, kx);
+                if (est > 0 && est < 0.97 * first && est < best) { best = est; best_ky = ky; best_kx = kx; }
+            }
+    eval(best_ky, best_kx);
 }
 
 struct LayerOffsets { std::vector<long long> p_off, wf_off, wb_off, twf_off, twb_off; };
@@ -556,6 +613,7 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
         int rc = choose_subtiles(g, pass == 1, o, N);
         if (rc != FTP_OK && pp.ctas == 2) { pp.ctas = 1; rc = choose_subtiles(g, pass == 1, o, N); }
         if (rc != FTP_OK) return rc;
+        if (pass == 1 && o.max_subtile == 0 && o.refine_backward) refine_backward_split(p, g, o);
         if (pass == 0 && !tcp) {
             // Filter staging: what the chosen sub-tiles leave of the shared memory holds, behind the
             // activation area, two halves of w_ch input channels' filters each (about 32 KB a half at
@@ -618,16 +676,7 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
         *redundancy = g.macs_untiled > 0 ? std::max(g.macs_done, bwd_done) / g.macs_untiled : 1.0;
 
     g.fwd.blocks = g.fwd.y.count * g.fwd.x.count * N;
-    // backward: `splits` blocks per user tile, each owning one partial gradient set
-    int min_items = 1 << 30;
-    for (int ty = 0; ty < gy; ++ty)
-        for (int tx = 0; tx < gx; ++tx) {
-            int items = N * (g.bwd.y.tile_begin[ty + 1] - g.bwd.y.tile_begin[ty]) *
-                        (g.bwd.x.tile_begin[tx + 1] - g.bwd.x.tile_begin[tx]);
-            min_items = std::min(min_items, items);
-        }
-    g.bwd.splits = std::max(1, std::min(min_items, kSmCount * g.bwd.ctas / (gy * gx)));
-    g.bwd.blocks = gy * gx * g.bwd.splits;
+    set_backward_blocks(g, N, gy, gx);
     // (tensor-core path, groups after the first: the blocks hold 8-channel planes of the padded channel count)
     g.bwd.scratch_floats = (size_t)N * (tcp && first > 1 ? round_up(p.maps[first - 1].C, 16) : p.maps[first - 1].C) *
                            g.bwd.y.scratch_off[g.bwd.y.count] *

@@ -159,6 +159,7 @@ struct PlanOpts {
     int strict_groups = 0;          // 1 = never cut a requested group
     int max_group_convs = 2;        // executed groups hold at most this many conv layers (0 = no limit)
     int cost_model = 1;             // 1 = the time model (pass_cost_terms) may replace the fixed rule's cuts, see build_plan
+    int refine_backward = 1;        // 1 = the time model may take a finer backward split that balances the blocks (refine_backward_split)
     int tc_ctas = 0;                // tensor-core path: blocks per SM, 1 or 2 (0 = two where every layer of the group allows it)
     int tensor_cores = 0;           // set by build_plan from the precision: shared-memory layouts of the bf16 path
 };

@@ -149,11 +149,14 @@ def test_cost_terms_of_a_single_conv_by_hand():
     assert t[3] == pytest.approx((in_floats + 16 * 256) * 4 / 1e6 / (R * Q))
     assert t[4] == 1 and t[5] == pytest.approx(16 * 256 / 1e6 / (R * Q)) and t[7] == 1
     assert est > 0
+    # backward: the one image's tile is cut into Rb x Qb stacks, one per block, so again every term is
+    # that of one stack on the critical path
     sb = plan.subtiles(1, 0)
-    assert sb["rows"] == 1 and sb["cols"] == 1                      # backward: the largest stack that fits
+    Rb, Qb = sb["rows"], sb["cols"]
+    assert sb["blocks"] == Rb * Qb <= 148 and 16 % Rb == 0 and 16 % Qb == 0
     tb, estb = plan.cost(1, 0, True)
-    assert tb[0] == pytest.approx(256 * 8 * 16 * 9 / 1e6)            # filter gradient: plain count
-    assert tb[1] == pytest.approx(512 * 32 * 16 * 9 / 1e6)           # input delta: 1 x 4 x 16 = 64 tasks, one round, 16 input channels each
+    assert tb[0] == pytest.approx(256 * 8 * 16 * 9 / 1e6 / (Rb * Qb))   # filter gradient: plain count
+    assert tb[1] == pytest.approx(512 * 32 * 16 * 9 / 1e6)           # input delta: at most 1 x 4 x 16 = 64 tasks, one round, 16 delta channels each
     assert tb[4] == pytest.approx((9 * 8 * 16 + 16) * 4 / 1e6)       # the stack's partial set
     assert plan.cost(1, 0, False)[0][1] == 0                         # no input delta asked for
     # twice the batch: twice the stacks on as many blocks, so every term but the launch doubles at most
@@ -217,19 +220,40 @@ def test_null_pointers_are_rejected_on_the_host():
 
 def test_delta_staging_is_granted_only_where_it_fits():
     """fp32 backward: a group with a fused conv+pool gets the 16-channel staging area when the
-    sub-tile split leaves room, a half or a quarter of it or none otherwise; groups without such a layer report 0.
-    (The GPU invariance test runs the two reduced settings.)"""
+    sub-tile split leaves room, a half or a quarter of it or none otherwise; groups without such a
+    layer report 0.  (Fixed-rule groups and the first split that fits, so that only the shared-memory
+    limit varies; the GPU invariance test runs the two reduced settings.)"""
     wl = synth.Workload("y8", tuple(synth.stack_yolo8()), 2, 3, 64, 96, (2, 2), ((1, 8),))
-    mk = lambda **kw: ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, **kw)
-    full, none, half = mk(), mk(smem_bytes=160000), mk(smem_bytes=100000)
-    assert full.exec_groups()[0] == none.exec_groups()[0] == half.exec_groups()[0] == (1, 4)
-    assert (full.delta_staging(0), mk(smem_bytes=180000).delta_staging(0), none.delta_staging(0), half.delta_staging(0)) == (16, 8, 0, 4)
-    assert none.subtiles(1, 0)["rows"] == full.subtiles(1, 0)["rows"]      # refused rather than paid for with smaller sub-tiles
-    for plan in (full, none, half):
-        for gi, (a, b) in enumerate(plan.exec_groups()):
-            has_pair = any(wl.layers[i].kind == "conv" and wl.layers[i + 1].kind == "pool" for i in range(a - 1, b - 1))
-            assert (plan.delta_staging(gi) > 0) <= has_pair
+    mk = lambda **kw: ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, max_subtile=64, cost_model=-1, **kw)
+    full, part, none = mk(), mk(smem_bytes=120000), mk(smem_bytes=100000)
+    for plan in (full, part, none):
+        assert plan.exec_groups() == [(1, 2), (3, 4), (5, 6), (7, 8)]
+    staging = lambda plan: [plan.delta_staging(g) for g in range(4)]
+    assert staging(full) == [16, 16, 0, 16]
+    assert staging(part) == [4, 8, 0, 16]
+    assert staging(none) == [0, 0, 0, 16]
+    for g in (0, 1):                                                        # refused rather than paid for with smaller sub-tiles
+        assert none.subtiles(1, g)["rows"] == full.subtiles(1, g)["rows"] and none.subtiles(1, g)["cols"] == full.subtiles(1, g)["cols"]
+    for plan in (full, part, none):
+        for gi in range(4):
             assert plan.subtiles(1, gi)["smem_bytes"] <= 225 * 1024
-    assert mk(precision=1).delta_staging(0) == 0                            # the bf16 path has no such area
+    assert ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=1).delta_staging(0) == 0   # the bf16 path has no such area
     with pytest.raises(binding.FtpError):
         full.delta_staging(99)
+
+
+def test_backward_split_is_refined_for_balance():
+    """Backward blocks share the stacks of a user tile; the planner may cut finer than the largest
+    sub-tiles that fit when that evens out the stacks per block.  C1, fp32: layer 5 alone fits as
+    3 x 2 sub-tiles per tile, i.e. 4 images x 6 = 24 stacks on 16 blocks (two for half of the blocks,
+    one for the rest); 4 x 2 gives every block two smaller stacks."""
+    wl = synth.workload("C1")
+    layers = wl.layers[4:5]
+    mk = lambda **kw: ftp.ftp_plan(layers, wl.N, 64, 104, 104, (3, 3), ((1, 1),), **kw)
+    first_fit, refined = mk(max_subtile=64).subtiles(1, 0), mk().subtiles(1, 0)
+    assert (first_fit["rows"], first_fit["cols"]) == (9, 6)
+    assert (refined["rows"], refined["cols"]) == (12, 6)
+    assert first_fit["blocks"] == refined["blocks"] == 144
+    assert (4 * 4 * 2) % 16 == 0 and (4 * 3 * 2) % 16 != 0
+    est = lambda **kw: mk(**kw).cost(1, 0, True)[1]
+    assert est() < 0.97 * est(max_subtile=64)
