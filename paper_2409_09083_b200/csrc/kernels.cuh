@@ -69,13 +69,42 @@ __device__ __forceinline__ void load_header(int* hdr, const GroupArgs& A, int r,
 __device__ __forceinline__ void load_input(float* buf, int cs, int pitch, int bh, int bw, int C,
                                            const float* __restrict__ src, int n, int H, int W, int oy, int ox)
 {
-    const int total = C * bh * bw;
-    for (int e = threadIdx.x; e < total; e += blockDim.x) {
-        int xx = e % bw, t = e / bw, yy = t % bh, c = t / bh;
-        int gy = oy + yy, gx = ox + xx;
-        float v = 0.f;
-        if (gy >= 0 && gy < H && gx >= 0 && gx < W) v = __ldg(src + (((size_t)n * C + c) * H + gy) * W + gx);
-        buf[c * cs + yy * pitch + xx] = v;
+    if (bw < 24) {
+        // narrow buffers: one element per thread and turn, whatever row it is in
+        const int total = C * bh * bw;
+        for (int e = threadIdx.x; e < total; e += blockDim.x) {
+            int xx = e % bw, t = e / bw, yy = t % bh, c = t / bh;
+            int gy = oy + yy, gx = ox + xx;
+            float v = 0.f;
+            if (gy >= 0 && gy < H && gx >= 0 && gx < W) v = __ldg(src + (((size_t)n * C + c) * H + gy) * W + gx);
+            buf[c * cs + yy * pitch + xx] = v;
+        }
+        return;
+    }
+    // one warp per buffer row (c, yy), lanes along the row: coalesced reads and no division per
+    // element; four rows are in flight per warp so that their loads overlap
+    constexpr int U = 4;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int rows = C * bh;
+    const float* img = src + (size_t)n * C * H * W;
+    for (int r0 = warp * U; r0 < rows; r0 += nwarps * U) {
+        const float* s[U]; float* d[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int r = min(r0 + u, rows - 1);
+            const int c = r / bh, yy = r - c * bh, gy = oy + yy;
+            d[u] = r0 + u < rows ? buf + c * cs + yy * pitch : nullptr;
+            s[u] = (gy >= 0 && gy < H) ? img + ((size_t)c * H + gy) * W + ox : nullptr;
+        }
+        for (int xx = lane; xx < bw; xx += 32) {
+            const bool in = ox + xx >= 0 && ox + xx < W;
+            float v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) v[u] = (in && s[u]) ? __ldg(s[u] + xx) : 0.f;
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (d[u]) d[u][xx] = v[u];
+        }
     }
 }
 
