@@ -34,6 +34,11 @@ SMALL = {
     "conv-pool": (W("e", (conv(3, 8, 3), pool()), 1, 3, 16, 24, (2, 2), ((1, 2),), x_dist="normal"), {}),
     "pool-first": (W("f", (pool(), conv(3, 8, 3), pool(), pool()), 1, 3, 32, 48, (2, 2), ((1, 4),), x_dist="normal"), {}),
     "pool|conv-split": (W("g", (conv(3, 6, 3), pool(), conv(6, 5, 3)), 3, 3, 12, 20, (3, 2), ((1, 1), (2, 3)), x_dist="normal"), {}),
+    # fused conv+pool ops whose delta is staged in more than one slice (20 and 24 channels, 16 at a time),
+    # with 7 x 7 and 5 x 5 windows, in one group and cut between them; filters staged a few channels at a time
+    "conv7-pool-conv5-pool": (W("h", (conv(4, 20, 7), pool(), conv(20, 24, 5), pool()), 1, 4, 12, 16, (2, 2), ((1, 4),), x_dist="normal"),
+                              dict(strict_groups=True)),
+    "conv7-pool|conv5-pool": (W("i", (conv(4, 20, 7), pool(), conv(20, 24, 5), pool()), 1, 4, 12, 16, (1, 2), ((1, 2), (3, 4)), x_dist="normal"), {}),
 }
 
 
