@@ -247,3 +247,40 @@ def test_cost_model_estimates_track_measured_pass_times(precision):
             assert best[g][ps] / 2.5 <= est <= best[g][ps] * 2.5, (g, ps, est, best[g][ps])
             tot_meas += best[g][ps]; tot_est += est
     assert tot_meas / 1.6 <= tot_est <= tot_meas * 1.6
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("precision", [0, 1])
+def test_step_can_be_captured_in_a_cuda_graph(precision):
+    """ftp_step only launches kernels on the caller's stream once the plan's tables are on the device
+    (first call): captured in a CUDA graph and replayed, three steps leave bit for bit the
+    parameters and the loss that three direct calls leave."""
+    wl = synth.workload("C0").with_(N=2)
+    x, params, target = synth.draw(wl, N=2)
+    plan = ftp.ftp_plan(wl.layers, 2, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=precision)
+    ws = plan.new_workspace("cuda")
+    xd, p0, td = (torch.from_numpy(a).cuda() for a in (x, params, target))
+    loss = torch.zeros(1, device="cuda")
+    dx = torch.empty_like(xd)
+    pd = p0.clone()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        ftp.ftp_step(plan, xd, pd, 0.05, ws, target=td, loss_out=loss, dx=dx, stream=s)      # uploads the tables
+    torch.cuda.synchronize()
+    pd.copy_(p0)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        ftp.ftp_step(plan, xd, pd, 0.05, ws, target=td, loss_out=loss, dx=dx, stream=s)
+    launches = plan.launch_count()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    plan.check(ws)
+    assert plan.launch_count() == launches                   # replays do not go through the library
+    p_graph, l_graph, dx_graph = pd.clone(), float(loss.item()), dx.clone()
+    pd.copy_(p0)
+    for _ in range(3):
+        ftp.ftp_step(plan, xd, pd, 0.05, ws, target=td, loss_out=loss, dx=dx)
+    torch.cuda.synchronize()
+    assert torch.equal(p_graph, pd) and l_graph == float(loss.item()) and torch.equal(dx_graph, dx)
+    assert not torch.equal(pd, p0)
