@@ -294,6 +294,21 @@ int ftp_step_host(ftp_plan* plan, const float* x_host, const float* target_host,
                   float lr, float* loss_host, float* dx, void* workspace, void* stream);
 
 /*
+ * Input pipeline for ftp_step_host (the paper's devices receive their tiles of the next image over the
+ * network while they compute, Section 5; here the next batch crosses PCIe while the current step runs).
+ * Copies x_host and target_host (pinned memory, shapes as in ftp_step_host) into the staging slot of the
+ * workspace that the last ftp_step_host call does not read, asynchronously on `copy_stream` (a
+ * cudaStream_t; NULL = the plan's own side stream), after the step that last read that slot.  The next
+ * ftp_step_host call that is given the SAME two host pointers waits for these copies on its stream
+ * instead of copying; a call with other pointers copies as usual and leaves the prefetched batch in
+ * place.  The host buffers must stay unchanged until that step's stream has been synchronised.  One
+ * batch can be in flight at a time: a second prefetch before the step overwrites the first.
+ * Returns FTP_ERR_ARG on a null or unaligned pointer, FTP_ERR_CUDA if a runtime call fails.
+ */
+int ftp_prefetch_host(ftp_plan* plan, const float* x_host, const float* target_host,
+                      void* workspace, void* copy_stream);
+
+/*
  * The two halves of ftp_step for data-parallel replicas (one process per GPU, the batch split
  * across them; Section 4.1 sums the partial gradient sets "once per batch", which across GPUs is
  * an all-reduce the caller runs between these two calls):

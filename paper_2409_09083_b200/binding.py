@@ -71,6 +71,8 @@ _lib.ftp_step.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp, _vp
 _lib.ftp_step.restype = _i
 _lib.ftp_step_host.argtypes = [_vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp, _vp, _vp]
 _lib.ftp_step_host.restype = _i
+_lib.ftp_prefetch_host.argtypes = [_vp, _vp, _vp, _vp, _vp]
+_lib.ftp_prefetch_host.restype = _i
 _lib.ftp_step_grad.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.ftp_step_grad.restype = _i
 _lib.ftp_loss_mse.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -265,6 +267,16 @@ def ftp_loss_mse_static(y, target, dy, loss_out, stream=None):
 
 def ftp_sgd(params, grad, lr, stream=None):
     _check(_lib.ftp_sgd(_ptr(params, "params"), _ptr(grad, "grad"), params.numel(), float(lr), _stream(stream)))
+
+
+def ftp_prefetch_host(plan, x_host, target_host, workspace, copy_stream=None):
+    """Starts copying the NEXT batch (pinned float32 CPU tensors) while the current step runs; the
+    ftp_step_host call given the same two tensors then waits for these copies instead of copying."""
+    for name, t in (("x_host", x_host), ("target_host", target_host)):
+        if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous float32 CPU tensor")
+    _check(_lib.ftp_prefetch_host(plan._h, x_host.data_ptr(), target_host.data_ptr(), workspace.data_ptr(),
+                                  _stream(copy_stream)))
 
 
 def ftp_step_host(plan, x_host, target_host, params, lr, loss_host, workspace, dx=None, stream=None):

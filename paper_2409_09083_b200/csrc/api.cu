@@ -386,6 +386,9 @@ void ftp_plan_destroy(ftp_plan* plan)
         cudaStreamDestroy(static_cast<cudaStream_t>(plan->copy_stream));
         cudaEventDestroy(static_cast<cudaEvent_t>(plan->ev_fork));
         cudaEventDestroy(static_cast<cudaEvent_t>(plan->ev_join));
+        cudaEventDestroy(static_cast<cudaEvent_t>(plan->ev_prefetch));
+        cudaEventDestroy(static_cast<cudaEvent_t>(plan->ev_slot_free[0]));
+        cudaEventDestroy(static_cast<cudaEvent_t>(plan->ev_slot_free[1]));
     }
     delete plan;
 }
@@ -517,6 +520,43 @@ int ftp_step(ftp_plan* plan, const float* x, const float* dy, const float* targe
     return step_impl(plan, x, dy, target, params, params, lr, nullptr, loss_out, dx, workspace, stream);
 }
 
+// Side stream and events of the host-batch entry points, created on first use.
+static int ensure_copy_stream(ftp_plan* plan)
+{
+    if (plan->copy_stream) return FTP_OK;
+    cudaStream_t cs;
+    cudaEvent_t e[5];
+    if (cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking) != cudaSuccess) return FTP_ERR_CUDA;
+    for (cudaEvent_t& ev : e)
+        if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return FTP_ERR_CUDA;
+    plan->copy_stream = cs; plan->ev_fork = e[0]; plan->ev_join = e[1]; plan->ev_prefetch = e[2];
+    plan->ev_slot_free[0] = e[3]; plan->ev_slot_free[1] = e[4];
+    return FTP_OK;
+}
+
+int ftp_prefetch_host(ftp_plan* plan, const float* x_host, const float* target_host, void* workspace, void* copy_stream)
+{
+    if (!plan || !x_host || !target_host || !workspace || !aligned256(workspace)) return FTP_ERR_ARG;
+    int rc = ensure_device(plan);
+    if (rc == FTP_OK) rc = ensure_copy_stream(plan);
+    if (rc != FTP_OK) return rc;
+    cudaStream_t cs = copy_stream ? static_cast<cudaStream_t>(copy_stream) : static_cast<cudaStream_t>(plan->copy_stream);
+    const MapShape& in = plan->maps.front();
+    const MapShape& out = plan->maps.back();
+    const int slot = 1 - plan->cur_slot;          // the slot the last (possibly still running) step does not read
+    float* xs = ws_ptr(workspace, plan->ws.x_stage_off + slot * plan->ws.x_stage_bytes);
+    float* ts = ws_ptr(workspace, plan->ws.t_stage_off + slot * plan->ws.t_stage_bytes);
+    // the step that last read this slot must be through with it
+    if (plan->slot_used[slot] && cudaStreamWaitEvent(cs, static_cast<cudaEvent_t>(plan->ev_slot_free[slot]), 0) != cudaSuccess)
+        return FTP_ERR_CUDA;
+    if (cudaMemcpyAsync(xs, x_host, (size_t)plan->N * in.C * in.H * in.W * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaMemcpyAsync(ts, target_host, (size_t)plan->N * out.C * out.H * out.W * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+        cudaEventRecord(static_cast<cudaEvent_t>(plan->ev_prefetch), cs) != cudaSuccess)
+        return FTP_ERR_CUDA;
+    plan->pre_x = x_host; plan->pre_t = target_host; plan->pre_slot = slot;
+    return FTP_OK;
+}
+
 int ftp_step_host(ftp_plan* plan, const float* x_host, const float* target_host, float* params, float lr,
                   float* loss_host, float* dx, void* workspace, void* stream)
 {
@@ -524,28 +564,34 @@ int ftp_step_host(ftp_plan* plan, const float* x_host, const float* target_host,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const MapShape& in = plan->maps.front();
     const MapShape& out = plan->maps.back();
-    float* xs = ws_ptr(workspace, plan->ws.x_stage_off);
-    float* ts = ws_ptr(workspace, plan->ws.t_stage_off);
     float* lv = ws_ptr(workspace, plan->ws.loss_val_off);
-    // The input goes first on the caller's stream; the target is only needed at the loss, so its copy
-    // runs on a side stream (created on first use) while the forward pass computes.
-    if (!plan->copy_stream) {
-        cudaStream_t cs; cudaEvent_t e0, e1;
-        if (cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking) != cudaSuccess ||
-            cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) != cudaSuccess ||
-            cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) != cudaSuccess)
-            return FTP_ERR_CUDA;
-        plan->copy_stream = cs; plan->ev_fork = e0; plan->ev_join = e1;
-    }
-    cudaStream_t cs = static_cast<cudaStream_t>(plan->copy_stream);
-    cudaEvent_t fork = static_cast<cudaEvent_t>(plan->ev_fork), join = static_cast<cudaEvent_t>(plan->ev_join);
-    if (cudaEventRecord(fork, st) != cudaSuccess || cudaStreamWaitEvent(cs, fork, 0) != cudaSuccess ||      // after earlier work on `stream`
-        cudaMemcpyAsync(ts, target_host, (size_t)plan->N * out.C * out.H * out.W * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
-        cudaEventRecord(join, cs) != cudaSuccess ||
-        cudaMemcpyAsync(xs, x_host, (size_t)plan->N * in.C * in.H * in.W * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return FTP_ERR_CUDA;
-    int rc = step_impl(plan, xs, nullptr, ts, params, params, lr, nullptr, lv, dx, workspace, stream, join);
+    int rc = ensure_copy_stream(plan);
     if (rc != FTP_OK) return rc;
+    const bool prefetched = plan->pre_slot >= 0 && plan->pre_x == x_host && plan->pre_t == target_host;
+    const int slot = prefetched ? plan->pre_slot : plan->cur_slot;
+    float* xs = ws_ptr(workspace, plan->ws.x_stage_off + slot * plan->ws.x_stage_bytes);
+    float* ts = ws_ptr(workspace, plan->ws.t_stage_off + slot * plan->ws.t_stage_bytes);
+    if (prefetched) {
+        // the batch is in (or on its way to) the other staging slot: wait for its copies only
+        if (cudaStreamWaitEvent(st, static_cast<cudaEvent_t>(plan->ev_prefetch), 0) != cudaSuccess) return FTP_ERR_CUDA;
+        plan->pre_slot = -1;
+        plan->cur_slot = slot;
+        rc = step_impl(plan, xs, nullptr, ts, params, params, lr, nullptr, lv, dx, workspace, stream);
+    } else {
+        // The input goes first on the caller's stream; the target is only needed at the loss, so its copy
+        // runs on the plan's side stream while the forward pass computes.
+        cudaStream_t cs = static_cast<cudaStream_t>(plan->copy_stream);
+        cudaEvent_t fork = static_cast<cudaEvent_t>(plan->ev_fork), join = static_cast<cudaEvent_t>(plan->ev_join);
+        if (cudaEventRecord(fork, st) != cudaSuccess || cudaStreamWaitEvent(cs, fork, 0) != cudaSuccess ||      // after earlier work on `stream`
+            cudaMemcpyAsync(ts, target_host, (size_t)plan->N * out.C * out.H * out.W * 4, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+            cudaEventRecord(join, cs) != cudaSuccess ||
+            cudaMemcpyAsync(xs, x_host, (size_t)plan->N * in.C * in.H * in.W * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return FTP_ERR_CUDA;
+        rc = step_impl(plan, xs, nullptr, ts, params, params, lr, nullptr, lv, dx, workspace, stream, join);
+    }
+    if (rc != FTP_OK) return rc;
+    if (cudaEventRecord(static_cast<cudaEvent_t>(plan->ev_slot_free[slot]), st) != cudaSuccess) return FTP_ERR_CUDA;
+    plan->slot_used[slot] = true;
     if (loss_host && cudaMemcpyAsync(loss_host, lv, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return FTP_ERR_CUDA;
     return FTP_OK;
 }

@@ -886,8 +886,10 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         p.loss_blocks = (int)std::min<size_t>(1024, (total + 1023) / 1024);
         ws.loss_off = take((size_t)p.loss_blocks * 4);
         ws.loss_val_off = take(4);
-        ws.t_stage_off = take(total * 4);
-        ws.x_stage_off = take((size_t)N * C * H * W * 4);
+        ws.t_stage_bytes = align_up(total * 4, 256);                      // two staging slots each (ftp_prefetch_host)
+        ws.x_stage_bytes = align_up((size_t)N * C * H * W * 4, 256);
+        ws.t_stage_off = take(2 * ws.t_stage_bytes);
+        ws.x_stage_off = take(2 * ws.x_stage_bytes);
     }
     size_t scratch = 0;
     for (const GroupPlan& g : p.groups) scratch = std::max(scratch, g.bwd.scratch_floats);

@@ -120,7 +120,8 @@ struct Workspace {                 // byte offsets, all 256-aligned
     size_t grad_off = 0;           // summed gradient (ftp_step keeps it internal)
     size_t loss_off = 0;           // per-block partial sums of the MSE
     size_t loss_val_off = 0;       // the loss value (ftp_step_host)
-    size_t x_stage_off = 0, t_stage_off = 0;   // device copies of a host batch (ftp_step_host)
+    size_t x_stage_off = 0, t_stage_off = 0;   // device copies of a host batch (ftp_step_host): two slots each, x_stage_bytes / t_stage_bytes apart
+    size_t x_stage_bytes = 0, t_stage_bytes = 0;
     size_t y32_off = 0;            // tensor-core path: fp32 NCHW copy of the last map for the loss (ftp_step with target)
     size_t err_off = 0;            // device error word of the tensor-core kernels (a bounded wait ran out)
     size_t total = 0;
@@ -149,6 +150,11 @@ struct ftp_plan {
     int loss_blocks = 0;
     // ftp_step_host: side stream and events that let the target's host-to-device copy overlap the forward pass
     void* copy_stream = nullptr; void* ev_fork = nullptr; void* ev_join = nullptr;
+    // ftp_prefetch_host: the batch copied ahead of its step into the staging slot the running step does not use
+    void* ev_prefetch = nullptr; void* ev_slot_free[2] = {nullptr, nullptr};
+    bool slot_used[2] = {false, false};
+    int cur_slot = 0, pre_slot = -1;
+    const float* pre_x = nullptr; const float* pre_t = nullptr;
 };
 
 namespace ftp {

@@ -284,3 +284,60 @@ def test_step_can_be_captured_in_a_cuda_graph(precision):
     torch.cuda.synchronize()
     assert torch.equal(p_graph, pd) and l_graph == float(loss.item()) and torch.equal(dx_graph, dx)
     assert not torch.equal(pd, p0)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("precision", [0, 1])
+def test_host_batches_with_and_without_prefetch(precision):
+    """ftp_step_host on four different host batches in a row: copying each batch inside its step,
+    prefetching every batch during the previous step (ftp_prefetch_host), and prefetching on a
+    caller's copy stream all leave bit for bit the parameters and losses of ftp_step on device
+    copies.  A step given other host pointers than the prefetched ones copies as usual, and the
+    prefetched batch is still there for the step after it."""
+    wl = synth.workload("C0").with_(N=2)
+    batches = [synth.draw(wl.with_(seed=s), N=2) for s in range(4)]
+    params = batches[0][1]
+    plan = ftp.ftp_plan(wl.layers, 2, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=precision)
+    ws = plan.new_workspace("cuda")
+    lr = 0.05
+
+    def run(mode):
+        pd = torch.from_numpy(params.copy()).cuda()
+        xs = [torch.from_numpy(b[0]).pin_memory() for b in batches]
+        ts = [torch.from_numpy(b[2]).pin_memory() for b in batches]
+        lh = [torch.zeros(1).pin_memory() for _ in batches]
+        copy_stream = torch.cuda.Stream() if mode == "own-stream" else None
+        losses = []
+        if mode == "device":
+            loss = torch.zeros(1, device="cuda")
+            for x, t in zip(xs, ts):
+                ftp.ftp_step(plan, x.cuda(), pd, lr, ws, target=t.cuda(), loss_out=loss)
+                losses.append(float(loss.item()))
+        elif mode == "plain":
+            for x, t, l in zip(xs, ts, lh):
+                ftp.ftp_step_host(plan, x, t, pd, lr, l, ws)
+        elif mode == "skipped":
+            # batch 1 is prefetched, then batch 0 runs without having been prefetched, then batch 1 finds its copy
+            ftp.ftp_prefetch_host(plan, xs[1], ts[1], ws)
+            ftp.ftp_step_host(plan, xs[0], ts[0], pd, lr, lh[0], ws)
+            ftp.ftp_step_host(plan, xs[1], ts[1], pd, lr, lh[1], ws)
+            for i in (2, 3):
+                ftp.ftp_step_host(plan, xs[i], ts[i], pd, lr, lh[i], ws)
+        else:
+            ftp.ftp_prefetch_host(plan, xs[0], ts[0], ws, copy_stream)
+            for i in range(4):
+                ftp.ftp_step_host(plan, xs[i], ts[i], pd, lr, lh[i], ws)
+                if i + 1 < 4:
+                    ftp.ftp_prefetch_host(plan, xs[i + 1], ts[i + 1], ws, copy_stream)
+        torch.cuda.synchronize()
+        plan.check(ws)
+        if mode != "device":
+            losses = [float(l[0]) for l in lh]
+        return pd.cpu().numpy(), losses
+
+    ref_p, ref_l = run("device")
+    assert len(set(ref_l)) == 4                                  # four different batches
+    for mode in ("plain", "prefetch", "own-stream", "skipped", "prefetch"):
+        p, l = run(mode)
+        assert np.array_equal(p, ref_p), mode
+        assert l == ref_l, mode
