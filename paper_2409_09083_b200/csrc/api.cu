@@ -226,7 +226,7 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
         a.scratch = ws_ptr(ws, p->ws.scratch_off);
         a.partial = ws_ptr(ws, g.partial_off);
         a.set_floats = (long long)g.param_floats;
-        a.splits = g.bwd.splits; a.tiles_x = p->grid_x;
+        
         a.need_dx = (gi > 0 || dx != nullptr) ? 1 : 0;
         { Timed t(p, st, 3, gi);
           const size_t smem = tc_smem(g.bwd.smem_bytes, g.bwd.ctas);
@@ -287,7 +287,7 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
         a.scratch = ws_ptr(ws, p->ws.scratch_off);
         a.partial = ws_ptr(ws, g.partial_off);
         a.param_floats = (long long)g.param_floats;
-        a.splits = g.bwd.splits; a.tiles_x = p->grid_x;
+        
         a.need_dx = (gi > 0 || dx != nullptr) ? 1 : 0;
         { Timed t(p, st, 3, gi);
           bwd_group_kernel<<<g.bwd.blocks, kThreads, g.bwd.smem_bytes, st>>>(a); }

@@ -27,7 +27,7 @@ struct GroupArgs {
     const int *yoff, *xoff, *ytile, *xtile;
     float*       partial;              // [blocks][param_floats] partial gradient sets of this group
     long long    param_floats;
-    int splits, tiles_x, need_dx;
+    int need_dx;
 };
 
 struct HaloSumArgs {
@@ -768,18 +768,17 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_group_kernel(const __grid_con
     unsigned char* smb = smem_raw + kSmemHeader;
     float* sm = reinterpret_cast<float*>(smb);
 
-    const int slot = blockIdx.x, tile = slot / A.splits, split = slot % A.splits;
-    const int ty = tile / A.tiles_x, tx = tile % A.tiles_x;
-    const int rb = A.ytile[ty], kr = A.ytile[ty + 1] - rb;
-    const int qb = A.xtile[tx], kq = A.xtile[tx + 1] - qb;
-    const int items = A.N * kr * kq;
-    const int lo = (int)((long long)split * items / A.splits), hi = (int)((long long)(split + 1) * items / A.splits);
+    // The sub-tile stacks of the whole batch, image by image and row by row, are dealt out evenly to
+    // the blocks; each block adds the filter gradients of its stacks into its own partial set.
+    const int slot = blockIdx.x;
+    const int items = A.N * A.R * A.Q;
+    const int lo = (int)((long long)slot * items / (int)gridDim.x), hi = (int)((long long)(slot + 1) * items / (int)gridDim.x);
     float* myset = A.partial + (size_t)slot * A.param_floats;
     const int nops = A.n_ops;
 
     for (int item = lo; item < hi; ++item) {
         const bool first = item == lo;
-        const int n = item / (kr * kq), r = rb + (item / kq) % kr, q = qb + item % kq;
+        const int n = item / (A.R * A.Q), r = (item / A.Q) % A.R, q = item % A.Q;
         load_header(hdr, A, r, q, false);
         __syncthreads();
 

@@ -37,7 +37,7 @@ struct TcGroupArgs {
     const int *yoff, *xoff, *ytile, *xtile;
     float*       partial;
     long long    set_floats;
-    int splits, tiles_x, need_dx;
+    int need_dx;
 };
 
 namespace tcd {
@@ -587,12 +587,11 @@ __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 2 : 1) bwd_group_tc_
     setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes, tmem_cols, stages);
     int* hdr = H->hdr;
 
-    const int slot = blockIdx.x, tile = slot / A.splits, split = slot % A.splits;
-    const int ty = tile / A.tiles_x, tx = tile % A.tiles_x;
-    const int rb = A.ytile[ty], kr = A.ytile[ty + 1] - rb;
-    const int qb = A.xtile[tx], kq = A.xtile[tx + 1] - qb;
-    const int items = A.N * kr * kq;
-    const int lo = (int)((long long)split * items / A.splits), hi = (int)((long long)(split + 1) * items / A.splits);
+    // The sub-tile stacks of the whole batch, image by image and row by row, are dealt out evenly to
+    // the blocks; each block adds the filter gradients of its stacks into its own partial set.
+    const int slot = blockIdx.x;
+    const int items = A.N * A.R * A.Q;
+    const int lo = (int)((long long)slot * items / (int)gridDim.x), hi = (int)((long long)(slot + 1) * items / (int)gridDim.x);
     float* myset = A.partial + (size_t)slot * A.set_floats;
     const int nops = A.n_ops;
 
@@ -616,7 +615,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 2 : 1) bwd_group_tc_
 
     for (int item = lo; item < hi; ++item) {
         const bool first = item == lo;
-        const int n = item / (kr * kq), r = rb + (item / kq) % kr, q = qb + item % kq;
+        const int n = item / (A.R * A.Q), r = (item / A.Q) % A.R, q = item % A.Q;
         __syncthreads();
         load_header(hdr, A, r, q, false);
         __syncthreads();

@@ -341,7 +341,7 @@ void count_macs(const GroupPlan& g, const PassPlan& pp, double* done, double* un
 // ---- cost terms of one pass of an executed group ----
 // Work on the critical path of one pass: every term is the total over all sub-tile stacks of the
 // pass divided by the number of stacks that run side by side (blocks in flight; in the backward
-// pass the blocks of the busiest user tile decide).  The planner's estimate of the pass time is a
+// pass the busiest block decides).  The planner's estimate of the pass time is a
 // weighted sum of the terms (see kCostWeights).  Terms, fp32 path (multiply-accumulates in units of
 // 1e6, bytes in MB, elements in units of 1e6):
 //   forward : 0 conv MACs, 1 conv+pool MACs, 2 filter MB read, 3 map MB read + written, 4 ops, 5 outputs, 7 one launch
@@ -451,12 +451,7 @@ void pass_cost_terms(const ftp_plan& p, const GroupPlan& g, bool backward, bool 
         const double slots = (double)kSmCount * pp.ctas;
         parallel = items / std::ceil(items / slots);
     } else {
-        int busiest = 1;
-        for (size_t a = 0; a + 1 < ty.tile_begin.size(); ++a)
-            for (size_t b = 0; b + 1 < tx.tile_begin.size(); ++b) {
-                const int it = N * (ty.tile_begin[a + 1] - ty.tile_begin[a]) * (tx.tile_begin[b + 1] - tx.tile_begin[b]);
-                busiest = std::max(busiest, (it + pp.splits - 1) / pp.splits);
-            }
+        const long long busiest = ((long long)items + pp.blocks - 1) / pp.blocks;       // stacks of the busiest block
         parallel = items / busiest;
     }
     for (int k = 0; k < kCostTerms - 1; ++k) f[k] = f[k] * N / parallel;
@@ -470,12 +465,12 @@ void pass_cost_terms(const ftp_plan& p, const GroupPlan& g, bool backward, bool 
 // 0.13-0.23 over the four (precision, pass) fits.
 const double kCostWeights[2][2][kCostTerms] = {
     {   // fp32: forward, backward
-        {6.542, 7.174, 18.76, 163.5, 3.134, 72.57, 0, 9.153},
-        {12.11, 2.713, 1.779, 288.3, 0, 258.7, 37.3, 11.19},
+        {6.444, 7.033, 18.79, 143.4, 5.824, 34.41, 0, 7.93},
+        {10.61, 3.967, 2.645, 274.6, 0, 261.3, 37.98, 5.55},
     },
     {   // bf16
-        {0, 1297, 34.79, 32.73, 3.082, 91.97, 235.4, 8.515},
-        {0.5158, 1.074, 0, 103.9, 22.5, 52.28, 6.621, 17.48},
+        {0, 1360, 34.42, 32.26, 3.056, 91.07, 229.4, 8.708},
+        {0.4465, 1.076, 0, 0, 78.93, 59.32, 6.233, 14.05},
     },
 };
 
@@ -487,24 +482,19 @@ double pass_estimate_us(int precision, bool backward, const double f[kCostTerms]
     return t;
 }
 
-// Backward launch shape: `splits` blocks per user tile, each owning one partial gradient set.
+// Backward launch shape: as many blocks as run at once (or as there are stacks), each owning one
+// partial gradient set; the stacks of the whole batch are dealt out evenly to them.
 void set_backward_blocks(GroupPlan& g, int N, int gy, int gx)
 {
-    int min_items = 1 << 30;
-    for (int ty = 0; ty < gy; ++ty)
-        for (int tx = 0; tx < gx; ++tx) {
-            int items = N * (g.bwd.y.tile_begin[ty + 1] - g.bwd.y.tile_begin[ty]) *
-                        (g.bwd.x.tile_begin[tx + 1] - g.bwd.x.tile_begin[tx]);
-            min_items = std::min(min_items, items);
-        }
-    g.bwd.splits = std::max(1, std::min(min_items, kSmCount * g.bwd.ctas / (gy * gx)));
-    g.bwd.blocks = gy * gx * g.bwd.splits;
+    (void)gy; (void)gx;
+    const long long items = (long long)N * g.bwd.y.count * g.bwd.x.count;
+    g.bwd.blocks = (int)std::max<long long>(1, std::min<long long>(items, (long long)kSmCount * g.bwd.ctas));
 }
 
 // Backward sub-tiling, second step.  choose_subtiles takes the largest sub-tiles that fit; the
-// blocks of a user tile then share its N x (sub-tiles per tile) stacks, and when that number does
-// not divide by the blocks the slowest block runs one stack more than the average.  A somewhat
-// finer split can even that out (8 stacks of 1/8 tile on 4 blocks beat 6 stacks of 1/6).  The
+// blocks then share the N x (sub-tiles of the map) stacks, and when that number does not divide by
+// the blocks the slowest block runs one stack more than the average.  A somewhat finer split can
+// even that out (296 stacks of 1/8 tile on 148 blocks beat 216 stacks of 1/6).  The
 // candidates up to three cuts finer per axis are compared by the time model's estimate of the
 // pass, which counts the stacks of the busiest block; the first split stays unless another is
 // estimated at least 3 % faster.

@@ -82,8 +82,7 @@ struct AxisTables {
 struct PassPlan {
     AxisTables y, x;
     size_t smem_bytes = 0;
-    int blocks = 0;                 // forward: R*Q*N ; backward: tiles * splits
-    int splits = 1;                 // backward: blocks per user tile
+    int blocks = 0;                 // forward: R*Q*N ; backward: min(R*Q*N, blocks that run at once), each with its own partial set
     int dz_ch = 0;                  // backward, fp32 path: channels of the delta staging area (see layout_backward)
     int stages = 2;                 // tensor-core path: stages of the filter ring
     int ctas = 1;                   // tensor-core path: blocks per SM (2 = each block takes half of the tensor memory)
