@@ -31,7 +31,7 @@ UNIT = "images/s"
 FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum of the fused backward kernel per launch (average over the launches of
 # a step), from the ncu captures summarised under profiles/ (workload C1 only; null for anything else)
-NCU_TRAFFIC = {("C1", "fp32"): 65.7e6, ("C1", "bf16"): 29.2e6}
+NCU_TRAFFIC = {("C1", "fp32"): 65.7e6, ("C1", "bf16"): 30.5e6}
 KIND = {0: "pack_filters", 1: "fwd_group", 2: "loss_delta", 3: "bwd_group", 4: "halo_sum", 5: "reduce_sgd"}
 
 
