@@ -17,14 +17,25 @@ namespace {
 
 inline float* ws_ptr(void* ws, size_t off) { return reinterpret_cast<float*>(static_cast<unsigned char*>(ws) + off); }
 
+// Largest conv window of an executed group (selects the kernel instantiation of the fp32 path).
+int max_window(const GroupPlan& g)
+{
+    int k = 1;
+    for (int i = 0; i < g.n_ops; ++i)
+        if (g.fwd_ops[i].kind != kOpPool) k = std::max(k, g.fwd_ops[i].k);
+    return k;
+}
+
 int ensure_device(ftp_plan* p)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return FTP_ERR_CUDA;
     if (p->dev_tables && p->dev_id == dev) return FTP_OK;
     if (p->dev_tables) { cudaFree(p->dev_tables); p->dev_tables = nullptr; }
-    if (cudaFuncSetAttribute(fwd_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(bwd_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
+    if (cudaFuncSetAttribute(fwd_group_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(fwd_group_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(bwd_group_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(bwd_group_kernel<7>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(fwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(fwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
@@ -201,7 +212,8 @@ int forward_impl(ftp_plan* p, const float* x, const float* params, float* y, voi
         GroupArgs a;
         fill_common(p, g, false, x, params, ws, a);
         { Timed t(p, st, 1, (int)gi);
-          fwd_group_kernel<<<dim3(a.R * a.Q, p->N), kThreads, g.fwd.smem_bytes, st>>>(a); }
+          if (max_window(g) <= 3) fwd_group_kernel<3><<<dim3(a.R * a.Q, p->N), kThreads, g.fwd.smem_bytes, st>>>(a);
+          else fwd_group_kernel<7><<<dim3(a.R * a.Q, p->N), kThreads, g.fwd.smem_bytes, st>>>(a); }
         if (!launched_ok()) return FTP_ERR_CUDA;
     }
     if (y) {
@@ -290,7 +302,8 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
         
         a.need_dx = (gi > 0 || dx != nullptr) ? 1 : 0;
         { Timed t(p, st, 3, gi);
-          bwd_group_kernel<<<g.bwd.blocks, kThreads, g.bwd.smem_bytes, st>>>(a); }
+          if (max_window(g) <= 3) bwd_group_kernel<3><<<g.bwd.blocks, kThreads, g.bwd.smem_bytes, st>>>(a);
+          else bwd_group_kernel<7><<<g.bwd.blocks, kThreads, g.bwd.smem_bytes, st>>>(a); }
         if (!launched_ok()) return FTP_ERR_CUDA;
         if (a.need_dx) {
             const MapShape& s = p->maps[g.first - 1];

@@ -403,7 +403,7 @@ __device__ __forceinline__ void delta_conv_staged(const float* __restrict__ D, c
     }
 }
 
-template <class Epilogue>
+template <int KMAX, class Epilogue>
 __device__ __forceinline__ void delta_conv_staged_k(int K, const float* D, const unsigned char* Darg, int d_cs, int d_pitch,
                                                     int zh, int zw, int vy0, int vx0, float* stage, int CH, const float* w,
                                                     int nd, int cin_pad, int cin, int ih, int iw, float* wst, Epilogue epi)
@@ -414,21 +414,23 @@ __device__ __forceinline__ void delta_conv_staged_k(int K, const float* D, const
         switch (K) {
         case 1: FTP_DELTA_CONV(1, true); break;
         case 3: FTP_DELTA_CONV(3, true); break;
-        case 5: FTP_DELTA_CONV(5, true); break;
-        default: FTP_DELTA_CONV(7, true); break;
+        default:
+            if constexpr (KMAX > 3) { if (K == 5) FTP_DELTA_CONV(5, true); else FTP_DELTA_CONV(7, true); }
+            break;
         }
     } else {
         switch (K) {
         case 1: FTP_DELTA_CONV(1, false); break;
         case 3: FTP_DELTA_CONV(3, false); break;
-        case 5: FTP_DELTA_CONV(5, false); break;
-        default: FTP_DELTA_CONV(7, false); break;
+        default:
+            if constexpr (KMAX > 3) { if (K == 5) FTP_DELTA_CONV(5, false); else FTP_DELTA_CONV(7, false); }
+            break;
         }
     }
 #undef FTP_DELTA_CONV
 }
 
-template <bool POOL_OUT, int MODE, class Epilogue>
+template <int KMAX, bool POOL_OUT, int MODE, class Epilogue>
 __device__ __forceinline__ void conv_tile_k(int K, const float* in, const unsigned char* arg, int in_cs, int in_pitch,
                                             int in_rows, int in_cols, int y_base, int x_base, const float* w, int cin,
                                             int cout_pad, const float* bias, int cout, float slope, int oh, int ow,
@@ -440,15 +442,17 @@ __device__ __forceinline__ void conv_tile_k(int K, const float* in, const unsign
         switch (K) {
         case 1: FTP_CONV_TILE(1, true); break;
         case 3: FTP_CONV_TILE(3, true); break;
-        case 5: FTP_CONV_TILE(5, true); break;
-        default: FTP_CONV_TILE(7, true); break;
+        default:
+            if constexpr (KMAX > 3) { if (K == 5) FTP_CONV_TILE(5, true); else FTP_CONV_TILE(7, true); }
+            break;
         }
     } else {
         switch (K) {
         case 1: FTP_CONV_TILE(1, false); break;
         case 3: FTP_CONV_TILE(3, false); break;
-        case 5: FTP_CONV_TILE(5, false); break;
-        default: FTP_CONV_TILE(7, false); break;
+        default:
+            if constexpr (KMAX > 3) { if (K == 5) FTP_CONV_TILE(5, false); else FTP_CONV_TILE(7, false); }
+            break;
         }
     }
 #undef FTP_CONV_TILE
@@ -637,7 +641,7 @@ __device__ __forceinline__ void filter_grad_thread(const float* __restrict__ d, 
     }
 }
 
-template <bool POOLED>
+template <int KMAX, bool POOLED>
 __device__ __forceinline__ void filter_grad_k(int K, const float* d, const unsigned char* arg, int d_cs, int d_pitch,
                                               const float* xin, int in_cs, int in_pitch, int cin, int cout, int oh,
                                               int ow, float* g, bool first)
@@ -658,8 +662,12 @@ __device__ __forceinline__ void filter_grad_k(int K, const float* d, const unsig
     switch (K) {
     case 1: filter_grad_tile<1, 4, 8, POOLED>(d, arg, d_cs, d_pitch, xin, in_cs, in_pitch, cin, cout, oh, ow, g, first); break;
     case 3: filter_grad_tile<3, 4, 2, POOLED>(d, arg, d_cs, d_pitch, xin, in_cs, in_pitch, cin, cout, oh, ow, g, first); break;
-    case 5: filter_grad_tile<5, 2, 1, POOLED>(d, arg, d_cs, d_pitch, xin, in_cs, in_pitch, cin, cout, oh, ow, g, first); break;
-    default: filter_grad_tile<7, 1, 1, POOLED>(d, arg, d_cs, d_pitch, xin, in_cs, in_pitch, cin, cout, oh, ow, g, first); break;
+    default:
+        if constexpr (KMAX > 3) {
+            if (K == 5) filter_grad_tile<5, 2, 1, POOLED>(d, arg, d_cs, d_pitch, xin, in_cs, in_pitch, cin, cout, oh, ow, g, first);
+            else filter_grad_tile<7, 1, 1, POOLED>(d, arg, d_cs, d_pitch, xin, in_cs, in_pitch, cin, cout, oh, ow, g, first);
+        }
+        break;
     }
 }
 
@@ -681,6 +689,8 @@ __device__ __forceinline__ void bias_grad_tile(const float* __restrict__ d, int 
 // ---------------------------------------------------------------------------------------------
 // Fused forward of one group: grid (R*Q, N), one sub-tile stack per block.
 // ---------------------------------------------------------------------------------------------
+// KMAX: largest conv window of the group (3: the 5x5 / 7x7 code paths are left out, which frees registers of the common ones).
+template <int KMAX>
 __global__ void __launch_bounds__(kThreads, 1) fwd_group_kernel(const __grid_constant__ GroupArgs A)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -744,12 +754,12 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_group_kernel(const __grid_con
             const float slope = op.slope;
             const float* bias = A.params + op.p_off + (size_t)op.cout * op.cin * op.k * op.k;
             if (op.kind == kOpConv)
-                conv_tile_k<false, kInPlain>(op.k, ib, nullptr, op.in_cs, op.in_pitch, oh + op.k - 1, 0, 0, 0,
+                conv_tile_k<KMAX, false, kInPlain>(op.k, ib, nullptr, op.in_cs, op.in_pitch, oh + op.k - 1, 0, 0, 0,
                                              A.wpk + op.wf_off, op.cin, op.cout_pad, bias, op.cout, slope, oh, ow,
                                              sm + op.w_off, op.w_ch,
                                              [&](int c, int ly, int lx, float z, int) { emit(c, ly, lx, leaky(z, slope), 0); });
             else
-                conv_tile_k<true, kInPlain>(op.k, ib, nullptr, op.in_cs, op.in_pitch, 2 * oh + op.k - 1, 0, 0, 0,
+                conv_tile_k<KMAX, true, kInPlain>(op.k, ib, nullptr, op.in_cs, op.in_pitch, 2 * oh + op.k - 1, 0, 0, 0,
                                             A.wpk + op.wf_off, op.cin, op.cout_pad, bias, op.cout, slope, 2 * oh, 2 * ow,
                                             sm + op.w_off, op.w_ch, emit);
         }
@@ -761,6 +771,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_group_kernel(const __grid_con
 // Fused backward of one group (adjoint form): each block owns one partial gradient set and walks
 // through its share of the (image, sub-tile) stacks of one user tile in a fixed order.
 // ---------------------------------------------------------------------------------------------
+template <int KMAX>
 __global__ void __launch_bounds__(kThreads, 1) bwd_group_kernel(const __grid_constant__ GroupArgs A)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -854,23 +865,23 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_group_kernel(const __grid_con
                 // input delta = correlation of the zero-extended output delta with the rotated filter:
                 // position u of the X buffer reads delta rows u + ky' - (K-1)
                 if (op.kind == kOpConv) {
-                    filter_grad_k<false>(op.k, D, nullptr, op.d_cs, op.d_pitch, X, op.in_cs, op.in_pitch, op.cin, op.cout,
+                    filter_grad_k<KMAX, false>(op.k, D, nullptr, op.d_cs, op.d_pitch, X, op.in_cs, op.in_pitch, op.cin, op.cout,
                                          oh, ow, gw, first);
                     bias_grad_tile(D, op.d_cs, op.d_pitch, op.cout, oh, ow, gw + (size_t)op.cout * op.cin * op.k * op.k, first);
                     if (need_in_delta)
-                        conv_tile_k<false, kInChecked>(op.k, D, nullptr, op.d_cs, op.d_pitch, oh, ow, vy0 - (op.k - 1),
+                        conv_tile_k<KMAX, false, kInChecked>(op.k, D, nullptr, op.d_cs, op.d_pitch, oh, ow, vy0 - (op.k - 1),
                                                        vx0 - (op.k - 1), A.wpk + op.wb_off, op.cout, op.cin_pad, nullptr,
                                                        op.cin, 0.f, ih, iw, sm + op.w_off, op.w_ch, put);
                 } else {
-                    filter_grad_k<true>(op.k, D, Darg, op.d_cs, op.d_pitch, X, op.in_cs, op.in_pitch, op.cin, op.cout,
+                    filter_grad_k<KMAX, true>(op.k, D, Darg, op.d_cs, op.d_pitch, X, op.in_cs, op.in_pitch, op.cin, op.cout,
                                         oh, ow, gw, first);
                     bias_grad_tile(D, op.d_cs, op.d_pitch, op.cout, oh, ow, gw + (size_t)op.cout * op.cin * op.k * op.k, first);
                     if (need_in_delta && op.dz_ch > 0)
-                        delta_conv_staged_k(op.k, D, Darg, op.d_cs, op.d_pitch, 2 * oh, 2 * ow, vy0, vx0, sm + op.dz_off, op.dz_ch,
+                        delta_conv_staged_k<KMAX>(op.k, D, Darg, op.d_cs, op.d_pitch, 2 * oh, 2 * ow, vy0, vx0, sm + op.dz_off, op.dz_ch,
                                             A.wpk + op.wb_off, op.cout, op.cin_pad, op.cin, ih, iw,
                                             op.w_ch > 0 ? sm + op.w_off : nullptr, put);
                     else if (need_in_delta)   // the pooled delta is expanded through the arg-max on the fly
-                        conv_tile_k<false, kInExpand>(op.k, D, Darg, op.d_cs, op.d_pitch, 2 * oh, 2 * ow, vy0 - (op.k - 1),
+                        conv_tile_k<KMAX, false, kInExpand>(op.k, D, Darg, op.d_cs, op.d_pitch, 2 * oh, 2 * ow, vy0 - (op.k - 1),
                                                       vx0 - (op.k - 1), A.wpk + op.wb_off, op.cout, op.cin_pad, nullptr,
                                                       op.cin, 0.f, ih, iw, nullptr, 0, put);
                 }
