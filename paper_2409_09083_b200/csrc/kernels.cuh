@@ -932,8 +932,8 @@ __global__ void halo_sum_kernel(const __grid_constant__ HaloSumArgs A)
     for (long long row = (long long)blockIdx.x * wpb + (threadIdx.x >> 5); row < rows; row += (long long)gridDim.x * wpb) {
         const int y = (int)(row % A.H); long long t = row / A.H;
         const int c = (int)(t % A.C); const int n = (int)(t / A.C);
-        const int r0 = ycover[2 * y], nr = min(ycover[2 * y + 1] - r0 + 1, 4);
-        int base[4], ch[4], dr[4];
+        const int r0 = ycover[2 * y], nr = ycover[2 * y + 1] - r0 + 1;
+        int base[4], ch[4], dr[4];       // the first four covering sub-tile rows (more only with very fine splits)
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const int r = min(r0 + k, A.R - 1);
@@ -952,6 +952,13 @@ __global__ void halo_sum_kernel(const __grid_constant__ HaloSumArgs A)
                         const int x1 = xspan[2 * q], w = xspan[2 * q + 1] - x1 + 1;
                         s += img[base[k] + xoff[q] * ch[k] + dr[k] * w + (x - x1)];
                     }
+            for (int k = 4; k < nr; ++k) {                 // same order, offsets worked out on the spot
+                const int r = r0 + k, y1 = yspan[2 * r], h = yspan[2 * r + 1] - y1 + 1;
+                for (int q = q0; q <= q1; ++q) {
+                    const int x1 = xspan[2 * q], w = xspan[2 * q + 1] - x1 + 1;
+                    s += img[A.C * yoff[r] * A.Wtot + xoff[q] * (A.C * h) + (c * h + (y - y1)) * w + (x - x1)];
+                }
+            }
             orow[x] = s;
         }
     }

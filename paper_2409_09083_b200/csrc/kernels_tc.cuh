@@ -782,7 +782,7 @@ __global__ void halo_sum_planes_kernel(const __grid_constant__ HaloSumArgs A)
     for (long long row = (long long)blockIdx.x * wpb + (threadIdx.x >> 5); row < rows; row += (long long)gridDim.x * wpb) {
         const int y = (int)(row % A.H); long long t = row / A.H;
         const int pl = (int)(t % planes); const int n = (int)(t / planes);
-        const int r0 = ycover[2 * y], nr = min(ycover[2 * y + 1] - r0 + 1, 4);
+        const int r0 = ycover[2 * y], nr = ycover[2 * y + 1] - r0 + 1;       // the first four covering rows are prepared, the rest walked
         int base[4], ch[4], dr[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -803,6 +803,16 @@ __global__ void halo_sum_planes_kernel(const __grid_constant__ HaloSumArgs A)
                         const float4 a = e[0], b = e[1];
                         s[0] += a.x; s[1] += a.y; s[2] += a.z; s[3] += a.w; s[4] += b.x; s[5] += b.y; s[6] += b.z; s[7] += b.w;
                     }
+            for (int k = 4; k < nr; ++k) {                 // very fine splits: same order, offsets worked out on the spot
+                const int r = r0 + k, y1 = yspan[2 * r], h = yspan[2 * r + 1] - y1 + 1;
+                for (int q = q0; q <= q1; ++q) {
+                    const int x1 = xspan[2 * q], w = xspan[2 * q + 1] - x1 + 1;
+                    const float4* e = reinterpret_cast<const float4*>(img + A.C * yoff[r] * A.Wtot + xoff[q] * (A.C * h) +
+                                                                      ((pl * h + (y - y1)) * w + (x - x1)) * 8);
+                    const float4 a = e[0], b = e[1];
+                    s[0] += a.x; s[1] += a.y; s[2] += a.z; s[3] += a.w; s[4] += b.x; s[5] += b.y; s[6] += b.z; s[7] += b.w;
+                }
+            }
             out[row * A.W + x] = tcd::pack8(s);
         }
     }

@@ -341,3 +341,41 @@ def test_host_batches_with_and_without_prefetch(precision):
         p, l = run(mode)
         assert np.array_equal(p, ref_p), mode
         assert l == ref_l, mode
+
+
+def _random_workload(rng):
+    """A small random stack of conv (1x1 / 3x3 / 5x5, 1-40 channels) and pool layers with a random
+    batch, extent, tile grid and grouping profile."""
+    layers, c = [], int(rng.integers(1, 6))
+    cin0, h, w = c, int(rng.integers(3, 9)) * 4, int(rng.integers(3, 9)) * 4
+    hh, ww = h, w
+    for _ in range(int(rng.integers(1, 5))):
+        if layers and layers[-1].kind == "conv" and hh % 2 == 0 and ww % 2 == 0 and min(hh, ww) >= 8 and rng.random() < 0.5:
+            layers.append(pool()); hh //= 2; ww //= 2
+        else:
+            co = int(rng.choice([1, 3, 8, 13, 24, 40]))
+            layers.append(conv(c, co, int(rng.choice([1, 3, 3, 3, 5])))); c = co
+    cuts = sorted(set(int(v) for v in rng.integers(1, len(layers) + 1, size=2)) | {len(layers)})
+    groups, a = [], 1
+    for b in cuts:
+        groups.append((a, b)); a = b + 1
+    grid = (int(rng.integers(1, min(4, hh) + 1)), int(rng.integers(1, min(4, ww) + 1)))
+    return W("rnd", tuple(layers), int(rng.integers(1, 4)), cin0, h, w, grid, tuple(groups), x_dist="normal")
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", range(24))
+def test_random_small_stacks_match_oracle(seed):
+    """Random layer stacks, shapes, grids and profiles under the planner's defaults (time-model cuts,
+    refined backward split, staged filters and deltas) and, every third case, with forced sub-tiling.
+    Dyadic values and slope 0.5 as in the mid-size cases: the forward is exact in fp32, so both sides
+    take the same leaky-ReLU and arg-max decisions (ties included: first maximum in window order)."""
+    rng = np.random.default_rng(1000 + seed)
+    wl = synth.with_slope(_random_workload(rng), 0.5)
+    opts = dict(max_subtile=int(rng.integers(2, 6))) if seed % 3 == 2 else {}
+    x, params, target = synth.draw_dyadic(wl, nnz=3)
+    ref = run_oracle(wl, x, params, target=target)
+    got = run_gpu(wl, x, params, target=target, **opts)
+    assert np.array_equal(got["y"].astype(np.float64), ref["y"]), wl
+    assert rel_err(got["dx"], ref["dx"]) <= FP32_TOL, wl
+    assert rel_err(got["dparams"], ref["dparams"]) <= FP32_TOL, wl
