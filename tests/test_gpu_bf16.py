@@ -300,3 +300,43 @@ def test_step_updates_parameters_like_the_oracle(name):
     plan.check(ws)
     assert np.array_equal(pd2.cpu().numpy(), new)
     assert float(lh[0]) == loss.item()
+
+
+def _random_workload(rng):
+    """A small random stack of conv (1x1 / 3x3 / 5x5, 1-40 channels) and pool layers with a random
+    batch, extent, tile grid and grouping profile (the generator of the fp32 random cases)."""
+    layers, c = [], int(rng.integers(1, 6))
+    cin0, h, w = c, int(rng.integers(3, 9)) * 4, int(rng.integers(3, 9)) * 4
+    hh, ww = h, w
+    for _ in range(int(rng.integers(1, 5))):
+        if layers and layers[-1].kind == "conv" and hh % 2 == 0 and ww % 2 == 0 and min(hh, ww) >= 8 and rng.random() < 0.5:
+            layers.append(pool()); hh //= 2; ww //= 2
+        else:
+            co = int(rng.choice([1, 3, 8, 13, 24, 40]))
+            layers.append(conv(c, co, int(rng.choice([1, 3, 3, 3, 5])))); c = co
+    cuts = sorted(set(int(v) for v in rng.integers(1, len(layers) + 1, size=2)) | {len(layers)})
+    groups, a = [], 1
+    for b in cuts:
+        groups.append((a, b)); a = b + 1
+    grid = (int(rng.integers(1, min(4, hh) + 1)), int(rng.integers(1, min(4, ww) + 1)))
+    return W("rnd", tuple(layers), int(rng.integers(1, 4)), cin0, h, w, grid, tuple(groups), x_dist="normal")
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_small_stacks_match_oracle(seed):
+    """Random shallow stacks, shapes, grids and profiles under the planner's defaults and, every third
+    case, with forced sub-tiling.  Stored values within one bf16 step of the oracle's; gradients in
+    the L2 norm (a rare arg-max or sign decision next to a rounding boundary may fall the other way,
+    which moves a delta to another pixel; see test_backward_matches_oracle)."""
+    rng = np.random.default_rng(1000 + seed)
+    wl = _random_workload(rng)
+    opts = dict(max_subtile=int(rng.integers(2, 6))) if seed % 3 == 2 else {}
+    x, params, target = synth.draw(wl, bias_std=0.3)
+    x, params = bf16_grid(x), bf16_grid(params)
+    c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    dy = np.random.default_rng(3).standard_normal((wl.N, c, h, w)).astype(np.float32)
+    ref = run_oracle(wl, x, params, dy=dy, store="bf16")
+    y, dx, dparams, plan = backward_bf16(wl, x, params, dy, **opts)
+    assert rel_err(y, ref["y"]) <= 1e-2, wl
+    assert l2_err(dx, ref["dx"]) <= 5e-2, wl
+    assert l2_err(dparams, ref["dparams"]) <= BF16_TOL, wl
