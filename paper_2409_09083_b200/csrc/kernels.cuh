@@ -677,9 +677,17 @@ __device__ __forceinline__ void bias_grad_tile(const float* __restrict__ d, int 
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const int npix = oh * ow;
+    // pixel p = lane, lane + 32, ... in row-major order; its (row, column) is stepped, not divided out
+    const int y0 = lane / ow, x0 = lane - y0 * ow, dy = 32 / ow, dx = 32 - dy * ow;
     for (int co = warp; co < cout; co += nwarps) {
+        const float* dc = d + co * d_cs;
         float s = 0.f;
-        for (int p = lane; p < npix; p += 32) s += d[co * d_cs + (p / ow) * d_pitch + p % ow];
+        int y = y0, x = x0;
+        for (int p = lane; p < npix; p += 32) {
+            s += dc[y * d_pitch + x];
+            x += dx; y += dy;
+            if (x >= ow) { x -= ow; ++y; }
+        }
 #pragma unroll
         for (int k = 16; k >= 1; k >>= 1) s += __shfl_xor_sync(0xffffffffu, s, k);
         if (lane == 0) gb[co] = first ? s : gb[co] + s;
