@@ -8,8 +8,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libftp.so")
 SOURCES = [os.path.join(CSRC, "api.cu"), os.path.join(CSRC, "noalloc.cu"), os.path.join(CSRC, "plan.cpp")]
-HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(CSRC, "plan.hpp"),
-           os.path.join(ROOT, "include", "ftp.h")]
+HEADERS = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".hpp", ".h"))) + \
+          [os.path.join(ROOT, "include", "ftp.h")]
 
 
 def _nvcc() -> str:
