@@ -269,7 +269,7 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
     auto flush = [&]() {
         if (!ra.n) return;
         Timed t(p, st, 5, -1);
-        reduce_sgd_tc_kernel<<<dim3(296, ra.n), 128, 0, st>>>(ra, sgd_params, lr, grad_out);
+        reduce_sgd_tc_kernel<<<dim3(1184, ra.n), 128, 0, st>>>(ra, sgd_params, lr, grad_out);
         ra.n = 0;
     };
     for (const GroupPlan& g : p->groups)

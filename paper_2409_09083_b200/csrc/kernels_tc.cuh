@@ -845,7 +845,7 @@ __global__ void reduce_sgd_tc_kernel(const __grid_constant__ TcReduceArgs A, flo
         }
         const float* src = L.partial + L.tgp_off + e;
         float s = 0.f;
-#pragma unroll 8
+#pragma unroll 16
         for (int k = 0; k < L.sets; ++k) s += src[(size_t)k * L.set_floats];
         if (grad_out) grad_out[dst] = s;
         if (params) params[dst] = params[dst] - lr * s;
