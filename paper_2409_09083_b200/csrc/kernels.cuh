@@ -953,13 +953,22 @@ __global__ void halo_sum_kernel(const __grid_constant__ HaloSumArgs A)
         for (int x = lane; x < A.W; x += 32) {
             const int q0 = xcover[2 * x], q1 = xcover[2 * x + 1];
             float s = 0.f;
+            // the first two covering sub-tile columns are handled without a loop, so that the loads of
+            // up to 4 x 2 blocks are in flight together (same order of the sums as the plain loops)
+            const int qb = min(q0 + 1, A.Q - 1);
+            const int xa1 = xspan[2 * q0], wa = xspan[2 * q0 + 1] - xa1 + 1, oa = xoff[q0];
+            const int xb1 = xspan[2 * qb], wb = xspan[2 * qb + 1] - xb1 + 1, ob = xoff[qb];
+            const bool two = q1 > q0;
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-                if (k < nr)
-                    for (int q = q0; q <= q1; ++q) {
+                if (k < nr) {
+                    s += img[base[k] + oa * ch[k] + dr[k] * wa + (x - xa1)];
+                    if (two) s += img[base[k] + ob * ch[k] + dr[k] * wb + (x - xb1)];
+                    for (int q = q0 + 2; q <= q1; ++q) {
                         const int x1 = xspan[2 * q], w = xspan[2 * q + 1] - x1 + 1;
                         s += img[base[k] + xoff[q] * ch[k] + dr[k] * w + (x - x1)];
                     }
+                }
             for (int k = 4; k < nr; ++k) {                 // same order, offsets worked out on the spot
                 const int r = r0 + k, y1 = yspan[2 * r], h = yspan[2 * r + 1] - y1 + 1;
                 for (int q = q0; q <= q1; ++q) {
