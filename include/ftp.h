@@ -68,9 +68,9 @@ typedef struct {
 } ftp_layer;
 
 /* A group as an inclusive 1-based layer range.  The paper's tuple (s, e)
- * "starting at the input to layer s and ending at the input to layer e"
- * (Section 4.2) is (first, last + 1).  Boundary data is exchanged only at the
- * input map of `first`. */
+ * spans the maps from the input of layer s to the input of layer e
+ * (Section 4.2); here that is (first, last + 1).  Boundary data is exchanged
+ * only at the input map of `first`. */
 typedef struct { int first, last; } ftp_group;
 
 typedef struct ftp_plan ftp_plan;   /* opaque, host-owned */

@@ -124,6 +124,53 @@ def _ptr(t, name, allow_none=False):
     return t.data_ptr()
 
 
+def _sized(*specs):
+    """Device pointers of tensors given as (tensor, name, element count[, allow_none]) after checking
+    that each holds exactly that many elements: the kernels index by the plan's shapes, so a tensor
+    of another size would be read or written out of bounds.  All sizes are checked before any
+    pointer is taken."""
+    for spec in specs:
+        t, name, count = spec[:3]
+        if t is not None and t.numel() != count:
+            raise ValueError(f"{name} has {t.numel()} elements, the plan needs {count}")
+    return [_ptr(spec[0], spec[1], len(spec) > 3 and spec[3]) for spec in specs]
+
+
+class _Ws:
+    """A workspace whose size has been checked; `.ptr` adds the device check, after the other arguments' sizes."""
+
+    def __init__(self, plan, workspace):
+        if workspace is None or not hasattr(workspace, "data_ptr"):
+            raise ValueError("workspace must be a CUDA tensor of at least plan.workspace_bytes bytes")
+        have = workspace.numel() * workspace.element_size()
+        if have < plan.workspace_bytes:
+            raise ValueError(f"workspace holds {have} bytes, the plan needs {plan.workspace_bytes}")
+        self.t = workspace
+
+    @property
+    def ptr(self):
+        if not self.t.is_cuda or not self.t.is_contiguous():
+            raise ValueError("workspace must be a contiguous CUDA tensor")
+        return self.t.data_ptr()
+
+
+def _workspace(plan, workspace):
+    return _Ws(plan, workspace)
+
+
+def _host(*specs):
+    """Host pointers of (tensor, name, element count) triples: sizes first, then layout."""
+    for t, name, count in specs:
+        if t is None:
+            raise ValueError(f"{name} must not be None")
+        if t.numel() != count:
+            raise ValueError(f"{name} has {t.numel()} elements, the plan needs {count}")
+    for t, name, _ in specs:
+        if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous float32 CPU tensor")
+    return [t.data_ptr() for t, _, _ in specs]
+
+
 def _stream(stream):
     if stream is None:
         return torch.cuda.current_stream().cuda_stream
@@ -162,6 +209,7 @@ class Plan:
         _check(_lib.ftp_plan_sizes(self._h, ctypes.byref(pf), ctypes.byref(wb), ctypes.byref(of),
                                    ctypes.byref(red)))
         self.param_floats, self.workspace_bytes, self.out_floats = pf.value, wb.value, of.value
+        self.in_floats = N * C * H * W
         self.redundancy = red.value
 
     def __del__(self):
@@ -219,7 +267,7 @@ class Plan:
 
     def check(self, workspace, stream=None):
         """Synchronise and raise FtpError(FTP_ERR_TIMEOUT) if a device-side wait of the bf16 path ran out."""
-        _check(_lib.ftp_plan_check(self._h, workspace.data_ptr(), _stream(stream)))
+        _check(_lib.ftp_plan_check(self._h, _workspace(self, workspace).ptr, _stream(stream)))
 
     def new_workspace(self, device="cuda"):
         return torch.empty(self.workspace_bytes, dtype=torch.uint8, device=device)
@@ -230,60 +278,73 @@ def ftp_plan(layers, N, C, H, W, tile_grid, groups, precision=FTP_FP32, **opts) 
 
 
 def ftp_forward(plan, x, params, y, workspace, stream=None):
-    _check(_lib.ftp_forward(plan._h, _ptr(x, "x"), _ptr(params, "params"), _ptr(y, "y", True),
-                            workspace.data_ptr(), _stream(stream)))
+    ws = _workspace(plan, workspace)
+    px, pp, py = _sized((x, "x", plan.in_floats), (params, "params", plan.param_floats), (y, "y", plan.out_floats, True))
+    _check(_lib.ftp_forward(plan._h, px, pp, py, ws.ptr, _stream(stream)))
 
 
 def ftp_backward(plan, x, dy, params, dx, dparams, workspace, stream=None):
-    _check(_lib.ftp_backward(plan._h, _ptr(x, "x"), _ptr(dy, "dy"), _ptr(params, "params"),
-                             _ptr(dx, "dx", True), _ptr(dparams, "dparams"), workspace.data_ptr(),
-                             _stream(stream)))
+    ws = _workspace(plan, workspace)
+    px, pdy, pp, pdx, pg = _sized((x, "x", plan.in_floats), (dy, "dy", plan.out_floats),
+                                  (params, "params", plan.param_floats), (dx, "dx", plan.in_floats, True),
+                                  (dparams, "dparams", plan.param_floats))
+    _check(_lib.ftp_backward(plan._h, px, pdy, pp, pdx, pg, ws.ptr, _stream(stream)))
 
 
 def ftp_step(plan, x, params, lr, workspace, dy=None, target=None, loss_out=None, dx=None, stream=None):
-    _check(_lib.ftp_step(plan._h, _ptr(x, "x"), _ptr(dy, "dy", True), _ptr(target, "target", True),
-                         _ptr(params, "params"), float(lr), _ptr(loss_out, "loss_out", True),
-                         _ptr(dx, "dx", True), workspace.data_ptr(), _stream(stream)))
+    ws = _workspace(plan, workspace)
+    px, pdy, pt, pp, pl, pdx = _sized((x, "x", plan.in_floats), (dy, "dy", plan.out_floats, True),
+                                      (target, "target", plan.out_floats, True), (params, "params", plan.param_floats),
+                                      (loss_out, "loss_out", 1, True), (dx, "dx", plan.in_floats, True))
+    _check(_lib.ftp_step(plan._h, px, pdy, pt, pp, float(lr), pl, pdx, ws.ptr, _stream(stream)))
 
 
 def ftp_step_grad(plan, x, params, dparams, workspace, dy=None, target=None, loss_out=None, dx=None, stream=None):
-    _check(_lib.ftp_step_grad(plan._h, _ptr(x, "x"), _ptr(dy, "dy", True), _ptr(target, "target", True),
-                              _ptr(params, "params"), _ptr(dparams, "dparams"), _ptr(loss_out, "loss_out", True),
-                              _ptr(dx, "dx", True), workspace.data_ptr(), _stream(stream)))
+    ws = _workspace(plan, workspace)
+    px, pdy, pt, pp, pg, pl, pdx = _sized((x, "x", plan.in_floats), (dy, "dy", plan.out_floats, True),
+                                          (target, "target", plan.out_floats, True),
+                                          (params, "params", plan.param_floats), (dparams, "dparams", plan.param_floats),
+                                          (loss_out, "loss_out", 1, True), (dx, "dx", plan.in_floats, True))
+    _check(_lib.ftp_step_grad(plan._h, px, pdy, pt, pp, pg, pl, pdx, ws.ptr, _stream(stream)))
 
 
 def ftp_loss_mse(plan, y, target, dy, loss_out, workspace, stream=None):
-    _check(_lib.ftp_loss_mse(plan._h, _ptr(y, "y"), _ptr(target, "target"), _ptr(dy, "dy", True),
-                             _ptr(loss_out, "loss_out", True), workspace.data_ptr(), _stream(stream)))
+    ws = _workspace(plan, workspace)
+    py, pt, pdy, pl = _sized((y, "y", plan.out_floats), (target, "target", plan.out_floats),
+                             (dy, "dy", plan.out_floats, True), (loss_out, "loss_out", 1, True))
+    _check(_lib.ftp_loss_mse(plan._h, py, pt, pdy, pl, ws.ptr, _stream(stream)))
 
 
 def ftp_loss_mse_static(y, target, dy, loss_out, stream=None):
     """MSE loss and delta without a plan, a workspace or any device allocation (see ftp.h)."""
-    if target.numel() != y.numel():
-        raise ValueError("y and target must have the same number of elements")
-    _check(_lib.ftp_loss_mse_static(_ptr(y, "y"), _ptr(target, "target"), _ptr(dy, "dy", True),
-                                    _ptr(loss_out, "loss_out", True), y.numel(), _stream(stream)))
+    if y is None or target is None:
+        raise ValueError("y and target must not be None")
+    py, pt, pdy, pl = _sized((y, "y", y.numel()), (target, "target", y.numel()), (dy, "dy", y.numel(), True),
+                             (loss_out, "loss_out", 1, True))
+    _check(_lib.ftp_loss_mse_static(py, pt, pdy, pl, y.numel(), _stream(stream)))
 
 
 def ftp_sgd(params, grad, lr, stream=None):
-    _check(_lib.ftp_sgd(_ptr(params, "params"), _ptr(grad, "grad"), params.numel(), float(lr), _stream(stream)))
+    if params is None:
+        raise ValueError("params must not be None")
+    pp, pg = _sized((params, "params", params.numel()), (grad, "grad", params.numel()))
+    _check(_lib.ftp_sgd(pp, pg, params.numel(), float(lr), _stream(stream)))
 
 
 def ftp_prefetch_host(plan, x_host, target_host, workspace, copy_stream=None):
     """Starts copying the NEXT batch (pinned float32 CPU tensors) while the current step runs; the
-    ftp_step_host call given the same two tensors then waits for these copies instead of copying."""
-    for name, t in (("x_host", x_host), ("target_host", target_host)):
-        if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
-            raise ValueError(f"{name} must be a contiguous float32 CPU tensor")
-    _check(_lib.ftp_prefetch_host(plan._h, x_host.data_ptr(), target_host.data_ptr(), workspace.data_ptr(),
-                                  _stream(copy_stream)))
+    ftp_step_host call given the same two tensors then waits for these copies instead of copying.
+    copy_stream=None selects the plan's own side stream (the NULL of the C-ABI), whatever stream is
+    current, so that the copies never queue behind the step they are meant to overlap."""
+    px, pt = _host((x_host, "x_host", plan.in_floats), (target_host, "target_host", plan.out_floats))
+    _check(_lib.ftp_prefetch_host(plan._h, px, pt, _workspace(plan, workspace).ptr,
+                                  None if copy_stream is None else _stream(copy_stream)))
 
 
 def ftp_step_host(plan, x_host, target_host, params, lr, loss_host, workspace, dx=None, stream=None):
     """x_host, target_host, loss_host: float32 CPU tensors (pinned memory recommended)."""
-    for name, t in (("x_host", x_host), ("target_host", target_host), ("loss_host", loss_host)):
-        if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
-            raise ValueError(f"{name} must be a contiguous float32 CPU tensor")
-    _check(_lib.ftp_step_host(plan._h, x_host.data_ptr(), target_host.data_ptr(), _ptr(params, "params"),
-                              float(lr), loss_host.data_ptr(), _ptr(dx, "dx", True), workspace.data_ptr(),
-                              _stream(stream)))
+    px, pt, pl = _host((x_host, "x_host", plan.in_floats), (target_host, "target_host", plan.out_floats),
+                       (loss_host, "loss_host", 1))
+    ws = _workspace(plan, workspace)
+    pp, pdx = _sized((params, "params", plan.param_floats), (dx, "dx", plan.in_floats, True))
+    _check(_lib.ftp_step_host(plan._h, px, pt, pp, float(lr), pl, pdx, ws.ptr, _stream(stream)))

@@ -38,7 +38,7 @@ inline Span forward_project(Span i, int K, int S, int P, int out_extent)
     return s;
 }
 
-// "Partitioned ... equally among the tiles": part i of n owns [floor(i*E/n), floor((i+1)*E/n) - 1].
+// Equal shares of a map's extent for the tiles (Section 4.2): part i of n owns [floor(i*E/n), floor((i+1)*E/n) - 1].
 std::vector<Span> equal_partition(int a0, int len, int parts)
 {
     std::vector<Span> out;

@@ -180,3 +180,38 @@ def draw_dyadic(wl: Workload, nnz: int = 3, N: Optional[int] = None):
     c, h, w = map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
     target = rng.standard_normal((n, c, h, w), dtype=np.float32)
     return x, params, target
+
+
+def draw_integer_relu(wl: Workload, N: Optional[int] = None):
+    """Inputs whose forward pass is exact in bfloat16 AND in fp32, for stacks with
+    slope 0 on every conv (use with_slope(wl, 0.0)): integer pixels in [0, 3];
+    every output channel's filter has exactly one tap of +1 and one of -1;
+    biases in {0, 1}.  A conv output is then a - b + bias for two values a, b of
+    its input map (or the zero padding), so with M the largest input value every
+    activation is an integer in [0, M + 1] after the ReLU: at most 3 + (number of
+    conv layers) over a whole stack, far below 256, the largest run of integers
+    that 8 significant bits hold.  A path that stores its maps in bf16 and one
+    that keeps them in fp64 therefore see identical maps, and every arg-max and
+    sign decision (exact ties included) is the same on both sides.  The target
+    is N(0,1)."""
+    rng = np.random.default_rng(wl.seed + 104729)
+    n = wl.N if N is None else N
+    x = rng.integers(0, 4, size=(n, wl.C, wl.H, wl.W)).astype(np.float32)
+    parts = []
+    for l in wl.layers:
+        if l.kind != "conv":
+            continue
+        fan = l.cin * l.k * l.k
+        F = np.zeros((l.cout, fan), dtype=np.float32)
+        for co in range(l.cout):
+            if fan >= 2:
+                plus, minus = rng.choice(fan, size=2, replace=False)
+                F[co, plus], F[co, minus] = 1.0, -1.0
+            else:
+                F[co, 0] = 1.0
+        parts.append(F.ravel())
+        parts.append(rng.integers(0, 2, size=l.cout).astype(np.float32))
+    params = np.concatenate(parts)
+    c, h, w = map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    target = rng.standard_normal((n, c, h, w), dtype=np.float32)
+    return x, params, target

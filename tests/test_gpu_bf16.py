@@ -340,3 +340,87 @@ def test_random_small_stacks_match_oracle(seed):
     assert rel_err(y, ref["y"]) <= 1e-2, wl
     assert l2_err(dx, ref["dx"]) <= 5e-2, wl
     assert l2_err(dparams, ref["dparams"]) <= BF16_TOL, wl
+
+
+# ---------------------------------------------------------------------------------------------
+# Whole-stack parity at the stated tolerance on decision-safe data
+# ---------------------------------------------------------------------------------------------
+SAFE = {
+    "yolo8-small": (FWD["yolo8-small"], None),
+    "yolo8-two-groups": (FWD["yolo8-two-groups"], None),
+    "yolo16-small": (FWD["yolo16-small"], None),
+    "C1": (synth.workload("C1"), None),                 # benchmark launch configurations, full batch
+    "C2": (synth.workload("C2"), None),
+    "C3": (synth.workload("C3"), (0, 15)),              # full batch on the GPU, loss delta on two images
+}
+
+
+@pytest.mark.parametrize("name", sorted(SAFE))
+def test_whole_stack_gradients_on_decision_safe_data(name):
+    """The whole plan, every group chained, at 2e-2 in the max norm.  The data (synth.draw_integer_relu,
+    slope 0) keeps every activation a small integer, which bf16 holds exactly: the forward pass is
+    bit-equal to the oracle's and both sides take the same arg-max and sign decisions, ties
+    included.  What is left to differ is the rounding of the deltas to bf16 (fp32 sums on one side,
+    fp64 on the other), which the tolerance covers."""
+    wl, images = SAFE[name]
+    wl = synth.with_slope(wl, 0.0)
+    x, params, target = synth.draw_integer_relu(wl)
+    c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    dy = np.random.default_rng(3).standard_normal((wl.N, c, h, w)).astype(np.float32)
+    sel = list(range(wl.N)) if images is None else list(images)
+    if images is not None:
+        keep = np.zeros(wl.N, dtype=bool)
+        keep[sel] = True
+        dy[~keep] = 0.0
+    y, dx, dparams, plan = backward_bf16(wl, x, params, dy)
+    ref = run_oracle(wl.with_(N=len(sel)), x[sel], params, dy=dy[sel], store="bf16")
+    plain = run_oracle(wl.with_(N=len(sel)), x[sel], params, dy=dy[sel])
+    assert np.array_equal(ref["y"], plain["y"])                     # storage rounding is the identity on these maps
+    assert np.array_equal(y[sel].astype(np.float64), ref["y"])      # forward: bit for bit
+    assert np.abs(ref["dparams"]).max() > 0 and np.abs(ref["dx"]).max() > 0
+    errs = per_layer_errors(list(wl.layers), dparams, ref["dparams"])
+    print(name, "exec groups", plan.exec_groups(), "dx", rel_err(dx[sel], ref["dx"]), errs)
+    assert rel_err(dx[sel], ref["dx"]) <= BF16_TOL
+    assert all(max(a, b) <= BF16_TOL for _, a, b in errs), errs
+    # the bf16 path against the PLAIN fp64 oracle as well: only the delta rounding separates them
+    assert rel_err(dx[sel], plain["dx"]) <= BF16_TOL
+    assert rel_err(dparams, plain["dparams"]) <= BF16_TOL
+
+
+def _crop_check_plain(wl, x, params, y_gpu, n, oy, ox, size):
+    """As _crop_check_bf16, against the plain fp64 oracle (no storage rounding anywhere)."""
+    from oracle import reference as orc
+    from oracle import spans
+    layers = list(wl.layers)
+    shapes = synth.map_shapes(layers, wl.C, wl.H, wl.W)
+    scale = wl.H // shapes[-1][1]
+
+    def crop_axis(o, extent_out, extent_in):
+        a, b = spans.forward_spans(layers, extent_out, (o, o + size - 1))[0]
+        a = (a // scale) * scale
+        b = min(extent_in, -(-(b + 1) // scale) * scale)
+        return a, b
+    y0, y1 = crop_axis(oy, shapes[-1][1], wl.H)
+    x0, x1 = crop_axis(ox, shapes[-1][2], wl.W)
+    maps, _ = orc.forward(layers, x[n:n + 1, :, y0:y1, x0:x1].astype(np.float64), params.astype(np.float64))
+    ref = maps[-1][0, :, oy - y0 // scale: oy - y0 // scale + size, ox - x0 // scale: ox - x0 // scale + size]
+    return float(np.abs(y_gpu[n, :, oy:oy + size, ox:ox + size] - ref).max())
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3"])
+def test_full_size_activations_against_the_plain_oracle(name):
+    """Activations have no routing ambiguity, so the bf16 path is held to 2e-2 against the PLAIN fp64
+    oracle here: the workloads' own inputs (U[0,1) pixels, He-normal filters, not moved to the bf16
+    grid), benchmark launch configuration, regions at map corners, tile boundaries and the interior."""
+    wl = synth.workload(name)
+    x, params, target = synth.draw(wl)
+    y, plan = forward_bf16(wl, x, params)
+    c, h, w = y.shape[1:]
+    scale = float(np.abs(y).max())
+    size, ty = 4, h // wl.grid[0]
+    worst = 0.0
+    for n, oy, ox in [(0, 0, 0), (wl.N - 1, h - size, w - size), (wl.N // 2, ty - 2, ty - 2), (0, h // 2, w // 3),
+                      (wl.N - 1, 0, w - size)]:
+        worst = max(worst, _crop_check_plain(wl, x, params, y, n, oy, ox, size) / scale)
+    print(name, "bf16 path vs plain fp64 oracle, worst sampled activation error", worst)
+    assert worst <= BF16_TOL

@@ -13,7 +13,7 @@ import pytest
 import torch
 
 import paper_2409_09083_b200 as ftp
-from paper_2409_09083_b200 import synth
+from paper_2409_09083_b200 import binding, synth
 from _util import (FP32_TOL, draw_unambiguous, rel_err, run_gpu, run_gpu_step, run_oracle)
 
 pytestmark = pytest.mark.gpu
@@ -323,6 +323,29 @@ def test_host_batches_with_and_without_prefetch(precision):
             ftp.ftp_step_host(plan, xs[1], ts[1], pd, lr, lh[1], ws)
             for i in (2, 3):
                 ftp.ftp_step_host(plan, xs[i], ts[i], pd, lr, lh[i], ws)
+        elif mode == "side-stream-current":
+            # a non-default stream is current: the steps run on it, the default prefetch still goes to the
+            # plan's own side stream (NULL at the C-ABI), not behind the step on the current stream
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            seen = []
+            real = binding._lib.ftp_prefetch_host
+
+            def spy(h, px, pt, pw, st):
+                seen.append(st)
+                return real(h, px, pt, pw, st)
+            spy.argtypes, spy.restype = real.argtypes, real.restype
+            binding._lib.ftp_prefetch_host = spy
+            try:
+                with torch.cuda.stream(side):
+                    ftp.ftp_prefetch_host(plan, xs[0], ts[0], ws)
+                    for i in range(4):
+                        ftp.ftp_step_host(plan, xs[i], ts[i], pd, lr, lh[i], ws)
+                        if i + 1 < 4:
+                            ftp.ftp_prefetch_host(plan, xs[i + 1], ts[i + 1], ws)
+            finally:
+                binding._lib.ftp_prefetch_host = real
+            assert seen == [None] * 4
         else:
             ftp.ftp_prefetch_host(plan, xs[0], ts[0], ws, copy_stream)
             for i in range(4):
@@ -337,10 +360,64 @@ def test_host_batches_with_and_without_prefetch(precision):
 
     ref_p, ref_l = run("device")
     assert len(set(ref_l)) == 4                                  # four different batches
-    for mode in ("plain", "prefetch", "own-stream", "skipped", "prefetch"):
+    for mode in ("plain", "prefetch", "own-stream", "skipped", "side-stream-current", "prefetch"):
         p, l = run(mode)
         assert np.array_equal(p, ref_p), mode
         assert l == ref_l, mode
+
+
+@pytest.mark.parametrize("precision", [0, 1])
+def test_step_grad_then_sgd_equals_step(precision):
+    """The two halves of the data-parallel step at world size 1: ftp_step_grad followed by ftp_sgd leaves
+    the parameters, the loss and the input gradient of ftp_step, bit for bit."""
+    wl = Y8
+    x, params, target = synth.draw(wl, bias_std=0.1)
+    lr = 0.05
+    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=precision)
+    ws = plan.new_workspace()
+    xd, td = torch.from_numpy(x).cuda(), torch.from_numpy(target).cuda()
+    pa, pb = torch.from_numpy(params.copy()).cuda(), torch.from_numpy(params.copy()).cuda()
+    la, lb = torch.zeros(1, device="cuda"), torch.zeros(1, device="cuda")
+    dxa, dxb = torch.empty_like(xd), torch.empty_like(xd)
+    ftp.ftp_step(plan, xd, pa, lr, ws, target=td, loss_out=la, dx=dxa)
+    grad = torch.full_like(pb, float("nan"))
+    ftp.ftp_step_grad(plan, xd, pb, grad, ws, target=td, loss_out=lb, dx=dxb)
+    torch.cuda.synchronize()
+    assert np.array_equal(pb.cpu().numpy(), params)                  # ftp_step_grad leaves the parameters alone
+    ftp.ftp_sgd(pb, grad, lr)
+    plan.check(ws)
+    assert np.array_equal(pa.cpu().numpy(), pb.cpu().numpy())
+    assert la.item() == lb.item()
+    assert np.array_equal(dxa.cpu().numpy(), dxb.cpu().numpy())
+    assert np.isfinite(grad.cpu().numpy()).all() and float(grad.abs().max()) > 0
+
+
+def test_two_half_batches_reproduce_the_full_batch_update():
+    """Data-parallel arithmetic on one GPU: the gradients of the two halves of a batch (ftp_step_grad on
+    each, as two ranks would), summed and applied by ftp_sgd with lr / 2, equal the full-batch update
+    within 1e-5 (each half's loss is the mean over its own images, so the full-batch gradient is the
+    mean of the two)."""
+    wl = Y8.with_(N=4)
+    x, params, target = synth.draw(wl, bias_std=0.1)
+    lr = 0.05
+    full = ftp.ftp_plan(wl.layers, 4, wl.C, wl.H, wl.W, wl.grid, wl.groups)
+    half = ftp.ftp_plan(wl.layers, 2, wl.C, wl.H, wl.W, wl.grid, wl.groups)
+    wsf, wsh = full.new_workspace(), half.new_workspace()
+    pf = torch.from_numpy(params.copy()).cuda()
+    ftp.ftp_step(full, torch.from_numpy(x).cuda(), pf, lr, wsf, target=torch.from_numpy(target).cuda())
+    ph = torch.from_numpy(params.copy()).cuda()
+    total = torch.zeros_like(ph)
+    for lo in (0, 2):
+        g = torch.empty_like(ph)
+        ftp.ftp_step_grad(half, torch.from_numpy(x[lo:lo + 2]).cuda(), ph, g, wsh,
+                          target=torch.from_numpy(target[lo:lo + 2]).cuda())
+        total += g                                                    # what the all-reduce does across ranks
+    ftp.ftp_sgd(ph, total, lr / 2)
+    torch.cuda.synchronize()
+    upd_full = pf.cpu().numpy().astype(np.float64) - params
+    upd_half = ph.cpu().numpy().astype(np.float64) - params
+    assert np.abs(upd_full).max() > 0
+    assert rel_err(upd_half, upd_full) <= 1e-5
 
 
 def _random_workload(rng):

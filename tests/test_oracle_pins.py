@@ -201,13 +201,41 @@ def test_batch_gradient_is_sum_of_per_image_gradients():
     assert np.allclose(full["dparams"], acc, rtol=1e-12, atol=1e-14)
 
 
-def test_result_independent_of_thread_count(monkeypatch):
-    layers = _tiny_net()
-    x, params, target = _draw(layers, 2, 2, 6, 8, 11)
-    a = orc.step(layers, x, params, lr=0.1, target=target)
-    b = orc.step(layers, x, params, lr=0.1, target=target)
-    assert np.array_equal(a["new_params"], b["new_params"])
-    assert np.array_equal(a["dx"], b["dx"])
+_THREAD_SCRIPT = """
+import sys
+import numpy as np
+sys.path.insert(0, sys.argv[1])
+from oracle import reference as orc
+from paper_2409_09083_b200 import synth
+layers = [synth.conv(2, 3, 3), synth.pool(), synth.conv(3, 4, 1), synth.conv(4, 2, 3)]
+rng = np.random.default_rng(11)
+x = rng.standard_normal((3, 2, 6, 8))
+params = rng.standard_normal(orc.param_count(layers)) * 0.5
+target = rng.standard_normal((3, 2, 3, 4))
+r = orc.step(layers, x, params, lr=0.1, target=target)
+np.savez(sys.argv[2], threads=orc.num_threads(), new_params=r["new_params"], dx=r["dx"], y=r["y"], loss=r["loss"])
+"""
+
+
+def test_result_independent_of_thread_count(tmp_path):
+    """The same step in fresh processes with 1, 2 and 5 OpenMP threads: the loops are parallel over
+    (image, output channel) only, so every sum keeps its order and the results are bit-identical."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script = tmp_path / "run.py"
+    script.write_text(_THREAD_SCRIPT)
+    got = {}
+    for threads in (1, 2, 5):
+        out = tmp_path / f"t{threads}.npz"
+        env = dict(os.environ, OMP_NUM_THREADS=str(threads), OMP_DYNAMIC="false")
+        subprocess.run([sys.executable, str(script), root, str(out)], check=True, env=env)
+        got[threads] = np.load(out)
+        assert int(got[threads]["threads"]) == threads          # the setting really reached the C loops
+    for threads in (2, 5):
+        for key in ("new_params", "dx", "y", "loss"):
+            assert np.array_equal(got[1][key], got[threads][key]), (threads, key)
 
 
 def test_round_bf16_matches_library_conversion_and_ties_go_to_even():
@@ -237,3 +265,70 @@ def test_bf16_storage_only_rounds_stored_maps():
     r64 = orc.step(lin, x, params, 0.0, target=target)
     err = np.abs(r["dparams"] - r64["dparams"]).max() / np.abs(r64["dparams"]).max()
     assert 0.0 < err <= 2e-2
+
+
+def _integer_case():
+    """A small conv / pool stack on data whose maps AND deltas are small integers."""
+    layers = [synth.conv(2, 4, 3, leaky=0.0), synth.pool(), synth.conv(4, 3, 1, leaky=0.0), synth.conv(3, 2, 3, leaky=0.0)]
+    wl = synth.Workload("int", tuple(layers), 2, 2, 8, 12, (1, 1), ((1, 4),))
+    x, params, _ = synth.draw_integer_relu(wl)
+    dy = np.random.default_rng(21).integers(-2, 3, size=(2, 2, 4, 6)).astype(np.float64)
+    return layers, x.astype(np.float64), params.astype(np.float64), dy
+
+
+def test_bf16_storage_is_the_identity_on_bf16_exact_data():
+    """Pin of the store="bf16" branch against the plain branch (itself pinned by finite differences
+    and a library autograd above): where every stored map and every delta in front of an activation
+    is exactly representable in bfloat16 (integers of magnitude <= 256), rounding them changes
+    nothing, so the two branches must agree BIT FOR BIT in every map, delta and gradient.  A mask
+    taken from the wrong tensor, `>=` instead of `>` at Z == 0, or a wrong slope in the store
+    branch breaks the equality."""
+    layers, x, params, dy = _integer_case()
+    plain = orc.step(layers, x, params, 0.25, dy=dy)
+    stored = orc.step(layers, x, params, 0.25, dy=dy, store="bf16")
+    # the premise, checked on the plain branch: integers that 8 significant bits hold
+    tape = orc.forward(layers, x, params)[1]
+    zero_preact = 0
+    for i, l in enumerate(layers):
+        m, d = plain["maps"][i + 1], plain["deltas"][i + 1]
+        assert np.array_equal(m, np.rint(m)) and np.abs(m).max() <= 256
+        assert np.array_equal(d, np.rint(d)) and np.abs(d).max() <= 256
+        if l.kind == "conv":
+            zero_preact += int(((tape[i] == 0.0) & (d != 0.0)).sum())
+    assert zero_preact > 0          # the Z == 0 rule is exercised with a non-zero delta
+    assert np.abs(plain["dparams"]).max() > 0 and np.abs(plain["dx"]).max() > 0
+    for a, b in zip(plain["maps"], stored["maps"]):
+        assert np.array_equal(a, b)
+    for a, b in zip(plain["deltas"], stored["deltas"]):
+        assert np.array_equal(a, b)
+    for key in ("y", "dx", "dparams", "new_params"):
+        assert np.array_equal(plain[key], stored[key]), key
+
+
+def test_bf16_storage_hand_evaluated_one_conv():
+    """One 1x1 conv, one channel, slope 0.1, evaluated by hand.  F = -1, b = 0.25, so Z = 0.25 - X:
+        X  = [[1, -2], [0.25, 3]]      Z = [[-0.75, 2.25], [0, -2.75]]
+    Derivative of the activation: 1 where Z > 0, else the slope (also at Z == 0):
+        mask = [[0.1, 1], [0.1, 0.1]]            (a mask taken from X instead would be [[1, .1], [1, 1]])
+        dY   = [[1.01, 1.01], [1.01, 1.3]]       dY * mask = [[0.101, 1.01], [0.101, 0.13]]
+    Rounded to 8 significant bits AFTER the mask:
+        0.101 = 0.808 * 2^-3 -> 207/256 * 2^-3 = 207/2048 = 0.10107421875
+        1.01  = 0.505 * 2^1  -> 129/256 * 2    = 129/128  = 1.0078125
+        0.13  = 0.52  * 2^-2 -> 133/256 / 4    = 133/1024 = 0.1298828125
+    (rounding dY first would give 1.0078125 * 0.1 = 0.10078125 and 1.296875 * 0.1 = 0.1296875).
+    Gradients are formed from the rounded delta:
+        db = 2 * 207/2048 + 129/128 + 133/1024                     = 1.33984375
+        dF = 1 * 207/2048 - 2 * 129/128 + 0.25 * 207/2048 + 3 * 133/1024 = -1.4996337890625
+        dX = F * dZ = -dZ"""
+    layers = [synth.conv(1, 1, 1, leaky=0.1)]
+    x = np.array([[1.0, -2.0], [0.25, 3.0]]).reshape(1, 1, 2, 2)
+    params = np.array([-1.0, 0.25])
+    dy = np.array([[1.01, 1.01], [1.01, 1.3]]).reshape(1, 1, 2, 2)
+    r = orc.step(layers, x, params, 0.0, dy=dy, store="bf16")
+    dz = np.array([[207 / 2048, 129 / 128], [207 / 2048, 133 / 1024]])
+    assert np.array_equal(r["dx"][0, 0], -dz)
+    assert r["dparams"][1] == 1.33984375
+    assert r["dparams"][0] == -1.4996337890625
+    # the forward half: Y = leaky(Z) stored in bf16; -0.075 = -0.6 * 2^-3 -> -154/256 / 8 = -0.0751953125,
+    # -0.275 = -0.55 * 2^-1 -> -141/256 / 2 = -0.275390625
+    assert np.array_equal(r["y"][0, 0], np.array([[-0.0751953125, 2.25], [0.0, -0.275390625]]))
