@@ -334,6 +334,20 @@ typedef struct { int kind; int group; float ms; } ftp_launch_time;
 int ftp_plan_timing(ftp_plan* plan, int enable);
 int ftp_plan_timing_read(ftp_plan* plan, int* n, ftp_launch_time* out, int capacity);
 
+/*
+ * Measurement aid for the roofline of the fp32 (CUDA-core) kernels, which are bound by the fp32
+ * multiply-add rate and not by memory (the fused stacks move about 9 MB per image for 15.8 GFLOP,
+ * Section 5 workload): launches a register-only loop of independent fp32 FMAs on every
+ * multiprocessor (two blocks of 512 threads each) on `stream`.  The caller times the launch with
+ * events; *flops receives the floating-point operations it performs (2 per FMA).
+ *   out        DEVICE, at least 1024 x (number of multiprocessors) floats, overwritten
+ *   iters      loop count per thread (128 FMAs per iteration)
+ * Returns FTP_ERR_ARG on a null pointer, iters <= 0 or a too-small `out`, FTP_ERR_CUDA if a runtime
+ * call fails.  The paper has no counterpart; it is here so that the fraction of peak is quoted
+ * against a number measured on the same device in the same run.
+ */
+int ftp_fma_peak(float* out, size_t out_count, long long iters, double* flops, void* stream);
+
 /* Number of kernels the library launched on the calling thread's behalf since
  * the plan was created (for launch accounting in benchmarks). */
 long long ftp_plan_launch_count(const ftp_plan* plan);

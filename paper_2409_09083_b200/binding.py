@@ -81,6 +81,8 @@ _lib.ftp_loss_mse_static.argtypes = [_vp, _vp, _vp, _vp, _sz, _vp]
 _lib.ftp_loss_mse_static.restype = _i
 _lib.ftp_sgd.argtypes = [_vp, _vp, _sz, ctypes.c_float, _vp]
 _lib.ftp_sgd.restype = _i
+_lib.ftp_fma_peak.argtypes = [_vp, _sz, ctypes.c_longlong, ctypes.POINTER(ctypes.c_double), _vp]
+_lib.ftp_fma_peak.restype = _i
 
 
 class ftp_launch_time(ctypes.Structure):
@@ -329,6 +331,14 @@ def ftp_sgd(params, grad, lr, stream=None):
         raise ValueError("params must not be None")
     pp, pg = _sized((params, "params", params.numel()), (grad, "grad", params.numel()))
     _check(_lib.ftp_sgd(pp, pg, params.numel(), float(lr), _stream(stream)))
+
+
+def ftp_fma_peak(out, iters, stream=None):
+    """Launches the register-only fp32 FMA loop (see ftp.h); returns the floating-point operations it performs."""
+    flops = ctypes.c_double()
+    (po,) = _sized((out, "out", out.numel()))
+    _check(_lib.ftp_fma_peak(po, out.numel(), int(iters), ctypes.byref(flops), _stream(stream)))
+    return flops.value
 
 
 def ftp_prefetch_host(plan, x_host, target_host, workspace, copy_stream=None):

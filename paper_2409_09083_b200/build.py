@@ -1,13 +1,18 @@
-"""Compile the CUDA library in-tree: paper_2409_09083_b200/libftp.so (sm_100a only)."""
+"""Compile the CUDA library in-tree: paper_2409_09083_b200/libftp.so (sm_100a only).
+
+Each source becomes an object under paper_2409_09083_b200/_build/ (compiled in parallel, rebuilt only
+when the source or a header is newer), then everything is linked into the shared library."""
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libftp.so")
-SOURCES = [os.path.join(CSRC, "api.cu"), os.path.join(CSRC, "noalloc.cu"), os.path.join(CSRC, "plan.cpp")]
+SOURCES = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cpp")))
 HEADERS = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".hpp", ".h"))) + \
           [os.path.join(ROOT, "include", "ftp.h")]
 
@@ -19,20 +24,38 @@ def _nvcc() -> str:
     return "nvcc"
 
 
+def _flags(verbose):
+    f = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
+         "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    return f + (["-Xptxas", "-v"] if verbose else [])
+
+
+def _compile(src, obj, verbose):
+    r = subprocess.run([_nvcc()] + _flags(verbose) + ["-c", src, "-o", obj], capture_output=True, text=True)
+    return src, r
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
-    deps = SOURCES + HEADERS
-    if (not force and os.path.exists(LIB)
-            and all(os.path.getmtime(LIB) >= os.path.getmtime(d) for d in deps)):
+    os.makedirs(OBJ, exist_ok=True)
+    newest_header = max(os.path.getmtime(h) for h in HEADERS)
+    jobs, objs = [], []
+    for src in SOURCES:
+        obj = os.path.join(OBJ, os.path.splitext(os.path.basename(src))[0] + ".o")
+        objs.append(obj)
+        if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), newest_header):
+            jobs.append((src, obj))
+    if not jobs and os.path.exists(LIB) and all(os.path.getmtime(LIB) >= os.path.getmtime(o) for o in objs):
         return LIB
-    cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3",
-           "-std=c++17", "-shared", "-Xcompiler", "-fPIC",
-           "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB] + SOURCES
-    if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-    subprocess.run(cmd, check=True)
+    with ThreadPoolExecutor(max_workers=max(1, min(len(jobs), os.cpu_count() or 1))) as pool:
+        results = list(pool.map(lambda j: _compile(j[0], j[1], verbose), jobs))
+    for src, r in results:
+        if verbose or r.returncode != 0:
+            sys.stderr.write(r.stdout + r.stderr)
+        if r.returncode != 0:
+            raise subprocess.CalledProcessError(r.returncode, f"nvcc -c {src}")
+    subprocess.run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB] + objs, check=True)
     return LIB
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force="-f" in sys.argv, verbose="-v" in sys.argv))
