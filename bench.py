@@ -32,7 +32,8 @@ FP32_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # dram__bytes_read.sum + dram__bytes_write.sum of the fused backward kernel per launch (average over the launches of
 # a step), from the ncu captures summarised under profiles/ (workload C1 only; null for anything else)
 NCU_TRAFFIC = {("C1", "fp32"): 65.7e6, ("C1", "bf16"): 30.5e6}
-KIND = {0: "pack_filters", 1: "fwd_group", 2: "loss_delta", 3: "bwd_group", 4: "halo_sum", 5: "reduce_sgd"}
+KIND = {0: "pack_filters", 1: "fwd_group", 2: "loss_delta", 3: "bwd_group", 4: "halo_sum", 5: "reduce_sgd",
+        6: "delta_act", 7: "filter_grad_rows", 8: "delta_conv_rows"}
 
 
 def measured_bf16_peak():

@@ -123,6 +123,13 @@ typedef struct {
                            layers by the planner's time model (ftp_plan_cost) and take the best one instead of the
                            max_group_convs rule's cuts when the model puts it at least 3 % ahead; -1: never.
                            Default: 1, unless max_group_convs is given (then only that rule applies) */
+    int stationary;       /* fp32 path: executed groups that hold ONE conv layer (with the pool after it, if any;
+                           1x1 or 3x3 window) can run weight-stationary instead of as fused sub-tile stacks: blocks
+                           keep a 64-channel slice of the filter, or a 64 x 32 slice of the filter gradient, on chip
+                           and stream pixel tiles through it, and the layer's maps cross the group boundary in
+                           global memory as at any group boundary (the paper's weight-dominated layers, Section 6).
+                           Default (0): groups whose conv has at least 32 input channels; 1: every such group
+                           whatever its channel count; -1: never */
 } ftp_plan_opts;
 
 /* ftp_plan_create with explicit planner options (NULL = defaults). */
@@ -135,6 +142,12 @@ int ftp_plan_create_opts(const ftp_layer* layers, int n_layers,
 /* The grouping profile that is executed (see ftp_plan_create): writes up to
  * `capacity` groups to groups_out (may be NULL) and the count to *n_groups. */
 int ftp_plan_exec_groups(const ftp_plan* plan, int* n_groups, ftp_group* groups_out, int capacity);
+
+/* How executed group `group` (0-based index into ftp_plan_exec_groups) runs: *stationary = 1 if it is a one-conv
+ * group run by the weight-stationary kernels (see ftp_plan_opts.stationary), 0 if as fused sub-tile stacks;
+ * *partial_sets (may be NULL) = the partial gradient sets of the group that the cross-tile reduction sums
+ * (Section 4.1).  FTP_ERR_ARG on a bad index or NULL. */
+int ftp_plan_group_mode(const ftp_plan* plan, int group, int* stationary, int* partial_sets);
 
 void ftp_plan_destroy(ftp_plan* plan);
 

@@ -40,7 +40,8 @@ _lib.ftp_plan_create.restype = _i
 
 class ftp_plan_opts(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_int), ("max_redundancy_pct", ctypes.c_int), ("max_subtile", ctypes.c_int),
-                ("smem_bytes", ctypes.c_int), ("strict_groups", ctypes.c_int), ("tc_blocks_per_sm", ctypes.c_int), ("max_group_convs", ctypes.c_int), ("cost_model", ctypes.c_int)]
+                ("smem_bytes", ctypes.c_int), ("strict_groups", ctypes.c_int), ("tc_blocks_per_sm", ctypes.c_int), ("max_group_convs", ctypes.c_int), ("cost_model", ctypes.c_int),
+                ("stationary", ctypes.c_int)]
 
 
 _lib.ftp_plan_create_opts.argtypes = [ctypes.POINTER(ftp_layer), _i, _i, _i, _i, _i, _i, _i,
@@ -49,6 +50,8 @@ _lib.ftp_plan_create_opts.argtypes = [ctypes.POINTER(ftp_layer), _i, _i, _i, _i,
 _lib.ftp_plan_create_opts.restype = _i
 _lib.ftp_plan_exec_groups.argtypes = [_vp, ctypes.POINTER(_i), ctypes.POINTER(ftp_group), _i]
 _lib.ftp_plan_exec_groups.restype = _i
+_lib.ftp_plan_group_mode.argtypes = [_vp, _i, ctypes.POINTER(_i), ctypes.POINTER(_i)]
+_lib.ftp_plan_group_mode.restype = _i
 _lib.ftp_plan_destroy.argtypes = [_vp]
 _lib.ftp_plan_destroy.restype = None
 _lib.ftp_plan_region.argtypes = [_vp, _i, _i, _i, _i, _i, ctypes.POINTER(_i * 4)]
@@ -199,11 +202,11 @@ class Plan:
     """Owner of an ftp_plan handle (ftp_plan_create / ftp_plan_destroy)."""
 
     def __init__(self, layers, N, C, H, W, grid, groups, precision=FTP_FP32, max_redundancy_pct=0, max_subtile=0,
-                 smem_bytes=0, strict_groups=False, tc_blocks_per_sm=0, max_group_convs=0, cost_model=0):
+                 smem_bytes=0, strict_groups=False, tc_blocks_per_sm=0, max_group_convs=0, cost_model=0, stationary=0):
         self._h = _vp()
         la, ga = _as_layers(layers), _as_groups(groups)
         opts = ftp_plan_opts(ctypes.sizeof(ftp_plan_opts), max_redundancy_pct, max_subtile, smem_bytes,
-                             1 if strict_groups else 0, tc_blocks_per_sm, max_group_convs, int(cost_model))
+                             1 if strict_groups else 0, tc_blocks_per_sm, max_group_convs, int(cost_model), int(stationary))
         _check(_lib.ftp_plan_create_opts(la, len(layers), N, C, H, W, grid[0], grid[1], ga, len(groups),
                                          precision, ctypes.byref(opts), ctypes.byref(self._h)))
         self.layers, self.shape, self.grid, self.groups = list(layers), (N, C, H, W), tuple(grid), list(groups)
@@ -227,6 +230,13 @@ class Plan:
         arr = (ftp_group * n.value)()
         _check(_lib.ftp_plan_exec_groups(self._h, ctypes.byref(n), arr, n.value))
         return [(g.first, g.last) for g in arr]
+
+    def group_mode(self, group):
+        """(stationary, partial_sets) of executed group `group`: whether the weight-stationary kernels run it,
+        and how many partial gradient sets the cross-tile reduction sums for it."""
+        st, sets = _i(), _i()
+        _check(_lib.ftp_plan_group_mode(self._h, group, ctypes.byref(st), ctypes.byref(sets)))
+        return bool(st.value), sets.value
 
     def region(self, pass_, group, map_index, ty, tx):
         """(x1, y1, x2, y2), inclusive, of user tile (ty, tx) at map X_{map_index}."""

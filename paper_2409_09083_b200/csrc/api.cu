@@ -10,6 +10,7 @@
 #include "kernels.cuh"
 #include "kernels_tc.cuh"
 #include "plan.hpp"
+#include "stationary.cuh"
 
 using namespace ftp;
 
@@ -39,7 +40,11 @@ int ensure_device(ftp_plan* p)
         cudaFuncSetAttribute(fwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(fwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(bwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess)
+        cudaFuncSetAttribute(bwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(conv_rows_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<1>::smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(conv_rows_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<3>::smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(filter_grad_rows_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FgGeom<1>::smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(filter_grad_rows_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, FgGeom<3>::smem_bytes) != cudaSuccess)
         return FTP_ERR_CUDA;
     const size_t bytes = p->tables.size() * sizeof(int);
     if (cudaMalloc(&p->dev_tables, bytes) != cudaSuccess) return FTP_ERR_CUDA;
@@ -202,6 +207,70 @@ int forward_tc(ftp_plan* p, const float* x, const float* params, float* y, void*
     return FTP_OK;
 }
 
+// One-conv group run weight-stationary (stationary.cuh): the convolution with bias, activation and, where a
+// pool follows, the 2x2 maximum and its arg-max, written to the group's output map.
+bool stationary_forward(ftp_plan* p, const GroupPlan& g, int gi, const float* x, const float* params, void* ws, cudaStream_t st)
+{
+    const OpDesc& op = g.fwd_ops[0];
+    ConvRowsArgs a{};
+    a.in = map_ptr(p, x, ws, g.first);
+    a.w = ws_ptr(ws, p->ws.wf_off) + op.wf_off;
+    a.bias = params + op.p_off + (size_t)op.cout * op.cin * op.k * op.k;
+    a.out = const_cast<float*>(map_ptr(p, x, ws, op.out_map));
+    a.arg = g.st.pool ? static_cast<unsigned char*>(ws) + p->ws.arg_off[op.out_map - 1] : nullptr;
+    a.N = p->N; a.Cin = op.cin; a.Cout = op.cout; a.CoutPad = op.cout_pad; a.H = op.in_H; a.W = op.in_W;
+    a.slope = op.slope; a.act = 1; a.pool = g.st.pool;
+    a.rp_img = (op.in_H + 1) / 2; a.x_tiles = (op.in_W + kStCols - 1) / kStCols; a.co_tiles = (op.cout + kStCoTile - 1) / kStCoTile;
+    { Timed t(p, st, 1, gi);
+      if (op.k == 3) conv_rows_kernel<3><<<g.st.fwd_blocks, kStThreads, StGeom<3>::smem_bytes, st>>>(a);
+      else conv_rows_kernel<1><<<g.st.fwd_blocks, kStThreads, StGeom<1>::smem_bytes, st>>>(a); }
+    return launched_ok();
+}
+
+// Backward of such a group: the delta in front of the activation at the conv's resolution, the partial filter
+// and bias gradients (one set per share of the pixels), and the input delta as the convolution of that
+// delta with the rotated filters (Section 4.1), written whole to `din` (may be null: not wanted).
+bool stationary_backward(ftp_plan* p, const GroupPlan& g, int gi, const float* x, const float* dout, float* din, void* ws,
+                         cudaStream_t st)
+{
+    const OpDesc& op = g.bwd_ops[0];
+    const int H = op.in_H, W = op.in_W;
+    float* dz = ws_ptr(ws, p->ws.dz_off);
+    const float* y = map_ptr(p, x, ws, op.out_map);
+    const unsigned char* arg = g.st.pool ? static_cast<unsigned char*>(ws) + p->ws.arg_off[op.out_map - 1] : nullptr;
+    const size_t count = (size_t)p->N * op.cout * op.out_H * op.out_W;
+    { Timed t(p, st, 6, gi);
+      const int blocks = (int)std::min<size_t>((count + 255) / 256, (size_t)kSmCount * 16);
+      delta_act_kernel<<<blocks, 256, 0, st>>>(dout, y, arg, dz, count, op.out_W, op.slope, g.st.pool); }
+    if (!launched_ok()) return false;
+    FilterGradRowsArgs f{};
+    f.dz = dz; f.x = map_ptr(p, x, ws, g.first);
+    f.partial = ws_ptr(ws, g.partial_off); f.set_floats = (long long)g.param_floats;
+    f.filter_off = op.gp_off; f.bias_off = op.gp_off + (long long)op.cout * op.cin * op.k * op.k;
+    f.N = p->N; f.Cin = op.cin; f.Cout = op.cout; f.H = H; f.W = W;
+    f.rp_img = (H + 1) / 2; f.x_tiles = (W + kStCols - 1) / kStCols;
+    f.stages = g.st.fg_stages; f.splits = g.st.fg_splits;
+    f.co_tiles = (op.cout + kFgCo - 1) / kFgCo; f.ci_tiles = (op.cin + kFgCi - 1) / kFgCi;
+    { Timed t(p, st, 7, gi);
+      if (op.k == 3) filter_grad_rows_kernel<3><<<g.st.fg_blocks, kStThreads, FgGeom<3>::smem_bytes, st>>>(f);
+      else filter_grad_rows_kernel<1><<<g.st.fg_blocks, kStThreads, FgGeom<1>::smem_bytes, st>>>(f); }
+    if (!launched_ok()) return false;
+    if (din) {
+        ConvRowsArgs a{};
+        a.in = dz;
+        a.w = ws_ptr(ws, p->ws.wb_off) + op.wb_off;
+        a.bias = nullptr; a.out = din; a.arg = nullptr;
+        a.N = p->N; a.Cin = op.cout; a.Cout = op.cin; a.CoutPad = op.cin_pad; a.H = H; a.W = W;
+        a.slope = 0.f; a.act = 0; a.pool = 0;
+        a.rp_img = (H + 1) / 2; a.x_tiles = (W + kStCols - 1) / kStCols; a.co_tiles = (op.cin + kStCoTile - 1) / kStCoTile;
+        { Timed t(p, st, 8, gi);
+          if (op.k == 3) conv_rows_kernel<3><<<g.st.dx_blocks, kStThreads, StGeom<3>::smem_bytes, st>>>(a);
+          else conv_rows_kernel<1><<<g.st.dx_blocks, kStThreads, StGeom<1>::smem_bytes, st>>>(a); }
+        if (!launched_ok()) return false;
+    }
+    return true;
+}
+
 int forward_impl(ftp_plan* p, const float* x, const float* params, float* y, void* ws, cudaStream_t st)
 {
     if (is_tc(p)) return forward_tc(p, x, params, y, ws, st);
@@ -209,6 +278,10 @@ int forward_impl(ftp_plan* p, const float* x, const float* params, float* y, voi
     if (rc != FTP_OK) return rc;
     for (size_t gi = 0; gi < p->groups.size(); ++gi) {
         const GroupPlan& g = p->groups[gi];
+        if (g.st.on) {
+            if (!stationary_forward(p, g, (int)gi, x, params, ws, st)) return FTP_ERR_CUDA;
+            continue;
+        }
         GroupArgs a;
         fill_common(p, g, false, x, params, ws, a);
         { Timed t(p, st, 1, (int)gi);
@@ -293,6 +366,12 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
     const int G = (int)p->groups.size();
     for (int gi = G - 1; gi >= 0; --gi) {
         const GroupPlan& g = p->groups[gi];
+        if (g.st.on) {
+            const float* dout = gi == G - 1 ? dy : ws_ptr(ws, p->ws.dmap_off[gi + 1]);
+            float* din = gi == 0 ? dx : ws_ptr(ws, p->ws.dmap_off[gi]);
+            if (!stationary_backward(p, g, gi, x, dout, din, ws, st)) return FTP_ERR_CUDA;
+            continue;
+        }
         GroupArgs a;
         fill_common(p, g, true, x, params, ws, a);
         a.dmap_out = gi == G - 1 ? dy : ws_ptr(ws, p->ws.dmap_off[gi + 1]);
@@ -361,6 +440,8 @@ int ftp_plan_create_opts(const ftp_layer* layers, int n_layers, int N, int C, in
         if (opts->max_group_convs) po.max_group_convs = opts->max_group_convs < 0 ? 0 : opts->max_group_convs;
         if (opts->cost_model < -1 || opts->cost_model > 1) return FTP_ERR_ARG;
         po.cost_model = opts->cost_model ? (opts->cost_model > 0 ? 1 : 0) : (opts->max_group_convs ? 0 : 1);
+        if (opts->stationary < -1 || opts->stationary > 1) return FTP_ERR_ARG;
+        po.stationary = opts->stationary;
     }
     ftp_plan* p = new (std::nothrow) ftp_plan();
     if (!p) return FTP_ERR_ARG;
@@ -387,6 +468,14 @@ int ftp_plan_exec_groups(const ftp_plan* plan, int* n_groups, ftp_group* groups_
     *n_groups = (int)plan->groups.size();
     if (groups_out)
         for (int i = 0; i < *n_groups && i < capacity; ++i) groups_out[i] = ftp_group{plan->groups[i].first, plan->groups[i].last};
+    return FTP_OK;
+}
+
+int ftp_plan_group_mode(const ftp_plan* plan, int group, int* stationary, int* partial_sets)
+{
+    if (!plan || !stationary || group < 0 || group >= (int)plan->groups.size()) return FTP_ERR_ARG;
+    *stationary = plan->groups[group].st.on;
+    if (partial_sets) *partial_sets = plan->groups[group].bwd.blocks;
     return FTP_OK;
 }
 
@@ -433,6 +522,17 @@ int ftp_plan_sizes(const ftp_plan* plan, size_t* param_floats, size_t* workspace
 int ftp_plan_subtiles(const ftp_plan* plan, int pass, int group, int* rows, int* cols, size_t* smem_bytes, int* blocks)
 {
     if (!plan || group < 0 || group >= (int)plan->groups.size() || pass < 0 || pass > 1) return FTP_ERR_ARG;
+    const GroupPlan& gp = plan->groups[group];
+    if (gp.st.on) {         // weight-stationary group: row-pair tiles of the whole batch x column tiles, 256-thread blocks
+        const OpDesc& op = gp.fwd_ops[0];
+        const int per = pass ? kFgRowPairs : kStRowPairs;
+        if (rows) *rows = (plan->N * ((op.in_H + 1) / 2) + per - 1) / per;
+        if (cols) *cols = (op.in_W + kStCols - 1) / kStCols;
+        if (smem_bytes) *smem_bytes = op.k == 3 ? (pass ? FgGeom<3>::smem_bytes : StGeom<3>::smem_bytes)
+                                                : (pass ? FgGeom<1>::smem_bytes : StGeom<1>::smem_bytes);
+        if (blocks) *blocks = pass ? gp.st.fg_blocks : gp.st.fwd_blocks;
+        return FTP_OK;
+    }
     const PassPlan& pp = pass ? plan->groups[group].bwd : plan->groups[group].fwd;
     if (rows) *rows = pp.y.count;
     if (cols) *cols = pp.x.count;

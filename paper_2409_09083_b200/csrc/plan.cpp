@@ -482,6 +482,19 @@ double pass_estimate_us(int precision, bool backward, const double f[kCostTerms]
     return t;
 }
 
+// Weight-stationary groups: multiply-accumulates at the measured rate of the kernels, the maps they move
+// at HBM speed, one launch overhead per kernel.
+double stationary_estimate_us(const ftp_plan& p, const GroupPlan& g, bool backward, bool need_dx)
+{
+    const OpDesc& op = g.fwd_ops[0];
+    const double px = (double)p.N * op.in_H * op.in_W;
+    const double flops = 2.0 * px * op.cin * op.cout * op.k * op.k;
+    const double rate = (op.k == 1 ? kStatTflops1x1 : kStatTflops) * 1e6;          // flop per microsecond
+    const double map_us = px * (op.cin + op.cout) * 4.0 / 6.5e6;                   // bytes at 6.5 TB/s
+    if (!backward) return flops / rate + map_us + 5.0;
+    return flops * (need_dx ? 2.0 : 1.0) / rate + 3.0 * map_us + 15.0;
+}
+
 // Backward launch shape: as many blocks as run at once (or as there are stacks), each owning one
 // partial gradient set; the stacks of the whole batch are dealt out evenly to them.
 void set_backward_blocks(GroupPlan& g, int N, int gy, int gx)
@@ -532,6 +545,37 @@ void refine_backward_split(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
                 if (est > 0 && est < 0.97 * first && est < best) { best = est; best_ky = ky; best_kx = kx; }
             }
     eval(best_ky, best_kx);
+}
+
+// Weight-stationary execution of a group that holds one conv layer (optionally with its pool), fp32
+// path: launch shapes of the three kernels.  The convolution cuts (row pairs of the whole batch) x
+// (columns) x (output channels) into blocks of 16 x 8 x 64; the filter gradient gives every 64 x 32
+// slice of (output, input) channels `fg_splits` blocks, each with an equal share of the pixel stages
+// and one partial set, so that about two rounds of blocks fill the GPU.
+void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
+{
+    g.st = StatPlan{};
+    if (p.precision != FTP_FP32 || o.stationary < 0 || g.n_ops != 1) return;
+    const OpDesc& op = g.fwd_ops[0];
+    if (op.kind == kOpPool || (op.k != 1 && op.k != 3)) return;
+    if (o.stationary == 0 && op.cin < kStatMinCin) return;
+    const int H = op.in_H, W = op.in_W;                        // the conv's resolution
+    const long long rp_total = (long long)p.N * ((H + 1) / 2);
+    const int x_tiles = (W + kStCols - 1) / kStCols;
+    const long long rp_tiles = (rp_total + kStRowPairs - 1) / kStRowPairs;
+    const long long fwd_blocks = rp_tiles * x_tiles * ((op.cout + kStCoTile - 1) / kStCoTile);
+    const long long dx_blocks = rp_tiles * x_tiles * ((op.cin + kStCoTile - 1) / kStCoTile);
+    const long long stages = (rp_total + kFgRowPairs - 1) / kFgRowPairs * x_tiles;
+    const long long slices = (long long)((op.cout + kFgCo - 1) / kFgCo) * ((op.cin + kFgCi - 1) / kFgCi);
+    if (fwd_blocks > 0x7fffffffLL || dx_blocks > 0x7fffffffLL || stages > 0x7fffffffLL || slices > 65535) return;
+    g.st.on = 1; g.st.k = op.k; g.st.pool = op.kind == kOpConvPool ? 1 : 0;
+    g.st.fwd_blocks = (int)fwd_blocks; g.st.dx_blocks = (int)dx_blocks;
+    g.st.fg_stages = (int)stages;
+    const long long slots = 4LL * kSmCount;                    // two rounds of two blocks per SM
+    g.st.fg_splits = (int)std::max<long long>(1, std::min<long long>(stages, slots / slices));
+    g.st.fg_blocks = (int)(slices * g.st.fg_splits);
+    g.bwd.blocks = g.st.fg_splits;                             // partial gradient sets of the group
+    g.bwd.scratch_floats = 0;                                  // the input delta is written whole, no overlapping parts to sum
 }
 
 struct LayerOffsets { std::vector<long long> p_off, wf_off, wb_off, twf_off, twb_off; };
@@ -671,6 +715,11 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
     g.bwd.scratch_floats = (size_t)N * (tcp && first > 1 ? round_up(p.maps[first - 1].C, 16) : p.maps[first - 1].C) *
                            g.bwd.y.scratch_off[g.bwd.y.count] *
                            g.bwd.x.scratch_off[g.bwd.x.count];
+    plan_stationary(p, g, o);
+    if (g.st.on) {                                  // no sub-tile stacks, no halo recomputation
+        g.macs_done = g.macs_untiled;
+        if (redundancy) *redundancy = 1.0;
+    }
 
     return FTP_OK;
 }
@@ -748,6 +797,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     // puts it at least 3 % ahead; the margin keeps the model's error (about 10 % per group) from
     // trading a measured-good default for a predicted tie.
     auto estimate = [&](const GroupPlan& g) {
+        if (g.st.on) return stationary_estimate_us(p, g, false, false) + stationary_estimate_us(p, g, true, g.first > 1);
         double f[kCostTerms];
         pass_cost_terms(p, g, false, false, f);
         double t = pass_estimate_us(precision, false, f);
@@ -881,9 +931,13 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         ws.t_stage_off = take(2 * ws.t_stage_bytes);
         ws.x_stage_off = take(2 * ws.x_stage_bytes);
     }
-    size_t scratch = 0;
-    for (const GroupPlan& g : p.groups) scratch = std::max(scratch, g.bwd.scratch_floats);
+    size_t scratch = 0, dz = 0;
+    for (const GroupPlan& g : p.groups) {
+        scratch = std::max(scratch, g.bwd.scratch_floats);
+        if (g.st.on) dz = std::max(dz, (size_t)N * g.fwd_ops[0].cout * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W);
+    }
     ws.scratch_off = take(scratch * 4);
+    ws.dz_off = take(dz * 4);
     ws.wf_off = take(p.wf_floats * (tcp ? 2 : 4));
     ws.wb_off = take(p.wb_floats * (tcp ? 2 : 4));
     ws.err_off = take(256);
@@ -898,7 +952,8 @@ int cost_terms(const ftp_plan& p, int pass, int group, int need_dx, double terms
 {
     if (group < 0 || group >= (int)p.groups.size() || pass < 0 || pass > 1 || !terms) return FTP_ERR_ARG;
     pass_cost_terms(p, p.groups[group], pass == 1, need_dx != 0, terms);
-    if (est_us) *est_us = pass_estimate_us(p.precision, pass == 1, terms);
+    if (est_us) *est_us = p.groups[group].st.on ? stationary_estimate_us(p, p.groups[group], pass == 1, need_dx != 0)
+                                                : pass_estimate_us(p.precision, pass == 1, terms);
     return FTP_OK;
 }
 

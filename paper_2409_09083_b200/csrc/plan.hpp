@@ -31,6 +31,16 @@ constexpr int kTcSmemBudget2 = 113 * 1024;// ... with two blocks per SM
 constexpr int kTcIssuers = 4;             // threads (lane 0 of warps 0..3) that issue MMAs, each for its own accumulators
 constexpr int kTcMaxUnits = 32;           // filter-gradient accumulators per pass (at least 16 columns each)
 constexpr int kTcTailEntries = 16;        // 16-byte entries appended to every tile plane
+// Weight-stationary kernels of one-conv groups (stationary.cuh): 256 threads, two blocks per SM.
+constexpr int kStThreads = 256;
+constexpr int kStCoTile  = 64;            // convolution: output channels per block (8 per thread)
+constexpr int kStRowPairs = 16;           // convolution: row pairs per block, 32 threads x (2 rows x 4 columns) each
+constexpr int kStCols    = 8;             // columns per block, both kernels
+constexpr int kFgCo = 64, kFgCi = 32;     // filter gradient: (output, input) channel slice of a block (8 x 1 per thread)
+constexpr int kFgRowPairs = 4;            // filter gradient: row pairs per pixel stage
+constexpr int kStatMinCin = 32;           // fewest input channels for which a one-conv group runs weight-stationary by default
+constexpr double kStatTflops = 40.0;      // measured rate of the weight-stationary kernels (3x3; 1x1 runs at kStatTflops1x1), for the planner's estimates
+constexpr double kStatTflops1x1 = 20.0;
 constexpr int kCostTerms = 8;             // terms of the planner's time estimate of one pass of a group
 
 struct Span { int a, b; };            // inclusive interval on one axis
@@ -93,8 +103,18 @@ struct PassPlan {
     int dev_ytile = 0, dev_xtile = 0;
 };
 
+// Weight-stationary execution of an executed group that holds one conv layer (stationary.cuh).
+struct StatPlan {
+    int on = 0;
+    int k = 0, pool = 0;
+    int fwd_blocks = 0, dx_blocks = 0;      // convolution launches: (row-pair tiles) x (column tiles) x (64-channel slices)
+    int fg_stages = 0, fg_splits = 0;       // filter gradient: pixel stages over the batch, and the shares they are dealt out in
+    int fg_blocks = 0;                      // (64 x 32 channel slices) x shares; a share is one partial gradient set
+};
+
 struct GroupPlan {
     int first = 0, last = 0;        // 1-based layers
+    StatPlan st;
     int n_ops = 0;
     OpDesc fwd_ops[kMaxOps];
     OpDesc bwd_ops[kMaxOps];
@@ -114,6 +134,7 @@ struct Workspace {                 // byte offsets, all 256-aligned
     std::vector<size_t> dmap_off;  // delta maps at group inputs of groups 1.. (index = group), and slot for dY
     size_t dy_off = 0;             // loss delta at the last map (ftp_step with target)
     size_t scratch_off = 0;
+    size_t dz_off = 0;             // weight-stationary groups: delta in front of the activation at the conv's resolution (largest such layer)
     size_t wf_off = 0, wb_off = 0; // packed filters
     size_t partial_off = 0;
     size_t grad_off = 0;           // summed gradient (ftp_step keeps it internal)
@@ -166,6 +187,7 @@ struct PlanOpts {
     int cost_model = 1;             // 1 = the time model (pass_cost_terms) may replace the fixed rule's cuts, see build_plan
     int refine_backward = 1;        // 1 = the time model may take a finer backward split that balances the blocks (refine_backward_split)
     int tc_ctas = 0;                // tensor-core path: blocks per SM, 1 or 2 (0 = two where every layer of the group allows it)
+    int stationary = 0;             // one-conv groups run weight-stationary: 0 = with at least kStatMinCin input channels, 1 = all, -1 = none
     int tensor_cores = 0;           // set by build_plan from the precision: shared-memory layouts of the bf16 path
 };
 // Builds everything but the device upload.  Returns FTP_OK or an error code.

@@ -1,44 +1,63 @@
 // Weight-stationary kernels of the fp32 path for executed groups that hold one conv layer
 // (optionally with the 2x2 max-pool after it).  The paper leaves weight-dominated layers to a
 // weight partitioning it names as future work (Section 6); here such a layer is cut along its
-// output channels and its pixels instead of into fused stacks: a block keeps a slice of the filter
+// channels and its pixels instead of into fused stacks: a block keeps a slice of the filter
 // (forward, input delta) or of the filter gradient (Section 4.1: feature-map tile convolved with the
-// delta tile) on chip and streams pixel tiles through it.
+// delta tile) on chip and streams pixel tiles through it.  The exchange with the neighbouring
+// groups goes through the full maps in global memory, as at every group boundary (Section 3).
 //
-//   conv_rows_kernel   out = conv(in, w) (+ bias, leaky ReLU, optional fused 2x2 max-pool with arg-max):
-//                      the forward convolution and, with the rotated filters, the input delta
-//   filter_grad_rows_kernel   partial filter and bias gradients of a slice of (output, input) channels
-//                      over a share of the pixels; the shares are summed by the cross-tile reduction
-//   delta_act_kernel   the delta in front of the activation, dZ = dY * leaky'(Y), at the conv's
-//                      resolution (routed through the arg-max where a pool follows)
+//   conv_rows_kernel         out = conv(in, w) (+ bias, leaky ReLU, optional fused 2x2 max-pool with
+//                            arg-max): the forward convolution and, with the rotated filters, the
+//                            input delta (Section 4.1)
+//   filter_grad_rows_kernel  partial filter and bias gradients of a (64 output, 32 input) channel
+//                            slice over a share of the pixels; the cross-tile reduction sums the shares
+//   delta_act_kernel         the delta in front of the activation, dZ = dY * leaky'(Y), at the conv's
+//                            resolution (routed through the arg-max where a pool follows)
 //
-// Thread tile of the convolution: 8 output channels x (2 rows x 4 columns).  Rows are taken in
-// pairs over the whole batch (image after image), so a tile of row pairs may span images and no
-// rows are wasted on maps whose height is not a multiple of the tile; every row pair keeps its own
-// four input rows in shared memory.  Each output value is accumulated over input channels in
-// ascending order and, per channel, over the window columns and then rows, the order of the fused
-// stack kernels, so both give the same bits.
+// Rows are taken in pairs over the whole batch (image after image), so a tile of row pairs may span
+// images and no rows are wasted on maps whose height is not a multiple of the tile; every row pair
+// keeps its own K + 1 input rows in shared memory.  Columns are taken eight at a time.
+// Each output value of the convolution is accumulated over input channels in ascending order and,
+// per channel, over the window columns and then rows: the order of the fused stack kernels, so both
+// give the same bits.
 #pragma once
 
 #include <cuda_runtime.h>
 
+#include "plan.hpp"
+
 namespace ftp {
+
+// Shared-memory geometry of one input stage of the convolution, in floats.  Column 0 of a block's
+// columns sits at offset 4 of a row (16-byte aligned for the 4-wide reads); the left halo uses offset
+// 3 and the right halo the first, otherwise unused, slot of the next row.  The stride between row
+// pairs is 8 or 24 modulo 32, so that the eight lanes of a quarter warp (two column quads of four row
+// pairs) read 4-wide without bank conflicts.
+template <int K> struct StGeom {
+    static constexpr int P = K / 2, RR = K + 1;
+    static constexpr int pitch = kStCols + (K > 1 ? 4 : 0);
+    static constexpr int rp_stride = K == 3 ? 56 : 24;
+    static constexpr int ci_stride = kStRowPairs * rp_stride;
+    static constexpr int ci_chunk = K == 3 ? 8 : 32;                 // input channels per stage
+    static constexpr int w_stage = ci_chunk * K * K * kStCoTile;     // floats
+    static constexpr int in_stage = ci_chunk * ci_stride;
+    static constexpr int smem_bytes = 2 * (w_stage + in_stage) * 4;
+    static constexpr int cols = kStCols + 2 * P;
+    static constexpr int npos = kStRowPairs * RR * cols;             // input positions of a stage per channel
+    static constexpr int pos_per_thread = (npos + kStThreads - 1) / kStThreads;
+};
 
 struct ConvRowsArgs {
     const float* in;        // [N][Cin][H][W]
-    const float* w;         // [Cin][K*K][CoutPad]: tap-major slices of 8-padded output channels
+    const float* w;         // [Cin][K*K][CoutPad]: per input channel and tap, the 8-padded output channels
     const float* bias;      // [Cout] or null
     float* out;             // [N][Cout][H][W], or the pooled map [N][Cout][H/2][W/2] when pool != 0
     unsigned char* arg;     // pool: arg-max (dy * 2 + dx, first maximum in row-major order) per pooled value
     int N, Cin, Cout, CoutPad, H, W;
-    float slope;            // leaky-ReLU slope; act == 0: no bias, no activation (input delta)
-    int act, pool;
-    int co_tile;            // output channels per block (multiple of 8)
-    int prp, pcq;           // row pairs and column quads per block: (co_tile / 8) * prp * pcq threads
-    int ci_chunk;           // input channels per shared-memory stage
+    float slope;            // leaky-ReLU slope (act != 0)
+    int act, pool;          // act == 0: plain sums (input delta)
     int rp_img;             // row pairs per image = ceil(H / 2)
     int x_tiles, co_tiles;  // blockIdx.x = (rp_tile * x_tiles + x_tile) * co_tiles + co_tile
-    int in_pitch, rp_stride, ci_stride;   // shared-memory geometry of an input stage, in floats
 };
 
 __device__ __forceinline__ void st_cp_async16(void* smem, const void* gmem, bool valid)
@@ -56,42 +75,35 @@ __device__ __forceinline__ void st_cp_async4(void* smem, const void* gmem, bool 
 __device__ __forceinline__ void st_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void st_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
 
-constexpr int kStMaxPos = 6;   // input positions (row, column of a stage) a thread copies per channel
-
-// K = 1 or 3 (stride 1, padding K/2).
+// K = 1 or 3 (stride 1, padding K / 2).  Thread tile: 8 output channels x (2 rows x 4 columns).
 template <int K>
-__global__ void __launch_bounds__(256, 2) conv_rows_kernel(const __grid_constant__ ConvRowsArgs A)
+__global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_constant__ ConvRowsArgs A)
 {
+    using G = StGeom<K>;
     extern __shared__ __align__(16) float st_smem[];
-    constexpr int KK = K * K, P = K / 2;
-    constexpr int RR = K + 1;                      // input rows of a row pair
-    const int tid = threadIdx.x, nthreads = blockDim.x;
-    const int npg = A.prp * A.pcq;
-    const int cg = tid / npg, pg = tid - cg * npg;
-    const int rp_l = pg / A.pcq, cq_l = pg - rp_l * A.pcq;
+    constexpr int KK = K * K, P = G::P, RR = G::RR;
+    const int tid = threadIdx.x;
+    const int cg = tid >> 5, pg = tid & 31;                  // a warp shares its 8 output channels: filter reads are broadcasts
+    const int rp_l = pg >> 1, cq_l = pg & 1;
     const int co_t = blockIdx.x % A.co_tiles;
     const int xt = (blockIdx.x / A.co_tiles) % A.x_tiles;
     const int rt = blockIdx.x / (A.co_tiles * A.x_tiles);
-    const int co0 = co_t * A.co_tile, x0 = xt * A.pcq * 4, rp0 = rt * A.prp;
-    const int TW = A.pcq * 4;
-    const int w_stage = A.ci_chunk * KK * A.co_tile;            // floats
-    const int in_stage = A.ci_chunk * A.ci_stride;
-    float* sw = st_smem;                                        // two weight stages
-    float* si = st_smem + 2 * w_stage;                          // two input stages
+    const int co0 = co_t * kStCoTile, x0 = xt * kStCols, rp0 = rt * kStRowPairs;
+    float* sw = st_smem;                                     // two filter stages
+    float* si = st_smem + 2 * G::w_stage;                    // two input stages
     const size_t plane = (size_t)A.H * A.W;
 
     // input positions this thread copies in every stage: (row pair, row, column) -> shared / global offsets
-    int pos_s[kStMaxPos]; long long pos_g[kStMaxPos]; unsigned pos_ok = 0;
-    const int cols = TW + 2 * P, npos = A.prp * RR * cols;
+    int pos_s[G::pos_per_thread]; long long pos_g[G::pos_per_thread]; unsigned pos_ok = 0;
 #pragma unroll
-    for (int e = 0; e < kStMaxPos; ++e) {
-        const int idx = tid + e * nthreads;
+    for (int e = 0; e < G::pos_per_thread; ++e) {
+        const int idx = tid + e * kStThreads;
         pos_s[e] = -1; pos_g[e] = 0;
-        if (idx < npos) {
-            const int c = idx % cols, t = idx / cols, r = t % RR, rl = t / RR;
+        if (idx < G::npos) {
+            const int c = idx % G::cols, t = idx / G::cols, r = t % RR, rl = t / RR;
             const int rp = rp0 + rl;
             const int n = rp / A.rp_img, y = (rp - n * A.rp_img) * 2 + r - P, x = x0 + c - P;
-            pos_s[e] = rl * A.rp_stride + r * A.in_pitch + c + (4 - P);
+            pos_s[e] = rl * G::rp_stride + r * G::pitch + c + (4 - P);
             if (n < A.N && y >= 0 && y < A.H && x >= 0 && x < A.W) {
                 pos_ok |= 1u << e;
                 pos_g[e] = (long long)n * A.Cin * plane + (long long)y * A.W + x;
@@ -99,76 +111,82 @@ __global__ void __launch_bounds__(256, 2) conv_rows_kernel(const __grid_constant
         }
     }
     auto load_stage = [&](int chunk) {
-        const int ci0 = chunk * A.ci_chunk, nci = min(A.ci_chunk, A.Cin - ci0);
-        float* dw = sw + (chunk & 1) * w_stage;
-        float* di = si + (chunk & 1) * in_stage;
-        // filters: rows of co_tile floats per (channel, tap)
-        const int q = A.co_tile / 4, n16 = nci * KK * q;
-        for (int i = tid; i < n16; i += nthreads) {
+        const int ci0 = chunk * G::ci_chunk, nci = min(G::ci_chunk, A.Cin - ci0);
+        float* dw = sw + (chunk & 1) * G::w_stage;
+        float* di = si + (chunk & 1) * G::in_stage;
+        // filters: a row of kStCoTile floats per (channel, tap)
+        constexpr int q = kStCoTile / 4;
+        for (int i = tid; i < nci * KK * q; i += kStThreads) {
             const int row = i / q, j = i - row * q;
             const int co = co0 + 4 * j;
-            st_cp_async16(dw + row * A.co_tile + 4 * j, A.w + ((size_t)ci0 * KK + row) * A.CoutPad + min(co, A.CoutPad - 4), co < A.CoutPad);
+            st_cp_async16(dw + row * kStCoTile + 4 * j, A.w + ((size_t)ci0 * KK + row) * A.CoutPad + min(co, A.CoutPad - 4), co < A.CoutPad);
         }
 #pragma unroll
-        for (int e = 0; e < kStMaxPos; ++e)
+        for (int e = 0; e < G::pos_per_thread; ++e)
             if (pos_s[e] >= 0) {
                 const bool ok = (pos_ok >> e) & 1u;
                 const float* src = A.in + pos_g[e] + (size_t)ci0 * plane;
                 float* dst = di + pos_s[e];
-                for (int ci = 0; ci < nci; ++ci) st_cp_async4(dst + ci * A.ci_stride, src + (size_t)ci * plane, ok);
+                for (int ci = 0; ci < nci; ++ci) st_cp_async4(dst + ci * G::ci_stride, src + (size_t)ci * plane, ok);
             }
         st_commit();
     };
 
-    float acc[2][4][8];
+    // Accumulators as pairs of neighbouring output channels: one packed multiply-add (two fp32 FMAs, each
+    // rounded like a scalar one) updates both, which halves the instructions the FMA pipe has to be fed with.
+    float2 acc[2][4][4];
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        const float b = (A.bias != nullptr && co0 + cg * 8 + c < A.Cout) ? __ldg(A.bias + co0 + cg * 8 + c) : 0.f;
+    for (int c = 0; c < 4; ++c) {
+        const int co = co0 + cg * 8 + 2 * c;
+        const float2 b = make_float2((A.bias != nullptr && co < A.Cout) ? __ldg(A.bias + co) : 0.f,
+                                     (A.bias != nullptr && co + 1 < A.Cout) ? __ldg(A.bias + co + 1) : 0.f);
 #pragma unroll
         for (int p = 0; p < 2; ++p)
 #pragma unroll
             for (int j = 0; j < 4; ++j) acc[p][j][c] = b;
     }
 
-    const int nchunks = (A.Cin + A.ci_chunk - 1) / A.ci_chunk;
-    const int my_in = rp_l * A.rp_stride + cq_l * 4 + 4;        // column 0 of this thread's quad (16-byte aligned)
+    const int nchunks = (A.Cin + G::ci_chunk - 1) / G::ci_chunk;
+    const int my_in = rp_l * G::rp_stride + cq_l * 4 + 4;    // column 0 of this thread's quad (16-byte aligned)
     load_stage(0);
     for (int chunk = 0; chunk < nchunks; ++chunk) {
         if (chunk + 1 < nchunks) { load_stage(chunk + 1); st_wait<1>(); } else st_wait<0>();
         __syncthreads();
-        const int nci = min(A.ci_chunk, A.Cin - chunk * A.ci_chunk);
-        const float* wb = sw + (chunk & 1) * w_stage + cg * 8;
-        const float* ib = si + (chunk & 1) * in_stage + my_in;
-        for (int ci = 0; ci < nci; ++ci) {
+        const int nci = min(G::ci_chunk, A.Cin - chunk * G::ci_chunk);
+        const float* wc = sw + (chunk & 1) * G::w_stage + cg * 8;
+        const float* ip = si + (chunk & 1) * G::in_stage + my_in;
+#pragma unroll 1
+        for (int ci = 0; ci < nci; ++ci, wc += KK * kStCoTile, ip += G::ci_stride) {
             float v[RR][4 + 2 * P];
-            const float* ip = ib + ci * A.ci_stride;
 #pragma unroll
             for (int r = 0; r < RR; ++r) {
-                const float4 m = *reinterpret_cast<const float4*>(ip + r * A.in_pitch);
-                if constexpr (P > 0) v[r][0] = ip[r * A.in_pitch - 1];
+                const float4 m = *reinterpret_cast<const float4*>(ip + r * G::pitch);
+                if constexpr (P > 0) v[r][0] = ip[r * G::pitch - 1];
                 v[r][P] = m.x; v[r][P + 1] = m.y; v[r][P + 2] = m.z; v[r][P + 3] = m.w;
-                if constexpr (P > 0) v[r][3 + 2 * P] = ip[r * A.in_pitch + 4];
+                if constexpr (P > 0) v[r][3 + 2 * P] = ip[r * G::pitch + 4];
             }
-            const float* wc = wb + ci * KK * A.co_tile;
 #pragma unroll
             for (int kx = 0; kx < K; ++kx)
 #pragma unroll
                 for (int ky = 0; ky < K; ++ky) {
-                    const float4 wa = *reinterpret_cast<const float4*>(wc + (ky * K + kx) * A.co_tile);
-                    const float4 wq = *reinterpret_cast<const float4*>(wc + (ky * K + kx) * A.co_tile + 4);
-                    const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wq.x, wq.y, wq.z, wq.w};
+                    const float4 wa = *reinterpret_cast<const float4*>(wc + (ky * K + kx) * kStCoTile);
+                    const float4 wq = *reinterpret_cast<const float4*>(wc + (ky * K + kx) * kStCoTile + 4);
+                    const float2 wv[4] = {make_float2(wa.x, wa.y), make_float2(wa.z, wa.w), make_float2(wq.x, wq.y), make_float2(wq.z, wq.w)};
 #pragma unroll
                     for (int p = 0; p < 2; ++p)
 #pragma unroll
-                        for (int j = 0; j < 4; ++j)
+                        for (int j = 0; j < 4; ++j) {
+                            const float2 vv = make_float2(v[p + ky][j + kx], v[p + ky][j + kx]);
 #pragma unroll
-                            for (int c = 0; c < 8; ++c) acc[p][j][c] = fmaf(v[p + ky][j + kx], wv[c], acc[p][j][c]);
+                            for (int c = 0; c < 4; ++c) acc[p][j][c] = __ffma2_rn(vv, wv[c], acc[p][j][c]);
+                        }
                 }
         }
         __syncthreads();
     }
 
     // epilogue
+    auto val = [&](int p, int j, int c) { return (c & 1) ? acc[p][j][c >> 1].y : acc[p][j][c >> 1].x; };
     const int rp = rp0 + rp_l;
     const int n = rp / A.rp_img, y = (rp - n * A.rp_img) * 2, x = x0 + cq_l * 4;
     if (n >= A.N || x >= A.W) return;
@@ -182,7 +200,7 @@ __global__ void __launch_bounds__(256, 2) conv_rows_kernel(const __grid_constant
                 if (y + p >= A.H) break;
                 float o[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) { const float z = acc[p][j][c]; o[j] = A.act ? (z > 0.f ? z : A.slope * z) : z; }
+                for (int j = 0; j < 4; ++j) { const float z = val(p, j, c); o[j] = A.act ? (z > 0.f ? z : A.slope * z) : z; }
                 float* dst = A.out + (((size_t)n * A.Cout + co) * A.H + y + p) * A.W + x;
                 if (x + 3 < A.W && (A.W & 3) == 0) *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[1], o[2], o[3]);
                 else
@@ -199,7 +217,7 @@ __global__ void __launch_bounds__(256, 2) conv_rows_kernel(const __grid_constant
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 if (x + 2 * h >= A.W) break;
-                float v00 = acc[0][2 * h][c], v01 = acc[0][2 * h + 1][c], v10 = acc[1][2 * h][c], v11 = acc[1][2 * h + 1][c];
+                float v00 = val(0, 2 * h, c), v01 = val(0, 2 * h + 1, c), v10 = val(1, 2 * h, c), v11 = val(1, 2 * h + 1, c);
                 v00 = v00 > 0.f ? v00 : A.slope * v00; v01 = v01 > 0.f ? v01 : A.slope * v01;
                 v10 = v10 > 0.f ? v10 : A.slope * v10; v11 = v11 > 0.f ? v11 : A.slope * v11;
                 float best = v00; int am = 0;
@@ -211,6 +229,175 @@ __global__ void __launch_bounds__(256, 2) conv_rows_kernel(const __grid_constant
                 if (A.arg) A.arg[gi] = (unsigned char)am;
             }
         }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Filter gradient.  Block: 64 output channels x 32 input channels; thread: 8 output channels x one
+// input channel x K*K taps, all sums in registers over the block's share of the pixel tiles
+// (4 row pairs x 8 columns each), in a fixed order.  The lanes of a warp hold consecutive input
+// channels: delta reads are broadcasts, input reads hit distinct banks (odd channel stride).
+// The sums of two neighbouring output channels share a register pair, and the delta is kept in shared
+// memory with the output channels of a pixel side by side, so that one packed multiply-add (two fp32
+// FMAs, each rounded like a scalar one) serves both channels.
+// ---------------------------------------------------------------------------------------------
+template <int K> struct FgGeom {
+    static constexpr int P = K / 2, RR = K + 1;
+    static constexpr int xpitch = kStCols + 2 * P;                       // input rows hold the columns -P .. 8 + P - 1
+    static constexpr int x_rp = RR * xpitch;
+    static constexpr int x_cs = (kFgRowPairs * x_rp) | 1;                // odd channel stride
+    static constexpr int x_stage = kFgCi * x_cs;
+    static constexpr int d_px = kFgCo + 4;                               // delta: [row pair][2 rows][8 columns][64 channels + 4]: the pad spreads
+    static constexpr int d_rp = 2 * kStCols * d_px;                      //   the copies of 8 columns x 4 channels over all banks
+    static constexpr int d_stage = kFgRowPairs * d_rp;
+    static constexpr int smem_bytes = 2 * (x_stage + d_stage) * 4;
+    static constexpr int xpos = kFgRowPairs * RR * xpitch;               // input positions per channel and stage
+};
+
+struct FilterGradRowsArgs {
+    const float* dz;        // [N][Cout][H][W]: delta in front of the activation
+    const float* x;         // [N][Cin][H][W]: the layer's input
+    float* partial;         // [splits][set_floats]; the layer's filter [Cout][Cin][K][K] at filter_off, its bias at bias_off
+    long long set_floats, filter_off, bias_off;
+    int N, Cin, Cout, H, W;
+    int rp_img, x_tiles;    // row pairs per image, column tiles
+    int stages;             // (row-pair tiles) x (column tiles) over the whole batch
+    int splits;             // shares of the stages; gridDim.x = co_tiles * ci_tiles * splits
+    int co_tiles, ci_tiles;
+};
+
+template <int K>
+__global__ void __launch_bounds__(kStThreads, 2) filter_grad_rows_kernel(const __grid_constant__ FilterGradRowsArgs A)
+{
+    using G = FgGeom<K>;
+    extern __shared__ __align__(16) float st_smem[];
+    constexpr int KK = K * K, P = G::P, RR = G::RR;
+    const int tid = threadIdx.x, lane = tid & 31, cg = tid >> 5;
+    const int split = blockIdx.x % A.splits;
+    const int ci_t = (blockIdx.x / A.splits) % A.ci_tiles;
+    const int co_t = blockIdx.x / (A.splits * A.ci_tiles);
+    const int co0 = co_t * kFgCo, ci0 = ci_t * kFgCi;
+    const int s_lo = (int)((long long)split * A.stages / A.splits), s_hi = (int)((long long)(split + 1) * A.stages / A.splits);
+    float* sx = st_smem;                       // two input stages
+    float* sd = st_smem + 2 * G::x_stage;      // two delta stages
+    const size_t plane = (size_t)A.H * A.W;
+
+    // what this thread copies in every stage: one position of the input window (threads 0 .. xpos - 1, all 32
+    // channels of it), and of the delta the column `dcol` of row (dq >> 1, dq & 1) for the channels dco, dco + 16, ...
+    const int xe = tid < G::xpos ? tid : 0;
+    const int xc = xe % G::xpitch, xr = (xe / G::xpitch) % RR, xrl = xe / (G::xpitch * RR);
+    const int dcol = tid & 7, dco = (tid >> 3) & 3, dq = tid >> 5;       // a warp copies 8 columns x 4 channels of one row
+    auto load_stage = [&](int s) {
+        const int rt = s / A.x_tiles, xt = s - rt * A.x_tiles;
+        const int rp0 = rt * kFgRowPairs, x0 = xt * kStCols;
+        float* dx = sx + (s & 1) * G::x_stage;
+        float* dd = sd + (s & 1) * G::d_stage;
+        if (tid < G::xpos) {
+            const int rp = rp0 + xrl, n = rp / A.rp_img, y = (rp - n * A.rp_img) * 2 + xr - P, x = x0 + xc - P;
+            const bool ok = n < A.N && y >= 0 && y < A.H && x >= 0 && x < A.W;
+            const float* src = ok ? A.x + ((size_t)n * A.Cin + ci0) * plane + (size_t)y * A.W + x : A.x;
+            float* dst = dx + xe;
+#pragma unroll 4
+            for (int ci = 0; ci < kFgCi; ++ci) {
+                const bool okc = ok && ci0 + ci < A.Cin;
+                st_cp_async4(dst + ci * G::x_cs, okc ? src + (size_t)ci * plane : A.x, okc);
+            }
+        }
+        {
+            const int rp = rp0 + (dq >> 1), n = rp / A.rp_img, y = (rp - n * A.rp_img) * 2 + (dq & 1), x = x0 + dcol;
+            const bool ok = n < A.N && y < A.H && x < A.W;
+            const float* src = ok ? A.dz + ((size_t)n * A.Cout + co0) * plane + (size_t)y * A.W + x : A.dz;
+            float* dst = dd + (dq * kStCols + dcol) * G::d_px;
+#pragma unroll 4
+            for (int co = dco; co < kFgCo; co += 4) {
+                const bool okc = ok && co0 + co < A.Cout;
+                st_cp_async4(dst + co, okc ? src + (size_t)co * plane : A.dz, okc);
+            }
+        }
+        st_commit();
+    };
+
+    float2 acc[4][KK];                         // (channel 2c, channel 2c + 1) of the thread's eight
+    float2 bsum[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        bsum[c] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int t = 0; t < KK; ++t) acc[c][t] = make_float2(0.f, 0.f);
+    }
+    const bool with_bias = ci_t == 0;          // one input-channel slice also sums the delta itself: the bias gradient
+
+    if (s_lo < s_hi) load_stage(s_lo);
+    for (int s = s_lo; s < s_hi; ++s) {
+        if (s + 1 < s_hi) { load_stage(s + 1); st_wait<1>(); } else st_wait<0>();
+        __syncthreads();
+        const float* xb = sx + (s & 1) * G::x_stage + lane * G::x_cs;
+        const float* db = sd + (s & 1) * G::d_stage + cg * 8;
+#pragma unroll 1
+        for (int rl = 0; rl < kFgRowPairs; ++rl)
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                float w[RR][4 + 2 * P];
+#pragma unroll
+                for (int r = 0; r < RR; ++r)
+#pragma unroll
+                    for (int c = 0; c < 4 + 2 * P; ++c) w[r][c] = xb[rl * G::x_rp + r * G::xpitch + 4 * q + c];
+#pragma unroll
+                for (int p = 0; p < 2; ++p)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float* dp = db + rl * G::d_rp + (p * kStCols + 4 * q + j) * G::d_px;
+                        const float4 da = *reinterpret_cast<const float4*>(dp);
+                        const float4 dq4 = *reinterpret_cast<const float4*>(dp + 4);
+                        const float2 d[4] = {make_float2(da.x, da.y), make_float2(da.z, da.w), make_float2(dq4.x, dq4.y), make_float2(dq4.z, dq4.w)};
+                        if (with_bias) {
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) bsum[c] = __fadd2_rn(bsum[c], d[c]);
+                        }
+#pragma unroll
+                        for (int ky = 0; ky < K; ++ky)
+#pragma unroll
+                            for (int kx = 0; kx < K; ++kx) {
+                                const float2 ww = make_float2(w[p + ky][j + kx], w[p + ky][j + kx]);
+#pragma unroll
+                                for (int c = 0; c < 4; ++c) acc[c][ky * K + kx] = __ffma2_rn(d[c], ww, acc[c][ky * K + kx]);
+                            }
+                    }
+            }
+        __syncthreads();
+    }
+
+    float* set = A.partial + (size_t)split * A.set_floats;
+    const int ci = ci0 + lane;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const int co = co0 + cg * 8 + c;
+        if (co >= A.Cout) break;
+        if (ci < A.Cin) {
+            float* dst = set + A.filter_off + ((size_t)co * A.Cin + ci) * KK;
+#pragma unroll
+            for (int t = 0; t < KK; ++t) dst[t] = (c & 1) ? acc[c >> 1][t].y : acc[c >> 1][t].x;
+        }
+        if (with_bias && lane == 0) set[A.bias_off + co] = (c & 1) ? bsum[c >> 1].y : bsum[c >> 1].x;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// dZ = dY * leaky'(Y) at the conv's resolution.  pool == 0: Y is the layer's output map, element by
+// element.  pool != 0: dY and Y are the pooled maps; each pooled delta goes to the arg-max position
+// of its 2x2 window and the other three positions get zero.
+// ---------------------------------------------------------------------------------------------
+__global__ void delta_act_kernel(const float* __restrict__ dy, const float* __restrict__ y, const unsigned char* __restrict__ arg,
+                                 float* __restrict__ dz, size_t count /*elements of dy*/, int OW /*pooled width*/, float slope, int pool)
+{
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < count; e += (size_t)gridDim.x * blockDim.x) {
+        const float v = dy[e] * (y[e] > 0.f ? 1.f : slope);
+        if (!pool) { dz[e] = v; continue; }
+        const size_t row = e / OW; const int px = (int)(e - row * OW);
+        const int am = arg[e];
+        float* o = dz + (row * 2) * (size_t)(2 * OW) + 2 * px;
+        *reinterpret_cast<float2*>(o) = make_float2(am == 0 ? v : 0.f, am == 1 ? v : 0.f);
+        *reinterpret_cast<float2*>(o + 2 * OW) = make_float2(am == 2 ? v : 0.f, am == 3 ? v : 0.f);
     }
 }
 

@@ -249,7 +249,7 @@ def test_backward_split_is_refined_for_balance():
     68 of the blocks, one for the rest); 4 x 2 gives 288 smaller stacks, two for nearly every block."""
     wl = synth.workload("C1")
     layers = wl.layers[4:5]
-    mk = lambda **kw: ftp.ftp_plan(layers, wl.N, 64, 104, 104, (3, 3), ((1, 1),), **kw)
+    mk = lambda **kw: ftp.ftp_plan(layers, wl.N, 64, 104, 104, (3, 3), ((1, 1),), stationary=-1, **kw)   # as fused stacks
     first_fit, refined = mk(max_subtile=64).subtiles(1, 0), mk().subtiles(1, 0)
     assert (first_fit["rows"], first_fit["cols"]) == (9, 6)
     assert (refined["rows"], refined["cols"]) == (12, 6)
@@ -258,5 +258,5 @@ def test_backward_split_is_refined_for_balance():
     est = lambda **kw: mk(**kw).cost(1, 0, True)[1]
     assert est() < 0.97 * est(max_subtile=64)
     # fewer stacks than blocks: one block per stack
-    small = ftp.ftp_plan(layers, 1, 64, 16, 16, (2, 2), ((1, 1),), max_subtile=64).subtiles(1, 0)
+    small = ftp.ftp_plan(layers, 1, 64, 16, 16, (2, 2), ((1, 1),), max_subtile=64, stationary=-1).subtiles(1, 0)
     assert small["blocks"] == small["rows"] * small["cols"]
