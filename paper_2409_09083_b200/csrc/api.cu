@@ -41,8 +41,11 @@ int ensure_device(ftp_plan* p)
         cudaFuncSetAttribute(fwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(conv_rows_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<1>::smem_bytes) != cudaSuccess ||
-        cudaFuncSetAttribute(conv_rows_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<3>::smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(conv_rows_kernel<1, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<1, 64>::smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(conv_rows_kernel<3, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<3, 64>::smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(conv_rows_kernel<1, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<1, 32>::smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(conv_rows_kernel<3, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<3, 32>::smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(thin_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kThinSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(filter_grad_rows_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FgGeom<1>::smem_bytes) != cudaSuccess ||
         cudaFuncSetAttribute(filter_grad_rows_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, FgGeom<3>::smem_bytes) != cudaSuccess)
         return FTP_ERR_CUDA;
@@ -207,6 +210,16 @@ int forward_tc(ftp_plan* p, const float* x, const float* params, float* y, void*
     return FTP_OK;
 }
 
+// Launches the row convolution with the block shape that fits the layer's output channels.
+void launch_conv_rows(ConvRowsArgs& a, int k, int ct, int blocks, cudaStream_t st)
+{
+    a.rp_img = (a.H + 1) / 2; a.x_tiles = (a.W + kStCols - 1) / kStCols; a.co_tiles = (a.Cout + ct - 1) / ct;
+    if (k == 3 && ct == 64) conv_rows_kernel<3, 64><<<blocks, kStThreads, StGeom<3, 64>::smem_bytes, st>>>(a);
+    else if (k == 3) conv_rows_kernel<3, 32><<<blocks, kStThreads, StGeom<3, 32>::smem_bytes, st>>>(a);
+    else if (ct == 64) conv_rows_kernel<1, 64><<<blocks, kStThreads, StGeom<1, 64>::smem_bytes, st>>>(a);
+    else conv_rows_kernel<1, 32><<<blocks, kStThreads, StGeom<1, 32>::smem_bytes, st>>>(a);
+}
+
 // One-conv group run weight-stationary (stationary.cuh): the convolution with bias, activation and, where a
 // pool follows, the 2x2 maximum and its arg-max, written to the group's output map.
 bool stationary_forward(ftp_plan* p, const GroupPlan& g, int gi, const float* x, const float* params, void* ws, cudaStream_t st)
@@ -220,21 +233,32 @@ bool stationary_forward(ftp_plan* p, const GroupPlan& g, int gi, const float* x,
     a.arg = g.st.pool ? static_cast<unsigned char*>(ws) + p->ws.arg_off[op.out_map - 1] : nullptr;
     a.N = p->N; a.Cin = op.cin; a.Cout = op.cout; a.CoutPad = op.cout_pad; a.H = op.in_H; a.W = op.in_W;
     a.slope = op.slope; a.act = 1; a.pool = g.st.pool;
-    a.rp_img = (op.in_H + 1) / 2; a.x_tiles = (op.in_W + kStCols - 1) / kStCols; a.co_tiles = (op.cout + kStCoTile - 1) / kStCoTile;
     { Timed t(p, st, 1, gi);
-      if (op.k == 3) conv_rows_kernel<3><<<g.st.fwd_blocks, kStThreads, StGeom<3>::smem_bytes, st>>>(a);
-      else conv_rows_kernel<1><<<g.st.fwd_blocks, kStThreads, StGeom<1>::smem_bytes, st>>>(a); }
+      launch_conv_rows(a, op.k, g.st.fwd_co_tile, g.st.fwd_blocks, st); }
     return launched_ok();
 }
 
 // Backward of such a group: the delta in front of the activation at the conv's resolution, the partial filter
 // and bias gradients (one set per share of the pixels), and the input delta as the convolution of that
 // delta with the rotated filters (Section 4.1), written whole to `din` (may be null: not wanted).
-bool stationary_backward(ftp_plan* p, const GroupPlan& g, int gi, const float* x, const float* dout, float* din, void* ws,
-                         cudaStream_t st)
+bool stationary_backward(ftp_plan* p, const GroupPlan& g, int gi, const float* x, const float* params, const float* dout, float* din,
+                         void* ws, cudaStream_t st)
 {
     const OpDesc& op = g.bwd_ops[0];
     const int H = op.in_H, W = op.in_W;
+    if (g.st.thin) {
+        ThinBwdArgs t{};
+        t.dyp = dout; t.yp = map_ptr(p, x, ws, op.out_map);
+        t.arg = static_cast<unsigned char*>(ws) + p->ws.arg_off[op.out_map - 1];
+        t.x = map_ptr(p, x, ws, g.first); t.filter = params + op.p_off; t.dx = din;
+        t.partial = ws_ptr(ws, g.partial_off); t.set_floats = (long long)g.param_floats;
+        t.filter_off = op.gp_off; t.bias_off = op.gp_off + (long long)op.cout * op.cin * 9;
+        t.N = p->N; t.Cin = op.cin; t.Cout = op.cout; t.OH = op.out_H; t.OW = op.out_W;
+        t.tiles_y = g.st.thin_tiles_y; t.tiles_x = g.st.thin_tiles_x; t.slope = op.slope;
+        { Timed tm(p, st, 3, gi);
+          thin_bwd_kernel<<<g.st.thin_blocks, kStThreads, kThinSmemBytes, st>>>(t); }
+        return launched_ok();
+    }
     float* dz = ws_ptr(ws, p->ws.dz_off);
     const float* y = map_ptr(p, x, ws, op.out_map);
     const unsigned char* arg = g.st.pool ? static_cast<unsigned char*>(ws) + p->ws.arg_off[op.out_map - 1] : nullptr;
@@ -262,10 +286,8 @@ bool stationary_backward(ftp_plan* p, const GroupPlan& g, int gi, const float* x
         a.bias = nullptr; a.out = din; a.arg = nullptr;
         a.N = p->N; a.Cin = op.cout; a.Cout = op.cin; a.CoutPad = op.cin_pad; a.H = H; a.W = W;
         a.slope = 0.f; a.act = 0; a.pool = 0;
-        a.rp_img = (H + 1) / 2; a.x_tiles = (W + kStCols - 1) / kStCols; a.co_tiles = (op.cin + kStCoTile - 1) / kStCoTile;
         { Timed t(p, st, 8, gi);
-          if (op.k == 3) conv_rows_kernel<3><<<g.st.dx_blocks, kStThreads, StGeom<3>::smem_bytes, st>>>(a);
-          else conv_rows_kernel<1><<<g.st.dx_blocks, kStThreads, StGeom<1>::smem_bytes, st>>>(a); }
+          launch_conv_rows(a, op.k, g.st.dx_co_tile, g.st.dx_blocks, st); }
         if (!launched_ok()) return false;
     }
     return true;
@@ -369,7 +391,7 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
         if (g.st.on) {
             const float* dout = gi == G - 1 ? dy : ws_ptr(ws, p->ws.dmap_off[gi + 1]);
             float* din = gi == 0 ? dx : ws_ptr(ws, p->ws.dmap_off[gi]);
-            if (!stationary_backward(p, g, gi, x, dout, din, ws, st)) return FTP_ERR_CUDA;
+            if (!stationary_backward(p, g, gi, x, params, dout, din, ws, st)) return FTP_ERR_CUDA;
             continue;
         }
         GroupArgs a;
@@ -525,11 +547,12 @@ int ftp_plan_subtiles(const ftp_plan* plan, int pass, int group, int* rows, int*
     const GroupPlan& gp = plan->groups[group];
     if (gp.st.on) {         // weight-stationary group: row-pair tiles of the whole batch x column tiles, 256-thread blocks
         const OpDesc& op = gp.fwd_ops[0];
-        const int per = pass ? kFgRowPairs : kStRowPairs;
+        const int per = pass ? kFgRowPairs : st_row_pairs(gp.st.fwd_co_tile);
         if (rows) *rows = (plan->N * ((op.in_H + 1) / 2) + per - 1) / per;
         if (cols) *cols = (op.in_W + kStCols - 1) / kStCols;
-        if (smem_bytes) *smem_bytes = op.k == 3 ? (pass ? FgGeom<3>::smem_bytes : StGeom<3>::smem_bytes)
-                                                : (pass ? FgGeom<1>::smem_bytes : StGeom<1>::smem_bytes);
+        const bool wide = gp.st.fwd_co_tile == 64;
+        if (smem_bytes) *smem_bytes = op.k == 3 ? (pass ? FgGeom<3>::smem_bytes : wide ? StGeom<3, 64>::smem_bytes : StGeom<3, 32>::smem_bytes)
+                                                : (pass ? FgGeom<1>::smem_bytes : wide ? StGeom<1, 64>::smem_bytes : StGeom<1, 32>::smem_bytes);
         if (blocks) *blocks = pass ? gp.st.fg_blocks : gp.st.fwd_blocks;
         return FTP_OK;
     }

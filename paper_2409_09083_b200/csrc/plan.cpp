@@ -489,7 +489,7 @@ double stationary_estimate_us(const ftp_plan& p, const GroupPlan& g, bool backwa
     const OpDesc& op = g.fwd_ops[0];
     const double px = (double)p.N * op.in_H * op.in_W;
     const double flops = 2.0 * px * op.cin * op.cout * op.k * op.k;
-    const double rate = (op.k == 1 ? kStatTflops1x1 : kStatTflops) * 1e6;          // flop per microsecond
+    const double rate = (op.k == 1 || g.st.thin ? kStatTflops1x1 : kStatTflops) * 1e6;   // flop per microsecond
     const double map_us = px * (op.cin + op.cout) * 4.0 / 6.5e6;                   // bytes at 6.5 TB/s
     if (!backward) return flops / rate + map_us + 5.0;
     return flops * (need_dx ? 2.0 : 1.0) / rate + 3.0 * map_us + 15.0;
@@ -558,24 +558,47 @@ void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     if (p.precision != FTP_FP32 || o.stationary < 0 || g.n_ops != 1) return;
     const OpDesc& op = g.fwd_ops[0];
     if (op.kind == kOpPool || (op.k != 1 && op.k != 3)) return;
-    if (o.stationary == 0 && op.cin < kStatMinCin) return;
+    const bool thin = op.kind == kOpConvPool && op.k == 3 && op.cin <= 4 && op.cout <= 32;
+    if (o.stationary == 0 && op.cin < kStatMinCin && !thin) return;
     const int H = op.in_H, W = op.in_W;                        // the conv's resolution
     const long long rp_total = (long long)p.N * ((H + 1) / 2);
     const int x_tiles = (W + kStCols - 1) / kStCols;
-    const long long rp_tiles = (rp_total + kStRowPairs - 1) / kStRowPairs;
-    const long long fwd_blocks = rp_tiles * x_tiles * ((op.cout + kStCoTile - 1) / kStCoTile);
-    const long long dx_blocks = rp_tiles * x_tiles * ((op.cin + kStCoTile - 1) / kStCoTile);
+    // blocks of 64 output channels x 16 row pairs, or of 32 x 32 where that wastes fewer channels or rows, i.e. takes
+    // fewer rounds of blocks (two blocks run per SM)
+    auto conv_blocks = [&](int cout, int ct) {
+        const int rpt = st_row_pairs(ct);
+        return (rp_total + rpt - 1) / rpt * x_tiles * ((cout + ct - 1) / ct);
+    };
+    auto pick_tile = [&](int cout) {
+        if (cout <= 32) return 32;
+        const long long slots = 2LL * kSmCount;
+        // both shapes do the same work per block (64 x 16 or 32 x 32 thread tiles): what differs is how many
+        // blocks the padded channel and row counts give, i.e. how many rounds of `slots` blocks
+        const long long r64 = (conv_blocks(cout, 64) + slots - 1) / slots, r32 = (conv_blocks(cout, 32) + slots - 1) / slots;
+        return r32 < r64 ? 32 : 64;
+    };
+    const int fwd_ct = pick_tile(op.cout), dx_ct = pick_tile(op.cin);
+    const long long fwd_blocks = conv_blocks(op.cout, fwd_ct), dx_blocks = conv_blocks(op.cin, dx_ct);
     const long long stages = (rp_total + kFgRowPairs - 1) / kFgRowPairs * x_tiles;
     const long long slices = (long long)((op.cout + kFgCo - 1) / kFgCo) * ((op.cin + kFgCi - 1) / kFgCi);
     if (fwd_blocks > 0x7fffffffLL || dx_blocks > 0x7fffffffLL || stages > 0x7fffffffLL || slices > 65535) return;
     g.st.on = 1; g.st.k = op.k; g.st.pool = op.kind == kOpConvPool ? 1 : 0;
     g.st.fwd_blocks = (int)fwd_blocks; g.st.dx_blocks = (int)dx_blocks;
+    g.st.fwd_co_tile = fwd_ct; g.st.dx_co_tile = dx_ct;
     g.st.fg_stages = (int)stages;
     const long long slots = 4LL * kSmCount;                    // two rounds of two blocks per SM
     g.st.fg_splits = (int)std::max<long long>(1, std::min<long long>(stages, slots / slices));
     g.st.fg_blocks = (int)(slices * g.st.fg_splits);
     g.bwd.blocks = g.st.fg_splits;                             // partial gradient sets of the group
     g.bwd.scratch_floats = 0;                                  // the input delta is written whole, no overlapping parts to sum
+    if (thin && o.stationary <= 0) {                           // (stationary = 1 forces the general kernels, for tests)
+        g.st.thin = 1;
+        g.st.thin_tiles_y = (op.out_H + kThinTileH - 1) / kThinTileH;
+        g.st.thin_tiles_x = (op.out_W + kThinTileW - 1) / kThinTileW;
+        const long long tiles = (long long)p.N * g.st.thin_tiles_y * g.st.thin_tiles_x;
+        g.st.thin_blocks = (int)std::min<long long>(tiles, 2LL * kSmCount);
+        g.bwd.blocks = g.st.thin_blocks;                       // one partial set per block
+    }
 }
 
 struct LayerOffsets { std::vector<long long> p_off, wf_off, wb_off, twf_off, twb_off; };
@@ -934,7 +957,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     size_t scratch = 0, dz = 0;
     for (const GroupPlan& g : p.groups) {
         scratch = std::max(scratch, g.bwd.scratch_floats);
-        if (g.st.on) dz = std::max(dz, (size_t)N * g.fwd_ops[0].cout * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W);
+        if (g.st.on && !g.st.thin) dz = std::max(dz, (size_t)N * g.fwd_ops[0].cout * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W);
     }
     ws.scratch_off = take(scratch * 4);
     ws.dz_off = take(dz * 4);

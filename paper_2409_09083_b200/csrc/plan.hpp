@@ -33,11 +33,14 @@ constexpr int kTcMaxUnits = 32;           // filter-gradient accumulators per pa
 constexpr int kTcTailEntries = 16;        // 16-byte entries appended to every tile plane
 // Weight-stationary kernels of one-conv groups (stationary.cuh): 256 threads, two blocks per SM.
 constexpr int kStThreads = 256;
-constexpr int kStCoTile  = 64;            // convolution: output channels per block (8 per thread)
-constexpr int kStRowPairs = 16;           // convolution: row pairs per block, 32 threads x (2 rows x 4 columns) each
+// convolution: 64 output channels x 16 row pairs per block (8 channels x 2 rows x 4 columns per thread), or 32 x 32 for layers
+// with at most 32 output channels
+// with at most 32 output channels or with so few blocks that the last round of 64-channel blocks would leave SMs idle
+constexpr int st_row_pairs(int co_tile) { return 1024 / co_tile; }
 constexpr int kStCols    = 8;             // columns per block, both kernels
 constexpr int kFgCo = 64, kFgCi = 32;     // filter gradient: (output, input) channel slice of a block (8 x 1 per thread)
 constexpr int kFgRowPairs = 4;            // filter gradient: row pairs per pixel stage
+constexpr int kThinTileH = 8, kThinTileW = 32;   // thin-input backward: pooled pixels per tile
 constexpr int kStatMinCin = 32;           // fewest input channels for which a one-conv group runs weight-stationary by default
 constexpr double kStatTflops = 40.0;      // measured rate of the weight-stationary kernels (3x3; 1x1 runs at kStatTflops1x1), for the planner's estimates
 constexpr double kStatTflops1x1 = 20.0;
@@ -106,8 +109,11 @@ struct PassPlan {
 // Weight-stationary execution of an executed group that holds one conv layer (stationary.cuh).
 struct StatPlan {
     int on = 0;
+    int thin = 0;                           // conv3x3 + pool with at most 4 input and 32 output channels: backward by thin_bwd_kernel
+    int thin_blocks = 0, thin_tiles_y = 0, thin_tiles_x = 0;
     int k = 0, pool = 0;
-    int fwd_blocks = 0, dx_blocks = 0;      // convolution launches: (row-pair tiles) x (column tiles) x (64-channel slices)
+    int fwd_blocks = 0, dx_blocks = 0;      // convolution launches: (row-pair tiles) x (column tiles) x (channel slices)
+    int fwd_co_tile = 64, dx_co_tile = 64;  // output channels per block of the two convolutions (64 or 32)
     int fg_stages = 0, fg_splits = 0;       // filter gradient: pixel stages over the batch, and the shares they are dealt out in
     int fg_blocks = 0;                      // (64 x 32 channel slices) x shares; a share is one partial gradient set
 };

@@ -33,17 +33,19 @@ namespace ftp {
 // 3 and the right halo the first, otherwise unused, slot of the next row.  The stride between row
 // pairs is 8 or 24 modulo 32, so that the eight lanes of a quarter warp (two column quads of four row
 // pairs) read 4-wide without bank conflicts.
-template <int K> struct StGeom {
+template <int K, int CO> struct StGeom {
     static constexpr int P = K / 2, RR = K + 1;
+    static constexpr int npg = kStThreads * 8 / CO;                  // pixel groups (2 rows x 4 columns) per block: 32 or 64
+    static constexpr int row_pairs = npg / 2;                        // row pairs per block: 16 or 32
     static constexpr int pitch = kStCols + (K > 1 ? 4 : 0);
     static constexpr int rp_stride = K == 3 ? 56 : 24;
-    static constexpr int ci_stride = kStRowPairs * rp_stride;
-    static constexpr int ci_chunk = K == 3 ? 8 : 32;                 // input channels per stage
-    static constexpr int w_stage = ci_chunk * K * K * kStCoTile;     // floats
+    static constexpr int ci_stride = row_pairs * rp_stride;
+    static constexpr int ci_chunk = (K == 3 ? 8 : 32) * CO / 64;     // input channels per stage
+    static constexpr int w_stage = ci_chunk * K * K * CO;            // floats
     static constexpr int in_stage = ci_chunk * ci_stride;
     static constexpr int smem_bytes = 2 * (w_stage + in_stage) * 4;
     static constexpr int cols = kStCols + 2 * P;
-    static constexpr int npos = kStRowPairs * RR * cols;             // input positions of a stage per channel
+    static constexpr int npos = row_pairs * RR * cols;               // input positions of a stage per channel
     static constexpr int pos_per_thread = (npos + kStThreads - 1) / kStThreads;
 };
 
@@ -75,20 +77,21 @@ __device__ __forceinline__ void st_cp_async4(void* smem, const void* gmem, bool 
 __device__ __forceinline__ void st_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void st_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
 
-// K = 1 or 3 (stride 1, padding K / 2).  Thread tile: 8 output channels x (2 rows x 4 columns).
-template <int K>
+// K = 1 or 3 (stride 1, padding K / 2); CO = 64 or 32 output channels per block (32 for layers with at most 32,
+// which then take twice the row pairs).  Thread tile: 8 output channels x (2 rows x 4 columns).
+template <int K, int CO>
 __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_constant__ ConvRowsArgs A)
 {
-    using G = StGeom<K>;
+    using G = StGeom<K, CO>;
     extern __shared__ __align__(16) float st_smem[];
     constexpr int KK = K * K, P = G::P, RR = G::RR;
     const int tid = threadIdx.x;
-    const int cg = tid >> 5, pg = tid & 31;                  // a warp shares its 8 output channels: filter reads are broadcasts
+    const int cg = tid / G::npg, pg = tid % G::npg;          // a warp shares its 8 output channels: filter reads are broadcasts
     const int rp_l = pg >> 1, cq_l = pg & 1;
     const int co_t = blockIdx.x % A.co_tiles;
     const int xt = (blockIdx.x / A.co_tiles) % A.x_tiles;
     const int rt = blockIdx.x / (A.co_tiles * A.x_tiles);
-    const int co0 = co_t * kStCoTile, x0 = xt * kStCols, rp0 = rt * kStRowPairs;
+    const int co0 = co_t * CO, x0 = xt * kStCols, rp0 = rt * G::row_pairs;
     float* sw = st_smem;                                     // two filter stages
     float* si = st_smem + 2 * G::w_stage;                    // two input stages
     const size_t plane = (size_t)A.H * A.W;
@@ -115,11 +118,11 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
         float* dw = sw + (chunk & 1) * G::w_stage;
         float* di = si + (chunk & 1) * G::in_stage;
         // filters: a row of kStCoTile floats per (channel, tap)
-        constexpr int q = kStCoTile / 4;
+        constexpr int q = CO / 4;
         for (int i = tid; i < nci * KK * q; i += kStThreads) {
             const int row = i / q, j = i - row * q;
             const int co = co0 + 4 * j;
-            st_cp_async16(dw + row * kStCoTile + 4 * j, A.w + ((size_t)ci0 * KK + row) * A.CoutPad + min(co, A.CoutPad - 4), co < A.CoutPad);
+            st_cp_async16(dw + row * CO + 4 * j, A.w + ((size_t)ci0 * KK + row) * A.CoutPad + min(co, A.CoutPad - 4), co < A.CoutPad);
         }
 #pragma unroll
         for (int e = 0; e < G::pos_per_thread; ++e)
@@ -155,8 +158,8 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
         const int nci = min(G::ci_chunk, A.Cin - chunk * G::ci_chunk);
         const float* wc = sw + (chunk & 1) * G::w_stage + cg * 8;
         const float* ip = si + (chunk & 1) * G::in_stage + my_in;
-#pragma unroll 1
-        for (int ci = 0; ci < nci; ++ci, wc += KK * kStCoTile, ip += G::ci_stride) {
+#pragma unroll(K == 1 ? 4 : 1)
+        for (int ci = 0; ci < nci; ++ci, wc += KK * CO, ip += G::ci_stride) {
             float v[RR][4 + 2 * P];
 #pragma unroll
             for (int r = 0; r < RR; ++r) {
@@ -169,8 +172,8 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
             for (int kx = 0; kx < K; ++kx)
 #pragma unroll
                 for (int ky = 0; ky < K; ++ky) {
-                    const float4 wa = *reinterpret_cast<const float4*>(wc + (ky * K + kx) * kStCoTile);
-                    const float4 wq = *reinterpret_cast<const float4*>(wc + (ky * K + kx) * kStCoTile + 4);
+                    const float4 wa = *reinterpret_cast<const float4*>(wc + (ky * K + kx) * CO);
+                    const float4 wq = *reinterpret_cast<const float4*>(wc + (ky * K + kx) * CO + 4);
                     const float2 wv[4] = {make_float2(wa.x, wa.y), make_float2(wa.z, wa.w), make_float2(wq.x, wq.y), make_float2(wq.z, wq.w)};
 #pragma unroll
                     for (int p = 0; p < 2; ++p)
@@ -398,6 +401,201 @@ __global__ void delta_act_kernel(const float* __restrict__ dy, const float* __re
         float* o = dz + (row * 2) * (size_t)(2 * OW) + 2 * px;
         *reinterpret_cast<float2*>(o) = make_float2(am == 0 ? v : 0.f, am == 1 ? v : 0.f);
         *reinterpret_cast<float2*>(o + 2 * OW) = make_float2(am == 2 ? v : 0.f, am == 3 ? v : 0.f);
+    }
+}
+
+}  // namespace ftp
+
+namespace ftp {
+
+// ---------------------------------------------------------------------------------------------
+// Backward of a thin-input conv3x3 + 2x2 max-pool group (at most 4 input and 32 output channels: the
+// first layer of an image network).  The pooled delta is sparse at the conv's resolution -- one
+// non-zero per 2x2 window, at the arg-max -- so the delta in front of the activation is never laid
+// out in global memory: a block stages, for a tile of 8 x 32 pooled pixels and a ring of one pooled
+// pixel around it, v = dY * leaky'(Y) and the arg-max of every output channel, plus the input patch
+// under it, and then
+//   filter gradient: lane = output channel; per pooled pixel the 3 x 3 x Cin input values around that
+//     channel's arg-max position meet v (27 multiply-adds instead of the 108 of the zero-extended
+//     delta); the warps of a block take the pixels of a tile in turn, and the block's sums over all its
+//     tiles form one partial gradient set (Section 4.1);
+//   input delta: thread = pooled pixel, i.e. 2 x 2 input pixels x Cin channels; per output channel
+//     the 4 x 4 neighbourhood of the zero-extended delta is rebuilt from the nine surrounding pooled
+//     values and meets the filter (correlation with the 180-degree-rotated filter written out as a
+//     gather, Section 4.1).
+// ---------------------------------------------------------------------------------------------
+constexpr int kThinTH = kThinTileH, kThinTW = kThinTileW;   // pooled pixels per tile
+constexpr int kThinPH = kThinTH + 2, kThinPW = kThinTW + 2;
+constexpr int kThinVs = 33, kThinAs = 36;             // strides of the staged v (floats) and arg-max (bytes) per pooled pixel
+constexpr int kThinXH = 2 * kThinTH + 2, kThinXW = 2 * kThinTW + 2, kThinXP = kThinXW + 1;   // input patch; odd pitch
+constexpr int kThinMaxCin = 4, kThinMaxCout = 32;
+constexpr int kThinSmemV = kThinPH * kThinPW * kThinVs;                  // floats
+constexpr int kThinSmemX = kThinMaxCin * kThinXH * kThinXP;              // floats
+constexpr int kThinSmemW = kThinMaxCout * 9 * 4;                         // floats: [co][tap][ci padded to 4]
+constexpr int kThinSmemBytes = (kThinSmemV + kThinSmemX + kThinSmemW) * 4 + kThinPH * kThinPW * kThinAs;
+
+struct ThinBwdArgs {
+    const float* dyp;           // [N][Cout][OH][OW] delta at the pooled map
+    const float* yp;            // [N][Cout][OH][OW] pooled output (sign of the activation at the arg-max)
+    const unsigned char* arg;   // [N][Cout][OH][OW]
+    const float* x;             // [N][Cin][2 OH][2 OW]
+    const float* filter;        // [Cout][Cin][3][3]
+    float* dx;                  // [N][Cin][2 OH][2 OW] or null
+    float* partial;             // [gridDim.x][set_floats]
+    long long set_floats, filter_off, bias_off;
+    int N, Cin, Cout, OH, OW;
+    int tiles_y, tiles_x;       // tiles per image
+    float slope;
+};
+
+__global__ void __launch_bounds__(kStThreads, 2) thin_bwd_kernel(const __grid_constant__ ThinBwdArgs A)
+{
+    extern __shared__ __align__(16) float st_smem[];
+    float* sv = st_smem;                                   // [pooled pixel][33]: v per output channel
+    float* sx = sv + kThinSmemV;                           // [ci][row][col]: input patch, global row 2 py0 - 1 at row 0
+    float* swt = sx + kThinSmemX;                          // [co][tap][4]
+    unsigned char* sa = reinterpret_cast<unsigned char*>(swt + kThinSmemW);   // [pooled pixel][36]
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int H = 2 * A.OH, W = 2 * A.OW;
+    const size_t pplane = (size_t)A.OH * A.OW, plane = (size_t)H * W;
+
+    for (int i = tid; i < kThinMaxCout * 9 * 4; i += kStThreads) {
+        const int ci = i & 3, tap = (i >> 2) % 9, co = i / 36;
+        swt[i] = (co < A.Cout && ci < A.Cin) ? __ldg(A.filter + ((size_t)co * A.Cin + ci) * 9 + tap) : 0.f;
+    }
+    float acc[kThinMaxCin - 1][9];                         // filter gradient of (output channel = lane, input channels 0..2)
+    float acc3[9];                                         // ... input channel 3 (only with four input channels)
+    float bsum = 0.f;
+#pragma unroll
+    for (int t = 0; t < 9; ++t) { acc[0][t] = acc[1][t] = acc[2][t] = 0.f; acc3[t] = 0.f; }
+
+    const int tiles_img = A.tiles_y * A.tiles_x, tiles = A.N * tiles_img;
+    const int t_lo = (int)((long long)blockIdx.x * tiles / gridDim.x), t_hi = (int)((long long)(blockIdx.x + 1) * tiles / gridDim.x);
+    for (int tile = t_lo; tile < t_hi; ++tile) {
+        const int n = tile / tiles_img, ty = (tile % tiles_img) / A.tiles_x, tx = tile % A.tiles_x;
+        const int py0 = ty * kThinTH, px0 = tx * kThinTW;
+        __syncthreads();                                   // the previous tile has been consumed
+        // stage v and arg-max: one warp per (channel, pooled row), lanes along the row
+        for (int r = warp; r < A.Cout * kThinPH; r += kStThreads / 32) {
+            const int co = r / kThinPH, ly = r - co * kThinPH, py = py0 + ly - 1;
+            const bool row_ok = py >= 0 && py < A.OH;
+            const size_t base = ((size_t)n * A.Cout + co) * pplane + (size_t)(row_ok ? py : 0) * A.OW;
+            for (int lx = lane; lx < kThinPW; lx += 32) {
+                const int px = px0 + lx - 1;
+                float v = 0.f; unsigned char a = 0;
+                if (row_ok && px >= 0 && px < A.OW) {
+                    v = __ldg(A.dyp + base + px) * (__ldg(A.yp + base + px) > 0.f ? 1.f : A.slope);
+                    a = A.arg[base + px];
+                }
+                sv[(ly * kThinPW + lx) * kThinVs + co] = v;
+                sa[(ly * kThinPW + lx) * kThinAs + co] = a;
+            }
+        }
+        // stage the input patch
+        for (int r = warp; r < A.Cin * kThinXH; r += kStThreads / 32) {
+            const int ci = r / kThinXH, lr = r - ci * kThinXH, y = 2 * py0 - 1 + lr;
+            const bool row_ok = y >= 0 && y < H;
+            const float* src = A.x + ((size_t)n * A.Cin + ci) * plane + (size_t)(row_ok ? y : 0) * W;
+            for (int lc = lane; lc < kThinXW; lc += 32) {
+                const int xg = 2 * px0 - 1 + lc;
+                sx[(ci * kThinXH + lr) * kThinXP + lc] = (row_ok && xg >= 0 && xg < W) ? __ldg(src + xg) : 0.f;
+            }
+        }
+        __syncthreads();
+
+        // filter gradient: lane = output channel, the warps take the tile's pooled pixels in turn
+        if (lane < A.Cout) {
+            for (int p = warp; p < kThinTH * kThinTW; p += kStThreads / 32) {
+                const int wy = p >> 5, wx = p & 31;
+                const int pi = (wy + 1) * kThinPW + wx + 1;
+                const float v = sv[pi * kThinVs + lane];
+                const int a = sa[pi * kThinAs + lane];
+                bsum += v;
+                // input position of tap (0, 0): rows 2 wy + ay (+ ky), columns 2 wx + ax (+ kx) of the patch
+                const float* xp = sx + (2 * wy + (a >> 1)) * kThinXP + 2 * wx + (a & 1);
+#pragma unroll
+                for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+                    for (int kx = 0; kx < 3; ++kx) {
+#pragma unroll
+                        for (int ci = 0; ci < kThinMaxCin - 1; ++ci)
+                            acc[ci][ky * 3 + kx] = fmaf(v, xp[(ci * kThinXH + ky) * kThinXP + kx], acc[ci][ky * 3 + kx]);
+                    }
+                if (A.Cin == 4) {
+#pragma unroll
+                    for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+                        for (int kx = 0; kx < 3; ++kx)
+                            acc3[ky * 3 + kx] = fmaf(v, xp[(3 * kThinXH + ky) * kThinXP + kx], acc3[ky * 3 + kx]);
+                }
+            }
+        }
+
+        // input delta: thread = pooled pixel (wy, wx) = 2 x 2 input pixels
+        if (A.dx) {
+            const int wy = tid >> 5, wx = tid & 31;
+            float o[kThinMaxCin][2][2];
+#pragma unroll
+            for (int ci = 0; ci < kThinMaxCin; ++ci) o[ci][0][0] = o[ci][0][1] = o[ci][1][0] = o[ci][1][1] = 0.f;
+            for (int co = 0; co < A.Cout; ++co) {
+                // zero-extended delta on rows 2 py - 1 .. 2 py + 2, columns 2 px - 1 .. 2 px + 2
+                float dz[4][4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int wr = (r + 1) >> 1, wc = (c + 1) >> 1;              // 0, 1, 1, 2
+                        const int want = (((r + 1) & 1) << 1) | ((c + 1) & 1);       // arg-max that puts the value there
+                        const int pi = (wy + wr) * kThinPW + wx + wc;
+                        dz[r][c] = (int)sa[pi * kThinAs + co] == want ? sv[pi * kThinVs + co] : 0.f;
+                    }
+#pragma unroll
+                for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+                    for (int kx = 0; kx < 3; ++kx) {
+                        const float4 wv = *reinterpret_cast<const float4*>(swt + (co * 9 + ky * 3 + kx) * 4);
+                        const float wc4[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+                        for (int i = 0; i < 2; ++i)
+#pragma unroll
+                            for (int j = 0; j < 2; ++j) {
+                                const float d = dz[i - ky + 2][j - kx + 2];
+#pragma unroll
+                                for (int ci = 0; ci < kThinMaxCin; ++ci) o[ci][i][j] = fmaf(wc4[ci], d, o[ci][i][j]);
+                            }
+                    }
+            }
+            const int py = py0 + wy, px = px0 + wx;
+            if (py < A.OH && px < A.OW) {
+#pragma unroll
+                for (int ci = 0; ci < kThinMaxCin; ++ci)
+                    if (ci < A.Cin) {
+                        float* dst = A.dx + ((size_t)n * A.Cin + ci) * plane + (size_t)(2 * py) * W + 2 * px;
+                        *reinterpret_cast<float2*>(dst) = make_float2(o[ci][0][0], o[ci][0][1]);
+                        *reinterpret_cast<float2*>(dst + W) = make_float2(o[ci][1][0], o[ci][1][1]);
+                    }
+            }
+        }
+    }
+
+    // the block's partial set: the eight warps' sums per (output channel, input channel, tap), added in warp order
+    __syncthreads();
+    float* red = st_smem;                                  // [warp][lane][40]
+    {
+        float* mine = red + (warp * 32 + lane) * 40;
+#pragma unroll
+        for (int t = 0; t < 9; ++t) { mine[t] = acc[0][t]; mine[9 + t] = acc[1][t]; mine[18 + t] = acc[2][t]; mine[27 + t] = acc3[t]; }
+        mine[36] = bsum;
+    }
+    __syncthreads();
+    float* set = A.partial + (size_t)blockIdx.x * A.set_floats;
+    for (int e = tid; e < A.Cout * 37; e += kStThreads) {
+        const int co = e / 37, k = e - co * 37;
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < kStThreads / 32; ++w) s += red[(w * 32 + co) * 40 + k];
+        if (k == 36) set[A.bias_off + co] = s;
+        else if (k / 9 < A.Cin) set[A.filter_off + ((size_t)co * A.Cin + k / 9) * 9 + k % 9] = s;
     }
 }
 
