@@ -225,6 +225,15 @@ def run_ours(args):
             for name in ("C1", "C2"):
                 sub = measure(ctx, name, args.precision)
                 with_bf16(name, sub)
+                if args.precision == "fp32":
+                    # the same step with the requested grouping profile executed as it is (fused sub-tile stacks
+                    # of whole requested groups), and with fused stacks only under the planner's own cuts
+                    for key, opts in (("requested_profile_as_is", dict(strict_groups=True, stationary=-1)),
+                                      ("fused_stacks_only", dict(stationary=-1))):
+                        try:
+                            sub[key] = measure(ctx, name, "fp32", light=True, **opts)
+                        except Exception as e:                # noqa: BLE001 - e.g. the requested groups do not fit as they are
+                            sub[key] = {"unavailable": str(e)}
                 line["workloads"][name] = {k: sub[k] for k in sub if k not in ("metric", "unit", "n_gpus", "higher_is_better", "scaling",
                                                                             "vs_baseline", "data", "fp32_fma_peak")}
         print(json.dumps(line))
@@ -232,8 +241,9 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def measure(ctx, name, precision, extras=True):
-    """Times the training step of one workload at one precision; returns the JSON line (rank 0) or None."""
+def measure(ctx, name, precision, extras=True, light=False, **plan_opts):
+    """Times the training step of one workload at one precision; returns the JSON line (rank 0) or None.
+    light: only the timed steps (for the comparison runs with other planner options, given as plan_opts)."""
     args, rank, world, local, dist = ctx["args"], ctx["rank"], ctx["world"], ctx["local"], ctx["dist"]
     ftp, dp, torch = ctx["ftp"], ctx["dp"], ctx["torch"]
     wl = synth.workload(name).with_(seed=rank)                # per-GPU batch is fixed: weak scaling
@@ -243,7 +253,7 @@ def measure(ctx, name, precision, extras=True):
     tcp = precision == "bf16"
     plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=1 if tcp else 0,
                         tc_blocks_per_sm=args.tc_blocks if tcp else 0, cost_model=args.cost_model,
-                        stationary=args.stationary, strict_groups=args.strict_groups)
+                        **dict(dict(stationary=args.stationary, strict_groups=args.strict_groups), **plan_opts))
     ws = plan.new_workspace()
     xd, pd, td = (torch.from_numpy(a).cuda() for a in (x, params, target))
     dx = torch.empty_like(xd)
@@ -295,13 +305,21 @@ def measure(ctx, name, precision, extras=True):
     t_begin = time.perf_counter()
     while True:
         repeats.append(timed_steps(lambda i: step()))
-        more = torch.tensor([1.0 if time.perf_counter() - t_begin < args.min_seconds and len(repeats) < 50 else 0.0], device="cuda")
+        budget = args.min_seconds * (0.25 if light else 1.0)
+        more = torch.tensor([1.0 if time.perf_counter() - t_begin < budget and len(repeats) < 50 else 0.0], device="cuda")
         if dist is not None:
             dist.broadcast(more, 0)
         if more.item() == 0.0:
             break
     launches = (plan.launch_count() - launches0) // len(repeats)
     total_ms = statistics.median(repeats)
+    if light:
+        if sampler:
+            sampler.stop()
+        return {"value": world * wl.N * steps / (total_ms / 1e3), "unit": UNIT, "ms_per_step": total_ms / steps,
+                "executed_groups": [list(g) for g in plan.exec_groups()],
+                "stationary_groups": [bool(plan.group_mode(i)[0]) for i in range(len(plan.exec_groups()))],
+                "gpu_launches": int(launches), "workspace_bytes": plan.workspace_bytes}
     # K more steps with an event pair around every launch of the library (ftp_plan_timing) for the per-kernel
     # breakdown and the launch durations of the roofline: the events do not change a kernel's duration, but
     # their records between the launches would lengthen the step, so they stay out of the timed steps.

@@ -375,6 +375,17 @@ long long ftp_plan_launch_count(const ftp_plan* plan);
  */
 int ftp_plan_check(ftp_plan* plan, void* workspace, void* stream);
 
+/*
+ * Diagnostic for the error path above (the paper has no counterpart): launches, on `stream`, one small
+ * kernel whose only thread waits on a barrier that nothing arrives on, through the same bounded-wait
+ * routine as the bf16 tile kernels but with a limit of about `limit_us` microseconds (1 .. 100000, counted
+ * in SM clock cycles at a nominal 2 GHz).  The wait runs out, the kernel sets the workspace's error word
+ * and returns; nothing faults and the context stays usable.  The next ftp_plan_check then reports
+ * FTP_ERR_TIMEOUT; the next ftp_forward / ftp_step* clears the word again.  bf16 plans only
+ * (FTP_ERR_PRECISION otherwise); FTP_ERR_ARG on a null or unaligned pointer or a limit out of range.
+ */
+int ftp_plan_wait_probe(ftp_plan* plan, void* workspace, int limit_us, void* stream);
+
 const char* ftp_strerror(int code);
 
 #ifdef __cplusplus

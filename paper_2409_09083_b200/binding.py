@@ -100,6 +100,8 @@ _lib.ftp_plan_launch_count.argtypes = [_vp]
 _lib.ftp_plan_launch_count.restype = ctypes.c_longlong
 _lib.ftp_plan_check.argtypes = [_vp, _vp, _vp]
 _lib.ftp_plan_check.restype = _i
+_lib.ftp_plan_wait_probe.argtypes = [_vp, _vp, _i, _vp]
+_lib.ftp_plan_wait_probe.restype = _i
 _lib.ftp_strerror.argtypes = [_i]
 _lib.ftp_strerror.restype = ctypes.c_char_p
 
@@ -280,6 +282,10 @@ class Plan:
     def check(self, workspace, stream=None):
         """Synchronise and raise FtpError(FTP_ERR_TIMEOUT) if a device-side wait of the bf16 path ran out."""
         _check(_lib.ftp_plan_check(self._h, _workspace(self, workspace).ptr, _stream(stream)))
+
+    def wait_probe(self, workspace, limit_us=2000, stream=None):
+        """Launches the kernel whose bounded wait runs out on purpose (see ftp_plan_wait_probe in ftp.h)."""
+        _check(_lib.ftp_plan_wait_probe(self._h, _workspace(self, workspace).ptr, int(limit_us), _stream(stream)))
 
     def new_workspace(self, device="cuda"):
         return torch.empty(self.workspace_bytes, dtype=torch.uint8, device=device)

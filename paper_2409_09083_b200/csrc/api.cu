@@ -793,6 +793,15 @@ int ftp_plan_check(ftp_plan* plan, void* workspace, void* stream)
     return word ? FTP_ERR_TIMEOUT : FTP_OK;
 }
 
+int ftp_plan_wait_probe(ftp_plan* plan, void* workspace, int limit_us, void* stream)
+{
+    if (!plan || !workspace || !aligned256(workspace) || limit_us <= 0 || limit_us > 100000) return FTP_ERR_ARG;
+    if (!is_tc(plan)) return FTP_ERR_PRECISION;
+    ++plan->launches;
+    tcd::wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(err_ptr(workspace, plan), (long long)limit_us * 2000);
+    return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
+}
+
 const char* ftp_strerror(int code)
 {
     switch (code) {

@@ -81,6 +81,19 @@ __device__ __forceinline__ bool wait_or_fail(Pipe& p, unsigned long long* bar, u
     return false;
 }
 
+// Exercises the give-up path of the bounded waits on its own: one thread sets up a barrier that nothing ever
+// arrives on and waits on it through the same routine as the tile kernels, with a limit of `limit_cycles`
+// instead of seconds; the wait runs out, the error word is set and the kernel returns.
+__global__ void wait_probe_kernel(int* error, long long limit_cycles)
+{
+    __shared__ unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+        if (!mbar_wait(smem_u32(&bar), 0, limit_cycles)) atomicExch(error, 1);
+    }
+}
+
 __device__ __forceinline__ uint4 pack8(const float* v)
 {
     __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);

@@ -935,11 +935,19 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
             ws.map_off[op.out_map - 1] = take((size_t)N * s.C * s.H * s.W * 4);
             if (op.kind == kOpConvPool) ws.arg_off[op.out_map - 1] = take((size_t)N * s.C * s.H * s.W);
         }
+    // Deltas at the inputs of the executed groups 1..: the backward pass of group gi reads the one at its output
+    // (index gi + 1) and writes the one at its input (index gi), so two areas, taken in turn, hold them all.
     ws.dmap_off.assign(n_exec, 0);
-    for (int gi = 1; gi < n_exec; ++gi) {
-        const MapShape& s = p.maps[p.groups[gi].first - 1];
-        ws.dmap_off[gi] = tcp ? take((size_t)N * round_up(s.C, 16) * s.H * s.W * 2)     // bf16 planes
-                              : take((size_t)N * s.C * s.H * s.W * 4);
+    {
+        size_t need[2] = {0, 0};
+        for (int gi = 1; gi < n_exec; ++gi) {
+            const MapShape& s = p.maps[p.groups[gi].first - 1];
+            const size_t bytes = tcp ? (size_t)N * round_up(s.C, 16) * s.H * s.W * 2     // bf16 planes
+                                     : (size_t)N * s.C * s.H * s.W * 4;
+            need[gi & 1] = std::max(need[gi & 1], bytes);
+        }
+        const size_t area[2] = {take(need[0]), take(need[1])};
+        for (int gi = 1; gi < n_exec; ++gi) ws.dmap_off[gi] = area[gi & 1];
     }
     {
         const MapShape& s = p.maps[n_layers];

@@ -124,16 +124,17 @@ __device__ __forceinline__ bool mbar_try(uint32_t mbar, uint32_t parity)
         : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Waits for the phase with the given parity to complete, for at most ~2 s; false = gave up.
-// Every wait of the tile kernels goes through here, so a missing arrival ends the kernel with an
-// error word instead of hanging it.
-__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity)
+// Waits for the phase with the given parity to complete, for at most `limit_cycles` SM clock cycles
+// (default: about 2 s) and 2^26 polls; false = gave up.  Every wait of the tile kernels goes through
+// here, so a missing arrival ends the kernel with an error word instead of hanging it.
+constexpr long long kWaitLimitCycles = 4000000000ll;
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, long long limit_cycles = kWaitLimitCycles)
 {
     if (mbar_try(mbar, parity)) return true;
     const long long t0 = clock64();
     for (int it = 0; it < (1 << 26); ++it) {
         if (mbar_try(mbar, parity)) return true;
-        if (clock64() - t0 > 4000000000ll) break;
+        if (clock64() - t0 > limit_cycles) break;
     }
     return false;
 }

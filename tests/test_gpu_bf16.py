@@ -424,3 +424,35 @@ def test_full_size_activations_against_the_plain_oracle(name):
         worst = max(worst, _crop_check_plain(wl, x, params, y, n, oy, ox, size) / scale)
     print(name, "bf16 path vs plain fp64 oracle, worst sampled activation error", worst)
     assert worst <= BF16_TOL
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    """The bf16 kernels never wait without a limit: a wait that runs out sets an error word that
+    ftp_plan_check turns into FTP_ERR_TIMEOUT.  The probe kernel waits, through the same routine but
+    with a limit of 2 ms, on a barrier nothing arrives on; afterwards an ordinary step on the same plan
+    and workspace runs, is checked clean and gives the result it gave before."""
+    from paper_2409_09083_b200 import binding
+    wl = synth.workload("C0")
+    x, params, target = synth.draw(wl, bias_std=0.3)
+    x, params = bf16_grid(x), bf16_grid(params)
+    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=BF16)
+    ws = plan.new_workspace()
+    xd, pd = torch.from_numpy(x).cuda(), torch.from_numpy(params).cuda()
+    y0 = torch.empty((1, 16, 16, 16), dtype=torch.float32, device="cuda")
+    ftp.ftp_forward(plan, xd, pd, y0, ws)
+    plan.check(ws)                                           # clean
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    plan.wait_probe(ws, limit_us=2000)
+    t1.record()
+    with pytest.raises(binding.FtpError) as e:
+        plan.check(ws)
+    assert e.value.code == -7 and "wait" in str(e.value)     # FTP_ERR_TIMEOUT
+    assert 0.5 <= t0.elapsed_time(t1) <= 50.0                # it waited about the limit, not the default seconds
+    y1 = torch.empty_like(y0)
+    ftp.ftp_forward(plan, xd, pd, y1, ws)                    # clears the error word
+    plan.check(ws)
+    assert torch.equal(y0, y1)
+    fp32_plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups)
+    with pytest.raises(binding.FtpError):
+        fp32_plan.wait_probe(fp32_plan.new_workspace())       # the fp32 path has no device-side waits
