@@ -10,7 +10,7 @@
 #include "kernels.cuh"
 #include "kernels_tc.cuh"
 #include "plan.hpp"
-#include "stationary.cuh"
+#include "stationary_args.hpp"
 
 using namespace ftp;
 
@@ -41,13 +41,7 @@ int ensure_device(ftp_plan* p)
         cudaFuncSetAttribute(fwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(conv_rows_kernel<1, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<1, 64>::smem_bytes) != cudaSuccess ||
-        cudaFuncSetAttribute(conv_rows_kernel<3, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<3, 64>::smem_bytes) != cudaSuccess ||
-        cudaFuncSetAttribute(conv_rows_kernel<1, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<1, 32>::smem_bytes) != cudaSuccess ||
-        cudaFuncSetAttribute(conv_rows_kernel<3, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<3, 32>::smem_bytes) != cudaSuccess ||
-        cudaFuncSetAttribute(thin_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kThinSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(filter_grad_rows_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FgGeom<1>::smem_bytes) != cudaSuccess ||
-        cudaFuncSetAttribute(filter_grad_rows_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, FgGeom<3>::smem_bytes) != cudaSuccess)
+        !st_prepare_device())
         return FTP_ERR_CUDA;
     const size_t bytes = p->tables.size() * sizeof(int);
     if (cudaMalloc(&p->dev_tables, bytes) != cudaSuccess) return FTP_ERR_CUDA;
@@ -210,16 +204,6 @@ int forward_tc(ftp_plan* p, const float* x, const float* params, float* y, void*
     return FTP_OK;
 }
 
-// Launches the row convolution with the block shape that fits the layer's output channels.
-void launch_conv_rows(ConvRowsArgs& a, int k, int ct, int blocks, cudaStream_t st)
-{
-    a.rp_img = (a.H + 1) / 2; a.x_tiles = (a.W + kStCols - 1) / kStCols; a.co_tiles = (a.Cout + ct - 1) / ct;
-    if (k == 3 && ct == 64) conv_rows_kernel<3, 64><<<blocks, kStThreads, StGeom<3, 64>::smem_bytes, st>>>(a);
-    else if (k == 3) conv_rows_kernel<3, 32><<<blocks, kStThreads, StGeom<3, 32>::smem_bytes, st>>>(a);
-    else if (ct == 64) conv_rows_kernel<1, 64><<<blocks, kStThreads, StGeom<1, 64>::smem_bytes, st>>>(a);
-    else conv_rows_kernel<1, 32><<<blocks, kStThreads, StGeom<1, 32>::smem_bytes, st>>>(a);
-}
-
 // One-conv group run weight-stationary (stationary.cuh): the convolution with bias, activation and, where a
 // pool follows, the 2x2 maximum and its arg-max, written to the group's output map.
 bool stationary_forward(ftp_plan* p, const GroupPlan& g, int gi, const float* x, const float* params, void* ws, cudaStream_t st)
@@ -234,7 +218,7 @@ bool stationary_forward(ftp_plan* p, const GroupPlan& g, int gi, const float* x,
     a.N = p->N; a.Cin = op.cin; a.Cout = op.cout; a.CoutPad = op.cout_pad; a.H = op.in_H; a.W = op.in_W;
     a.slope = op.slope; a.act = 1; a.pool = g.st.pool;
     { Timed t(p, st, 1, gi);
-      launch_conv_rows(a, op.k, g.st.fwd_co_tile, g.st.fwd_blocks, st); }
+      st_launch_conv_rows(a, op.k, g.st.fwd_co_tile, g.st.fwd_blocks, st); }
     return launched_ok();
 }
 
@@ -256,7 +240,7 @@ bool stationary_backward(ftp_plan* p, const GroupPlan& g, int gi, const float* x
         t.N = p->N; t.Cin = op.cin; t.Cout = op.cout; t.OH = op.out_H; t.OW = op.out_W;
         t.tiles_y = g.st.thin_tiles_y; t.tiles_x = g.st.thin_tiles_x; t.slope = op.slope;
         { Timed tm(p, st, 3, gi);
-          thin_bwd_kernel<<<g.st.thin_blocks, kStThreads, kThinSmemBytes, st>>>(t); }
+          st_launch_thin_bwd(t, g.st.thin_blocks, st); }
         return launched_ok();
     }
     float* dz = ws_ptr(ws, p->ws.dz_off);
@@ -264,20 +248,16 @@ bool stationary_backward(ftp_plan* p, const GroupPlan& g, int gi, const float* x
     const unsigned char* arg = g.st.pool ? static_cast<unsigned char*>(ws) + p->ws.arg_off[op.out_map - 1] : nullptr;
     const size_t count = (size_t)p->N * op.cout * op.out_H * op.out_W;
     { Timed t(p, st, 6, gi);
-      const int blocks = (int)std::min<size_t>((count + 255) / 256, (size_t)kSmCount * 16);
-      delta_act_kernel<<<blocks, 256, 0, st>>>(dout, y, arg, dz, count, op.out_W, op.slope, g.st.pool); }
+      st_launch_delta_act(dout, y, arg, dz, count, op.out_W, op.slope, g.st.pool, st); }
     if (!launched_ok()) return false;
     FilterGradRowsArgs f{};
     f.dz = dz; f.x = map_ptr(p, x, ws, g.first);
     f.partial = ws_ptr(ws, g.partial_off); f.set_floats = (long long)g.param_floats;
     f.filter_off = op.gp_off; f.bias_off = op.gp_off + (long long)op.cout * op.cin * op.k * op.k;
     f.N = p->N; f.Cin = op.cin; f.Cout = op.cout; f.H = H; f.W = W;
-    f.rp_img = (H + 1) / 2; f.x_tiles = (W + kStCols - 1) / kStCols;
     f.stages = g.st.fg_stages; f.splits = g.st.fg_splits;
-    f.co_tiles = (op.cout + kFgCo - 1) / kFgCo; f.ci_tiles = (op.cin + kFgCi - 1) / kFgCi;
     { Timed t(p, st, 7, gi);
-      if (op.k == 3) filter_grad_rows_kernel<3><<<g.st.fg_blocks, kStThreads, FgGeom<3>::smem_bytes, st>>>(f);
-      else filter_grad_rows_kernel<1><<<g.st.fg_blocks, kStThreads, FgGeom<1>::smem_bytes, st>>>(f); }
+      st_launch_filter_grad_rows(f, op.k, g.st.fg_blocks, st); }
     if (!launched_ok()) return false;
     if (din) {
         ConvRowsArgs a{};
@@ -287,7 +267,7 @@ bool stationary_backward(ftp_plan* p, const GroupPlan& g, int gi, const float* x
         a.N = p->N; a.Cin = op.cout; a.Cout = op.cin; a.CoutPad = op.cin_pad; a.H = H; a.W = W;
         a.slope = 0.f; a.act = 0; a.pool = 0;
         { Timed t(p, st, 8, gi);
-          launch_conv_rows(a, op.k, g.st.dx_co_tile, g.st.dx_blocks, st); }
+          st_launch_conv_rows(a, op.k, g.st.dx_co_tile, g.st.dx_blocks, st); }
         if (!launched_ok()) return false;
     }
     return true;
@@ -550,9 +530,7 @@ int ftp_plan_subtiles(const ftp_plan* plan, int pass, int group, int* rows, int*
         const int per = pass ? kFgRowPairs : st_row_pairs(gp.st.fwd_co_tile);
         if (rows) *rows = (plan->N * ((op.in_H + 1) / 2) + per - 1) / per;
         if (cols) *cols = (op.in_W + kStCols - 1) / kStCols;
-        const bool wide = gp.st.fwd_co_tile == 64;
-        if (smem_bytes) *smem_bytes = op.k == 3 ? (pass ? FgGeom<3>::smem_bytes : wide ? StGeom<3, 64>::smem_bytes : StGeom<3, 32>::smem_bytes)
-                                                : (pass ? FgGeom<1>::smem_bytes : wide ? StGeom<1, 64>::smem_bytes : StGeom<1, 32>::smem_bytes);
+        if (smem_bytes) *smem_bytes = pass ? st_filter_grad_smem_bytes(op.k) : st_conv_smem_bytes(op.k, gp.st.fwd_co_tile);
         if (blocks) *blocks = pass ? gp.st.fg_blocks : gp.st.fwd_blocks;
         return FTP_OK;
     }

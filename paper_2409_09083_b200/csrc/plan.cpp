@@ -579,14 +579,18 @@ void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     };
     const int fwd_ct = pick_tile(op.cout), dx_ct = pick_tile(op.cin);
     const long long fwd_blocks = conv_blocks(op.cout, fwd_ct), dx_blocks = conv_blocks(op.cin, dx_ct);
-    const long long stages = (rp_total + kFgRowPairs - 1) / kFgRowPairs * x_tiles;
-    const long long slices = (long long)((op.cout + kFgCo - 1) / kFgCo) * ((op.cin + kFgCi - 1) / kFgCi);
+    // filter gradient: 3 x 3 in stages of 4 row pairs x 8 columns and 64 x 32 channel slices; 1 x 1 as a contraction over
+    // stages of 32 flat pixels of an image and 64 x 128 channel slices
+    const long long stages = op.k == 1 ? (long long)p.N * ((H * W + kFg1Px - 1) / kFg1Px)
+                                       : (rp_total + kFgRowPairs - 1) / kFgRowPairs * x_tiles;
+    const long long slices = op.k == 1 ? (long long)((op.cout + kFg1Co - 1) / kFg1Co) * ((op.cin + kFg1Ci - 1) / kFg1Ci)
+                                       : (long long)((op.cout + kFgCo - 1) / kFgCo) * ((op.cin + kFgCi - 1) / kFgCi);
     if (fwd_blocks > 0x7fffffffLL || dx_blocks > 0x7fffffffLL || stages > 0x7fffffffLL || slices > 65535) return;
     g.st.on = 1; g.st.k = op.k; g.st.pool = op.kind == kOpConvPool ? 1 : 0;
     g.st.fwd_blocks = (int)fwd_blocks; g.st.dx_blocks = (int)dx_blocks;
     g.st.fwd_co_tile = fwd_ct; g.st.dx_co_tile = dx_ct;
     g.st.fg_stages = (int)stages;
-    const long long slots = 4LL * kSmCount;                    // two rounds of two blocks per SM
+    const long long slots = (op.k == 1 ? 6LL : 4LL) * kSmCount;   // two rounds of the blocks that run at once (2 per SM; 1 x 1: 3)
     g.st.fg_splits = (int)std::max<long long>(1, std::min<long long>(stages, slots / slices));
     g.st.fg_blocks = (int)(slices * g.st.fg_splits);
     g.bwd.blocks = g.st.fg_splits;                             // partial gradient sets of the group

@@ -40,6 +40,7 @@ constexpr int st_row_pairs(int co_tile) { return 1024 / co_tile; }
 constexpr int kStCols    = 8;             // columns per block, both kernels
 constexpr int kFgCo = 64, kFgCi = 32;     // filter gradient: (output, input) channel slice of a block (8 x 1 per thread)
 constexpr int kFgRowPairs = 4;            // filter gradient: row pairs per pixel stage
+constexpr int kFg1Co = 64, kFg1Ci = 128, kFg1Px = 32;   // filter gradient of a 1 x 1 conv: channel slice of a block, pixels per stage
 constexpr int kThinTileH = 8, kThinTileW = 32;   // thin-input backward: pooled pixels per tile
 constexpr int kStatMinCin = 32;           // fewest input channels for which a one-conv group runs weight-stationary by default
 constexpr double kStatTflops = 40.0;      // measured rate of the weight-stationary kernels (3x3; 1x1 runs at kStatTflops1x1), for the planner's estimates

@@ -25,6 +25,7 @@
 #include <cuda_runtime.h>
 
 #include "plan.hpp"
+#include "stationary_args.hpp"
 
 namespace ftp {
 
@@ -45,21 +46,6 @@ template <int K, int CO> struct StGeom {
     static constexpr int in_stage = ci_chunk * ci_stride;
     static constexpr int smem_bytes = 2 * (w_stage + in_stage) * 4;
     static constexpr int cols = kStCols + 2 * P;
-    static constexpr int npos = row_pairs * RR * cols;               // input positions of a stage per channel
-    static constexpr int pos_per_thread = (npos + kStThreads - 1) / kStThreads;
-};
-
-struct ConvRowsArgs {
-    const float* in;        // [N][Cin][H][W]
-    const float* w;         // [Cin][K*K][CoutPad]: per input channel and tap, the 8-padded output channels
-    const float* bias;      // [Cout] or null
-    float* out;             // [N][Cout][H][W], or the pooled map [N][Cout][H/2][W/2] when pool != 0
-    unsigned char* arg;     // pool: arg-max (dy * 2 + dx, first maximum in row-major order) per pooled value
-    int N, Cin, Cout, CoutPad, H, W;
-    float slope;            // leaky-ReLU slope (act != 0)
-    int act, pool;          // act == 0: plain sums (input delta)
-    int rp_img;             // row pairs per image = ceil(H / 2)
-    int x_tiles, co_tiles;  // blockIdx.x = (rp_tile * x_tiles + x_tile) * co_tiles + co_tile
 };
 
 __device__ __forceinline__ void st_cp_async16(void* smem, const void* gmem, bool valid)
@@ -74,12 +60,19 @@ __device__ __forceinline__ void st_cp_async4(void* smem, const void* gmem, bool 
     const int bytes = valid ? 4 : 0;
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" :: "r"(s), "l"(gmem), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void st_cp_async8(void* smem, const void* gmem, bool valid)
+{
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    const int bytes = valid ? 8 : 0;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" :: "r"(s), "l"(gmem), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void st_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void st_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
 
 // K = 1 or 3 (stride 1, padding K / 2); CO = 64 or 32 output channels per block (32 for layers with at most 32,
 // which then take twice the row pairs).  Thread tile: 8 output channels x (2 rows x 4 columns).
-template <int K, int CO>
+// VEC = floats per copy of the input columns: 4 where the map's rows are 16-byte aligned (width a multiple of 4), else 2 or 1.
+template <int K, int CO, int VEC>
 __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_constant__ ConvRowsArgs A)
 {
     using G = StGeom<K, CO>;
@@ -96,20 +89,31 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
     float* si = st_smem + 2 * G::w_stage;                    // two input stages
     const size_t plane = (size_t)A.H * A.W;
 
-    // input positions this thread copies in every stage: (row pair, row, column) -> shared / global offsets
-    int pos_s[G::pos_per_thread]; long long pos_g[G::pos_per_thread]; unsigned pos_ok = 0;
+    // What this thread copies of the input in every stage.  A row of a row pair is copied as its left halo
+    // column (3 x 3 only), its eight columns in pieces of VEC floats and its right halo column; piece i of the
+    // block is (row pair, row, piece of the row).
+    constexpr int vec = VEC;
+    constexpr int per_row = kStCols / vec + 2 * P, nitems = G::row_pairs * RR * per_row;
+    constexpr int max_items = (nitems + kStThreads - 1) / kStThreads;
+    int it_s[max_items]; long long it_g[max_items]; unsigned it_ok = 0, it_halo = 0;
 #pragma unroll
-    for (int e = 0; e < G::pos_per_thread; ++e) {
+    for (int e = 0; e < max_items; ++e) {
         const int idx = tid + e * kStThreads;
-        pos_s[e] = -1; pos_g[e] = 0;
-        if (idx < G::npos) {
-            const int c = idx % G::cols, t = idx / G::cols, r = t % RR, rl = t / RR;
+        it_s[e] = -1; it_g[e] = 0;
+        if (idx < nitems) {
+            const int piece = idx % per_row, t = idx / per_row, r = t % RR, rl = t / RR;
+            // column of the piece relative to the block's first column, and whether it is a single halo column
+            int c; bool halo = false;
+            if (P && piece == 0) { c = -1; halo = true; }
+            else if (P && piece == per_row - 1) { c = kStCols; halo = true; }
+            else c = (piece - P) * vec;
             const int rp = rp0 + rl;
-            const int n = rp / A.rp_img, y = (rp - n * A.rp_img) * 2 + r - P, x = x0 + c - P;
-            pos_s[e] = rl * G::rp_stride + r * G::pitch + c + (4 - P);
-            if (n < A.N && y >= 0 && y < A.H && x >= 0 && x < A.W) {
-                pos_ok |= 1u << e;
-                pos_g[e] = (long long)n * A.Cin * plane + (long long)y * A.W + x;
+            const int n = rp / A.rp_img, y = (rp - n * A.rp_img) * 2 + r - P, x = x0 + c;
+            it_s[e] = rl * G::rp_stride + r * G::pitch + c + 4;
+            if (halo) it_halo |= 1u << e;
+            if (n < A.N && y >= 0 && y < A.H && x >= 0 && x < A.W) {     // a piece lies wholly inside or outside the row
+                it_ok |= 1u << e;
+                it_g[e] = (long long)n * A.Cin * plane + (long long)y * A.W + x;
             }
         }
     }
@@ -117,7 +121,7 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
         const int ci0 = chunk * G::ci_chunk, nci = min(G::ci_chunk, A.Cin - ci0);
         float* dw = sw + (chunk & 1) * G::w_stage;
         float* di = si + (chunk & 1) * G::in_stage;
-        // filters: a row of kStCoTile floats per (channel, tap)
+        // filters: a row of CO floats per (channel, tap)
         constexpr int q = CO / 4;
         for (int i = tid; i < nci * KK * q; i += kStThreads) {
             const int row = i / q, j = i - row * q;
@@ -125,12 +129,15 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
             st_cp_async16(dw + row * CO + 4 * j, A.w + ((size_t)ci0 * KK + row) * A.CoutPad + min(co, A.CoutPad - 4), co < A.CoutPad);
         }
 #pragma unroll
-        for (int e = 0; e < G::pos_per_thread; ++e)
-            if (pos_s[e] >= 0) {
-                const bool ok = (pos_ok >> e) & 1u;
-                const float* src = A.in + pos_g[e] + (size_t)ci0 * plane;
-                float* dst = di + pos_s[e];
-                for (int ci = 0; ci < nci; ++ci) st_cp_async4(dst + ci * G::ci_stride, src + (size_t)ci * plane, ok);
+        for (int e = 0; e < max_items; ++e)
+            if (it_s[e] >= 0) {
+                const bool ok = (it_ok >> e) & 1u;
+                const float* src = A.in + it_g[e] + (size_t)ci0 * plane;
+                float* dst = di + it_s[e];
+                const int w = ((it_halo >> e) & 1u) ? 1 : vec;
+                if (w == 4) for (int ci = 0; ci < nci; ++ci) st_cp_async16(dst + ci * G::ci_stride, src + (size_t)ci * plane, ok);
+                else if (w == 2) for (int ci = 0; ci < nci; ++ci) st_cp_async8(dst + ci * G::ci_stride, src + (size_t)ci * plane, ok);
+                else for (int ci = 0; ci < nci; ++ci) st_cp_async4(dst + ci * G::ci_stride, src + (size_t)ci * plane, ok);
             }
         st_commit();
     };
@@ -244,6 +251,7 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
 // memory with the output channels of a pixel side by side, so that one packed multiply-add (two fp32
 // FMAs, each rounded like a scalar one) serves both channels.
 // ---------------------------------------------------------------------------------------------
+static_assert(2 * kFgRowPairs == kStThreads / 32, "one warp per delta row of a stage");
 template <int K> struct FgGeom {
     static constexpr int P = K / 2, RR = K + 1;
     static constexpr int xpitch = kStCols + 2 * P;                       // input rows hold the columns -P .. 8 + P - 1
@@ -255,18 +263,6 @@ template <int K> struct FgGeom {
     static constexpr int d_stage = kFgRowPairs * d_rp;
     static constexpr int smem_bytes = 2 * (x_stage + d_stage) * 4;
     static constexpr int xpos = kFgRowPairs * RR * xpitch;               // input positions per channel and stage
-};
-
-struct FilterGradRowsArgs {
-    const float* dz;        // [N][Cout][H][W]: delta in front of the activation
-    const float* x;         // [N][Cin][H][W]: the layer's input
-    float* partial;         // [splits][set_floats]; the layer's filter [Cout][Cin][K][K] at filter_off, its bias at bias_off
-    long long set_floats, filter_off, bias_off;
-    int N, Cin, Cout, H, W;
-    int rp_img, x_tiles;    // row pairs per image, column tiles
-    int stages;             // (row-pair tiles) x (column tiles) over the whole batch
-    int splits;             // shares of the stages; gridDim.x = co_tiles * ci_tiles * splits
-    int co_tiles, ci_tiles;
 };
 
 template <int K>
@@ -286,10 +282,10 @@ __global__ void __launch_bounds__(kStThreads, 2) filter_grad_rows_kernel(const _
     const size_t plane = (size_t)A.H * A.W;
 
     // what this thread copies in every stage: one position of the input window (threads 0 .. xpos - 1, all 32
-    // channels of it), and of the delta the column `dcol` of row (dq >> 1, dq & 1) for the channels dco, dco + 16, ...
+    // channels of it), and of the delta the column `dcol` of its warp's row for the channels dco, dco + 4, ...
     const int xe = tid < G::xpos ? tid : 0;
     const int xc = xe % G::xpitch, xr = (xe / G::xpitch) % RR, xrl = xe / (G::xpitch * RR);
-    const int dcol = tid & 7, dco = (tid >> 3) & 3, dq = tid >> 5;       // a warp copies 8 columns x 4 channels of one row
+    const int dcol = tid & 7, dco = (tid >> 3) & 3, dq = tid >> 5;       // warp dq copies row (dq >> 1, dq & 1): 8 columns x 4 channels at a time
     auto load_stage = [&](int s) {
         const int rt = s / A.x_tiles, xt = s - rt * A.x_tiles;
         const int rp0 = rt * kFgRowPairs, x0 = xt * kStCols;
@@ -386,6 +382,100 @@ __global__ void __launch_bounds__(kStThreads, 2) filter_grad_rows_kernel(const _
 }
 
 // ---------------------------------------------------------------------------------------------
+// Filter gradient of a 1 x 1 conv: a plain contraction over pixels, dW[co][ci] = sum_p dZ[co][p] X[ci][p].
+// Block: 64 output x 128 input channels; thread: 4 output x 8 input channels (two groups of four, 64
+// channels apart, so that the 16 lanes that differ in input channels read consecutive 16-byte pieces).
+// A stage is 32 consecutive pixels of one image, kept in shared memory pixel-major ([pixel][channel],
+// padded by 4) for both operands; the sums of two neighbouring input channels share a register pair.
+// ---------------------------------------------------------------------------------------------
+constexpr int kF1Co = kFg1Co, kF1Ci = kFg1Ci, kF1Px = kFg1Px;
+constexpr int kF1Ds = kF1Co + 4, kF1Xs = kF1Ci + 4;                     // floats per pixel of the delta / input stage
+constexpr int kF1Stage = kF1Px * (kF1Ds + kF1Xs);                       // floats
+constexpr int kF1SmemBytes = 2 * kF1Stage * 4;
+
+__global__ void __launch_bounds__(kStThreads, 3) filter_grad_1x1_kernel(const __grid_constant__ FilterGradRowsArgs A)
+{
+    extern __shared__ __align__(16) float st_smem[];
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int cig = tid & 15, cog = tid >> 4;              // a warp: 16 input-channel groups x 2 output-channel groups
+    const int split = blockIdx.x % A.splits;
+    const int ci_t = (blockIdx.x / A.splits) % A.ci_tiles;
+    const int co_t = blockIdx.x / (A.splits * A.ci_tiles);
+    const int co0 = co_t * kF1Co, ci0 = ci_t * kF1Ci;
+    const int HW = A.H * A.W, per_img = (HW + kF1Px - 1) / kF1Px;     // stages = N * per_img (A.stages)
+    const int s_lo = (int)((long long)split * A.stages / A.splits), s_hi = (int)((long long)(split + 1) * A.stages / A.splits);
+
+    // copies: a warp takes 8 pixels x 4 channels at a time (conflict-free with the padded pixel stride)
+    const int cpx = lane & 7, cch = lane >> 3, cw = tid >> 5;
+    auto load_stage = [&](int s) {
+        const int n = s / per_img, p0 = (s - n * per_img) * kF1Px;
+        float* sd = st_smem + (s & 1) * kF1Stage;
+        float* sx = sd + kF1Px * kF1Ds;
+        const float* dsrc = A.dz + ((size_t)n * A.Cout + co0) * HW + p0;
+        const float* xsrc = A.x + ((size_t)n * A.Cin + ci0) * HW + p0;
+        // tasks: (pixel octet q of 4) x (channel quad): delta 4 x 16, input 4 x 32
+        for (int t = cw; t < 4 * (kF1Co / 4); t += kStThreads / 32) {
+            const int q = t & 3, ch = (t >> 2) * 4 + cch, p = q * 8 + cpx;
+            const bool ok = p0 + p < HW && co0 + ch < A.Cout;
+            st_cp_async4(sd + p * kF1Ds + ch, ok ? dsrc + (size_t)ch * HW + p : A.dz, ok);
+        }
+        for (int t = cw; t < 4 * (kF1Ci / 4); t += kStThreads / 32) {
+            const int q = t & 3, ch = (t >> 2) * 4 + cch, p = q * 8 + cpx;
+            const bool ok = p0 + p < HW && ci0 + ch < A.Cin;
+            st_cp_async4(sx + p * kF1Xs + ch, ok ? xsrc + (size_t)ch * HW + p : A.x, ok);
+        }
+        st_commit();
+    };
+
+    float2 acc[4][4];                          // [output channel][pair of input channels]
+    float bsum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[c][i] = make_float2(0.f, 0.f);
+    const bool with_bias = ci_t == 0 && cig == 0;
+
+    if (s_lo < s_hi) load_stage(s_lo);
+    for (int s = s_lo; s < s_hi; ++s) {
+        if (s + 1 < s_hi) { load_stage(s + 1); st_wait<1>(); } else st_wait<0>();
+        __syncthreads();
+        const float* dp = st_smem + (s & 1) * kF1Stage + cog * 4;
+        const float* xp = st_smem + (s & 1) * kF1Stage + kF1Px * kF1Ds + cig * 4;
+#pragma unroll 4
+        for (int p = 0; p < kF1Px; ++p) {
+            const float4 d = *reinterpret_cast<const float4*>(dp + p * kF1Ds);
+            const float4 xa = *reinterpret_cast<const float4*>(xp + p * kF1Xs);
+            const float4 xb = *reinterpret_cast<const float4*>(xp + p * kF1Xs + 64);
+            const float2 xv[4] = {make_float2(xa.x, xa.y), make_float2(xa.z, xa.w), make_float2(xb.x, xb.y), make_float2(xb.z, xb.w)};
+            const float dv[4] = {d.x, d.y, d.z, d.w};
+            if (with_bias) { bsum[0] += d.x; bsum[1] += d.y; bsum[2] += d.z; bsum[3] += d.w; }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const float2 dd = make_float2(dv[c], dv[c]);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[c][i] = __ffma2_rn(dd, xv[i], acc[c][i]);
+            }
+        }
+        __syncthreads();
+    }
+
+    float* set = A.partial + (size_t)split * A.set_floats;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const int co = co0 + cog * 4 + c;
+        if (co >= A.Cout) break;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int ci = ci0 + cig * 4 + (i >> 1) * 64 + (i & 1) * 2;
+            float* dst = set + A.filter_off + (size_t)co * A.Cin + ci;
+            if (ci < A.Cin) dst[0] = acc[c][i].x;
+            if (ci + 1 < A.Cin) dst[1] = acc[c][i].y;
+        }
+        if (with_bias) set[A.bias_off + co] = bsum[c];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // dZ = dY * leaky'(Y) at the conv's resolution.  pool == 0: Y is the layer's output map, element by
 // element.  pool != 0: dY and Y are the pooled maps; each pooled delta goes to the arg-max position
 // of its 2x2 window and the other three positions get zero.
@@ -433,20 +523,6 @@ constexpr int kThinSmemV = kThinPH * kThinPW * kThinVs;                  // floa
 constexpr int kThinSmemX = kThinMaxCin * kThinXH * kThinXP;              // floats
 constexpr int kThinSmemW = kThinMaxCout * 9 * 4;                         // floats: [co][tap][ci padded to 4]
 constexpr int kThinSmemBytes = (kThinSmemV + kThinSmemX + kThinSmemW) * 4 + kThinPH * kThinPW * kThinAs;
-
-struct ThinBwdArgs {
-    const float* dyp;           // [N][Cout][OH][OW] delta at the pooled map
-    const float* yp;            // [N][Cout][OH][OW] pooled output (sign of the activation at the arg-max)
-    const unsigned char* arg;   // [N][Cout][OH][OW]
-    const float* x;             // [N][Cin][2 OH][2 OW]
-    const float* filter;        // [Cout][Cin][3][3]
-    float* dx;                  // [N][Cin][2 OH][2 OW] or null
-    float* partial;             // [gridDim.x][set_floats]
-    long long set_floats, filter_off, bias_off;
-    int N, Cin, Cout, OH, OW;
-    int tiles_y, tiles_x;       // tiles per image
-    float slope;
-};
 
 __global__ void __launch_bounds__(kStThreads, 2) thin_bwd_kernel(const __grid_constant__ ThinBwdArgs A)
 {
