@@ -266,8 +266,11 @@ def measure(ctx, name, precision, extras=True, light=False, **plan_opts):
         if world == 1:
             ftp.ftp_step(plan, xd, pd, wl.lr, ws, target=td, loss_out=loss, dx=dx)
         else:
-            ftp.ftp_step_grad(plan, xd, pd, grad, ws, target=td, loss_out=loss, dx=dx)
-            dp.allreduce_and_update(grad, wl.lr, world, dist.all_reduce, lambda g, lr: ftp.ftp_sgd(pd, g, lr))
+            # every executed group's gradient slice is all-reduced on a communication stream as soon as it is
+            # complete, while the groups before it are back-propagated; the update follows the last slice
+            ex = dp.cuda_overlap(torch, dist, grad, world)
+            ftp.ftp_step_grad_groups(plan, xd, pd, grad, ws, ex.ready, target=td, loss_out=loss, dx=dx)
+            ex.finish(wl.lr, lambda g, lr: ftp.ftp_sgd(pd, g, lr), join=ex.join)
 
     def barrier():
         if dist is not None:

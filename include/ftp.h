@@ -323,8 +323,8 @@ int ftp_prefetch_host(ftp_plan* plan, const float* x_host, const float* target_h
 
 /*
  * The two halves of ftp_step for data-parallel replicas (one process per GPU, the batch split
- * across them; Section 4.1 sums the partial gradient sets "once per batch", which across GPUs is
- * an all-reduce the caller runs between these two calls):
+ * across them; Section 4.1 sums the partial gradient sets one time for each batch, which across GPUs
+ * is an all-reduce the caller runs between these two calls):
  * ftp_step_grad = ftp_step without the update: forward, loss delta, backward, and the fixed-order
  *   sum of this GPU's partial sets written to dparams (device, same layout as params).
  * ftp_sgd = params[i] -= lr * grad[i] for i < count (device pointers).
@@ -333,6 +333,22 @@ int ftp_step_grad(ftp_plan* plan, const float* x, const float* dy, const float* 
                   const float* params, float* dparams, float* loss_out, float* dx,
                   void* workspace, void* stream);
 int ftp_sgd(float* params, const float* grad, size_t count, float lr, void* stream);
+
+/*
+ * ftp_step_grad that tells the caller when the gradient of each executed group is complete, so that its
+ * all-reduce can run while the groups before it are still being back-propagated (the paper's devices send
+ * their partial sets to the common device at the end of the batch, Section 4.1; between GPUs the sets of the
+ * last layers can travel while the first layers still compute).  Groups finish in reverse order.  Right
+ * after the launches that write parameters [param_begin, param_begin + param_floats) of dparams have been
+ * put on `stream`, `ready` is called ON THE HOST, in the calling thread: the work is queued, not done, so the
+ * callee orders its own work behind it (record an event on `stream`, make the communication stream wait for
+ * it).  Every parameter is reported exactly once.  The sums are the same, in the same order, as
+ * ftp_step_grad's: dparams is bit-identical.  `ready` may be NULL (then this is ftp_step_grad).
+ */
+typedef void (*ftp_group_ready_fn)(void* user, int group, long long param_begin, long long param_floats);
+int ftp_step_grad_groups(ftp_plan* plan, const float* x, const float* dy, const float* target,
+                         const float* params, float* dparams, float* loss_out, float* dx,
+                         void* workspace, void* stream, ftp_group_ready_fn ready, void* user);
 
 /*
  * Per-launch device timing for benchmarks.  ftp_plan_timing(plan, 1) makes every later call on

@@ -78,6 +78,9 @@ _lib.ftp_prefetch_host.argtypes = [_vp, _vp, _vp, _vp, _vp]
 _lib.ftp_prefetch_host.restype = _i
 _lib.ftp_step_grad.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.ftp_step_grad.restype = _i
+GROUP_READY_FN = ctypes.CFUNCTYPE(None, _vp, _i, ctypes.c_longlong, ctypes.c_longlong)
+_lib.ftp_step_grad_groups.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, GROUP_READY_FN, _vp]
+_lib.ftp_step_grad_groups.restype = _i
 _lib.ftp_loss_mse.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.ftp_loss_mse.restype = _i
 _lib.ftp_loss_mse_static.argtypes = [_vp, _vp, _vp, _vp, _sz, _vp]
@@ -324,6 +327,28 @@ def ftp_step_grad(plan, x, params, dparams, workspace, dy=None, target=None, los
                                           (params, "params", plan.param_floats), (dparams, "dparams", plan.param_floats),
                                           (loss_out, "loss_out", 1, True), (dx, "dx", plan.in_floats, True))
     _check(_lib.ftp_step_grad(plan._h, px, pdy, pt, pp, pg, pl, pdx, ws.ptr, _stream(stream)))
+
+
+def ftp_step_grad_groups(plan, x, params, dparams, workspace, ready, dy=None, target=None, loss_out=None, dx=None, stream=None):
+    """ftp_step_grad that calls ready(group, param_begin, param_floats) on the host as soon as the launches that
+    complete an executed group's slice of dparams are queued on the stream (groups finish in reverse order)."""
+    ws = _workspace(plan, workspace)
+    px, pdy, pt, pp, pg, pl, pdx = _sized((x, "x", plan.in_floats), (dy, "dy", plan.out_floats, True),
+                                          (target, "target", plan.out_floats, True),
+                                          (params, "params", plan.param_floats), (dparams, "dparams", plan.param_floats),
+                                          (loss_out, "loss_out", 1, True), (dx, "dx", plan.in_floats, True))
+    errors = []
+
+    def trampoline(_user, group, begin, count):
+        try:
+            ready(int(group), int(begin), int(count))
+        except BaseException as e:            # noqa: BLE001 - must not unwind through the C frames
+            errors.append(e)
+    cb = GROUP_READY_FN(trampoline)
+    rc = _lib.ftp_step_grad_groups(plan._h, px, pdy, pt, pp, pg, pl, pdx, ws.ptr, _stream(stream), cb, None)
+    if errors:
+        raise errors[0]
+    _check(rc)
 
 
 def ftp_loss_mse(plan, y, target, dy, loss_out, workspace, stream=None):

@@ -321,6 +321,22 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
           if (g.bwd.ctas == 2) bwd_group_tc_kernel<256><<<g.bwd.blocks, 256, smem, st>>>(a, tile_bytes, kTcTmemCols / 2, g.bwd.stages);
           else bwd_group_tc_kernel<512><<<g.bwd.blocks, 512, smem, st>>>(a, tile_bytes, kTcTmemCols, g.bwd.stages); }
         if (!launched_ok()) return FTP_ERR_CUDA;
+        if (p->group_ready && g.param_floats) {       // ftp_step_grad_groups: this group's sets are summed right away
+            TcReduceArgs rg{};
+            for (int i = 0; i < g.n_ops; ++i) {
+                const OpDesc& op = g.bwd_ops[i];
+                if (op.kind == kOpPool) continue;
+                rg.l[rg.n++] = TcReduceLayer{op.p_off, ws_ptr(ws, g.partial_off), (long long)g.param_floats, op.tgp_off,
+                                             g.bwd.blocks, op.cin, op.cout, op.k, op.cin16, op.cout16};
+            }
+            { Timed t(p, st, 5, gi);
+              reduce_sgd_tc_kernel<<<dim3(1184, rg.n), 128, 0, st>>>(rg, nullptr, 0.f, grad_out); }
+            if (!launched_ok()) return FTP_ERR_CUDA;
+            long long floats = 0;
+            for (int i = 0; i < g.n_ops; ++i)
+                if (g.bwd_ops[i].kind != kOpPool) floats += (long long)g.bwd_ops[i].cout * g.bwd_ops[i].cin * g.bwd_ops[i].k * g.bwd_ops[i].k + g.bwd_ops[i].cout;
+            p->group_ready(p->group_ready_user, gi, g.param_begin, floats);
+        }
         if (a.need_dx) {
             const MapShape& s = p->maps[g.first - 1];
             const bool planes = g.first > 1;          // group input is a saved bf16 map: deltas travel as planes too
@@ -340,6 +356,7 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
             if (!launched_ok()) return FTP_ERR_CUDA;
         }
     }
+    if (p->group_ready) return launched_ok() ? FTP_OK : FTP_ERR_CUDA;      // summed group by group above
     TcReduceArgs ra{};
     auto flush = [&]() {
         if (!ra.n) return;
@@ -359,6 +376,24 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
     return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
 }
 
+// ftp_step_grad_groups: the sum of ONE executed group's partial sets, launched as soon as its backward pass is
+// queued, and the caller's notification.  Same per-parameter sums as the reduction over all groups.
+int reduce_group_and_notify(ftp_plan* p, int gi, float* grad_out, void* ws, cudaStream_t st)
+{
+    const GroupPlan& g = p->groups[gi];
+    if (g.param_floats == 0) return FTP_OK;
+    ReduceArgs ra{};
+    ra.n = 1;
+    ra.g[0] = ReduceGroup{g.param_begin, (long long)g.param_floats, ws_ptr(ws, g.partial_off), g.bwd.blocks};
+    const long long first = g.param_begin, total = g.param_begin + (long long)g.param_floats;
+    const int blocks = (int)std::min<long long>(((long long)g.param_floats + 255) / 256, (long long)kSmCount * 16);
+    { Timed t(p, st, 5, gi);
+      reduce_sgd_kernel<<<blocks, 256, 0, st>>>(ra, first, total, nullptr, 0.f, grad_out); }
+    if (!launched_ok()) return FTP_ERR_CUDA;
+    p->group_ready(p->group_ready_user, gi, first, (long long)g.param_floats);
+    return FTP_OK;
+}
+
 // Backward of all groups in reverse order, halo sums at the group inputs, then the cross-tile
 // reduction; `sgd_params` non-null applies the update in the same kernel.
 int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* params, float* dx, float* grad_out,
@@ -372,6 +407,7 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
             const float* dout = gi == G - 1 ? dy : ws_ptr(ws, p->ws.dmap_off[gi + 1]);
             float* din = gi == 0 ? dx : ws_ptr(ws, p->ws.dmap_off[gi]);
             if (!stationary_backward(p, g, gi, x, params, dout, din, ws, st)) return FTP_ERR_CUDA;
+            if (p->group_ready) { const int rc = reduce_group_and_notify(p, gi, grad_out, ws, st); if (rc != FTP_OK) return rc; }
             continue;
         }
         GroupArgs a;
@@ -386,6 +422,7 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
           if (max_window(g) <= 3) bwd_group_kernel<3><<<g.bwd.blocks, kThreads, g.bwd.smem_bytes, st>>>(a);
           else bwd_group_kernel<7><<<g.bwd.blocks, kThreads, g.bwd.smem_bytes, st>>>(a); }
         if (!launched_ok()) return FTP_ERR_CUDA;
+        if (p->group_ready) { const int rc = reduce_group_and_notify(p, gi, grad_out, ws, st); if (rc != FTP_OK) return rc; }
         if (a.need_dx) {
             const MapShape& s = p->maps[g.first - 1];
             HaloSumArgs h{};
@@ -402,6 +439,7 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
             if (!launched_ok()) return FTP_ERR_CUDA;
         }
     }
+    if (p->group_ready) return FTP_OK;       // every group's sets were summed right after its backward pass
     ReduceArgs ra{};
     for (const GroupPlan& g : p->groups) {
         if (g.param_floats == 0) continue;
@@ -411,7 +449,7 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
         const long long total = (long long)p->param_floats;
         const int blocks = (int)std::min<long long>((total + 255) / 256, (long long)kSmCount * 16);
         { Timed t(p, st, 5, -1);
-          reduce_sgd_kernel<<<blocks, 256, 0, st>>>(ra, total, sgd_params, lr, grad_out); }
+          reduce_sgd_kernel<<<blocks, 256, 0, st>>>(ra, 0, total, sgd_params, lr, grad_out); }
         if (!launched_ok()) return FTP_ERR_CUDA;
     }
     return FTP_OK;
@@ -715,6 +753,17 @@ int ftp_step_grad(ftp_plan* plan, const float* x, const float* dy, const float* 
 {
     if (!dparams) return FTP_ERR_ARG;
     return step_impl(plan, x, dy, target, params, nullptr, 0.f, dparams, loss_out, dx, workspace, stream);
+}
+
+int ftp_step_grad_groups(ftp_plan* plan, const float* x, const float* dy, const float* target, const float* params,
+                         float* dparams, float* loss_out, float* dx, void* workspace, void* stream,
+                         ftp_group_ready_fn ready, void* user)
+{
+    if (!plan || !dparams) return FTP_ERR_ARG;
+    plan->group_ready = ready; plan->group_ready_user = user;
+    const int rc = step_impl(plan, x, dy, target, params, nullptr, 0.f, dparams, loss_out, dx, workspace, stream);
+    plan->group_ready = nullptr; plan->group_ready_user = nullptr;
+    return rc;
 }
 
 int ftp_sgd(float* params, const float* grad, size_t count, float lr, void* stream)

@@ -1005,10 +1005,11 @@ __global__ void pack_filters_kernel(const __grid_constant__ PackArgs A, const fl
 
 // Cross-tile reduction of the partial gradient sets in a fixed order, fused with the update
 // (Section 4.1: the sets are summed once per batch and the result updates F_l).
-__global__ void reduce_sgd_kernel(const __grid_constant__ ReduceArgs A, long long total, float* __restrict__ params,
+__global__ void reduce_sgd_kernel(const __grid_constant__ ReduceArgs A, long long first, long long total, float* __restrict__ params,
                                   float lr, float* __restrict__ grad_out)
 {
-    for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    // parameters first .. total - 1 (the groups of A cover them)
+    for (long long e = first + blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
         int g = 0;
         while (g + 1 < A.n && e >= A.g[g + 1].begin) ++g;
         const long long local = e - A.g[g].begin;

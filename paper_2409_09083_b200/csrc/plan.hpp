@@ -182,6 +182,8 @@ struct ftp_plan {
     bool slot_used[2] = {false, false};
     int cur_slot = 0, pre_slot = -1;
     const float* pre_x = nullptr; const float* pre_t = nullptr;
+    // ftp_step_grad_groups: called on the host right after the launches that complete an executed group's summed gradient
+    ftp_group_ready_fn group_ready = nullptr; void* group_ready_user = nullptr;
 };
 
 namespace ftp {

@@ -392,6 +392,46 @@ def test_step_grad_then_sgd_equals_step(precision):
     assert np.isfinite(grad.cpu().numpy()).all() and float(grad.abs().max()) > 0
 
 
+@pytest.mark.parametrize("precision", [0, 1])
+@pytest.mark.parametrize("stationary", [0, -1])
+def test_group_by_group_gradient_is_the_same_gradient(precision, stationary):
+    """ftp_step_grad_groups reports every executed group's slice of the gradient once, last group first, and
+    leaves bit for bit the gradient, loss and input gradient of ftp_step_grad; the slices, handed to the
+    overlapped exchange at world size 1, give the update of ftp_step."""
+    from paper_2409_09083_b200 import dp
+    wl = Y8.with_(groups=((1, 4), (5, 8)))
+    x, params, target = synth.draw(wl, bias_std=0.1)
+    lr = 0.05
+    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=precision, stationary=stationary)
+    ws = plan.new_workspace()
+    xd, td = torch.from_numpy(x).cuda(), torch.from_numpy(target).cuda()
+    pd = torch.from_numpy(params.copy()).cuda()
+    ga, gb = torch.full_like(pd, float("nan")), torch.full_like(pd, float("nan"))
+    la, lb = torch.zeros(1, device="cuda"), torch.zeros(1, device="cuda")
+    dxa, dxb = torch.empty_like(xd), torch.empty_like(xd)
+    ftp.ftp_step_grad(plan, xd, pd, ga, ws, target=td, loss_out=la, dx=dxa)
+    ex = dp.OverlappedExchange(gb, 1, all_reduce=None)
+    ftp.ftp_step_grad_groups(plan, xd, pd, gb, ws, ex.ready, target=td, loss_out=lb, dx=dxb)
+    plan.check(ws)
+    groups = [g for g, _, c in ex.slices]
+    assert groups == sorted(groups, reverse=True) and len(set(groups)) == len(groups)
+    assert len(groups) == len(plan.exec_groups())                       # every executed group of this stack holds a conv
+    assert sum(c for _, _, c in ex.slices) == plan.param_floats
+    assert np.array_equal(ga.cpu().numpy(), gb.cpu().numpy())
+    assert la.item() == lb.item() and np.array_equal(dxa.cpu().numpy(), dxb.cpu().numpy())
+    ex.finish(lr, lambda g, lr_eff: ftp.ftp_sgd(pd, g, lr_eff))
+    pa = torch.from_numpy(params.copy()).cuda()
+    ftp.ftp_step(plan, xd, pa, lr, ws, target=td)
+    torch.cuda.synchronize()
+    assert np.array_equal(pa.cpu().numpy(), pd.cpu().numpy())
+
+    def boom(group, begin, count):
+        raise KeyError("from the callback")
+    with pytest.raises(KeyError):                                        # an exception in the callback surfaces after the call
+        ftp.ftp_step_grad_groups(plan, xd, pd, gb, ws, boom, target=td)
+    torch.cuda.synchronize()
+
+
 def test_two_half_batches_reproduce_the_full_batch_update():
     """Data-parallel arithmetic on one GPU: the gradients of the two halves of a batch (ftp_step_grad on
     each, as two ranks would), summed and applied by ftp_sgd with lr / 2, equal the full-batch update
