@@ -43,6 +43,17 @@ int ensure_device(ftp_plan* p)
         cudaFuncSetAttribute(bwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         !st_prepare_device())
         return FTP_ERR_CUDA;
+    if (!p->grad_stream) {
+        cudaStream_t gs;
+        if (cudaStreamCreateWithFlags(&gs, cudaStreamNonBlocking) != cudaSuccess) return FTP_ERR_CUDA;
+        p->grad_stream = gs;
+        for (int i = 0; i < 2; ++i) {
+            cudaEvent_t a, b;
+            if (cudaEventCreateWithFlags(&a, cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&b, cudaEventDisableTiming) != cudaSuccess) return FTP_ERR_CUDA;
+            p->ev_dz[i] = a; p->ev_fg[i] = b;
+        }
+    }
     const size_t bytes = p->tables.size() * sizeof(int);
     if (cudaMalloc(&p->dev_tables, bytes) != cudaSuccess) return FTP_ERR_CUDA;
     if (cudaMemcpy(p->dev_tables, p->tables.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess) return FTP_ERR_CUDA;
@@ -243,22 +254,39 @@ bool stationary_backward(ftp_plan* p, const GroupPlan& g, int gi, const float* x
           st_launch_thin_bwd(t, g.st.thin_blocks, st); }
         return launched_ok();
     }
-    float* dz = ws_ptr(ws, p->ws.dz_off);
+    // The filter gradient and the input delta both read dZ and nothing else of each other, so the filter gradient
+    // runs on the plan's side stream: the blocks of one kernel fill the SMs that the last, partly filled round of the
+    // other leaves idle.  dZ areas are taken in turn; an area is reused only after the filter gradient that read it.
+    // (With per-launch timing or per-group notification on, everything stays on the caller's stream.)
+    const bool side = !p->timing && !p->group_ready && din != nullptr;
+    const int turn = p->dz_turn++ & 1;
+    cudaStream_t gs = side ? static_cast<cudaStream_t>(p->grad_stream) : st;
+    float* dz = ws_ptr(ws, p->ws.dz_off + (size_t)turn * p->ws.dz_bytes);
     const float* y = map_ptr(p, x, ws, op.out_map);
     const unsigned char* arg = g.st.pool ? static_cast<unsigned char*>(ws) + p->ws.arg_off[op.out_map - 1] : nullptr;
     const size_t count = (size_t)p->N * op.cout * op.out_H * op.out_W;
+    if (p->fg_pending[turn]) {
+        if (cudaStreamWaitEvent(st, static_cast<cudaEvent_t>(p->ev_fg[turn]), 0) != cudaSuccess) return false;
+        p->fg_pending[turn] = false;
+    }
     { Timed t(p, st, 6, gi);
       st_launch_delta_act(dout, y, arg, dz, count, op.out_W, op.slope, g.st.pool, st); }
     if (!launched_ok()) return false;
+    if (side && (cudaEventRecord(static_cast<cudaEvent_t>(p->ev_dz[turn]), st) != cudaSuccess ||
+                 cudaStreamWaitEvent(gs, static_cast<cudaEvent_t>(p->ev_dz[turn]), 0) != cudaSuccess)) return false;
     FilterGradRowsArgs f{};
     f.dz = dz; f.x = map_ptr(p, x, ws, g.first);
     f.partial = ws_ptr(ws, g.partial_off); f.set_floats = (long long)g.param_floats;
     f.filter_off = op.gp_off; f.bias_off = op.gp_off + (long long)op.cout * op.cin * op.k * op.k;
     f.N = p->N; f.Cin = op.cin; f.Cout = op.cout; f.H = H; f.W = W;
     f.stages = g.st.fg_stages; f.splits = g.st.fg_splits;
-    { Timed t(p, st, 7, gi);
-      st_launch_filter_grad_rows(f, op.k, g.st.fg_blocks, st); }
+    { Timed t(p, gs, 7, gi);
+      st_launch_filter_grad_rows(f, op.k, g.st.fg_blocks, gs); }
     if (!launched_ok()) return false;
+    if (side) {
+        if (cudaEventRecord(static_cast<cudaEvent_t>(p->ev_fg[turn]), gs) != cudaSuccess) return false;
+        p->fg_pending[turn] = true;
+    }
     if (din) {
         ConvRowsArgs a{};
         a.in = dz;
@@ -439,6 +467,11 @@ int backward_impl(ftp_plan* p, const float* x, const float* dy, const float* par
             if (!launched_ok()) return FTP_ERR_CUDA;
         }
     }
+    for (int turn = 0; turn < 2; ++turn)     // the filter gradients on the side stream join here
+        if (p->fg_pending[turn]) {
+            if (cudaStreamWaitEvent(st, static_cast<cudaEvent_t>(p->ev_fg[turn]), 0) != cudaSuccess) return FTP_ERR_CUDA;
+            p->fg_pending[turn] = false;
+        }
     if (p->group_ready) return FTP_OK;       // every group's sets were summed right after its backward pass
     ReduceArgs ra{};
     for (const GroupPlan& g : p->groups) {
@@ -524,6 +557,13 @@ void ftp_plan_destroy(ftp_plan* plan)
     if (!plan) return;
     ftp_plan_timing(plan, 0);
     if (plan->dev_tables) cudaFree(plan->dev_tables);
+    if (plan->grad_stream) {
+        cudaStreamDestroy(static_cast<cudaStream_t>(plan->grad_stream));
+        for (int i = 0; i < 2; ++i) {
+            cudaEventDestroy(static_cast<cudaEvent_t>(plan->ev_dz[i]));
+            cudaEventDestroy(static_cast<cudaEvent_t>(plan->ev_fg[i]));
+        }
+    }
     if (plan->copy_stream) {
         cudaStreamDestroy(static_cast<cudaStream_t>(plan->copy_stream));
         cudaEventDestroy(static_cast<cudaEvent_t>(plan->ev_fork));

@@ -590,8 +590,10 @@ void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     g.st.fwd_blocks = (int)fwd_blocks; g.st.dx_blocks = (int)dx_blocks;
     g.st.fwd_co_tile = fwd_ct; g.st.dx_co_tile = dx_ct;
     g.st.fg_stages = (int)stages;
-    const long long slots = (op.k == 1 ? 6LL : 4LL) * kSmCount;   // two rounds of the blocks that run at once (2 per SM; 1 x 1: 3)
-    g.st.fg_splits = (int)std::max<long long>(1, std::min<long long>(stages, slots / slices));
+    // one round of the blocks that run at once (2 per SM; 1 x 1: 3): the input-delta convolution on the other stream fills
+    // what a round leaves idle, and every share costs a partial set that the reduction has to read; at least 4 stages a share
+    const long long slots = (op.k == 1 ? 3LL : 2LL) * kSmCount;
+    g.st.fg_splits = (int)std::max<long long>(1, std::min<long long>(std::max<long long>(1, stages / 4), slots / slices));
     g.st.fg_blocks = (int)(slices * g.st.fg_splits);
     g.bwd.blocks = g.st.fg_splits;                             // partial gradient sets of the group
     g.bwd.scratch_floats = 0;                                  // the input delta is written whole, no overlapping parts to sum
@@ -972,7 +974,8 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         if (g.st.on && !g.st.thin) dz = std::max(dz, (size_t)N * g.fwd_ops[0].cout * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W);
     }
     ws.scratch_off = take(scratch * 4);
-    ws.dz_off = take(dz * 4);
+    ws.dz_bytes = align_up(dz * 4, 256);
+    ws.dz_off = take(2 * ws.dz_bytes);
     ws.wf_off = take(p.wf_floats * (tcp ? 2 : 4));
     ws.wb_off = take(p.wb_floats * (tcp ? 2 : 4));
     ws.err_off = take(256);

@@ -141,7 +141,8 @@ struct Workspace {                 // byte offsets, all 256-aligned
     std::vector<size_t> dmap_off;  // delta maps at group inputs of groups 1.. (index = group), and slot for dY
     size_t dy_off = 0;             // loss delta at the last map (ftp_step with target)
     size_t scratch_off = 0;
-    size_t dz_off = 0;             // weight-stationary groups: delta in front of the activation at the conv's resolution (largest such layer)
+    size_t dz_off = 0, dz_bytes = 0;   // weight-stationary groups: two areas (taken in turn) for the delta in front of the activation at
+                                       // the conv's resolution, each as large as the largest such layer needs
     size_t wf_off = 0, wb_off = 0; // packed filters
     size_t partial_off = 0;
     size_t grad_off = 0;           // summed gradient (ftp_step keeps it internal)
@@ -182,6 +183,10 @@ struct ftp_plan {
     bool slot_used[2] = {false, false};
     int cur_slot = 0, pre_slot = -1;
     const float* pre_x = nullptr; const float* pre_t = nullptr;
+    // weight-stationary groups: the filter gradients run on a side stream beside the input-delta convolutions
+    void* grad_stream = nullptr; void* ev_dz[2] = {nullptr, nullptr}; void* ev_fg[2] = {nullptr, nullptr};
+    bool fg_pending[2] = {false, false};
+    int dz_turn = 0;
     // ftp_step_grad_groups: called on the host right after the launches that complete an executed group's summed gradient
     ftp_group_ready_fn group_ready = nullptr; void* group_ready_user = nullptr;
 };
