@@ -37,7 +37,10 @@ bool conv_attr()
 bool st_prepare_device()
 {
     return conv_attr<1, 64>() && conv_attr<3, 64>() && conv_attr<1, 32>() && conv_attr<3, 32>() &&
-           cudaFuncSetAttribute(thin_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kThinSmemBytes) == cudaSuccess &&
+           cudaFuncSetAttribute(thin_bwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kThinSmemBytes) == cudaSuccess &&
+           cudaFuncSetAttribute(thin_bwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kThinSmemBytes) == cudaSuccess &&
+           cudaFuncSetAttribute(thin_bwd_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kThinSmemBytes) == cudaSuccess &&
+           cudaFuncSetAttribute(thin_bwd_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kThinSmemBytes) == cudaSuccess &&
            cudaFuncSetAttribute(filter_grad_1x1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kF1SmemBytes) == cudaSuccess &&
            cudaFuncSetAttribute(filter_grad_rows_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, FgGeom<3>::smem_bytes) == cudaSuccess;
 }
@@ -80,7 +83,13 @@ void st_launch_delta_act(const float* dy, const float* y, const unsigned char* a
 
 void st_launch_thin_bwd(const ThinBwdArgs& a, int blocks, void* stream)
 {
-    thin_bwd_kernel<<<blocks, kStThreads, kThinSmemBytes, static_cast<cudaStream_t>(stream)>>>(a);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    switch (a.Cin) {
+    case 1: thin_bwd_kernel<1><<<blocks, kStThreads, kThinSmemBytes, st>>>(a); break;
+    case 2: thin_bwd_kernel<2><<<blocks, kStThreads, kThinSmemBytes, st>>>(a); break;
+    case 3: thin_bwd_kernel<3><<<blocks, kStThreads, kThinSmemBytes, st>>>(a); break;
+    default: thin_bwd_kernel<4><<<blocks, kStThreads, kThinSmemBytes, st>>>(a); break;
+    }
 }
 
 }  // namespace ftp

@@ -524,6 +524,7 @@ constexpr int kThinSmemX = kThinMaxCin * kThinXH * kThinXP;              // floa
 constexpr int kThinSmemW = kThinMaxCout * 9 * 4;                         // floats: [co][tap][ci padded to 4]
 constexpr int kThinSmemBytes = (kThinSmemV + kThinSmemX + kThinSmemW) * 4 + kThinPH * kThinPW * kThinAs;
 
+template <int CIN>
 __global__ void __launch_bounds__(kStThreads, 2) thin_bwd_kernel(const __grid_constant__ ThinBwdArgs A)
 {
     extern __shared__ __align__(16) float st_smem[];
@@ -537,13 +538,14 @@ __global__ void __launch_bounds__(kStThreads, 2) thin_bwd_kernel(const __grid_co
 
     for (int i = tid; i < kThinMaxCout * 9 * 4; i += kStThreads) {
         const int ci = i & 3, tap = (i >> 2) % 9, co = i / 36;
-        swt[i] = (co < A.Cout && ci < A.Cin) ? __ldg(A.filter + ((size_t)co * A.Cin + ci) * 9 + tap) : 0.f;
+        swt[i] = (co < A.Cout && ci < CIN) ? __ldg(A.filter + ((size_t)co * CIN + ci) * 9 + tap) : 0.f;
     }
-    float acc[kThinMaxCin - 1][9];                         // filter gradient of (output channel = lane, input channels 0..2)
-    float acc3[9];                                         // ... input channel 3 (only with four input channels)
+    float acc[CIN][9];                                     // filter gradient of (output channel = lane, input channel, tap)
     float bsum = 0.f;
 #pragma unroll
-    for (int t = 0; t < 9; ++t) { acc[0][t] = acc[1][t] = acc[2][t] = 0.f; acc3[t] = 0.f; }
+    for (int ci = 0; ci < CIN; ++ci)
+#pragma unroll
+        for (int t = 0; t < 9; ++t) acc[ci][t] = 0.f;
 
     const int tiles_img = A.tiles_y * A.tiles_x, tiles = A.N * tiles_img;
     const int t_lo = (int)((long long)blockIdx.x * tiles / gridDim.x), t_hi = (int)((long long)(blockIdx.x + 1) * tiles / gridDim.x);
@@ -551,27 +553,27 @@ __global__ void __launch_bounds__(kStThreads, 2) thin_bwd_kernel(const __grid_co
         const int n = tile / tiles_img, ty = (tile % tiles_img) / A.tiles_x, tx = tile % A.tiles_x;
         const int py0 = ty * kThinTH, px0 = tx * kThinTW;
         __syncthreads();                                   // the previous tile has been consumed
-        // stage v and arg-max: one warp per (channel, pooled row), lanes along the row
-        for (int r = warp; r < A.Cout * kThinPH; r += kStThreads / 32) {
-            const int co = r / kThinPH, ly = r - co * kThinPH, py = py0 + ly - 1;
-            const bool row_ok = py >= 0 && py < A.OH;
-            const size_t base = ((size_t)n * A.Cout + co) * pplane + (size_t)(row_ok ? py : 0) * A.OW;
-            for (int lx = lane; lx < kThinPW; lx += 32) {
-                const int px = px0 + lx - 1;
+        // stage v and arg-max: one warp per output channel at a time, lanes along the 10 x 34 pooled pixels of the tile
+        for (int co = warp; co < A.Cout; co += kStThreads / 32) {
+            const size_t base = ((size_t)n * A.Cout + co) * pplane;
+            for (int e = lane; e < kThinPH * kThinPW; e += 32) {
+                const int ly = e / kThinPW, lx = e - ly * kThinPW;
+                const int py = py0 + ly - 1, px = px0 + lx - 1;
                 float v = 0.f; unsigned char a = 0;
-                if (row_ok && px >= 0 && px < A.OW) {
-                    v = __ldg(A.dyp + base + px) * (__ldg(A.yp + base + px) > 0.f ? 1.f : A.slope);
-                    a = A.arg[base + px];
+                if (py >= 0 && py < A.OH && px >= 0 && px < A.OW) {
+                    const size_t gi = base + (size_t)py * A.OW + px;
+                    v = __ldg(A.dyp + gi) * (__ldg(A.yp + gi) > 0.f ? 1.f : A.slope);
+                    a = A.arg[gi];
                 }
-                sv[(ly * kThinPW + lx) * kThinVs + co] = v;
-                sa[(ly * kThinPW + lx) * kThinAs + co] = a;
+                sv[e * kThinVs + co] = v;
+                sa[e * kThinAs + co] = a;
             }
         }
         // stage the input patch
-        for (int r = warp; r < A.Cin * kThinXH; r += kStThreads / 32) {
+        for (int r = warp; r < CIN * kThinXH; r += kStThreads / 32) {
             const int ci = r / kThinXH, lr = r - ci * kThinXH, y = 2 * py0 - 1 + lr;
             const bool row_ok = y >= 0 && y < H;
-            const float* src = A.x + ((size_t)n * A.Cin + ci) * plane + (size_t)(row_ok ? y : 0) * W;
+            const float* src = A.x + ((size_t)n * CIN + ci) * plane + (size_t)(row_ok ? y : 0) * W;
             for (int lc = lane; lc < kThinXW; lc += 32) {
                 const int xg = 2 * px0 - 1 + lc;
                 sx[(ci * kThinXH + lr) * kThinXP + lc] = (row_ok && xg >= 0 && xg < W) ? __ldg(src + xg) : 0.f;
@@ -590,30 +592,33 @@ __global__ void __launch_bounds__(kStThreads, 2) thin_bwd_kernel(const __grid_co
                 // input position of tap (0, 0): rows 2 wy + ay (+ ky), columns 2 wx + ax (+ kx) of the patch
                 const float* xp = sx + (2 * wy + (a >> 1)) * kThinXP + 2 * wx + (a & 1);
 #pragma unroll
-                for (int ky = 0; ky < 3; ++ky)
-#pragma unroll
-                    for (int kx = 0; kx < 3; ++kx) {
-#pragma unroll
-                        for (int ci = 0; ci < kThinMaxCin - 1; ++ci)
-                            acc[ci][ky * 3 + kx] = fmaf(v, xp[(ci * kThinXH + ky) * kThinXP + kx], acc[ci][ky * 3 + kx]);
-                    }
-                if (A.Cin == 4) {
+                for (int ci = 0; ci < CIN; ++ci)
 #pragma unroll
                     for (int ky = 0; ky < 3; ++ky)
 #pragma unroll
                         for (int kx = 0; kx < 3; ++kx)
-                            acc3[ky * 3 + kx] = fmaf(v, xp[(3 * kThinXH + ky) * kThinXP + kx], acc3[ky * 3 + kx]);
-                }
+                            acc[ci][ky * 3 + kx] = fmaf(v, xp[(ci * kThinXH + ky) * kThinXP + kx], acc[ci][ky * 3 + kx]);
             }
         }
 
         // input delta: thread = pooled pixel (wy, wx) = 2 x 2 input pixels
         if (A.dx) {
             const int wy = tid >> 5, wx = tid & 31;
-            float o[kThinMaxCin][2][2];
+            float o[CIN][2][2];
 #pragma unroll
-            for (int ci = 0; ci < kThinMaxCin; ++ci) o[ci][0][0] = o[ci][0][1] = o[ci][1][0] = o[ci][1][1] = 0.f;
+            for (int ci = 0; ci < CIN; ++ci) o[ci][0][0] = o[ci][0][1] = o[ci][1][0] = o[ci][1][1] = 0.f;
+#pragma unroll 2
             for (int co = 0; co < A.Cout; ++co) {
+                // the nine pooled values around the pixel and their arg-max
+                float v9[3][3]; int a9[3][3];
+#pragma unroll
+                for (int dy = 0; dy < 3; ++dy)
+#pragma unroll
+                    for (int dx = 0; dx < 3; ++dx) {
+                        const int pi = (wy + dy) * kThinPW + wx + dx;
+                        v9[dy][dx] = sv[pi * kThinVs + co];
+                        a9[dy][dx] = sa[pi * kThinAs + co];
+                    }
                 // zero-extended delta on rows 2 py - 1 .. 2 py + 2, columns 2 px - 1 .. 2 px + 2
                 float dz[4][4];
 #pragma unroll
@@ -622,8 +627,7 @@ __global__ void __launch_bounds__(kStThreads, 2) thin_bwd_kernel(const __grid_co
                     for (int c = 0; c < 4; ++c) {
                         const int wr = (r + 1) >> 1, wc = (c + 1) >> 1;              // 0, 1, 1, 2
                         const int want = (((r + 1) & 1) << 1) | ((c + 1) & 1);       // arg-max that puts the value there
-                        const int pi = (wy + wr) * kThinPW + wx + wc;
-                        dz[r][c] = (int)sa[pi * kThinAs + co] == want ? sv[pi * kThinVs + co] : 0.f;
+                        dz[r][c] = a9[wr][wc] == want ? v9[wr][wc] : 0.f;
                     }
 #pragma unroll
                 for (int ky = 0; ky < 3; ++ky)
@@ -637,19 +641,18 @@ __global__ void __launch_bounds__(kStThreads, 2) thin_bwd_kernel(const __grid_co
                             for (int j = 0; j < 2; ++j) {
                                 const float d = dz[i - ky + 2][j - kx + 2];
 #pragma unroll
-                                for (int ci = 0; ci < kThinMaxCin; ++ci) o[ci][i][j] = fmaf(wc4[ci], d, o[ci][i][j]);
+                                for (int ci = 0; ci < CIN; ++ci) o[ci][i][j] = fmaf(wc4[ci], d, o[ci][i][j]);
                             }
                     }
             }
             const int py = py0 + wy, px = px0 + wx;
             if (py < A.OH && px < A.OW) {
 #pragma unroll
-                for (int ci = 0; ci < kThinMaxCin; ++ci)
-                    if (ci < A.Cin) {
-                        float* dst = A.dx + ((size_t)n * A.Cin + ci) * plane + (size_t)(2 * py) * W + 2 * px;
-                        *reinterpret_cast<float2*>(dst) = make_float2(o[ci][0][0], o[ci][0][1]);
-                        *reinterpret_cast<float2*>(dst + W) = make_float2(o[ci][1][0], o[ci][1][1]);
-                    }
+                for (int ci = 0; ci < CIN; ++ci) {
+                    float* dst = A.dx + ((size_t)n * CIN + ci) * plane + (size_t)(2 * py) * W + 2 * px;
+                    *reinterpret_cast<float2*>(dst) = make_float2(o[ci][0][0], o[ci][0][1]);
+                    *reinterpret_cast<float2*>(dst + W) = make_float2(o[ci][1][0], o[ci][1][1]);
+                }
             }
         }
     }
@@ -660,18 +663,21 @@ __global__ void __launch_bounds__(kStThreads, 2) thin_bwd_kernel(const __grid_co
     {
         float* mine = red + (warp * 32 + lane) * 40;
 #pragma unroll
-        for (int t = 0; t < 9; ++t) { mine[t] = acc[0][t]; mine[9 + t] = acc[1][t]; mine[18 + t] = acc[2][t]; mine[27 + t] = acc3[t]; }
+        for (int ci = 0; ci < CIN; ++ci)
+#pragma unroll
+            for (int t = 0; t < 9; ++t) mine[ci * 9 + t] = acc[ci][t];
         mine[36] = bsum;
     }
     __syncthreads();
     float* set = A.partial + (size_t)blockIdx.x * A.set_floats;
     for (int e = tid; e < A.Cout * 37; e += kStThreads) {
         const int co = e / 37, k = e - co * 37;
+        if (k < 36 && k >= CIN * 9) continue;
         float s = 0.f;
 #pragma unroll
         for (int w = 0; w < kStThreads / 32; ++w) s += red[(w * 32 + co) * 40 + k];
         if (k == 36) set[A.bias_off + co] = s;
-        else if (k / 9 < A.Cin) set[A.filter_off + ((size_t)co * A.Cin + k / 9) * 9 + k % 9] = s;
+        else set[A.filter_off + ((size_t)co * CIN + k / 9) * 9 + k % 9] = s;
     }
 }
 
