@@ -130,6 +130,10 @@ typedef struct {
                            global memory as at any group boundary (the paper's weight-dominated layers, Section 6).
                            Default (0): groups whose conv has at least 32 input channels; 1: every such group
                            whatever its channel count; -1: never */
+    int tc_tma;           /* bf16 path: how the tiles of maps saved as bf16 planes reach shared memory.  Default (0): tensor
+                           copies by the TMA engine (cp.async.bulk.tensor, one box per 8-channel plane, zeros outside the map;
+                           the tensor maps cover the calling GPU's own memory only and no copy is multicast); -1: plain
+                           loads by the threads */
 } ftp_plan_opts;
 
 /* ftp_plan_create with explicit planner options (NULL = defaults). */

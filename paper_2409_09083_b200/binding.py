@@ -41,7 +41,7 @@ _lib.ftp_plan_create.restype = _i
 class ftp_plan_opts(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_int), ("max_redundancy_pct", ctypes.c_int), ("max_subtile", ctypes.c_int),
                 ("smem_bytes", ctypes.c_int), ("strict_groups", ctypes.c_int), ("tc_blocks_per_sm", ctypes.c_int), ("max_group_convs", ctypes.c_int), ("cost_model", ctypes.c_int),
-                ("stationary", ctypes.c_int)]
+                ("stationary", ctypes.c_int), ("tc_tma", ctypes.c_int)]
 
 
 _lib.ftp_plan_create_opts.argtypes = [ctypes.POINTER(ftp_layer), _i, _i, _i, _i, _i, _i, _i,
@@ -207,11 +207,11 @@ class Plan:
     """Owner of an ftp_plan handle (ftp_plan_create / ftp_plan_destroy)."""
 
     def __init__(self, layers, N, C, H, W, grid, groups, precision=FTP_FP32, max_redundancy_pct=0, max_subtile=0,
-                 smem_bytes=0, strict_groups=False, tc_blocks_per_sm=0, max_group_convs=0, cost_model=0, stationary=0):
+                 smem_bytes=0, strict_groups=False, tc_blocks_per_sm=0, max_group_convs=0, cost_model=0, stationary=0, tc_tma=0):
         self._h = _vp()
         la, ga = _as_layers(layers), _as_groups(groups)
         opts = ftp_plan_opts(ctypes.sizeof(ftp_plan_opts), max_redundancy_pct, max_subtile, smem_bytes,
-                             1 if strict_groups else 0, tc_blocks_per_sm, max_group_convs, int(cost_model), int(stationary))
+                             1 if strict_groups else 0, tc_blocks_per_sm, max_group_convs, int(cost_model), int(stationary), int(tc_tma))
         _check(_lib.ftp_plan_create_opts(la, len(layers), N, C, H, W, grid[0], grid[1], ga, len(groups),
                                          precision, ctypes.byref(opts), ctypes.byref(self._h)))
         self.layers, self.shape, self.grid, self.groups = list(layers), (N, C, H, W), tuple(grid), list(groups)

@@ -1,4 +1,5 @@
 // C-ABI entry points: argument checks, lazy upload of the plan tables, kernel launches.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -136,6 +137,42 @@ inline int* err_ptr(void* ws, const ftp_plan* p) { return reinterpret_cast<int*>
 // one block, more than a third for two.
 inline size_t tc_smem(size_t need, int ctas) { return std::max(need, (size_t)(ctas == 2 ? 77 : 120) * 1024); }
 
+// cuTensorMapEncodeTiled, obtained through the runtime (the library does not link against the driver library).
+typedef CUresult (*tensor_map_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                         const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                         CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+tensor_map_encode_fn tensor_map_encoder()
+{
+    static tensor_map_encode_fn fn = []() -> tensor_map_encode_fn {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) return nullptr;
+        return reinterpret_cast<tensor_map_encode_fn>(sym);
+    }();
+    return fn;
+}
+
+// Tensor map of a saved bf16 map [N][planes][H][W][8 channels] of THIS GPU's memory, with one tile plane
+// (box_h rows x box_w columns x 8 channels) as the box and zeros outside the map.  false: not encodable
+// (the kernel then copies the tile with plain loads).
+bool encode_plane_map(unsigned char out[128], const void* base, int N, int planes, int H, int W, int box_h, int box_w)
+{
+    tensor_map_encode_fn enc = tensor_map_encoder();
+    if (!enc || box_h > 256 || box_w > 256 || box_h < 1 || box_w < 1) return false;
+    static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+    const cuuint64_t dims[4] = {8, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N * planes};
+    const cuuint64_t strides[3] = {16, (cuuint64_t)W * 16, (cuuint64_t)H * W * 16};      // bytes, dimensions 1..3
+    const cuuint32_t box[4] = {8, (cuuint32_t)box_w, (cuuint32_t)box_h, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUtensorMap m;
+    if (enc(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    std::memcpy(out, &m, 128);
+    return true;
+}
+
 void fill_common_tc(const ftp_plan* p, const GroupPlan& g, bool backward, const float* x, const float* params,
                     void* ws, TcGroupArgs& a)
 {
@@ -160,6 +197,20 @@ void fill_common_tc(const ftp_plan* p, const GroupPlan& g, bool backward, const 
     a.wpk = reinterpret_cast<const __nv_bfloat16*>(ws_ptr(ws, backward ? p->ws.wb_off : p->ws.wf_off));
     a.params = params;
     a.error = err_ptr(ws, p);
+    // tiles of maps stored as bf16 planes arrive by TMA: the group input (forward), every op's input (backward)
+    a.use_tma = 0;
+    if (p->tc_tma) {
+        const int n_maps = backward ? g.n_ops : 1;
+        for (int i = 0; i < n_maps; ++i) {
+            const OpDesc& op = a.op[i];
+            if (i == 0 && a.in_f32) continue;                          // the network input is fp32 NCHW: converted by the threads
+            const MapShape& s = p->maps[op.in_map - 1];
+            const int planes = (s.C + 15) / 16 * 2;
+            const int bh = backward ? op.t_x_Hp : op.t_in_Hp, bw = backward ? op.t_x_Wp : op.t_in_Wp;
+            if (planes != op.cin16 / 8) continue;
+            if (encode_plane_map(a.tmap[i], a.map[i], p->N, planes, s.H, s.W, bh, bw)) a.use_tma |= 1u << i;
+        }
+    }
 }
 
 int pack_filters_tc(ftp_plan* p, const float* params, void* ws, cudaStream_t st)
@@ -515,6 +566,8 @@ int ftp_plan_create_opts(const ftp_layer* layers, int n_layers, int N, int C, in
         po.cost_model = opts->cost_model ? (opts->cost_model > 0 ? 1 : 0) : (opts->max_group_convs ? 0 : 1);
         if (opts->stationary < -1 || opts->stationary > 1) return FTP_ERR_ARG;
         po.stationary = opts->stationary;
+        if (opts->tc_tma < -1 || opts->tc_tma > 0) return FTP_ERR_ARG;
+        po.tc_tma = opts->tc_tma;
     }
     ftp_plan* p = new (std::nothrow) ftp_plan();
     if (!p) return FTP_ERR_ARG;

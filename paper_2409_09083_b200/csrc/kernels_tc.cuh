@@ -29,6 +29,12 @@ struct TcGroupArgs {
     const __nv_bfloat16* wpk;            // packed filters (forward or rotated arrangement)
     const float* params;
     int* error;                          // set to 1 when a bounded wait ran out
+    // Tensor maps (128 bytes each, CUtensorMap) of the bf16 maps that tiles are copied from by TMA: [0] the group
+    // input (forward), [i] the input map of op i (backward); use_tma bit i says whether entry i is valid.
+    // A map is seen as the 4-dimensional tensor [image x plane][row][column][8 channels]; a box is one plane of
+    // a tile (rows x columns of the tile's pitch), positions outside the map arrive as zeros (the padding).
+    alignas(64) unsigned char tmap[kMaxOps][128];
+    unsigned use_tma;
     // backward only
     const void*  dmap_out;               // delta at the group's output map: fp32 NCHW (from the caller / the loss), or
     int          dmap_planes;            //   bf16 planes written by halo_sum_planes_kernel (dmap_planes = 1)
@@ -50,6 +56,7 @@ struct Header {
     unsigned long long full[kTcMaxStages];          // weight stage filled (transaction bytes)
     unsigned long long empty[kTcMaxStages];         // weight stage consumed (tcgen05.commit)
     unsigned long long done;                     // all MMAs of a pass completed
+    unsigned long long tile_bar;                 // a tile copied by TMA has arrived (transaction bytes)
     uint32_t tmem_base;
     int stage_mask, stage_shift;                 // filter ring: stages - 1 and log2(stages)
     int tmem_cols;                               // columns this block allocated (512, or 256 with two blocks per SM)
@@ -69,6 +76,7 @@ struct Pipe {
     uint32_t ring;          // shared-memory address of the weight ring
     uint32_t stages_done;   // weight stages produced / consumed so far by this thread's role
     uint32_t passes_done;   // passes completed so far
+    uint32_t tiles_done;    // tiles received by TMA so far
     int* error;
 };
 
@@ -222,7 +230,7 @@ struct Tile {
 };
 __device__ __forceinline__ Tile make_tile(unsigned char* tiles, int off, int planes, int Hp, int Wp)
 {
-    return Tile{tiles + off, planes, Hp, Wp, (uint32_t)(Hp * Wp + kTcTailEntries) * 16u};
+    return Tile{tiles + off, planes, Hp, Wp, (uint32_t)tc_plane_bytes(Hp, Wp)};
 }
 
 // Load the header of sub-tile (r, q): spans and owned cells at every map of the group.
@@ -269,6 +277,25 @@ __device__ __forceinline__ void load_tile(const Tile& T, int bh, int bw, int fil
     }
 }
 
+// The same fill by TMA for a map stored as bf16 planes: one box of Hp x Wp entries per plane, starting at map
+// position (oy, ox) of image n (negative and beyond-the-edge positions arrive as zeros: the padding).  Columns
+// beyond the sub-tile's own width then hold the map's neighbouring values instead of zeros; they only meet
+// accumulator rows that are discarded, or zeros of the other operand, like the tile's tail.  One thread issues
+// the copies; every thread waits (bounded) for the bytes to arrive.  All threads must make the call.
+__device__ __forceinline__ void load_tile_tma(Pipe& p, const Tile& T, const void* tmap, int n, int oy, int ox)
+{
+    fence_async_smem();           // earlier writes of this block to the tile's area are ordered before the copies
+    __syncthreads();
+    const uint32_t bar = smem_u32(&p.h->tile_bar);
+    if (threadIdx.x == 0) {
+        mbar_expect_tx(bar, (uint32_t)T.planes * (uint32_t)(T.Hp * T.Wp) * 16u);
+        for (int pl = 0; pl < T.planes; ++pl)
+            tma_load_4d(smem_u32(T.base + (size_t)pl * T.plane), tmap, 0, ox, oy, n * T.planes + pl, bar);
+    }
+    wait_or_fail(p, &p.h->tile_bar, p.tiles_done & 1);
+    p.tiles_done++;
+}
+
 // Zero every entry of rows [0, bh) x cols [0, bw) of a tile outside the rectangle [y0,y1] x [x0,x1].
 __device__ __forceinline__ void zero_outside(const Tile& T, int bh, int bw, int y0, int y1, int x0, int x1)
 {
@@ -295,6 +322,7 @@ __device__ __forceinline__ void setup(Header* h, Pipe& p, unsigned char* smem, i
         h->stage_mask = stages - 1; h->stage_shift = stages == 4 ? 2 : 1;
         for (int s = 0; s < kTcMaxStages; ++s) { mbar_init(smem_u32(&h->full[s]), 1); mbar_init(smem_u32(&h->empty[s]), kTcIssuers); }
         mbar_init(smem_u32(&h->done), kTcIssuers);
+        mbar_init(smem_u32(&h->tile_bar), 1);
         h->failed = 0;
         fence_mbar_init();
     }
@@ -305,7 +333,7 @@ __device__ __forceinline__ void setup(Header* h, Pipe& p, unsigned char* smem, i
     fence_before_sync();
     __syncthreads();
     fence_after_sync();
-    p.h = h; p.ring = smem_u32(smem + kTcHeader); p.stages_done = 0; p.passes_done = 0; p.error = error;
+    p.h = h; p.ring = smem_u32(smem + kTcHeader); p.stages_done = 0; p.passes_done = 0; p.tiles_done = 0; p.error = error;
 }
 
 __device__ __forceinline__ void teardown(Header* h)
@@ -472,6 +500,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 2 : 1) fwd_group_tc_
     unsigned char* tiles = smem_raw + (kTcHeader + stages * kTcStageBytes);
     Pipe pipe;
     setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes, tmem_cols, stages);
+    const bool tma_ok = (smem_u32(smem_raw) & 127u) == 0;       // tensor copies want 128-byte aligned destinations
     int* hdr = H->hdr;
     const int items = A.N * A.R * A.Q;
 
@@ -483,8 +512,10 @@ __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 2 : 1) fwd_group_tc_
             const OpDesc& op = A.op[0];
             const int oh = hdr[8 + 1] - hdr[8 + 0] + 1, ow = hdr[8 + 3] - hdr[8 + 2] + 1;
             const int bh = (oh - 1) * op.S + op.keff, bw = (ow - 1) * op.S + op.keff;
-            load_tile(make_tile(tiles, op.t_in_off, op.cin16 / 8, op.t_in_Hp, op.t_in_Wp), bh, bw, bw, A.map[0], A.in_f32 != 0,
-                      A.in_C, n, op.in_H, op.in_W, hdr[8 + 0] * op.S - op.pad, hdr[8 + 2] * op.S - op.pad);
+            const Tile IN = make_tile(tiles, op.t_in_off, op.cin16 / 8, op.t_in_Hp, op.t_in_Wp);
+            if ((A.use_tma & 1u) && tma_ok) load_tile_tma(pipe, IN, A.tmap[0], n, hdr[8 + 0] * op.S - op.pad, hdr[8 + 2] * op.S - op.pad);
+            else load_tile(IN, bh, bw, bw, A.map[0], A.in_f32 != 0, A.in_C, n, op.in_H, op.in_W, hdr[8 + 0] * op.S - op.pad,
+                           hdr[8 + 2] * op.S - op.pad);
         }
         for (int i = 0; i < A.n_ops; ++i) {
             const OpDesc& op = A.op[i];
@@ -598,6 +629,7 @@ __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 2 : 1) bwd_group_tc_
     unsigned char* tiles = smem_raw + (kTcHeader + stages * kTcStageBytes);
     Pipe pipe;
     setup(H, pipe, smem_raw, A.error, (size_t)tile_bytes, tmem_cols, stages);
+    const bool tma_ok = (smem_u32(smem_raw) & 127u) == 0;       // tensor copies want 128-byte aligned destinations
     int* hdr = H->hdr;
 
     // The sub-tile stacks of the whole batch, image by image and row by row, are dealt out evenly to
@@ -681,7 +713,8 @@ __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 2 : 1) bwd_group_tc_
             const int vy0 = hi_[0] - oy, vx0 = hi_[2] - ox;                     // its offset inside the X tile
             const Tile X = make_tile(tiles, op.t_x_off, op.cin16 / 8, op.t_x_Hp, op.t_x_Wp);
             const Tile DZ = make_tile(tiles, op.t_dz_off, op.t_dz_planes, op.t_dz_Hp, op.t_dz_Wp);
-            load_tile(X, bh, bw, X.Wp, A.map[i], i == 0 && A.in_f32, A.in_C, n, op.in_H, op.in_W, oy, ox);
+            if (((A.use_tma >> i) & 1u) && tma_ok) load_tile_tma(pipe, X, A.tmap[i], n, oy, ox);
+            else load_tile(X, bh, bw, X.Wp, A.map[i], i == 0 && A.in_f32, A.in_C, n, op.in_H, op.in_W, oy, ox);
             const bool to_scratch = i == 0;
             Tile PD{};
             const OpDesc& pv = A.op[i > 0 ? i - 1 : 0];

@@ -197,7 +197,7 @@ size_t layout_forward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& t
         const int oh = ty.maxext[i + 1], ow = tx.maxext[i + 1];
         op.t_in_Hp = (oh - 1) * op.S + op.keff;
         op.t_in_Wp = (ow - 1) * op.S + op.keff;
-        const size_t plane = ((size_t)op.t_in_Hp * op.t_in_Wp + kTcTailEntries) * 16;
+        const size_t plane = tc_plane_bytes(op.t_in_Hp, op.t_in_Wp);
         size[i] = (size_t)(op.cin16 / 8) * plane;
         slack = std::max(slack, tc_slack(op.t_in_Wp, 0, plane));
     }
@@ -228,8 +228,8 @@ size_t layout_backward_tc(GroupPlan& g, const AxisTables& ty, const AxisTables& 
             op.t_dz_planes = op.cout16 <= 64 ? 8 : round_up(op.cout16, 128) / 8;
             op.t_x_Hp = coh + a; op.t_x_Wp = op.t_dz_Wp;
         }
-        const size_t dplane = ((size_t)op.t_dz_Hp * op.t_dz_Wp + kTcTailEntries) * 16;
-        const size_t xplane = ((size_t)op.t_x_Hp * op.t_x_Wp + kTcTailEntries) * 16;
+        const size_t dplane = tc_plane_bytes(op.t_dz_Hp, op.t_dz_Wp);
+        const size_t xplane = tc_plane_bytes(op.t_x_Hp, op.t_x_Wp);
         dsize[i] = (size_t)op.t_dz_planes * dplane;
         xsize[i] = (size_t)(op.cin16 / 8) * xplane;
         slack = std::max(slack, std::max(tc_slack(op.t_dz_Wp, 0, dplane), tc_slack(op.t_x_Wp, 0, xplane)));
@@ -769,6 +769,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     popts.tensor_cores = tcp ? 1 : 0;
     p.layers.assign(layers, layers + n_layers);
     p.N = N; p.grid_y = gy; p.grid_x = gx; p.precision = precision;
+    p.tc_tma = opts.tc_tma < 0 ? 0 : 1;
 
     // layer validation and map shapes X_1 .. X_{L+1}
     p.maps.clear();

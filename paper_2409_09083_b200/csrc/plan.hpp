@@ -31,6 +31,12 @@ constexpr int kTcSmemBudget2 = 113 * 1024;// ... with two blocks per SM
 constexpr int kTcIssuers = 4;             // threads (lane 0 of warps 0..3) that issue MMAs, each for its own accumulators
 constexpr int kTcMaxUnits = 32;           // filter-gradient accumulators per pass (at least 16 columns each)
 constexpr int kTcTailEntries = 16;        // 16-byte entries appended to every tile plane
+// Bytes from one 8-channel plane of a shared-memory tile to the next: Hp x Wp entries of 16 bytes and the tail, rounded to
+// 128 bytes so that every plane can be the destination of a tensor (TMA) copy.
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+constexpr size_t tc_plane_bytes(int Hp, int Wp) { return ((((size_t)Hp * Wp + kTcTailEntries) * 16) + 127) / 128 * 128; }
 // Weight-stationary kernels of one-conv groups (stationary.cuh): 256 threads, two blocks per SM.
 constexpr int kStThreads = 256;
 // convolution: 64 output channels x 16 row pairs per block (8 channels x 2 rows x 4 columns per thread), or 32 x 32 for layers
@@ -163,6 +169,7 @@ struct ftp_plan {
     std::vector<ftp_group> user_groups;     // the requested grouping profile
     std::vector<ftp::GroupPlan> groups;     // the executed groups (a requested group may be cut, see build_plan)
     int N = 0, grid_y = 0, grid_x = 0, precision = 0;
+    int tc_tma = 1;                         // bf16 path: tiles of saved bf16 maps are copied by TMA (0: by the threads)
     size_t param_floats = 0;
     size_t wf_floats = 0, wb_floats = 0;    // packed filters (tensor-core path: counted in bf16 elements)
     ftp::Workspace ws;
@@ -201,6 +208,7 @@ struct PlanOpts {
     int cost_model = 1;             // 1 = the time model (pass_cost_terms) may replace the fixed rule's cuts, see build_plan
     int refine_backward = 1;        // 1 = the time model may take a finer backward split that balances the blocks (refine_backward_split)
     int tc_ctas = 0;                // tensor-core path: blocks per SM, 1 or 2 (0 = two where every layer of the group allows it)
+    int tc_tma = 0;                 // bf16 path: 0 = tiles of saved maps arrive by TMA (cp.async.bulk.tensor), -1 = copied by the threads
     int stationary = 0;             // one-conv groups run weight-stationary: 0 = with at least kStatMinCin input channels, 1 = all, -1 = none
     int tensor_cores = 0;           // set by build_plan from the precision: shared-memory layouts of the bf16 path
 };

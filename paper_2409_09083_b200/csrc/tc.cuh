@@ -147,5 +147,14 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uin
                  :: "r"(dst_smem), "l"(src), "r"(bytes), "r"(mbar) : "memory");
 }
 
+// Tensor (TMA) copy of one box of a 4-dimensional tensor map from global memory to this CTA's shared memory
+// (128-byte aligned); coordinates innermost first; elements outside the tensor arrive as zeros; completion is
+// signalled on `mbar` as transaction bytes.  No multicast: the box goes to this CTA only.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst_smem, const void* tmap, int c0, int c1, int c2, int c3, uint32_t mbar)
+{
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 :: "r"(dst_smem), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(mbar) : "memory");
+}
+
 }  // namespace tc
 }  // namespace ftp

@@ -180,7 +180,9 @@ def test_result_does_not_depend_on_grid_or_groups_and_is_reproducible():
                 # planner options: whole requested groups fused, one conv per group, two blocks per SM, forced sub-tiling
                 dict(grid=(2, 2), opts=dict(max_group_convs=-1)), dict(grid=(3, 2), opts=dict(max_group_convs=1)),
                 dict(grid=(3, 3), opts=dict(cost_model=1)), dict(grid=(3, 3), opts=dict(cost_model=-1)),
-                dict(grid=(2, 3), opts=dict(tc_blocks_per_sm=2)), dict(grid=(2, 3), opts=dict(tc_blocks_per_sm=1, max_subtile=3))]
+                dict(grid=(2, 3), opts=dict(tc_blocks_per_sm=2)), dict(grid=(2, 3), opts=dict(tc_blocks_per_sm=1, max_subtile=3)),
+                # tiles copied by the threads instead of by TMA tensor copies (the default)
+                dict(grid=(3, 3), opts=dict(tc_tma=-1)), dict(grid=(2, 2), groups=((1, 4), (5, 8)), opts=dict(tc_tma=-1, max_subtile=5))]
     for v in variants:
         opts = v.pop("opts", {})
         y, dx, dparams, plan = backward_bf16(wl.with_(**v), x, params, dy, **opts)
@@ -456,3 +458,16 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
     fp32_plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups)
     with pytest.raises(binding.FtpError):
         fp32_plan.wait_probe(fp32_plan.new_workspace())       # the fp32 path has no device-side waits
+
+
+def test_tma_and_thread_copies_of_the_tiles_give_the_same_bits():
+    """The tiles of maps saved as bf16 planes reach shared memory by TMA tensor copies (zeros outside the map come
+    from the copy engine) or, with tc_tma=-1, by plain loads of the threads: same activations and gradients, bit for
+    bit, also with sub-tiles whose spans start outside the map (negative coordinates) and ragged last tiles."""
+    wl = W("y8", tuple(synth.stack_yolo8()), 2, 3, 88, 104, (5, 7), ((1, 2), (3, 8)))
+    x, params, target = synth.draw(wl, bias_std=0.1)
+    dy = np.random.default_rng(1).standard_normal((wl.N, 128, 11, 13)).astype(np.float32)
+    a = backward_bf16(wl, x, params, dy)
+    b = backward_bf16(wl, x, params, dy, tc_tma=-1)
+    for u, v in zip(a[:3], b[:3]):
+        assert np.array_equal(u, v)
