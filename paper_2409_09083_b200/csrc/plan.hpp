@@ -49,8 +49,8 @@ constexpr int kFgRowPairs = 4;            // filter gradient: row pairs per pixe
 constexpr int kFg1Co = 64, kFg1Ci = 128, kFg1Px = 32;   // filter gradient of a 1 x 1 conv: channel slice of a block, pixels per stage
 constexpr int kThinTileH = 8, kThinTileW = 32;   // thin-input backward: pooled pixels per tile
 constexpr int kStatMinCin = 32;           // fewest input channels for which a one-conv group runs weight-stationary by default
-constexpr double kStatTflops = 40.0;      // measured rate of the weight-stationary kernels (3x3; 1x1 runs at kStatTflops1x1), for the planner's estimates
-constexpr double kStatTflops1x1 = 20.0;
+constexpr double kStatTflops = 45.0;      // measured rate of the weight-stationary kernels on B200 (3x3 layers), for the planner's estimates
+constexpr double kStatTflops1x1 = 25.0;   // ... of the 1x1 kernels and of the thin first layer (dense-equivalent)
 constexpr int kCostTerms = 8;             // terms of the planner's time estimate of one pass of a group
 
 struct Span { int a, b; };            // inclusive interval on one axis
