@@ -160,8 +160,10 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
     const int my_in = rp_l * G::rp_stride + cq_l * 4 + 4;    // column 0 of this thread's quad (16-byte aligned)
     load_stage(0);
     for (int chunk = 0; chunk < nchunks; ++chunk) {
-        if (chunk + 1 < nchunks) { load_stage(chunk + 1); st_wait<1>(); } else st_wait<0>();
+        // one barrier per chunk: behind it every thread has left the previous chunk, whose buffer the next copies fill
+        st_wait<0>();
         __syncthreads();
+        if (chunk + 1 < nchunks) load_stage(chunk + 1);
         const int nci = min(G::ci_chunk, A.Cin - chunk * G::ci_chunk);
         const float* wc = sw + (chunk & 1) * G::w_stage + cg * 8;
         const float* ip = si + (chunk & 1) * G::in_stage + my_in;
@@ -192,7 +194,6 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
                         }
                 }
         }
-        __syncthreads();
     }
 
     // epilogue
@@ -328,8 +329,9 @@ __global__ void __launch_bounds__(kStThreads, 2) filter_grad_rows_kernel(const _
 
     if (s_lo < s_hi) load_stage(s_lo);
     for (int s = s_lo; s < s_hi; ++s) {
-        if (s + 1 < s_hi) { load_stage(s + 1); st_wait<1>(); } else st_wait<0>();
-        __syncthreads();
+        st_wait<0>();
+        __syncthreads();                      // also the release of the other buffer, which the next copies fill
+        if (s + 1 < s_hi) load_stage(s + 1);
         const float* xb = sx + (s & 1) * G::x_stage + lane * G::x_cs;
         const float* db = sd + (s & 1) * G::d_stage + cg * 8;
 #pragma unroll 1
@@ -363,7 +365,6 @@ __global__ void __launch_bounds__(kStThreads, 2) filter_grad_rows_kernel(const _
                             }
                     }
             }
-        __syncthreads();
     }
 
     float* set = A.partial + (size_t)split * A.set_floats;
@@ -437,8 +438,9 @@ __global__ void __launch_bounds__(kStThreads, 3) filter_grad_1x1_kernel(const __
 
     if (s_lo < s_hi) load_stage(s_lo);
     for (int s = s_lo; s < s_hi; ++s) {
-        if (s + 1 < s_hi) { load_stage(s + 1); st_wait<1>(); } else st_wait<0>();
-        __syncthreads();
+        st_wait<0>();
+        __syncthreads();                      // also the release of the other buffer, which the next copies fill
+        if (s + 1 < s_hi) load_stage(s + 1);
         const float* dp = st_smem + (s & 1) * kF1Stage + cog * 4;
         const float* xp = st_smem + (s & 1) * kF1Stage + kF1Px * kF1Ds + cig * 4;
 #pragma unroll 4
@@ -456,7 +458,6 @@ __global__ void __launch_bounds__(kStThreads, 3) filter_grad_1x1_kernel(const __
                 for (int i = 0; i < 4; ++i) acc[c][i] = __ffma2_rn(dd, xv[i], acc[c][i]);
             }
         }
-        __syncthreads();
     }
 
     float* set = A.partial + (size_t)split * A.set_floats;
