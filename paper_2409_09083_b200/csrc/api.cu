@@ -12,6 +12,7 @@
 #include "kernels_tc.cuh"
 #include "plan.hpp"
 #include "stationary_args.hpp"
+#include "tc_stationary.cuh"
 
 using namespace ftp;
 
@@ -42,6 +43,7 @@ int ensure_device(ftp_plan* p)
         cudaFuncSetAttribute(fwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(filter_grad_tc_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcFgSmemBudget) != cudaSuccess ||
         !st_prepare_device())
         return FTP_ERR_CUDA;
     if (!p->grad_stream) {
@@ -379,6 +381,66 @@ int forward_impl(ftp_plan* p, const float* x, const float* params, float* y, voi
     return FTP_OK;
 }
 
+// Backward pass of a one-conv bf16 group behind the first layer: dz planes at the conv's resolution, the filter
+// gradient by the weight-stationary tensor-core kernel over bands of the whole batch (one partial set per pixel
+// share), and the delta at the group's input.
+bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& a, void* ws, cudaStream_t st)
+{
+    const OpDesc& op = g.bwd_ops[0];
+    const TcFgPlan& t = g.tfg;
+    uint4* dz = reinterpret_cast<uint4*>(ws_ptr(ws, p->ws.dz_off));
+    DeltaActPlanesArgs d{};
+    d.dmap = a.dmap_out; d.dmap_planes = a.dmap_planes;
+    d.y = static_cast<const uint4*>(a.map[1]);
+    d.arg = reinterpret_cast<const unsigned long long*>(a.arg[0]);
+    d.dz = dz;
+    d.N = p->N; d.cout = op.cout; d.cout16 = op.cout16; d.out_H = op.out_H; d.out_W = op.out_W;
+    d.pool = op.kind == kOpConvPool ? 1 : 0;
+    d.slope = op.slope;
+    const size_t total = (size_t)p->N * (op.cout16 / 8) * op.out_H * op.out_W;
+    { Timed tm(p, st, 6, gi);
+      delta_act_planes_kernel<<<(int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16), 256, 0, st>>>(d); }
+    if (!launched_ok()) return false;
+
+    TcFilterGradArgs f{};
+    if (!encode_plane_map(f.tmap_dz, dz, p->N, op.cout16 / 8, op.in_H, op.in_W, t.R, t.Wp) ||
+        !encode_plane_map(f.tmap_x, a.map[0], p->N, op.cin16 / 8, op.in_H, op.in_W, t.R + t.k - 1, t.Wp))
+        return false;
+    f.partial = a.partial; f.set_floats = a.set_floats; f.tgp_off = op.tgp_off;
+    f.error = a.error;
+    f.N = p->N; f.K = t.k; f.cout16 = op.cout16; f.cin16 = op.cin16;
+    f.Ms = t.Ms; f.slices = t.slices; f.ncols = t.ncols; f.nci = t.nci;
+    f.R = t.R; f.Wp = t.Wp; f.bands_img = t.bands_img; f.bands = t.bands; f.shares = t.shares;
+    f.dz_plane = t.dz_plane; f.x_plane = t.x_plane; f.stage_bytes = t.stage_bytes;
+    { Timed tm(p, st, 7, gi);
+      filter_grad_tc_rows_kernel<<<t.blocks, kTcFgThreads, t.smem_bytes, st>>>(f); }
+    if (!launched_ok()) return false;
+
+    // input delta: the forward kernel on the conv with the channel counts exchanged (dz planes in, delta planes out)
+    TcGroupArgs b;
+    std::memset(&b, 0, sizeof(b));
+    const PassPlan& pp = g.dxp;
+    b.n_ops = 1; b.R = pp.y.count; b.Q = pp.x.count; b.N = p->N;
+    b.op[0] = g.dx_op;
+    b.map[0] = dz;
+    b.map[1] = ws_ptr(ws, p->ws.dmap_off[gi]);
+    b.map_out[1] = reinterpret_cast<__nv_bfloat16*>(ws_ptr(ws, p->ws.dmap_off[gi]));
+    b.yspan = p->dev_tables + pp.dev_yspan; b.xspan = p->dev_tables + pp.dev_xspan;
+    b.ycell = p->dev_tables + pp.dev_ycell; b.xcell = p->dev_tables + pp.dev_xcell;
+    b.wpk = reinterpret_cast<const __nv_bfloat16*>(ws_ptr(ws, p->ws.wb_off));
+    b.params = nullptr;                               // no bias; the op's slope of 1 makes the activation the identity
+    b.error = a.error;
+    if (p->tc_tma && encode_plane_map(b.tmap[0], dz, p->N, g.dx_op.cin16 / 8, g.dx_op.in_H, g.dx_op.in_W, g.dx_op.t_in_Hp, g.dx_op.t_in_Wp))
+        b.use_tma = 1u;
+    { Timed tm(p, st, 8, gi);
+      const size_t smem = tc_smem(pp.smem_bytes, pp.ctas);
+      const int items = b.R * b.Q * p->N;
+      const int blocks = std::min(items, kSmCount * pp.ctas), tile_bytes = (int)(smem - tc_fixed_bytes(pp.stages));
+      if (pp.ctas == 2) fwd_group_tc_kernel<256><<<blocks, 256, smem, st>>>(b, tile_bytes, kTcTmemCols / 2, pp.stages);
+      else fwd_group_tc_kernel<512><<<blocks, 512, smem, st>>>(b, tile_bytes, kTcTmemCols, pp.stages); }
+    return launched_ok();
+}
+
 int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* params, float* dx, float* grad_out,
                 float* sgd_params, float lr, void* ws, cudaStream_t st)
 {
@@ -394,6 +456,11 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
         a.set_floats = (long long)g.param_floats;
         
         a.need_dx = (gi > 0 || dx != nullptr) ? 1 : 0;
+        if (g.tfg.on) {
+            // one conv behind the first layer: the filter gradient by the weight-stationary kernel, the delta at the group's input as a
+            // convolution of dz with the rotated filters (written whole: nothing to sum afterwards)
+            if (!tc_filter_grad(p, g, gi, a, ws, st)) return FTP_ERR_CUDA;
+        } else
         { Timed t(p, st, 3, gi);
           const size_t smem = tc_smem(g.bwd.smem_bytes, g.bwd.ctas);
           const int tile_bytes = (int)(smem - tc_fixed_bytes(g.bwd.stages));
@@ -406,7 +473,7 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
                 const OpDesc& op = g.bwd_ops[i];
                 if (op.kind == kOpPool) continue;
                 rg.l[rg.n++] = TcReduceLayer{op.p_off, ws_ptr(ws, g.partial_off), (long long)g.param_floats, op.tgp_off,
-                                             g.bwd.blocks, op.cin, op.cout, op.k, op.cin16, op.cout16};
+                                             g.sets(), op.cin, op.cout, op.k, op.cin16, op.cout16};
             }
             { Timed t(p, st, 5, gi);
               reduce_sgd_tc_kernel<<<dim3(1184, rg.n), 128, 0, st>>>(rg, nullptr, 0.f, grad_out); }
@@ -416,7 +483,7 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
                 if (g.bwd_ops[i].kind != kOpPool) floats += (long long)g.bwd_ops[i].cout * g.bwd_ops[i].cin * g.bwd_ops[i].k * g.bwd_ops[i].k + g.bwd_ops[i].cout;
             p->group_ready(p->group_ready_user, gi, g.param_begin, floats);
         }
-        if (a.need_dx) {
+        if (a.need_dx && !g.tfg.on) {
             const MapShape& s = p->maps[g.first - 1];
             const bool planes = g.first > 1;          // group input is a saved bf16 map: deltas travel as planes too
             HaloSumArgs h{};
@@ -449,7 +516,7 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
             if (op.kind == kOpPool) continue;
             if (ra.n == kMaxOps * 2) flush();
             ra.l[ra.n++] = TcReduceLayer{op.p_off, ws_ptr(ws, g.partial_off), (long long)g.param_floats, op.tgp_off,
-                                         g.bwd.blocks, op.cin, op.cout, op.k, op.cin16, op.cout16};
+                                         g.sets(), op.cin, op.cout, op.k, op.cin16, op.cout16};
         }
     flush();
     return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
@@ -600,8 +667,8 @@ int ftp_plan_exec_groups(const ftp_plan* plan, int* n_groups, ftp_group* groups_
 int ftp_plan_group_mode(const ftp_plan* plan, int group, int* stationary, int* partial_sets)
 {
     if (!plan || !stationary || group < 0 || group >= (int)plan->groups.size()) return FTP_ERR_ARG;
-    *stationary = plan->groups[group].st.on;
-    if (partial_sets) *partial_sets = plan->groups[group].bwd.blocks;
+    *stationary = plan->groups[group].st.on ? 1 : plan->groups[group].tfg.on ? 2 : 0;
+    if (partial_sets) *partial_sets = plan->groups[group].sets();
     return FTP_OK;
 }
 

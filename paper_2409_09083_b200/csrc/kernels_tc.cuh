@@ -569,9 +569,9 @@ __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 2 : 1) fwd_group_tc_
                 __syncthreads();
                 continue;
             }
-            // bias of this op -> shared memory (zero for the padded channels)
-            const float* bias = A.params + op.p_off + (size_t)op.cout * op.cin * op.k * op.k;
-            for (int c = threadIdx.x; c < op.cout16; c += blockDim.x) H->bias[c] = c < op.cout ? __ldg(bias + c) : 0.f;
+            // bias of this op -> shared memory (zero for the padded channels; no parameters: a convolution without bias)
+            const float* bias = A.params ? A.params + op.p_off + (size_t)op.cout * op.cin * op.k * op.k : nullptr;
+            for (int c = threadIdx.x; c < op.cout16; c += blockDim.x) H->bias[c] = (bias && c < op.cout) ? __ldg(bias + c) : 0.f;
             tc::fence_async_smem();      // tile written with ordinary stores, read by the tensor core
             __syncthreads();
             const float slope = op.slope;

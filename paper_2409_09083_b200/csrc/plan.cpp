@@ -607,6 +607,85 @@ void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     }
 }
 
+// bf16 path: whether a conv layer runs as a group of its own with the weight-stationary filter gradient: window 1
+// or 3, rows of at most 256 tile entries, a saved bf16 map as input, i.e. not the first layer.  (Measured on B200
+// this beats the fused sub-tile stacks for every such layer of the YOLO stacks, by 2x to 6x for the backward pass of
+// the layers with 128 channels and more, whose per-sub-tile gradient flush it removes.)
+bool tc_stationary_conv(const ftp_plan& p, int li /*0-based*/, const PlanOpts& o)
+{
+    const ftp_layer& l = p.layers[li];
+    if (p.precision != FTP_BF16_FP32ACC || o.stationary < 0 || l.kind != FTP_CONV || li == 0) return false;
+    return (l.k == 1 || l.k == 3) && p.maps[li].W + l.k - 1 <= 256;
+}
+
+// Launch shape of the weight-stationary filter gradient of a one-conv bf16 group (tc_stationary.cuh): slices of
+// Ms output x ncols input channels (all window positions of a slice fit the 512 tensor-memory columns), bands of
+// R rows chosen for the fewest K steps among those whose two stages fit in shared memory, and as many pixel
+// shares as fill the SMs once.
+void plan_tc_filter_grad(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
+{
+    g.tfg = TcFgPlan{};
+    if (g.n_ops != 1 || g.bwd_ops[0].kind == kOpPool || !tc_stationary_conv(p, g.first - 1, o)) return;
+    const OpDesc& op = g.bwd_ops[0];
+    TcFgPlan t;
+    const int H = op.in_H, W = op.in_W, K = op.k;
+    t.k = K; t.Wp = W + K - 1;
+    t.Ms = op.cout16 <= 64 ? 64 : 128;
+    t.slices = (op.cout16 + t.Ms - 1) / t.Ms;
+    t.ncols = std::min(op.cin16, K == 1 ? 256 : 48);
+    t.nci = (op.cin16 + t.ncols - 1) / t.ncols;
+    long long best = -1;
+    for (int R = 1; R <= std::min(H, 64); ++R) {
+        const size_t dzp = align_up(((size_t)R * t.Wp + 16) * 16, 128), xp = align_up(((size_t)(R + K - 1) * t.Wp + 32) * 16, 128);
+        const size_t stage = (size_t)(t.Ms / 8) * dzp + (size_t)(t.ncols / 8) * xp;
+        if (kTcFgHeader + 2 * stage > (size_t)kTcFgSmemBudget || R + K - 1 > 256) break;
+        const long long cost = (long long)((H + R - 1) / R) * ((R * t.Wp + 15) / 16 * 16 + 32);
+        if (best < 0 || cost <= best) {
+            best = cost; t.R = R; t.dz_plane = (int)dzp; t.x_plane = (int)xp; t.stage_bytes = (int)stage;
+        }
+    }
+    if (best < 0) return;
+    t.smem_bytes = kTcFgHeader + 2 * t.stage_bytes;
+    t.bands_img = (H + t.R - 1) / t.R;
+    const long long bands = (long long)p.N * t.bands_img;
+    if (bands > 0x7fffffffLL) return;
+    t.bands = (int)bands;
+    const int roles = t.slices * t.nci;
+    t.shares = (int)std::max<long long>(1, std::min<long long>(bands, kSmCount / roles));
+    t.blocks = roles * t.shares;
+    // the input delta: convolution of dz (cout16 channels) with the rotated filters at the conv's resolution, no bias,
+    // no activation (slope 1), planned as the forward pass of a one-op group of its own
+    GroupPlan d{};
+    d.n_ops = 1;
+    OpDesc& c = d.fwd_ops[0];
+    c = op;
+    c.kind = kOpConv; c.S = 1; c.keff = K; c.slope = 1.0f; c.prev_has_act = 0;
+    c.cin = op.cout; c.cout = op.cin; c.cin16 = op.cout16; c.cout16 = op.cin16;
+    c.out_H = H; c.out_W = W;
+    c.twf_off = op.twb_off;
+    d.bwd_ops[0] = c;
+    d.tile_y = equal_partition(0, H, p.grid_y);
+    d.tile_x = equal_partition(0, W, p.grid_x);
+    const int max_ch = std::max(c.cin16, c.cout16);
+    d.fwd.ctas = o.tc_ctas == 0 ? (max_ch <= 64 ? 2 : 1) : (o.tc_ctas == 2 && max_ch <= 256 ? 2 : 1);
+    d.fwd.stages = 2;
+    int rc = choose_subtiles(d, false, o, p.N);
+    if (rc != FTP_OK && d.fwd.ctas == 2) { d.fwd.ctas = 1; rc = choose_subtiles(d, false, o, p.N); }
+    if (rc != FTP_OK) return;
+    {
+        const size_t budget = std::min<size_t>(d.fwd.ctas == 2 ? kTcSmemBudget2 : kTcSmemBudget, (size_t)o.smem_bytes + 2048);
+        const size_t bytes4 = layout_forward_tc(d, d.fwd.y, d.fwd.x, kTcMaxStages);
+        if (bytes4 <= budget) { d.fwd.stages = kTcMaxStages; d.fwd.smem_bytes = bytes4; }
+        else d.fwd.smem_bytes = layout_forward_tc(d, d.fwd.y, d.fwd.x, d.fwd.stages);
+    }
+    d.fwd.blocks = d.fwd.y.count * d.fwd.x.count * p.N;
+    g.dxp = d.fwd;
+    g.dx_op = d.fwd_ops[0];
+    t.on = 1;
+    g.tfg = t;
+    g.bwd.scratch_floats = 0;       // no per-sub-tile input deltas
+}
+
 struct LayerOffsets { std::vector<long long> p_off, wf_off, wb_off, twf_off, twb_off; };
 
 // Builds the ops, the sub-tiling and the block counts of one executed group (layers first..last).
@@ -745,6 +824,7 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
                            g.bwd.y.scratch_off[g.bwd.y.count] *
                            g.bwd.x.scratch_off[g.bwd.x.count];
     plan_stationary(p, g, o);
+    plan_tc_filter_grad(p, g, o);
     if (g.st.on) {                                  // no sub-tile stacks, no halo recomputation
         g.macs_done = g.macs_untiled;
         if (redundancy) *redundancy = 1.0;
@@ -846,9 +926,12 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
             int hi = std::min(last, start + kMaxOps - 1);
             if (!opts.strict_groups && opts.max_group_convs > 0) {
                 int convs = 0, end = start - 1;
+                bool alone_before = false;
                 while (end + 1 <= hi) {
                     const bool is_conv = p.layers[end].kind == FTP_CONV;
                     if (is_conv && convs == opts.max_group_convs) break;
+                    if (is_conv && convs > 0 && (alone_before || tc_stationary_conv(p, end, popts))) break;   // runs as a group of its own
+                    if (is_conv) alone_before = tc_stationary_conv(p, end, popts);
                     if (is_conv && convs > 0 && p.layers[end - 1].kind == FTP_MAXPOOL) break;
                     if (is_conv) ++convs;
                     ++end;
@@ -884,8 +967,11 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
             for (int s = last; s >= first; --s) {
                 if (s > first && p.layers[s - 2].kind == FTP_CONV && p.layers[s - 1].kind == FTP_MAXPOOL) continue;
                 int convs = 0;
+                bool alone = false;
                 for (int e = s; e <= std::min(last, s + kMaxOps - 1); ++e) {
                     if (p.layers[e - 1].kind == FTP_CONV && ++convs > kCostMaxConvs) break;
+                    if (p.layers[e - 1].kind == FTP_CONV) alone = alone || tc_stationary_conv(p, e - 1, popts);
+                    if (alone && convs > 1) break;             // such a conv is a group of its own
                     if (e < last && p.layers[e - 1].kind == FTP_CONV && p.layers[e].kind == FTP_MAXPOOL) continue;
                     if (best[e + 1] >= inf) continue;
                     GroupPlan g;
@@ -915,7 +1001,8 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     p.tables.clear();
     auto push = [&](const std::vector<int>& v) { int o = (int)p.tables.size(); p.tables.insert(p.tables.end(), v.begin(), v.end()); return o; };
     for (GroupPlan& g : p.groups)
-        for (PassPlan* pp : {&g.fwd, &g.bwd}) {
+        for (PassPlan* pp : {&g.fwd, &g.bwd, &g.dxp}) {
+            if (pp == &g.dxp && !g.tfg.on) continue;
             pp->dev_yspan = push(pp->y.span);   pp->dev_xspan = push(pp->x.span);
             pp->dev_ycell = push(pp->y.cell);   pp->dev_xcell = push(pp->x.cell);
             pp->dev_yoff = push(pp->y.scratch_off); pp->dev_xoff = push(pp->x.scratch_off);
@@ -973,15 +1060,16 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     for (const GroupPlan& g : p.groups) {
         scratch = std::max(scratch, g.bwd.scratch_floats);
         if (g.st.on && !g.st.thin) dz = std::max(dz, (size_t)N * g.fwd_ops[0].cout * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W);
+        if (g.tfg.on) dz = std::max(dz, (size_t)N * g.fwd_ops[0].cout16 * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W / 2);   // bf16
     }
     ws.scratch_off = take(scratch * 4);
     ws.dz_bytes = align_up(dz * 4, 256);
-    ws.dz_off = take(2 * ws.dz_bytes);
+    ws.dz_off = take((tcp ? 1 : 2) * ws.dz_bytes);
     ws.wf_off = take(p.wf_floats * (tcp ? 2 : 4));
     ws.wb_off = take(p.wb_floats * (tcp ? 2 : 4));
     ws.err_off = take(256);
     ws.partial_off = off;
-    for (GroupPlan& g : p.groups) g.partial_off = take((size_t)g.bwd.blocks * g.param_floats * 4);
+    for (GroupPlan& g : p.groups) g.partial_off = take((size_t)g.sets() * g.param_floats * 4);
     ws.grad_off = take(p.param_floats * 4);
     ws.total = off;
     return FTP_OK;

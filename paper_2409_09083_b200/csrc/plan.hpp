@@ -125,9 +125,30 @@ struct StatPlan {
     int fg_blocks = 0;                      // (64 x 32 channel slices) x shares; a share is one partial gradient set
 };
 
+// bf16 path, one-conv groups behind the first layer: the filter gradient by the weight-stationary tensor-core kernel
+// (tc_stationary.cuh); the input delta as a plain convolution of dz with the rotated filters, which the forward
+// kernel runs (every sub-tile writes the cells it owns, so there are no overlapping parts to sum).
+struct TcFgPlan {
+    int on = 0;
+    int k = 0, Ms = 0, slices = 0;          // output channels per block (64 or 128), number of slices
+    int ncols = 0, nci = 0;                 // input channels per block (multiple of 16), number of slices
+    int R = 0, Wp = 0;                      // rows of a band, pitch of its tiles (W + k - 1)
+    int bands_img = 0, bands = 0;           // bands per image and in the batch
+    int shares = 0;                         // pixel shares = partial gradient sets of the group
+    int blocks = 0;                         // slices * nci * shares
+    int dz_plane = 0, x_plane = 0;          // bytes between the planes of the two tiles
+    int stage_bytes = 0, smem_bytes = 0;
+};
+constexpr int kTcFgHeader = 1024;             // barriers, tensor-memory slot, a core matrix of ones
+constexpr int kTcFgSmemBudget = 200 * 1024;   // header + two stages
+
 struct GroupPlan {
     int first = 0, last = 0;        // 1-based layers
     StatPlan st;
+    TcFgPlan tfg;
+    PassPlan dxp;                   // tfg.on: sub-tiling of the input-delta convolution (run by the forward kernel on dx_op)
+    OpDesc dx_op;                   //         the conv with the channel counts exchanged: dz planes in, input delta planes out
+    int sets() const { return tfg.on ? tfg.shares : bwd.blocks; }   // partial gradient sets the reduction sums
     int n_ops = 0;
     OpDesc fwd_ops[kMaxOps];
     OpDesc bwd_ops[kMaxOps];

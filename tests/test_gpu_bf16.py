@@ -84,9 +84,11 @@ def l2_err(a, o):
     return float(np.linalg.norm(a - o) / max(np.linalg.norm(o), 1e-300))
 
 
+@pytest.mark.parametrize("route", ["default", "fused"])
 @pytest.mark.parametrize("name", sorted(FWD))
-def test_backward_matches_oracle(name):
-    """Shallow stacks: max-norm parity of every gradient.  Deep stacks: one stored activation that
+def test_backward_matches_oracle(name, route):
+    """Both routes of the backward pass (default: conv layers behind the first as groups of their own with the
+    weight-stationary filter gradient; fused: sub-tile stacks only).  Shallow stacks: max-norm parity of every gradient.  Deep stacks: one stored activation that
     lands one bf16 step beside the oracle's (fp32 vs fp64 summation next to a rounding boundary)
     perturbs its successors, and after several layers some pooling windows pick another winner on
     the two sides; a max-norm cannot absorb a delta that moved to another pixel, so whole-stack
@@ -97,7 +99,9 @@ def test_backward_matches_oracle(name):
     c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
     dy = np.random.default_rng(3).standard_normal((wl.N, c, h, w)).astype(np.float32)
     ref = run_oracle(wl, x, params, dy=dy, store="bf16")
-    y, dx, dparams, plan = backward_bf16(wl, x, params, dy)
+    y, dx, dparams, plan = backward_bf16(wl, x, params, dy, stationary=-1 if route == "fused" else 0)
+    modes = [plan.group_mode(i)[0] for i in range(len(plan.exec_groups()))]
+    assert all(m == 0 for m in modes) if route == "fused" else modes[0] == 0
     if name in DEEP:
         assert l2_err(dx, ref["dx"]) <= (5e-2 if "yolo8" in name else 0.3)
         assert l2_err(dparams, ref["dparams"]) <= (BF16_TOL if "yolo8" in name else 0.2)
@@ -333,6 +337,7 @@ def test_random_small_stacks_match_oracle(seed):
     rng = np.random.default_rng(1000 + seed)
     wl = _random_workload(rng)
     opts = dict(max_subtile=int(rng.integers(2, 6))) if seed % 3 == 2 else {}
+    if seed % 2: opts["stationary"] = -1               # every other case: fused sub-tile stacks only
     x, params, target = synth.draw(wl, bias_std=0.3)
     x, params = bf16_grid(x), bf16_grid(params)
     c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
@@ -357,13 +362,14 @@ SAFE = {
 }
 
 
-@pytest.mark.parametrize("name", sorted(SAFE))
+@pytest.mark.parametrize("name", sorted(SAFE) + ["yolo8-small/fused", "yolo16-small/fused", "C1/fused"])
 def test_whole_stack_gradients_on_decision_safe_data(name):
     """The whole plan, every group chained, at 2e-2 in the max norm.  The data (synth.draw_integer_relu,
     slope 0) keeps every activation a small integer, which bf16 holds exactly: the forward pass is
     bit-equal to the oracle's and both sides take the same arg-max and sign decisions, ties
     included.  What is left to differ is the rounding of the deltas to bf16 (fp32 sums on one side,
     fp64 on the other), which the tolerance covers."""
+    name, _, route = name.partition("/")
     wl, images = SAFE[name]
     wl = synth.with_slope(wl, 0.0)
     x, params, target = synth.draw_integer_relu(wl)
@@ -374,7 +380,9 @@ def test_whole_stack_gradients_on_decision_safe_data(name):
         keep = np.zeros(wl.N, dtype=bool)
         keep[sel] = True
         dy[~keep] = 0.0
-    y, dx, dparams, plan = backward_bf16(wl, x, params, dy)
+    y, dx, dparams, plan = backward_bf16(wl, x, params, dy, stationary=-1 if route == "fused" else 0)
+    modes = [plan.group_mode(i)[0] for i in range(len(plan.exec_groups()))]
+    assert (2 in modes) != (route == "fused")            # the route asked for is the one that ran
     ref = run_oracle(wl.with_(N=len(sel)), x[sel], params, dy=dy[sel], store="bf16")
     plain = run_oracle(wl.with_(N=len(sel)), x[sel], params, dy=dy[sel])
     assert np.array_equal(ref["y"], plain["y"])                     # storage rounding is the identity on these maps
