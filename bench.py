@@ -40,7 +40,8 @@ KIND = {0: ("pack_filters", None), 1: ("fwd_group", 1), 2: ("loss_delta", None),
         5: ("reduce_sgd", None), 6: ("delta_act", None), 7: ("filter_grad_rows", 1), 8: ("delta_conv_rows", 1)}
 KERNEL = {("fwd_group", "fp32"): "fwd_group_kernel / conv_rows_kernel", ("bwd_group", "fp32"): "bwd_group_kernel / thin_bwd_kernel",
           ("filter_grad_rows", "fp32"): "filter_grad_rows_kernel", ("delta_conv_rows", "fp32"): "conv_rows_kernel (input delta)",
-          ("fwd_group", "bf16"): "fwd_group_tc_kernel", ("bwd_group", "bf16"): "bwd_group_tc_kernel"}
+          ("fwd_group", "bf16"): "fwd_group_tc_kernel", ("bwd_group", "bf16"): "bwd_group_tc_kernel",
+          ("filter_grad_rows", "bf16"): "filter_grad_tc_rows_kernel", ("delta_conv_rows", "bf16"): "fwd_group_tc_kernel (input delta)"}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
 # under profiles/ (static: null for every kernel / workload without a capture of the current code)
 NCU_TRAFFIC = {("C3", "fp32", "fwd_group"): 128.5e6, ("C3", "fp32", "filter_grad_rows"): 245.9e6,
@@ -415,7 +416,7 @@ def measure(ctx, name, precision, extras=True, light=False, **plan_opts):
                          "timing": f"value: median of {len(repeats)} repeats of K steps without per-launch events; breakdown and roofline: "
                                    "K more steps with an event pair around every launch",
                          "repeats": len(repeats), "workspace_bytes": plan.workspace_bytes, "redundancy_fwd": plan.redundancy})
-    cfg["workload"] += f"; executed as groups {' '.join(exec_desc)} (* = one-conv group run weight-stationary)"
+    cfg["workload"] += f"; executed as groups {' '.join(exec_desc)} (* = one-conv group run weight-stationary{', its filter gradient on the bf16 path' if tcp else ''})"
     line = {"metric": METRIC, "value": world * wl.N * steps / (total_ms / 1e3), "unit": UNIT, "n_gpus": world,
             "steps": steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if tcp else "f32", "data": "synthetic",
