@@ -44,6 +44,7 @@ int ensure_device(ftp_plan* p)
         cudaFuncSetAttribute(bwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(filter_grad_tc_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcFgSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(conv_tc_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcFgSmemBudget) != cudaSuccess ||
         !st_prepare_device())
         return FTP_ERR_CUDA;
     if (!p->grad_stream) {
@@ -175,6 +176,45 @@ bool encode_plane_map(unsigned char out[128], const void* base, int N, int plane
     return true;
 }
 
+// Tensor map of bf16 planes [N x planes][H][pitch_w][8] of THIS GPU's memory for the banded kernels: columns
+// 0 .. W-1 of every row (W < pitch_w: a column range that starts at `base`), seen as rows of 2 W eight-byte elements
+// (two per pixel) so that a box row of box_w pixels is one contiguous run; zeros outside.  box_w <= 128.
+bool encode_rows_map(unsigned char out[128], const void* base, int N, int planes, int H, int W, int pitch_w, int box_h, int box_w)
+{
+    tensor_map_encode_fn enc = tensor_map_encoder();
+    if (!enc || box_h > 256 || box_w > 128 || box_h < 1 || box_w < 1) return false;
+    const cuuint64_t dims[3] = {2 * (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N * planes};
+    const cuuint64_t strides[2] = {(cuuint64_t)pitch_w * 16, (cuuint64_t)H * pitch_w * 16};
+    const cuuint32_t box[3] = {2 * (cuuint32_t)box_w, (cuuint32_t)box_h, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUtensorMap m;
+    if (enc(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    std::memcpy(out, &m, 128);
+    return true;
+}
+
+// One launch of the banded convolution kernel: `in` planes (cin16 channels) -> `out` planes (cout16 channels).
+bool launch_tc_conv(ftp_plan* p, const TcConvPlan& c, int kind, int gi, const void* in, const __nv_bfloat16* w, const float* bias,
+                    void* out, unsigned char* arg, int K, int cin16, int cout16, int cout, int H, int W, bool pool, float slope,
+                    int* error, cudaStream_t st)
+{
+    TcConvRowsArgs a{};
+    if (!encode_rows_map(a.tmap_x, in, p->N, cin16 / 8, H, W, W, c.R + K - 1, c.Wp)) return false;
+    a.w = w;
+    a.bias = bias; a.out = static_cast<uint4*>(out); a.arg = reinterpret_cast<unsigned long long*>(arg);
+    a.error = error;
+    a.N = p->N; a.K = K; a.cin16 = cin16; a.cout16 = cout16; a.cout = cout; a.H = H; a.W = W; a.pool = pool ? 1 : 0;
+    a.slope = slope;
+    a.Ns = c.Ns; a.slices = c.slices; a.R = c.R; a.Wp = c.Wp; a.bands_img = c.bands_img; a.nblk = c.nblk; a.kpc = c.kpc;
+    a.ncc = c.ncc; a.Cw = c.Cw; a.items = c.items; a.pool_planes = c.pool_planes; a.nbuf = c.nbuf;
+    a.x_plane = c.x_plane; a.stage_bytes = c.stage_bytes; a.stages = c.stages;
+    { Timed tm(p, st, kind, gi);
+      conv_tc_rows_kernel<<<c.blocks, kTcConvThreads, c.smem_bytes, st>>>(a); }
+    return launched_ok();
+}
+
 void fill_common_tc(const ftp_plan* p, const GroupPlan& g, bool backward, const float* x, const float* params,
                     void* ws, TcGroupArgs& a)
 {
@@ -231,7 +271,8 @@ int pack_filters_tc(ftp_plan* p, const float* params, void* ws, cudaStream_t st)
             const OpDesc& op = g.fwd_ops[i];
             if (op.kind == kOpPool) continue;
             if (pa.n == kMaxOps * 2) flush();
-            pa.l[pa.n++] = TcPackLayer{op.p_off, op.twf_off, op.cin, op.cout, op.k, op.cin16, op.cout16};
+            pa.l[pa.n++] = TcPackLayer{op.p_off, op.twf_off, op.cin, op.cout, op.k, op.cin16, op.cout16,
+                                       g.banded() ? 1 : 0, g.cf.Ns, g.cf.kpc, g.cd.Ns, g.cd.kpc};
         }
     flush();
     return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
@@ -246,6 +287,15 @@ int forward_tc(ftp_plan* p, const float* x, const float* params, float* y, void*
         const GroupPlan& g = p->groups[gi];
         TcGroupArgs a;
         fill_common_tc(p, g, false, x, params, ws, a);
+        if (g.banded()) {                       // one conv behind the first layer: the banded kernel
+            const OpDesc& op = g.fwd_ops[0];
+            const __nv_bfloat16* wf = reinterpret_cast<const __nv_bfloat16*>(ws_ptr(ws, p->ws.wf_off)) + op.twf_off;
+            if (!launch_tc_conv(p, g.cf, 1, (int)gi, a.map[0], wf, params + op.p_off + (size_t)op.cout * op.cin * op.k * op.k,
+                                a.map_out[1], a.arg[0], op.k, op.cin16, op.cout16, op.cout, op.in_H, op.in_W,
+                                op.kind == kOpConvPool, op.slope, a.error, st))
+                return FTP_ERR_CUDA;
+            continue;
+        }
         const int items = a.R * a.Q * p->N;
         { Timed t(p, st, 1, (int)gi);
           const size_t smem = tc_smem(g.fwd.smem_bytes, g.fwd.ctas);
@@ -403,9 +453,12 @@ bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& 
     if (!launched_ok()) return false;
 
     TcFilterGradArgs f{};
-    if (!encode_plane_map(f.tmap_dz, dz, p->N, op.cout16 / 8, op.in_H, op.in_W, t.R, t.Wp) ||
-        !encode_plane_map(f.tmap_x, a.map[0], p->N, op.cin16 / 8, op.in_H, op.in_W, t.R + t.k - 1, t.Wp))
-        return false;
+    for (int cc = 0; cc < t.ncc; ++cc)          // one dz map per column chunk: its columns only, zeros behind them
+        if (!encode_rows_map(f.tmap_dz[cc], dz + (size_t)cc * t.Cw, p->N, op.cout16 / 8, op.in_H, std::min(t.Cw, op.in_W - cc * t.Cw),
+                             op.in_W, t.R, t.Wp))
+            return false;
+    if (!encode_rows_map(f.tmap_x, a.map[0], p->N, op.cin16 / 8, op.in_H, op.in_W, op.in_W, t.R + t.k - 1, t.Wp)) return false;
+    f.ncc = t.ncc; f.Cw = t.Cw;
     f.partial = a.partial; f.set_floats = a.set_floats; f.tgp_off = op.tgp_off;
     f.error = a.error;
     f.N = p->N; f.K = t.k; f.cout16 = op.cout16; f.cin16 = op.cin16;
@@ -416,7 +469,12 @@ bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& 
       filter_grad_tc_rows_kernel<<<t.blocks, kTcFgThreads, t.smem_bytes, st>>>(f); }
     if (!launched_ok()) return false;
 
-    // input delta: the forward kernel on the conv with the channel counts exchanged (dz planes in, delta planes out)
+    // input delta: the convolution of dz with the rotated filters (dz planes in, delta planes out)
+    if (g.banded()) {
+        const __nv_bfloat16* wb = reinterpret_cast<const __nv_bfloat16*>(ws_ptr(ws, p->ws.wb_off)) + op.twb_off;
+        return launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, ws_ptr(ws, p->ws.dmap_off[gi]), nullptr, t.k, op.cout16, op.cin16, op.cin,
+                              op.in_H, op.in_W, false, 1.0f, a.error, st);
+    }
     TcGroupArgs b;
     std::memset(&b, 0, sizeof(b));
     const PassPlan& pp = g.dxp;

@@ -931,7 +931,12 @@ __global__ void planes_to_nchw_kernel(const __nv_bfloat16* __restrict__ src, flo
 // Filters -> the two packed bf16 arrangements of the tensor-core kernels:
 //   wf[tap][cin16/8][cout16][8]   B operand of the forward pass   (rows = cout, K = cin)
 //   wb[tap'][cout16/8][cin16][8]  B operand of the delta pass, tap' = K*K-1-tap (rotated 180 degrees; rows = cin, K = cout)
-struct TcPackLayer { long long p_off, w_off; int cin, cout, k, cin16, cout16; };
+// Layers run by the banded kernels (sliced != 0) get instead, per pass, the arrangement in which the filters one block
+// needs for one chunk of input channels are contiguous (one bulk copy):
+//   wf[slice][chunk][tap][kpc_f][ns_f][8]    rows = output channels slice*ns_f .., K = input channels (chunk*kpc_f + j)*8 ..
+//   wb[slice][chunk][tap'][kpc_d][ns_d][8]   rows = input channels slice*ns_d ..,  K = output channels (chunk*kpc_d + j)*8 ..
+// with zeros beyond the layer's channel counts.
+struct TcPackLayer { long long p_off, w_off; int cin, cout, k, cin16, cout16; int sliced, ns_f, kpc_f, ns_d, kpc_d; };
 struct TcPackArgs { int n; TcPackLayer l[kMaxOps * 2]; };
 
 __global__ void pack_filters_tc_kernel(const __grid_constant__ TcPackArgs A, const float* __restrict__ params,
@@ -939,6 +944,26 @@ __global__ void pack_filters_tc_kernel(const __grid_constant__ TcPackArgs A, con
 {
     const TcPackLayer L = A.l[blockIdx.y];
     const int KK = L.k * L.k;
+    if (L.sliced) {
+        const int nch_f = (L.cin16 / 8 + L.kpc_f - 1) / L.kpc_f, nch_d = (L.cout16 / 8 + L.kpc_d - 1) / L.kpc_d;
+        const long long per_f = (long long)((L.cout16 + L.ns_f - 1) / L.ns_f) * nch_f * KK * L.kpc_f * L.ns_f * 8;
+        const long long per_d = (long long)((L.cin16 + L.ns_d - 1) / L.ns_d) * nch_d * KK * L.kpc_d * L.ns_d * 8;
+        for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < per_f + per_d; e += (long long)gridDim.x * blockDim.x) {
+            const bool fwd = e < per_f;
+            const int ns = fwd ? L.ns_f : L.ns_d, kpc = fwd ? L.kpc_f : L.kpc_d, nch = fwd ? nch_f : nch_d;
+            long long t = fwd ? e : e - per_f;
+            const int c8 = (int)(t % 8); t /= 8;
+            const int r = (int)(t % ns); t /= ns;
+            const int j = (int)(t % kpc); t /= kpc;
+            const int tap = (int)(t % KK); t /= KK;
+            const int c = (int)(t % nch); const int sl = (int)(t / nch);
+            const int row = sl * ns + r, kch = (c * kpc + j) * 8 + c8;            // output row of the GEMM, contraction channel
+            const int co = fwd ? row : kch, ci = fwd ? kch : row;
+            const float v = (co < L.cout && ci < L.cin) ? params[L.p_off + ((long long)co * L.cin + ci) * KK + (fwd ? tap : KK - 1 - tap)] : 0.f;
+            if (fwd) wf[L.w_off + e] = __float2bfloat16(v); else wb[L.w_off + (e - per_f)] = __float2bfloat16(v);
+        }
+        return;
+    }
     const long long per = (long long)KK * L.cin16 * L.cout16;
     for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < 2 * per; e += (long long)gridDim.x * blockDim.x) {
         if (e < per) {

@@ -615,7 +615,57 @@ bool tc_stationary_conv(const ftp_plan& p, int li /*0-based*/, const PlanOpts& o
 {
     const ftp_layer& l = p.layers[li];
     if (p.precision != FTP_BF16_FP32ACC || o.stationary < 0 || l.kind != FTP_CONV || li == 0) return false;
-    return (l.k == 1 || l.k == 3) && p.maps[li].W + l.k - 1 <= 256;
+    return (l.k == 1 || l.k == 3) && p.maps[li].W <= kTcMaxColChunks * 126;
+}
+
+// Column chunks of a band: as few as keep the tile pitch (chunk + k - 1) within the 128 pixels of a TMA box row,
+// of equal (even) width.
+void tc_col_chunks(int W, int* ncc, int* Cw)
+{
+    *ncc = (W + 125) / 126;
+    *Cw = ((W + *ncc - 1) / *ncc + 1) / 2 * 2;
+    if (*Cw > W) *Cw = W;
+}
+
+// Launch shape of the banded convolution kernel for a conv with `cout16` output and `cin16` input channels (padded)
+// on N maps of H x W: bands as tall as the accumulators allow (512 columns = blocks of 128 entries x Ns channels),
+// among those the height with the fewest rounds of blocks over the SMs; as many stages as fit.
+TcConvPlan plan_tc_conv(int N, int H, int W, int K, int cin16, int cout16, bool pool)
+{
+    TcConvPlan c;
+    tc_col_chunks(W, &c.ncc, &c.Cw);
+    c.Wp = c.Cw + K - 1;
+    c.Ns = std::min(cout16, 128);
+    c.slices = (cout16 + c.Ns - 1) / c.Ns;
+    // slices of at most 64 channels: items of 256 columns in two alternating buffers (narrow MMAs leave the tensor
+    // core idle while an item is read back); wider slices: one buffer of 512 columns (their filters are read per item)
+    c.nbuf = c.Ns <= 64 ? 2 : 1;
+    const int max_blk = std::min(8, kTcTmemCols / c.nbuf / c.Ns);
+    c.kpc = K == 1 ? std::min(cin16 / 8, 8) : 2;
+    const int step = pool ? 2 : 1;
+    const int r_max = std::min((max_blk * 128) / c.Wp, H) / step * step;
+    if (r_max < step) return c;
+    double best = -1;
+    for (int R = step; R <= r_max; R += step) {
+        const int bands = (H + R - 1) / R * c.ncc, nblk = (R * c.Wp + 127) / 128;
+        const long long items = (long long)N * bands * c.slices;
+        const double cost = (double)((items + kSmCount - 1) / kSmCount) * (nblk + 0.5);      // rounds x (MMAs + fixed part) of a block
+        if (best < 0 || cost <= best) { best = cost; c.R = R; c.nblk = nblk; c.bands_img = bands; }
+    }
+    const size_t entries = std::max<size_t>((size_t)(c.R + K - 1) * c.Wp, (size_t)c.nblk * 128 + (size_t)(K - 1) * c.Wp + K);
+    c.x_plane = (int)align_up(entries * 16, 128);
+    c.stage_bytes = c.kpc * c.x_plane + (K == 1 ? c.kpc : 2 * K * K) * c.Ns * 16;
+    const size_t staging = pool ? kTcPoolStageBytes : 0;                                     // the band as stored, 16 channels or more at a time
+    c.stages = (int)std::min<size_t>(4, ((size_t)kTcFgSmemBudget - kTcFgHeader - staging) / c.stage_bytes);
+    c.pool_planes = pool ? (int)(kTcPoolStageBytes / ((size_t)c.nblk * 128 * 16)) / 2 * 2 : 0;
+    if (c.stages < 2 || (pool && c.pool_planes < 2)) return c;
+    c.smem_bytes = kTcFgHeader + c.stages * c.stage_bytes + (int)staging;
+    const long long items = (long long)N * c.bands_img * c.slices;
+    if (items > 0x7fffffffLL) return c;
+    c.items = (int)items;
+    c.blocks = (int)std::min<long long>(items, kSmCount);
+    c.on = 1;
+    return c;
 }
 
 // Launch shape of the weight-stationary filter gradient of a one-conv bf16 group (tc_stationary.cuh): slices of
@@ -629,7 +679,8 @@ void plan_tc_filter_grad(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     const OpDesc& op = g.bwd_ops[0];
     TcFgPlan t;
     const int H = op.in_H, W = op.in_W, K = op.k;
-    t.k = K; t.Wp = W + K - 1;
+    tc_col_chunks(W, &t.ncc, &t.Cw);
+    t.k = K; t.Wp = t.Cw + K - 1;
     t.Ms = op.cout16 <= 64 ? 64 : 128;
     t.slices = (op.cout16 + t.Ms - 1) / t.Ms;
     t.ncols = std::min(op.cin16, K == 1 ? 256 : 48);
@@ -646,7 +697,7 @@ void plan_tc_filter_grad(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     }
     if (best < 0) return;
     t.smem_bytes = kTcFgHeader + 2 * t.stage_bytes;
-    t.bands_img = (H + t.R - 1) / t.R;
+    t.bands_img = (H + t.R - 1) / t.R * t.ncc;
     const long long bands = (long long)p.N * t.bands_img;
     if (bands > 0x7fffffffLL) return;
     t.bands = (int)bands;
@@ -681,6 +732,10 @@ void plan_tc_filter_grad(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     d.fwd.blocks = d.fwd.y.count * d.fwd.x.count * p.N;
     g.dxp = d.fwd;
     g.dx_op = d.fwd_ops[0];
+    if (o.stationary != 2) {        // (2: banded filter gradient only, for comparisons)
+        g.cf = plan_tc_conv(p.N, H, W, K, op.cin16, op.cout16, op.kind == kOpConvPool);
+        g.cd = plan_tc_conv(p.N, H, W, K, op.cout16, op.cin16, false);
+    }
     t.on = 1;
     g.tfg = t;
     g.bwd.scratch_floats = 0;       // no per-sub-tile input deltas
@@ -873,8 +928,8 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
             lo.wf_off[i] = wf; wf += (long long)l.cin * l.k * l.k * cout_pad;
             lo.wb_off[i] = wb; wb += (long long)l.cout * l.k * l.k * cin_pad;
             if (tcp && (l.cin > kTcTmemCols || l.cout > kTcTmemCols)) return FTP_ERR_LAYERS;
-            lo.twf_off[i] = lo.twb_off[i] = twf;        // both packed layouts hold k*k*cin16*cout16 elements
-            twf += (long long)l.k * l.k * round_up(l.cin, 16) * round_up(l.cout, 16);
+            lo.twf_off[i] = lo.twb_off[i] = twf;        // both packed layouts hold k*k*cin16*cout16 elements; room for the
+            twf += (long long)l.k * l.k * round_up(l.cin, 128) * round_up(l.cout, 128);   // banded kernels' padded slices
         } else if (l.kind == FTP_MAXPOOL) {
             if (l.k != 2 || l.stride != 2 || l.pad != 0 || in.H % 2 || in.W % 2) return FTP_ERR_LAYERS;
             p.maps.push_back(MapShape{in.C, in.H / 2, in.W / 2});

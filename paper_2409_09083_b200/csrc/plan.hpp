@@ -132,13 +132,30 @@ struct TcFgPlan {
     int on = 0;
     int k = 0, Ms = 0, slices = 0;          // output channels per block (64 or 128), number of slices
     int ncols = 0, nci = 0;                 // input channels per block (multiple of 16), number of slices
-    int R = 0, Wp = 0;                      // rows of a band, pitch of its tiles (W + k - 1)
+    int R = 0, Wp = 0;                      // rows of a band, pitch of its tiles (Cw + k - 1)
+    int ncc = 1, Cw = 0;                    // column chunks of a row band (maps wider than 126 pixels) and their width
     int bands_img = 0, bands = 0;           // bands per image and in the batch
     int shares = 0;                         // pixel shares = partial gradient sets of the group
     int blocks = 0;                         // slices * nci * shares
     int dz_plane = 0, x_plane = 0;          // bytes between the planes of the two tiles
     int stage_bytes = 0, smem_bytes = 0;
 };
+// Banded tensor-core convolution of a one-conv bf16 group (conv_tc_rows_kernel): forward pass and input delta.
+struct TcConvPlan {
+    int on = 0;
+    int Ns = 0, slices = 0;                 // output channels per block, number of slices
+    int R = 0, Wp = 0, bands_img = 0;       // rows per band, tile pitch, bands (row bands x column chunks) per image
+    int ncc = 1, Cw = 0;                    // column chunks of a row band (maps wider than 126 pixels) and their width
+    int nblk = 0;                           // accumulator blocks (128 tile entries each) of a full band
+    int kpc = 0;                            // 8-channel input planes per chunk
+    int x_plane = 0, stage_bytes = 0, stages = 0, smem_bytes = 0;
+    int items = 0;                          // N * bands_img * slices
+    int blocks = 0;                         // persistent blocks: min(items, SMs)
+    int pool_planes = 0;                    // fused pool: 8-channel planes the staging area holds
+    int nbuf = 1;                           // accumulator buffers (2 for slices of at most 64 channels)
+};
+constexpr int kTcPoolStageBytes = 32 * 1024;  // staging area of the fused pool in the banded convolution
+constexpr int kTcMaxColChunks = 8;            // a band spans at most 126 columns (a TMA box row of 128 pixels with the halo): wider maps are cut into chunks
 constexpr int kTcFgHeader = 1024;             // barriers, tensor-memory slot, a core matrix of ones
 constexpr int kTcFgSmemBudget = 200 * 1024;   // header + two stages
 
@@ -148,6 +165,8 @@ struct GroupPlan {
     TcFgPlan tfg;
     PassPlan dxp;                   // tfg.on: sub-tiling of the input-delta convolution (run by the forward kernel on dx_op)
     OpDesc dx_op;                   //         the conv with the channel counts exchanged: dz planes in, input delta planes out
+    TcConvPlan cf, cd;              // tfg.on: the forward convolution and the input-delta convolution as banded kernels
+    bool banded() const { return tfg.on && cf.on && cd.on; }   // both run banded: the layer's filters are packed for them
     int sets() const { return tfg.on ? tfg.shares : bwd.blocks; }   // partial gradient sets the reduction sums
     int n_ops = 0;
     OpDesc fwd_ops[kMaxOps];

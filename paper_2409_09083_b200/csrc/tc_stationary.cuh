@@ -22,9 +22,14 @@
 
 namespace ftp {
 
+// Tensor maps of bf16 planes [N x C16/8][H][W][8] as the TMA engine sees them here: 3-dimensional, rows of 2 W
+// eight-byte elements (a pixel's 8 channels = two elements), so that a box row is one contiguous run of Wp pixels
+// instead of Wp separate 16-byte pieces; a box row holds at most 256 elements, i.e. Wp <= 128 pixels.
 struct TcFilterGradArgs {
-    alignas(64) unsigned char tmap_dz[128];   // [N x cout16/8][H][W][8] bf16, box = 8 x Wp x R
-    alignas(64) unsigned char tmap_x[128];    // [N x cin16/8][H][W][8] bf16,  box = 8 x Wp x (R + K - 1)
+    // dz planes, one map per column chunk: the chunk's columns only (base moved to its first column, extent = its
+    // width), so that the box (Wp pixels x R rows) reads zeros behind the chunk's last column
+    alignas(64) unsigned char tmap_dz[kTcMaxColChunks][128];
+    alignas(64) unsigned char tmap_x[128];    // the layer's input planes, box = Wp pixels x (R + K - 1) rows
     float* partial;                           // partial sets of the group
     long long set_floats, tgp_off;            // floats per set, offset of this layer inside a set
     int* error;
@@ -32,6 +37,7 @@ struct TcFilterGradArgs {
     int Ms, slices;                           // output channels per block (64 or 128) and number of such slices
     int ncols, nci;                           // input channels per block (multiple of 16) and number of such slices
     int R, Wp, bands_img, bands, shares;      // rows per band, tile pitch, bands per image / in the batch, pixel shares
+    int ncc, Cw;                              // column chunks per row band and their width (Wp = Cw + K - 1)
     int dz_plane, x_plane, stage_bytes;       // bytes between planes of the two tiles, bytes of one stage
 };
 
@@ -144,15 +150,16 @@ __global__ void __launch_bounds__(kTcFgThreads, 1) filter_grad_tc_rows_kernel(co
         for (int i = 0; i < nb; ++i) {
             const int s = i & 1;
             if (!wait(&H->empty[s], ((uint32_t)(i >> 1) & 1u) ^ 1u)) break;
-            const int b = b_lo + i, n = b / A.bands_img, y0 = (b - n * A.bands_img) * A.R;
+            const int b = b_lo + i, n = b / A.bands_img, bi = b - n * A.bands_img;
+            const int cc = bi % A.ncc, y0 = (bi / A.ncc) * A.R, x0 = cc * A.Cw;
             unsigned char* dzs = stages + (size_t)s * A.stage_bytes;
             unsigned char* xs = dzs + (size_t)mp * A.dz_plane;
             const uint32_t bar = smem_u32(&H->full[s]);
             mbar_expect_tx(bar, (uint32_t)((nd * A.R + np * (A.R + K - 1)) * A.Wp) * 16u);
             for (int pl = 0; pl < nd; ++pl)
-                tma_load_4d(smem_u32(dzs + (size_t)pl * A.dz_plane), A.tmap_dz, 0, 0, y0, n * (A.cout16 / 8) + slice * mp + pl, bar);
+                tma_load_3d(smem_u32(dzs + (size_t)pl * A.dz_plane), A.tmap_dz[cc], 0, y0, n * (A.cout16 / 8) + slice * mp + pl, bar);
             for (int pl = 0; pl < np; ++pl)
-                tma_load_4d(smem_u32(xs + (size_t)pl * A.x_plane), A.tmap_x, 0, -(K / 2), y0 - K / 2, n * (A.cin16 / 8) + ci0 / 8 + pl, bar);
+                tma_load_3d(smem_u32(xs + (size_t)pl * A.x_plane), A.tmap_x, 2 * (x0 - K / 2), y0 - K / 2, n * (A.cin16 / 8) + ci0 / 8 + pl, bar);
             ++issued[s];
         }
         if (H->failed)       // gave up somewhere: let the copies already under way land before the block leaves
@@ -226,6 +233,285 @@ __global__ void __launch_bounds__(kTcFgThreads, 1) filter_grad_tc_rows_kernel(co
     fence_before_sync();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, (uint32_t)kTcTmemCols);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Convolution of a one-conv group over bands of rows (forward pass, and the input delta as the convolution of dz
+// with the rotated filters).  A work item is a band of R rows x Cw columns of one image x a slice of Ns output
+// channels: up to 512 / Ns accumulator blocks of 128 consecutive tile entries (pitch Wp = Cw + K - 1, so the entries
+// of a block are pixels of consecutive rows with K - 1 discarded positions between them) stay in tensor memory
+// while the input channels stream past in chunks: per chunk one tile of `kpc` 8-channel planes of the band (with
+// its K - 1 halo rows, TMA tensor copies) and the filters of those channels for the slice (one bulk copy),
+// through a ring of stages.  Window position (ky, kx) moves the A operand by ky * Wp + kx entries.  Against the
+// fused sub-tile kernel, whose sub-tiles follow the tile grid (64 pixels a tile on the deepest maps) and which
+// streams all filters of the layer once per 128 pixels, the filters read per pixel shrink by the number of
+// accumulator blocks and the pixels per block no longer depend on the grid.
+//
+// Persistent blocks (one per SM) walk over the items; the warps have fixed roles: warps 0-7 read the accumulators
+// back (bias, leaky ReLU, bf16 planes; with a fused 2x2 pool through a small staging area, 16 channels or more at
+// a time, first maximum in window order, with the arg-max bytes the backward pass routes deltas by), lane 0 of
+// warps 8-11 issues the MMAs (each for its own accumulator blocks), lane 0 of warp 12 issues the copies and runs
+// ahead into the next item while the accumulators of the current one are read back.
+// ---------------------------------------------------------------------------------------------
+struct TcConvRowsArgs {
+    alignas(64) unsigned char tmap_x[128];    // input planes (rows of 2 W eight-byte elements): box = Wp pixels x (R + K - 1) rows
+    const __nv_bfloat16* w;                   // filters of the layer, [slice][chunk][window position][kpc][Ns][8]: the
+                                              //   filters a block needs for one chunk are one contiguous run
+    const float* bias;                        // cout floats, or null
+    uint4* out;                               // output planes [N][cout16/8][OH][OW] (OH = H / 2 with the pool)
+    unsigned long long* arg;                  // pool: arg-max bytes in the same arrangement
+    int* error;
+    int N, K, cin16, cout16, cout, H, W, pool;
+    float slope;
+    int Ns, slices;                           // output channels per item, number of slices
+    int R, Wp, bands_img, nblk;               // rows per band, tile pitch, bands per image, accumulator blocks of a full band
+    int ncc, Cw;                              // column chunks per row band and their width (even with the pool; Wp = Cw + K - 1)
+    int kpc;                                  // 8-channel planes per chunk (2 for 3x3)
+    int x_plane, stage_bytes, stages;
+    int items;                                // N * bands_img * slices
+    int pool_planes;                          // pool: 8-channel planes the staging area holds (even)
+    int nbuf;                                 // accumulator buffers (2: items of at most 256 columns alternate between the halves
+                                              //   of the tensor memory, so the MMAs of one run while the other is read back)
+};
+
+constexpr int kTcConvMaxStages = 4;
+constexpr int kTcConvEpiWarps = 8;
+constexpr int kTcConvThreads = (kTcConvEpiWarps + kTcIssuers + 1) * 32;
+
+__global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const __grid_constant__ TcConvRowsArgs A)
+{
+    using namespace tc;
+    extern __shared__ __align__(1024) unsigned char cv_smem[];
+    struct Hdr {
+        unsigned long long full[kTcConvMaxStages], empty[kTcConvMaxStages];
+        unsigned long long done[2];     // the MMAs of an item have completed (one commit per issuer), per accumulator buffer
+        unsigned long long tfree[2];    // its accumulators have been read back (one arrival per epilogue warp)
+        unsigned long long drain;       // all MMAs of the block have completed
+        uint32_t tmem_base;
+        volatile int failed;
+        volatile int epi_stop;          // the epilogue warps' common view of `failed` (they meet at named barriers)
+        float bias[128];
+    };
+    static_assert(sizeof(Hdr) <= kTcFgHeader, "header does not fit");
+    Hdr* H = reinterpret_cast<Hdr*>(cv_smem);
+    unsigned char* stages = cv_smem + kTcFgHeader;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int K = A.K, KK = K * K;
+    const int kplanes = A.cin16 / 8, nchunks = (kplanes + A.kpc - 1) / A.kpc;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTcConvMaxStages; ++s) { mbar_init(smem_u32(&H->full[s]), 1); mbar_init(smem_u32(&H->empty[s]), kTcIssuers); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&H->done[i]), kTcIssuers); mbar_init(smem_u32(&H->tfree[i]), kTcConvEpiWarps); }
+        mbar_init(smem_u32(&H->drain), kTcIssuers);
+        H->failed = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) { __syncwarp(); tmem_alloc(smem_u32(&H->tmem_base), (uint32_t)kTcTmemCols); }
+    tcd::zero_bytes(stages, (size_t)A.stages * A.stage_bytes);       // what the copies never write is read as zeros
+    fence_async_smem();
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem = H->tmem_base;
+
+    auto wait = [&](unsigned long long* bar, uint32_t parity) {
+        if (H->failed) return false;
+        if (mbar_wait(smem_u32(bar), parity)) return true;
+        H->failed = 1;
+        atomicExch(A.error, 1);
+        return false;
+    };
+    if ((smem_u32(cv_smem) & 127u) != 0) {                  // tensor copies want 128-byte aligned destinations
+        if (threadIdx.x == 0) { H->failed = 1; atomicExch(A.error, 1); }
+        __syncthreads();
+    }
+    // item -> (slice, image, band origin); every role walks the same sequence of items
+    struct Item { int slice, n, y0, x0, rows, cw, co0, cols, nblk; };
+    auto item_of = [&](int it) {
+        Item I;
+        I.slice = it % A.slices;
+        const int band = it / A.slices;
+        I.n = band / A.bands_img;
+        const int bi = band - I.n * A.bands_img;
+        I.y0 = (bi / A.ncc) * A.R; I.x0 = (bi % A.ncc) * A.Cw;
+        I.rows = min(A.R, A.H - I.y0); I.cw = min(A.Cw, A.W - I.x0);
+        I.co0 = I.slice * A.Ns; I.cols = min(A.Ns, A.cout16 - I.co0);
+        I.nblk = (I.rows * A.Wp + 127) >> 7;
+        return I;
+    };
+    const uint32_t w_tap = (uint32_t)A.kpc * (uint32_t)A.Ns * 16u;                      // filter bytes of one window position
+    const uint32_t w_chunk = (uint32_t)KK * w_tap;
+
+    if (warp == kTcConvEpiWarps + kTcIssuers) {
+        if (lane == 0) {
+            // producer
+            int issued[kTcConvMaxStages] = {0, 0, 0, 0};
+            uint32_t g = 0;                                                             // chunks issued so far
+            for (int it = blockIdx.x; it < A.items && !H->failed; it += gridDim.x) {
+                const Item I = item_of(it);
+                for (int c = 0; c < nchunks; ++c, ++g) {
+                    const int s = (int)(g % (uint32_t)A.stages);
+                    if (!wait(&H->empty[s], ((g / (uint32_t)A.stages) & 1u) ^ 1u)) break;
+                    const int kp0 = c * A.kpc, np = min(A.kpc, kplanes - kp0);
+                    unsigned char* xs = stages + (size_t)s * A.stage_bytes;
+                    unsigned char* ws = xs + (size_t)A.kpc * A.x_plane;
+                    const uint32_t bar = smem_u32(&H->full[s]);
+                    mbar_expect_tx(bar, (uint32_t)(np * (A.R + K - 1) * A.Wp) * 16u + w_chunk);
+                    for (int pl = 0; pl < np; ++pl)
+                        tma_load_3d(smem_u32(xs + (size_t)pl * A.x_plane), A.tmap_x, 2 * (I.x0 - K / 2), I.y0 - K / 2,
+                                    I.n * kplanes + kp0 + pl, bar);
+                    bulk_g2s(smem_u32(ws), A.w + ((size_t)I.slice * nchunks + c) * (w_chunk / 2), w_chunk, bar);
+                    ++issued[s];
+                }
+            }
+            if (H->failed)       // gave up somewhere: let the copies already under way land before the block leaves
+                for (int s = 0; s < A.stages; ++s)
+                    if (issued[s] > 0) mbar_wait(smem_u32(&H->full[s]), (uint32_t)(issued[s] - 1) & 1u, 200000000ll);
+        }
+    } else if (warp >= kTcConvEpiWarps) {
+        if (lane == 0) {
+            // MMA issue: every issuer takes every kTcIssuers-th accumulator block; K-major operands: 8 pixels (or 8
+            // output channels) x 16 bytes per core matrix, the next 8 rows 128 bytes on, the next 8 channels one plane on
+            const int iw = warp - kTcConvEpiWarps;
+            const uint32_t a_hi = desc_hi(128), b_hi = desc_hi(128);
+            const uint32_t xstep = 2u * ((uint32_t)A.x_plane >> 4), wstep = 2u * (uint32_t)A.Ns;   // one K step, 16-byte units
+            const uint32_t w_tap16 = w_tap >> 4;
+            uint32_t g = 0, k = 0;
+            for (int it = blockIdx.x; it < A.items && !H->failed; it += gridDim.x, ++k) {
+                const Item I = item_of(it);
+                const uint32_t idesc = make_idesc(128, I.cols, false, false);
+                const uint32_t buf = k % (uint32_t)A.nbuf, use = k / (uint32_t)A.nbuf;  // accumulator buffer and how often it was used
+                if (use > 0 && !wait(&H->tfree[buf], (use - 1) & 1u)) break;            // its accumulators have been read back
+                fence_after_sync();
+                for (int c = 0; c < nchunks; ++c, ++g) {
+                    const int s = (int)(g % (uint32_t)A.stages);
+                    if (!wait(&H->full[s], (g / (uint32_t)A.stages) & 1u)) break;
+                    fence_after_sync();
+                    const int nks = min(A.kpc, kplanes - c * A.kpc) >> 1;
+                    const uint32_t xaddr = smem_u32(stages + (size_t)s * A.stage_bytes), waddr = xaddr + (uint32_t)(A.kpc * A.x_plane);
+                    const uint32_t b_lo0 = desc_lo(waddr, (uint32_t)A.Ns * 16u);
+                    // (the thread that issues is the bottleneck of a narrow MMA: descriptors advance by adds only)
+                    for (int b = iw; b < I.nblk; b += kTcIssuers) {
+                        const uint32_t tcol = tmem + buf * 256u + (uint32_t)(b * A.Ns);
+                        uint32_t a_row = desc_lo(xaddr + (uint32_t)b * 2048u, (uint32_t)A.x_plane), b_t = b_lo0;
+                        bool acc = c > 0;
+                        for (int ky = 0; ky < K; ++ky, a_row += (uint32_t)A.Wp) {
+                            uint32_t a_t = a_row;
+                            for (int kx = 0; kx < K; ++kx, ++a_t, b_t += w_tap16) {
+                                uint32_t a_lo = a_t, b_lo = b_t;
+                                for (int ks = 0; ks < nks; ++ks) {
+                                    mma_bf16(tcol, desc64(a_hi, a_lo), desc64(b_hi, b_lo), idesc, acc);
+                                    acc = true; a_lo += xstep; b_lo += wstep;
+                                }
+                            }
+                        }
+                    }
+                    mma_commit(smem_u32(&H->empty[s]));
+                }
+                mma_commit(smem_u32(&H->done[buf]));
+            }
+            mma_commit(smem_u32(&H->drain));
+        }
+    } else {
+        // epilogue warps: lane quarter q = warp % 4 of every accumulator block; the two warps of a quarter take
+        // alternate blocks
+        const int q = warp & 3, half = warp >> 2;
+        const int oplanes = A.cout16 / 8;
+        const float slope = A.slope;
+        const int E = A.nblk * 128;                                   // entries per plane of the pooling layout
+        uint4* S = reinterpret_cast<uint4*>(stages + (size_t)A.stages * A.stage_bytes);
+        const int et = threadIdx.x;                                   // 0 .. 255
+        uint32_t k = 0;
+        for (int it = blockIdx.x; it < A.items; it += gridDim.x, ++k) {
+            const Item I = item_of(it);
+            asm volatile("bar.sync 1, 256;" ::: "memory");            // every warp is through with the bias of the item before
+            for (int c = et; c < A.Ns; c += 256) H->bias[c] = (A.bias && I.co0 + c < A.cout) ? __ldg(A.bias + I.co0 + c) : 0.f;
+            if (et == 0) H->epi_stop = H->failed;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (H->epi_stop) break;                                   // the same answer for all 256 threads: they leave together
+            const uint32_t buf = k % (uint32_t)A.nbuf, use = k / (uint32_t)A.nbuf;
+            const uint32_t tbuf = tmem + buf * 256u;
+            wait(&H->done[buf], use & 1u);                            // (ran out: the item is written from whatever is there; the error word is set)
+            fence_after_sync();
+            if (!A.pool) {
+                for (int b = half; b < I.nblk; b += 2) {
+                    const int p = b * 128 + q * 32 + lane;
+                    const int r = p / A.Wp, c = p - r * A.Wp;
+                    const bool valid = r < I.rows && c < I.cw;
+                    uint4* o = A.out + (((size_t)I.n * oplanes + (I.co0 >> 3)) * A.H + I.y0 + r) * A.W + I.x0 + c;
+                    for (int c0 = 0; c0 < I.cols; c0 += 16) {
+                        float v[16];
+                        tmem_ld16(tbuf + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * A.Ns + c0), v);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) { const float z = v[j] + H->bias[c0 + j]; v[j] = z > 0.f ? z : slope * z; }
+                        if (valid) {
+                            o[(size_t)(c0 >> 3) * A.H * A.W] = tcd::pack8(v);
+                            o[(size_t)((c0 >> 3) + 1) * A.H * A.W] = tcd::pack8(v + 8);
+                        }
+                    }
+                }
+            } else {
+                const int OH = A.H / 2, OW = A.W / 2, prs = I.rows / 2, pcs = I.cw / 2;
+                for (int pl0 = 0; pl0 < (I.cols >> 3); pl0 += A.pool_planes) {
+                    const int npl = min(A.pool_planes, (I.cols >> 3) - pl0);
+                    // the band as it would be stored, planes pl0 .. pl0 + npl - 1
+                    for (int b = half; b < I.nblk; b += 2) {
+                        const int p = b * 128 + q * 32 + lane;
+                        for (int c0 = pl0 * 8; c0 < (pl0 + npl) * 8; c0 += 16) {
+                            float v[16];
+                            tmem_ld16(tbuf + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * A.Ns + c0), v);
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) { const float z = v[j] + H->bias[c0 + j]; v[j] = z > 0.f ? z : slope * z; }
+                            S[(size_t)((c0 >> 3) - pl0) * E + p] = tcd::pack8(v);
+                            S[(size_t)((c0 >> 3) - pl0 + 1) * E + p] = tcd::pack8(v + 8);
+                        }
+                    }
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    // one thread per pooled pixel and plane; the four window members are compared as stored, two
+                    // channels (a bf16 pair) per instruction: a later member wins only if it is greater
+                    const int npix = prs * pcs, total = npl * npix;
+                    for (int e = et; e < total; e += 256) {
+                        const int pl = e / npix, pix = e - pl * npix, pr = pix / pcs, pc = pix - pr * pcs;
+                        const uint4* s4 = S + (size_t)pl * E + (size_t)(2 * pr) * A.Wp + 2 * pc;
+                        const uint4 m0 = s4[0], m1 = s4[1], m2 = s4[A.Wp], m3 = s4[A.Wp + 1];
+                        const uint32_t* w0 = &m0.x; const uint32_t* w1 = &m1.x; const uint32_t* w2 = &m2.x; const uint32_t* w3 = &m3.x;
+                        uint32_t best[4], code[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint32_t m = w0[j], a = 0u;
+                            const uint32_t cand[3] = {w1[j], w2[j], w3[j]};
+#pragma unroll
+                            for (int w = 0; w < 3; ++w) {
+                                const uint32_t gt = __hgt2_mask(*reinterpret_cast<const __nv_bfloat162*>(&cand[w]),
+                                                                *reinterpret_cast<const __nv_bfloat162*>(&m));
+                                m = (cand[w] & gt) | (m & ~gt);
+                                a = (((uint32_t)(w + 1) * 0x00010001u) & gt) | (a & ~gt);
+                            }
+                            best[j] = m; code[j] = a;
+                        }
+                        // arg-max bytes: channel 2j in the low half of code[j], channel 2j + 1 in the high half
+                        const unsigned long long am = (unsigned long long)__byte_perm(code[0], code[1], 0x6420) |
+                                                      ((unsigned long long)__byte_perm(code[2], code[3], 0x6420) << 32);
+                        const size_t gi = (((size_t)I.n * oplanes + (I.co0 >> 3) + pl0 + pl) * OH + (I.y0 >> 1) + pr) * OW + (I.x0 >> 1) + pc;
+                        A.out[gi] = make_uint4(best[0], best[1], best[2], best[3]);
+                        A.arg[gi] = am;
+                    }
+                    asm volatile("bar.sync 1, 256;" ::: "memory");    // the staging area is free for the next planes
+                }
+            }
+            fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&H->tfree[buf]));
+        }
+    }
+    __syncthreads();
+    // every MMA of the block has completed before the tensor memory goes back (also when a wait gave up)
+    if (warp == 0) {
+        if (lane == 0) mbar_wait(smem_u32(&H->drain), 0, 200000000ll);
+        __syncwarp();
+        fence_after_sync();
+        tmem_dealloc(tmem, (uint32_t)kTcTmemCols);
+    }
 }
 
 }  // namespace ftp

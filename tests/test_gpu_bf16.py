@@ -186,14 +186,30 @@ def test_result_does_not_depend_on_grid_or_groups_and_is_reproducible():
                 dict(grid=(3, 3), opts=dict(cost_model=1)), dict(grid=(3, 3), opts=dict(cost_model=-1)),
                 dict(grid=(2, 3), opts=dict(tc_blocks_per_sm=2)), dict(grid=(2, 3), opts=dict(tc_blocks_per_sm=1, max_subtile=3)),
                 # tiles copied by the threads instead of by TMA tensor copies (the default)
-                dict(grid=(3, 3), opts=dict(tc_tma=-1)), dict(grid=(2, 2), groups=((1, 4), (5, 8)), opts=dict(tc_tma=-1, max_subtile=5))]
+                dict(grid=(3, 3), opts=dict(tc_tma=-1)), dict(grid=(2, 2), groups=((1, 4), (5, 8)), opts=dict(tc_tma=-1, max_subtile=5)),
+                # fused sub-tile stacks only
+                dict(grid=(3, 3), opts=dict(stationary=-1)), dict(grid=(4, 2), groups=((1, 4), (5, 8)), opts=dict(stationary=-1))]
+    def routes(plan):
+        """Which kernel family computes each layer: the order of the fp32 sums of an output value is fixed
+        within a family (fused sub-tile stacks: window positions outermost; banded kernels: input channels
+        outermost), whatever the grid, the groups and the sub-tiles."""
+        return {layer: plan.group_mode(i)[0] for i, (a, b) in enumerate(plan.exec_groups()) for layer in range(a, b + 1)}
+    base_routes = routes(base[3])
     for v in variants:
         opts = v.pop("opts", {})
         y, dx, dparams, plan = backward_bf16(wl.with_(**v), x, params, dy, **opts)
-        assert np.array_equal(y, base[0])                             # same arithmetic per output value
-        # deltas inside a group are rounded to bf16 per sub-tile before overlapping parts are summed
-        assert rel_err(dx, base[1]) <= BF16_TOL, v
-        assert rel_err(dparams, base[2]) <= BF16_TOL, v
+        if routes(plan) == base_routes:
+            assert np.array_equal(y, base[0]), v                      # same arithmetic per output value
+            # deltas inside a group are rounded to bf16 per sub-tile before overlapping parts are summed
+            assert rel_err(dx, base[1]) <= BF16_TOL, v
+            assert rel_err(dparams, base[2]) <= BF16_TOL, v
+        else:
+            # another order of the fp32 sums: a stored value may land one bf16 step aside, and a pool window or a
+            # sign decision next to such a value may then fall the other way, which moves a delta to another pixel
+            # (see test_backward_matches_oracle): L2 norms
+            assert rel_err(y, base[0]) <= 1e-2, v
+            assert l2_err(dx, base[1]) <= 5e-2, v
+            assert l2_err(dparams, base[2]) <= BF16_TOL, v
 
 
 def _crop_check_bf16(wl, x, params, y_gpu, n, oy, ox, size):
