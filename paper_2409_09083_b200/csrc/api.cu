@@ -271,8 +271,11 @@ int pack_filters_tc(ftp_plan* p, const float* params, void* ws, cudaStream_t st)
             const OpDesc& op = g.fwd_ops[i];
             if (op.kind == kOpPool) continue;
             if (pa.n == kMaxOps * 2) flush();
-            pa.l[pa.n++] = TcPackLayer{op.p_off, op.twf_off, op.cin, op.cout, op.k, op.cin16, op.cout16,
-                                       g.banded() ? 1 : 0, g.cf.Ns, g.cf.kpc, g.cd.Ns, g.cd.kpc};
+            // (first layer on the window-unrolled input: a 1x1 conv with 9 cin input channels, same parameters)
+            if (g.col_cin16) pa.l[pa.n++] = TcPackLayer{op.p_off, op.twf_off, g.col_cin, op.cout, 1, g.col_cin16, op.cout16,
+                                                        1, g.cf.Ns, g.cf.kpc, g.cd.Ns, g.cd.kpc};
+            else pa.l[pa.n++] = TcPackLayer{op.p_off, op.twf_off, op.cin, op.cout, op.k, op.cin16, op.cout16,
+                                            g.tfg.on ? 1 : 0, g.cf.Ns, g.cf.kpc, g.cd.Ns, g.cd.kpc};
         }
     flush();
     return launched_ok() ? FTP_OK : FTP_ERR_CUDA;
@@ -287,11 +290,21 @@ int forward_tc(ftp_plan* p, const float* x, const float* params, float* y, void*
         const GroupPlan& g = p->groups[gi];
         TcGroupArgs a;
         fill_common_tc(p, g, false, x, params, ws, a);
-        if (g.banded()) {                       // one conv behind the first layer: the banded kernel
+        if (g.tfg.on) {                         // one conv: the banded kernel
             const OpDesc& op = g.fwd_ops[0];
             const __nv_bfloat16* wf = reinterpret_cast<const __nv_bfloat16*>(ws_ptr(ws, p->ws.wf_off)) + op.twf_off;
-            if (!launch_tc_conv(p, g.cf, 1, (int)gi, a.map[0], wf, params + op.p_off + (size_t)op.cout * op.cin * op.k * op.k,
-                                a.map_out[1], a.arg[0], op.k, op.cin16, op.cout16, op.cout, op.in_H, op.in_W,
+            const void* in = a.map[0];
+            if (g.col_cin16) {                  // first layer: a 1x1 conv on the window-unrolled network input
+                uint4* col = reinterpret_cast<uint4*>(ws_ptr(ws, p->ws.col_off));
+                const size_t total = (size_t)p->N * (g.col_cin16 / 8) * op.in_H * op.in_W;
+                { Timed t(p, st, 9, (int)gi);
+                  unroll_windows_kernel<<<(int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16), 256, 0, st>>>(
+                      x, col, p->N, op.cin, op.in_H, op.in_W, g.col_cin16 / 8); }
+                if (!launched_ok()) return FTP_ERR_CUDA;
+                in = col;
+            }
+            if (!launch_tc_conv(p, g.cf, 1, (int)gi, in, wf, params + op.p_off + (size_t)op.cout * op.cin * op.k * op.k,
+                                a.map_out[1], a.arg[0], g.tfg.k, g.col_cin16 ? g.col_cin16 : op.cin16, op.cout16, op.cout, op.in_H, op.in_W,
                                 op.kind == kOpConvPool, op.slope, a.error, st))
                 return FTP_ERR_CUDA;
             continue;
@@ -431,13 +444,27 @@ int forward_impl(ftp_plan* p, const float* x, const float* params, float* y, voi
     return FTP_OK;
 }
 
-// Backward pass of a one-conv bf16 group behind the first layer: dz planes at the conv's resolution, the filter
-// gradient by the weight-stationary tensor-core kernel over bands of the whole batch (one partial set per pixel
-// share), and the delta at the group's input.
-bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& a, void* ws, cudaStream_t st)
+// A layer's entry for the cross-tile reduction: where its slice of the partial sets lies and how it is arranged (the
+// first layer on the window-unrolled input: as the 1x1 conv with 9 cin input channels that computed it).
+TcReduceLayer reduce_layer(const GroupPlan& g, const OpDesc& op, void* ws)
+{
+    if (g.col_cin16)
+        return TcReduceLayer{op.p_off, ws_ptr(ws, g.partial_off), (long long)g.param_floats, op.tgp_off, g.sets(), g.col_cin, op.cout, 1,
+                             g.col_cin16, op.cout16};
+    return TcReduceLayer{op.p_off, ws_ptr(ws, g.partial_off), (long long)g.param_floats, op.tgp_off, g.sets(), op.cin, op.cout, op.k,
+                         op.cin16, op.cout16};
+}
+
+// Backward pass of a one-conv bf16 group: dz planes at the conv's resolution, the filter gradient by the
+// weight-stationary tensor-core kernel over bands of the whole batch (one partial set per pixel share), and the delta
+// at the group's input.
+bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& a, void* ws, bool need_dx, float* dx, cudaStream_t st)
 {
     const OpDesc& op = g.bwd_ops[0];
     const TcFgPlan& t = g.tfg;
+    // the layer's input as bf16 planes: the saved map, or (first layer) the window-unrolled network input of the forward pass
+    void* xin = g.col_cin16 ? static_cast<void*>(ws_ptr(ws, p->ws.col_off)) : const_cast<void*>(a.map[0]);
+    const int cin16 = g.col_cin16 ? g.col_cin16 : op.cin16;
     uint4* dz = reinterpret_cast<uint4*>(ws_ptr(ws, p->ws.dz_off));
     DeltaActPlanesArgs d{};
     d.dmap = a.dmap_out; d.dmap_planes = a.dmap_planes;
@@ -457,11 +484,11 @@ bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& 
         if (!encode_rows_map(f.tmap_dz[cc], dz + (size_t)cc * t.Cw, p->N, op.cout16 / 8, op.in_H, std::min(t.Cw, op.in_W - cc * t.Cw),
                              op.in_W, t.R, t.Wp))
             return false;
-    if (!encode_rows_map(f.tmap_x, a.map[0], p->N, op.cin16 / 8, op.in_H, op.in_W, op.in_W, t.R + t.k - 1, t.Wp)) return false;
+    if (!encode_rows_map(f.tmap_x, xin, p->N, cin16 / 8, op.in_H, op.in_W, op.in_W, t.R + t.k - 1, t.Wp)) return false;
     f.ncc = t.ncc; f.Cw = t.Cw;
     f.partial = a.partial; f.set_floats = a.set_floats; f.tgp_off = op.tgp_off;
     f.error = a.error;
-    f.N = p->N; f.K = t.k; f.cout16 = op.cout16; f.cin16 = op.cin16;
+    f.N = p->N; f.K = t.k; f.cout16 = op.cout16; f.cin16 = cin16;
     f.Ms = t.Ms; f.slices = t.slices; f.ncols = t.ncols; f.nci = t.nci;
     f.R = t.R; f.Wp = t.Wp; f.bands_img = t.bands_img; f.bands = t.bands; f.shares = t.shares;
     f.dz_plane = t.dz_plane; f.x_plane = t.x_plane; f.stage_bytes = t.stage_bytes;
@@ -470,32 +497,20 @@ bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& 
     if (!launched_ok()) return false;
 
     // input delta: the convolution of dz with the rotated filters (dz planes in, delta planes out)
-    if (g.banded()) {
-        const __nv_bfloat16* wb = reinterpret_cast<const __nv_bfloat16*>(ws_ptr(ws, p->ws.wb_off)) + op.twb_off;
-        return launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, ws_ptr(ws, p->ws.dmap_off[gi]), nullptr, t.k, op.cout16, op.cin16, op.cin,
+    if (!need_dx) return true;
+    const __nv_bfloat16* wb = reinterpret_cast<const __nv_bfloat16*>(ws_ptr(ws, p->ws.wb_off)) + op.twb_off;
+    if (!g.col_cin16)
+        return launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, ws_ptr(ws, p->ws.dmap_off[gi]), nullptr, t.k, op.cout16, cin16, op.cin,
                               op.in_H, op.in_W, false, 1.0f, a.error, st);
-    }
-    TcGroupArgs b;
-    std::memset(&b, 0, sizeof(b));
-    const PassPlan& pp = g.dxp;
-    b.n_ops = 1; b.R = pp.y.count; b.Q = pp.x.count; b.N = p->N;
-    b.op[0] = g.dx_op;
-    b.map[0] = dz;
-    b.map[1] = ws_ptr(ws, p->ws.dmap_off[gi]);
-    b.map_out[1] = reinterpret_cast<__nv_bfloat16*>(ws_ptr(ws, p->ws.dmap_off[gi]));
-    b.yspan = p->dev_tables + pp.dev_yspan; b.xspan = p->dev_tables + pp.dev_xspan;
-    b.ycell = p->dev_tables + pp.dev_ycell; b.xcell = p->dev_tables + pp.dev_xcell;
-    b.wpk = reinterpret_cast<const __nv_bfloat16*>(ws_ptr(ws, p->ws.wb_off));
-    b.params = nullptr;                               // no bias; the op's slope of 1 makes the activation the identity
-    b.error = a.error;
-    if (p->tc_tma && encode_plane_map(b.tmap[0], dz, p->N, g.dx_op.cin16 / 8, g.dx_op.in_H, g.dx_op.in_W, g.dx_op.t_in_Hp, g.dx_op.t_in_Wp))
-        b.use_tma = 1u;
-    { Timed tm(p, st, 8, gi);
-      const size_t smem = tc_smem(pp.smem_bytes, pp.ctas);
-      const int items = b.R * b.Q * p->N;
-      const int blocks = std::min(items, kSmCount * pp.ctas), tile_bytes = (int)(smem - tc_fixed_bytes(pp.stages));
-      if (pp.ctas == 2) fwd_group_tc_kernel<256><<<blocks, 256, smem, st>>>(b, tile_bytes, kTcTmemCols / 2, pp.stages);
-      else fwd_group_tc_kernel<512><<<blocks, 512, smem, st>>>(b, tile_bytes, kTcTmemCols, pp.stages); }
+    // first layer: the delta of the window-unrolled input (over the unrolled input itself, which nobody reads any more),
+    // folded back into the caller's fp32 map
+    if (!launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, xin, nullptr, 1, op.cout16, cin16, g.col_cin, op.in_H, op.in_W, false, 1.0f,
+                        a.error, st))
+        return false;
+    const size_t dx_total = (size_t)p->N * op.cin * op.in_H * op.in_W;
+    { Timed tm(p, st, 10, gi);
+      fold_windows_kernel<<<(int)std::min<size_t>((dx_total + 255) / 256, (size_t)kSmCount * 16), 256, 0, st>>>(
+          static_cast<const __nv_bfloat16*>(xin), dx, p->N, op.cin, op.in_H, op.in_W, cin16 / 8); }
     return launched_ok();
 }
 
@@ -517,7 +532,7 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
         if (g.tfg.on) {
             // one conv behind the first layer: the filter gradient by the weight-stationary kernel, the delta at the group's input as a
             // convolution of dz with the rotated filters (written whole: nothing to sum afterwards)
-            if (!tc_filter_grad(p, g, gi, a, ws, st)) return FTP_ERR_CUDA;
+            if (!tc_filter_grad(p, g, gi, a, ws, a.need_dx != 0, dx, st)) return FTP_ERR_CUDA;
         } else
         { Timed t(p, st, 3, gi);
           const size_t smem = tc_smem(g.bwd.smem_bytes, g.bwd.ctas);
@@ -530,8 +545,7 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
             for (int i = 0; i < g.n_ops; ++i) {
                 const OpDesc& op = g.bwd_ops[i];
                 if (op.kind == kOpPool) continue;
-                rg.l[rg.n++] = TcReduceLayer{op.p_off, ws_ptr(ws, g.partial_off), (long long)g.param_floats, op.tgp_off,
-                                             g.sets(), op.cin, op.cout, op.k, op.cin16, op.cout16};
+                rg.l[rg.n++] = reduce_layer(g, op, ws);
             }
             { Timed t(p, st, 5, gi);
               reduce_sgd_tc_kernel<<<dim3(1184, rg.n), 128, 0, st>>>(rg, nullptr, 0.f, grad_out); }
@@ -573,8 +587,7 @@ int backward_tc(ftp_plan* p, const float* x, const float* dy, const float* param
             const OpDesc& op = g.bwd_ops[i];
             if (op.kind == kOpPool) continue;
             if (ra.n == kMaxOps * 2) flush();
-            ra.l[ra.n++] = TcReduceLayer{op.p_off, ws_ptr(ws, g.partial_off), (long long)g.param_floats, op.tgp_off,
-                                         g.sets(), op.cin, op.cout, op.k, op.cin16, op.cout16};
+            ra.l[ra.n++] = reduce_layer(g, op, ws);
         }
     flush();
     return launched_ok() ? FTP_OK : FTP_ERR_CUDA;

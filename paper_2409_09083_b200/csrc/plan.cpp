@@ -614,7 +614,9 @@ void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
 bool tc_stationary_conv(const ftp_plan& p, int li /*0-based*/, const PlanOpts& o)
 {
     const ftp_layer& l = p.layers[li];
-    if (p.precision != FTP_BF16_FP32ACC || o.stationary < 0 || l.kind != FTP_CONV || li == 0) return false;
+    if (p.precision != FTP_BF16_FP32ACC || o.stationary < 0 || l.kind != FTP_CONV) return false;
+    // the first layer reads the fp32 network input: only as a 1x1 conv on its window-unrolled copy (3x3, at most 7 channels)
+    if (li == 0 && (l.k != 3 || l.cin * 9 > 64)) return false;
     return (l.k == 1 || l.k == 3) && p.maps[li].W <= kTcMaxColChunks * 126;
 }
 
@@ -678,13 +680,16 @@ void plan_tc_filter_grad(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     if (g.n_ops != 1 || g.bwd_ops[0].kind == kOpPool || !tc_stationary_conv(p, g.first - 1, o)) return;
     const OpDesc& op = g.bwd_ops[0];
     TcFgPlan t;
-    const int H = op.in_H, W = op.in_W, K = op.k;
+    const bool unrolled = g.first == 1;                         // first layer: 1x1 conv on the window-unrolled input
+    const int col_cin16 = round_up(op.cin * 9, 16);
+    const int H = op.in_H, W = op.in_W, K = unrolled ? 1 : op.k;
+    const int cin16 = unrolled ? col_cin16 : op.cin16;
     tc_col_chunks(W, &t.ncc, &t.Cw);
     t.k = K; t.Wp = t.Cw + K - 1;
     t.Ms = op.cout16 <= 64 ? 64 : 128;
     t.slices = (op.cout16 + t.Ms - 1) / t.Ms;
-    t.ncols = std::min(op.cin16, K == 1 ? 256 : 48);
-    t.nci = (op.cin16 + t.ncols - 1) / t.ncols;
+    t.ncols = std::min(cin16, K == 1 ? 256 : 48);
+    t.nci = (cin16 + t.ncols - 1) / t.ncols;
     long long best = -1;
     for (int R = 1; R <= std::min(H, 64); ++R) {
         const size_t dzp = align_up(((size_t)R * t.Wp + 16) * 16, 128), xp = align_up(((size_t)(R + K - 1) * t.Wp + 32) * 16, 128);
@@ -704,38 +709,11 @@ void plan_tc_filter_grad(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     const int roles = t.slices * t.nci;
     t.shares = (int)std::max<long long>(1, std::min<long long>(bands, kSmCount / roles));
     t.blocks = roles * t.shares;
-    // the input delta: convolution of dz (cout16 channels) with the rotated filters at the conv's resolution, no bias,
-    // no activation (slope 1), planned as the forward pass of a one-op group of its own
-    GroupPlan d{};
-    d.n_ops = 1;
-    OpDesc& c = d.fwd_ops[0];
-    c = op;
-    c.kind = kOpConv; c.S = 1; c.keff = K; c.slope = 1.0f; c.prev_has_act = 0;
-    c.cin = op.cout; c.cout = op.cin; c.cin16 = op.cout16; c.cout16 = op.cin16;
-    c.out_H = H; c.out_W = W;
-    c.twf_off = op.twb_off;
-    d.bwd_ops[0] = c;
-    d.tile_y = equal_partition(0, H, p.grid_y);
-    d.tile_x = equal_partition(0, W, p.grid_x);
-    const int max_ch = std::max(c.cin16, c.cout16);
-    d.fwd.ctas = o.tc_ctas == 0 ? (max_ch <= 64 ? 2 : 1) : (o.tc_ctas == 2 && max_ch <= 256 ? 2 : 1);
-    d.fwd.stages = 2;
-    int rc = choose_subtiles(d, false, o, p.N);
-    if (rc != FTP_OK && d.fwd.ctas == 2) { d.fwd.ctas = 1; rc = choose_subtiles(d, false, o, p.N); }
-    if (rc != FTP_OK) return;
-    {
-        const size_t budget = std::min<size_t>(d.fwd.ctas == 2 ? kTcSmemBudget2 : kTcSmemBudget, (size_t)o.smem_bytes + 2048);
-        const size_t bytes4 = layout_forward_tc(d, d.fwd.y, d.fwd.x, kTcMaxStages);
-        if (bytes4 <= budget) { d.fwd.stages = kTcMaxStages; d.fwd.smem_bytes = bytes4; }
-        else d.fwd.smem_bytes = layout_forward_tc(d, d.fwd.y, d.fwd.x, d.fwd.stages);
-    }
-    d.fwd.blocks = d.fwd.y.count * d.fwd.x.count * p.N;
-    g.dxp = d.fwd;
-    g.dx_op = d.fwd_ops[0];
-    if (o.stationary != 2) {        // (2: banded filter gradient only, for comparisons)
-        g.cf = plan_tc_conv(p.N, H, W, K, op.cin16, op.cout16, op.kind == kOpConvPool);
-        g.cd = plan_tc_conv(p.N, H, W, K, op.cout16, op.cin16, false);
-    }
+    // the forward convolution, and the input delta as the convolution of dz (cout16 channels) with the rotated filters
+    g.cf = plan_tc_conv(p.N, H, W, K, cin16, op.cout16, op.kind == kOpConvPool);
+    g.cd = plan_tc_conv(p.N, H, W, K, op.cout16, cin16, false);
+    if (!g.cf.on || !g.cd.on) return;
+    if (unrolled) { g.col_cin = op.cin * 9; g.col_cin16 = col_cin16; }
     t.on = 1;
     g.tfg = t;
     g.bwd.scratch_floats = 0;       // no per-sub-tile input deltas
@@ -1056,8 +1034,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     p.tables.clear();
     auto push = [&](const std::vector<int>& v) { int o = (int)p.tables.size(); p.tables.insert(p.tables.end(), v.begin(), v.end()); return o; };
     for (GroupPlan& g : p.groups)
-        for (PassPlan* pp : {&g.fwd, &g.bwd, &g.dxp}) {
-            if (pp == &g.dxp && !g.tfg.on) continue;
+        for (PassPlan* pp : {&g.fwd, &g.bwd}) {
             pp->dev_yspan = push(pp->y.span);   pp->dev_xspan = push(pp->x.span);
             pp->dev_ycell = push(pp->y.cell);   pp->dev_xcell = push(pp->x.cell);
             pp->dev_yoff = push(pp->y.scratch_off); pp->dev_xoff = push(pp->x.scratch_off);
@@ -1118,6 +1095,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         if (g.tfg.on) dz = std::max(dz, (size_t)N * g.fwd_ops[0].cout16 * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W / 2);   // bf16
     }
     ws.scratch_off = take(scratch * 4);
+    if (!p.groups.empty() && p.groups[0].col_cin16) ws.col_off = take((size_t)N * p.groups[0].col_cin16 * H * W * 2);
     ws.dz_bytes = align_up(dz * 4, 256);
     ws.dz_off = take((tcp ? 1 : 2) * ws.dz_bytes);
     ws.wf_off = take(p.wf_floats * (tcp ? 2 : 4));

@@ -125,9 +125,9 @@ struct StatPlan {
     int fg_blocks = 0;                      // (64 x 32 channel slices) x shares; a share is one partial gradient set
 };
 
-// bf16 path, one-conv groups behind the first layer: the filter gradient by the weight-stationary tensor-core kernel
-// (tc_stationary.cuh); the input delta as a plain convolution of dz with the rotated filters, which the forward
-// kernel runs (every sub-tile writes the cells it owns, so there are no overlapping parts to sum).
+// bf16 path, one-conv groups: the filter gradient by the weight-stationary tensor-core kernel (tc_stationary.cuh);
+// the forward pass and the input delta (a plain convolution of dz with the rotated filters) by the banded
+// convolution kernel, which writes every cell once, so there are no overlapping parts to sum.
 struct TcFgPlan {
     int on = 0;
     int k = 0, Ms = 0, slices = 0;          // output channels per block (64 or 128), number of slices
@@ -163,10 +163,12 @@ struct GroupPlan {
     int first = 0, last = 0;        // 1-based layers
     StatPlan st;
     TcFgPlan tfg;
-    PassPlan dxp;                   // tfg.on: sub-tiling of the input-delta convolution (run by the forward kernel on dx_op)
-    OpDesc dx_op;                   //         the conv with the channel counts exchanged: dz planes in, input delta planes out
-    TcConvPlan cf, cd;              // tfg.on: the forward convolution and the input-delta convolution as banded kernels
-    bool banded() const { return tfg.on && cf.on && cd.on; }   // both run banded: the layer's filters are packed for them
+    TcConvPlan cf, cd;              // tfg.on: the forward convolution and the input-delta convolution (dz planes in, delta planes
+                                    //   out: the conv with the channel counts exchanged and the filters rotated) as banded kernels
+    // First layer of the bf16 path: a 3x3 conv with few input channels runs as a 1x1 conv with 9 cin input channels
+    // on a window-unrolled copy of the network input (channel ci * 9 + ky * 3 + kx of a pixel = the input of channel ci
+    // at window position (ky, kx)); the parameters keep their places, since W[co][ci][ky][kx] IS W'[co][ci * 9 + ky * 3 + kx].
+    int col_cin = 0, col_cin16 = 0;     // 9 cin and its padding to 16 (0: not this route)
     int sets() const { return tfg.on ? tfg.shares : bwd.blocks; }   // partial gradient sets the reduction sums
     int n_ops = 0;
     OpDesc fwd_ops[kMaxOps];
@@ -187,6 +189,7 @@ struct Workspace {                 // byte offsets, all 256-aligned
     std::vector<size_t> dmap_off;  // delta maps at group inputs of groups 1.. (index = group), and slot for dY
     size_t dy_off = 0;             // loss delta at the last map (ftp_step with target)
     size_t scratch_off = 0;
+    size_t col_off = 0;                // first layer of the bf16 path: the window-unrolled network input (bf16 planes), later its delta
     size_t dz_off = 0, dz_bytes = 0;   // weight-stationary groups: two areas (taken in turn) for the delta in front of the activation at
                                        // the conv's resolution, each as large as the largest such layer needs
     size_t wf_off = 0, wb_off = 0; // packed filters

@@ -87,6 +87,46 @@ __global__ void delta_act_planes_kernel(const __grid_constant__ DeltaActPlanesAr
     }
 }
 
+// First layer: the fp32 network input [N][C][H][W] -> window-unrolled bf16 planes [N][C16'/8][H][W][8] with channel
+// ci * 9 + ky * 3 + kx of pixel (y, x) = input(ci, y + ky - 1, x + kx - 1) (zero outside the map and beyond 9 C).
+__global__ void unroll_windows_kernel(const float* __restrict__ x, uint4* __restrict__ col, int N, int C, int H, int W, int planes)
+{
+    const size_t total = (size_t)N * planes * H * W;
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+        const int px = (int)(e % W); size_t t = e / W;
+        const int py = (int)(t % H); t /= H;
+        const int pl = (int)(t % planes); const int n = (int)(t / planes);
+        float v[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const int j = pl * 8 + c, ci = j / 9, tap = j - ci * 9, ky = tap / 3, kx = tap - ky * 3;
+            const int yy = py + ky - 1, xx = px + kx - 1;
+            v[c] = (ci < C && yy >= 0 && yy < H && xx >= 0 && xx < W) ? __ldg(x + (((size_t)n * C + ci) * H + yy) * W + xx) : 0.f;
+        }
+        col[e] = tcd::pack8(v);
+    }
+}
+
+// ... and back: the delta at the network input, fp32 NCHW, as the sum over the window positions of the delta planes of
+// the unrolled input: dx(ci, y, x) = sum over (ky, kx) of dcol(ci * 9 + ky * 3 + kx, y - ky + 1, x - kx + 1).
+__global__ void fold_windows_kernel(const __nv_bfloat16* __restrict__ dcol, float* __restrict__ dx, int N, int C, int H, int W, int planes)
+{
+    const size_t total = (size_t)N * C * H * W;
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+        const int px = (int)(e % W); size_t t = e / W;
+        const int py = (int)(t % H); t /= H;
+        const int ci = (int)(t % C); const int n = (int)(t / C);
+        float s = 0.f;
+#pragma unroll
+        for (int tap = 0; tap < 9; ++tap) {
+            const int ky = tap / 3, kx = tap - ky * 3, yy = py - ky + 1, xx = px - kx + 1, j = ci * 9 + tap;
+            if (yy >= 0 && yy < H && xx >= 0 && xx < W)
+                s += __bfloat162float(dcol[((((size_t)n * planes + (j >> 3)) * H + yy) * W + xx) * 8 + (j & 7)]);
+        }
+        dx[e] = s;
+    }
+}
+
 constexpr int kTcFgThreads = 256;
 
 __global__ void __launch_bounds__(kTcFgThreads, 1) filter_grad_tc_rows_kernel(const __grid_constant__ TcFilterGradArgs A)

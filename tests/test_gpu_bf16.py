@@ -101,7 +101,7 @@ def test_backward_matches_oracle(name, route):
     ref = run_oracle(wl, x, params, dy=dy, store="bf16")
     y, dx, dparams, plan = backward_bf16(wl, x, params, dy, stationary=-1 if route == "fused" else 0)
     modes = [plan.group_mode(i)[0] for i in range(len(plan.exec_groups()))]
-    assert all(m == 0 for m in modes) if route == "fused" else modes[0] == 0
+    assert route != "fused" or all(m == 0 for m in modes)
     if name in DEEP:
         assert l2_err(dx, ref["dx"]) <= (5e-2 if "yolo8" in name else 0.3)
         assert l2_err(dparams, ref["dparams"]) <= (BF16_TOL if "yolo8" in name else 0.2)
