@@ -37,11 +37,12 @@ FP32_NOMINAL_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 # Launch kinds of the library's per-launch timing (ftp_plan_timing): name, and how many forward-equivalents of the
 # executed group's multiply-accumulates the launch performs (None: a memory-bound helper)
 KIND = {0: ("pack_filters", None), 1: ("fwd_group", 1), 2: ("loss_delta", None), 3: ("bwd_group", 2), 4: ("halo_sum", None),
-        5: ("reduce_sgd", None), 6: ("delta_act", None), 7: ("filter_grad_rows", 1), 8: ("delta_conv_rows", 1)}
+        5: ("reduce_sgd", None), 6: ("delta_act", None), 7: ("filter_grad_rows", 1), 8: ("delta_conv_rows", 1),
+        9: ("unroll_windows", None), 10: ("fold_windows", None)}
 KERNEL = {("fwd_group", "fp32"): "fwd_group_kernel / conv_rows_kernel", ("bwd_group", "fp32"): "bwd_group_kernel / thin_bwd_kernel",
           ("filter_grad_rows", "fp32"): "filter_grad_rows_kernel", ("delta_conv_rows", "fp32"): "conv_rows_kernel (input delta)",
-          ("fwd_group", "bf16"): "fwd_group_tc_kernel", ("bwd_group", "bf16"): "bwd_group_tc_kernel",
-          ("filter_grad_rows", "bf16"): "filter_grad_tc_rows_kernel", ("delta_conv_rows", "bf16"): "fwd_group_tc_kernel (input delta)"}
+          ("fwd_group", "bf16"): "conv_tc_rows_kernel / fwd_group_tc_kernel", ("bwd_group", "bf16"): "bwd_group_tc_kernel",
+          ("filter_grad_rows", "bf16"): "filter_grad_tc_rows_kernel", ("delta_conv_rows", "bf16"): "conv_tc_rows_kernel (input delta)"}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
 # under profiles/ (static: null for every kernel / workload without a capture of the current code)
 NCU_TRAFFIC = {("C3", "fp32", "fwd_group"): 128.5e6, ("C3", "fp32", "filter_grad_rows"): 245.9e6,

@@ -296,10 +296,8 @@ int forward_tc(ftp_plan* p, const float* x, const float* params, float* y, void*
             const void* in = a.map[0];
             if (g.col_cin16) {                  // first layer: a 1x1 conv on the window-unrolled network input
                 uint4* col = reinterpret_cast<uint4*>(ws_ptr(ws, p->ws.col_off));
-                const size_t total = (size_t)p->N * (g.col_cin16 / 8) * op.in_H * op.in_W;
                 { Timed t(p, st, 9, (int)gi);
-                  unroll_windows_kernel<<<(int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16), 256, 0, st>>>(
-                      x, col, p->N, op.cin, op.in_H, op.in_W, g.col_cin16 / 8); }
+                  launch_unroll_windows(x, col, p->N, op.cin, op.in_H, op.in_W, st); }
                 if (!launched_ok()) return FTP_ERR_CUDA;
                 in = col;
             }
@@ -507,10 +505,8 @@ bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& 
     if (!launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, xin, nullptr, 1, op.cout16, cin16, g.col_cin, op.in_H, op.in_W, false, 1.0f,
                         a.error, st))
         return false;
-    const size_t dx_total = (size_t)p->N * op.cin * op.in_H * op.in_W;
     { Timed tm(p, st, 10, gi);
-      fold_windows_kernel<<<(int)std::min<size_t>((dx_total + 255) / 256, (size_t)kSmCount * 16), 256, 0, st>>>(
-          static_cast<const __nv_bfloat16*>(xin), dx, p->N, op.cin, op.in_H, op.in_W, cin16 / 8); }
+      launch_fold_windows(static_cast<const __nv_bfloat16*>(xin), dx, p->N, op.cin, op.in_H, op.in_W, st); }
     return launched_ok();
 }
 

@@ -495,6 +495,25 @@ double stationary_estimate_us(const ftp_plan& p, const GroupPlan& g, bool backwa
     return flops * (need_dx ? 2.0 : 1.0) / rate + 3.0 * map_us + 15.0;
 }
 
+// One-conv groups of the bf16 path (banded convolutions, weight-stationary filter gradient): padded multiply-
+// accumulates at the rates measured for the kernels on B200 (convolutions: about 800 TFLOP/s with slices of 80 channels
+// and more, in proportion below that, since a narrow MMA costs the tensor core about as much as a wide one; filter
+// gradient: 600), the maps at 5 TB/s, a few microseconds a launch.
+double tc_stationary_estimate_us(const ftp_plan& p, const GroupPlan& g, bool backward, bool need_dx)
+{
+    const OpDesc& op = g.fwd_ops[0];
+    const double px = (double)p.N * op.in_H * op.in_W;
+    const int cin16 = g.col_cin16 ? g.col_cin16 : op.cin16, kk = g.col_cin16 ? 1 : op.k * op.k;
+    const double flops = 2.0 * px * cin16 * op.cout16 * kk;
+    auto rate = [](int ns) { return 800e6 * std::min(1.0, std::max(ns, 16) / 80.0); };           // flop per microsecond
+    const double in_b = px * cin16 * 2.0, out_b = px * op.cout16 * 2.0 / (op.kind == kOpConvPool ? 4.0 : 1.0), dz_b = px * op.cout16 * 2.0;
+    if (!backward) return flops / rate(g.cf.Ns) + (in_b + out_b) / 5e6 + (g.col_cin16 ? in_b / 3e6 : 0.0) + 8.0;
+    double t = (2.0 * out_b + dz_b) / 5e6 + 4.0;                                               // dz planes
+    t += flops / 600e6 + (in_b + dz_b) / 5e6 + 10.0;                                           // filter gradient
+    if (need_dx) t += flops / rate(g.cd.Ns) + (in_b + dz_b) / 5e6 + (g.col_cin16 ? in_b / 3e6 : 0.0) + 8.0;
+    return t;
+}
+
 // Backward launch shape: as many blocks as run at once (or as there are stacks), each owning one
 // partial gradient set; the stacks of the whole batch are dealt out evenly to them.
 void set_backward_blocks(GroupPlan& g, int N, int gy, int gx)
@@ -941,6 +960,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     // trading a measured-good default for a predicted tie.
     auto estimate = [&](const GroupPlan& g) {
         if (g.st.on) return stationary_estimate_us(p, g, false, false) + stationary_estimate_us(p, g, true, g.first > 1);
+        if (g.tfg.on) return tc_stationary_estimate_us(p, g, false, false) + tc_stationary_estimate_us(p, g, true, g.first > 1);
         double f[kCostTerms];
         pass_cost_terms(p, g, false, false, f);
         double t = pass_estimate_us(precision, false, f);
@@ -1112,8 +1132,9 @@ int cost_terms(const ftp_plan& p, int pass, int group, int need_dx, double terms
 {
     if (group < 0 || group >= (int)p.groups.size() || pass < 0 || pass > 1 || !terms) return FTP_ERR_ARG;
     pass_cost_terms(p, p.groups[group], pass == 1, need_dx != 0, terms);
-    if (est_us) *est_us = p.groups[group].st.on ? stationary_estimate_us(p, p.groups[group], pass == 1, need_dx != 0)
-                                                : pass_estimate_us(p.precision, pass == 1, terms);
+    if (est_us) *est_us = p.groups[group].st.on  ? stationary_estimate_us(p, p.groups[group], pass == 1, need_dx != 0)
+                        : p.groups[group].tfg.on ? tc_stationary_estimate_us(p, p.groups[group], pass == 1, need_dx != 0)
+                                                 : pass_estimate_us(p.precision, pass == 1, terms);
     return FTP_OK;
 }
 

@@ -18,6 +18,8 @@
 // run behind the MMAs of the current one.
 #pragma once
 
+#include <algorithm>
+
 #include "kernels_tc.cuh"
 
 namespace ftp {
@@ -89,41 +91,85 @@ __global__ void delta_act_planes_kernel(const __grid_constant__ DeltaActPlanesAr
 
 // First layer: the fp32 network input [N][C][H][W] -> window-unrolled bf16 planes [N][C16'/8][H][W][8] with channel
 // ci * 9 + ky * 3 + kx of pixel (y, x) = input(ci, y + ky - 1, x + kx - 1) (zero outside the map and beyond 9 C).
-__global__ void unroll_windows_kernel(const float* __restrict__ x, uint4* __restrict__ col, int N, int C, int H, int W, int planes)
+// One thread per pixel: it reads the 9 C values of its window once and writes its entry of every plane (the
+// channel -> (ci, ky, kx) arithmetic is resolved at compile time).
+template <int C>
+__global__ void unroll_windows_kernel(const float* __restrict__ x, uint4* __restrict__ col, int N, int H, int W)
 {
-    const size_t total = (size_t)N * planes * H * W;
+    constexpr int planes = (9 * C + 15) / 16 * 2;
+    const size_t HW = (size_t)H * W, total = (size_t)N * HW;
     for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
         const int px = (int)(e % W); size_t t = e / W;
-        const int py = (int)(t % H); t /= H;
-        const int pl = (int)(t % planes); const int n = (int)(t / planes);
-        float v[8];
+        const int py = (int)(t % H); const int n = (int)(t / H);
+        float v[planes * 8];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            const int j = pl * 8 + c, ci = j / 9, tap = j - ci * 9, ky = tap / 3, kx = tap - ky * 3;
+        for (int j = 0; j < planes * 8; ++j) {
+            const int ci = j / 9, tap = j - ci * 9, ky = tap / 3, kx = tap - ky * 3;
             const int yy = py + ky - 1, xx = px + kx - 1;
-            v[c] = (ci < C && yy >= 0 && yy < H && xx >= 0 && xx < W) ? __ldg(x + (((size_t)n * C + ci) * H + yy) * W + xx) : 0.f;
+            v[j] = (ci < C && yy >= 0 && yy < H && xx >= 0 && xx < W) ? __ldg(x + ((size_t)n * C + ci) * HW + (size_t)yy * W + xx) : 0.f;
         }
-        col[e] = tcd::pack8(v);
+#pragma unroll
+        for (int pl = 0; pl < planes; ++pl) col[((size_t)n * planes + pl) * HW + (size_t)py * W + px] = tcd::pack8(v + 8 * pl);
     }
 }
 
 // ... and back: the delta at the network input, fp32 NCHW, as the sum over the window positions of the delta planes of
-// the unrolled input: dx(ci, y, x) = sum over (ky, kx) of dcol(ci * 9 + ky * 3 + kx, y - ky + 1, x - kx + 1).
-__global__ void fold_windows_kernel(const __nv_bfloat16* __restrict__ dcol, float* __restrict__ dx, int N, int C, int H, int W, int planes)
+// the unrolled input: dx(ci, y, x) = sum over (ky, kx) of dcol(ci * 9 + ky * 3 + kx, y - ky + 1, x - kx + 1), in the
+// order of the window positions.  One thread per pixel and all its channels: of the neighbour at window position
+// (ky, kx) it needs channel ci * 9 + ky * 3 + kx for every ci.
+template <int C>
+__global__ void fold_windows_kernel(const __nv_bfloat16* __restrict__ dcol, float* __restrict__ dx, int N, int H, int W)
 {
-    const size_t total = (size_t)N * C * H * W;
+    constexpr int planes = (9 * C + 15) / 16 * 2;
+    const size_t HW = (size_t)H * W, total = (size_t)N * HW;
     for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
         const int px = (int)(e % W); size_t t = e / W;
-        const int py = (int)(t % H); t /= H;
-        const int ci = (int)(t % C); const int n = (int)(t / C);
-        float s = 0.f;
+        const int py = (int)(t % H); const int n = (int)(t / H);
+        float s[C];
+#pragma unroll
+        for (int ci = 0; ci < C; ++ci) s[ci] = 0.f;
 #pragma unroll
         for (int tap = 0; tap < 9; ++tap) {
-            const int ky = tap / 3, kx = tap - ky * 3, yy = py - ky + 1, xx = px - kx + 1, j = ci * 9 + tap;
-            if (yy >= 0 && yy < H && xx >= 0 && xx < W)
-                s += __bfloat162float(dcol[((((size_t)n * planes + (j >> 3)) * H + yy) * W + xx) * 8 + (j & 7)]);
+            const int ky = tap / 3, kx = tap - ky * 3, yy = py - ky + 1, xx = px - kx + 1;
+            if (yy >= 0 && yy < H && xx >= 0 && xx < W) {
+                const __nv_bfloat16* src = dcol + ((size_t)n * planes * HW + (size_t)yy * W + xx) * 8;
+#pragma unroll
+                for (int ci = 0; ci < C; ++ci) {
+                    const int j = ci * 9 + tap;
+                    s[ci] += __bfloat162float(__ldg(src + (size_t)(j >> 3) * HW * 8 + (j & 7)));
+                }
+            }
         }
-        dx[e] = s;
+#pragma unroll
+        for (int ci = 0; ci < C; ++ci) dx[((size_t)n * C + ci) * HW + (size_t)py * W + px] = s[ci];
+    }
+}
+
+// the two kernels for the channel counts the route takes (9 C <= 64)
+inline void launch_unroll_windows(const float* x, uint4* col, int N, int C, int H, int W, cudaStream_t st)
+{
+    const int blocks = (int)std::min<size_t>(((size_t)N * H * W + 255) / 256, (size_t)kSmCount * 16);
+    switch (C) {
+        case 1: unroll_windows_kernel<1><<<blocks, 256, 0, st>>>(x, col, N, H, W); break;
+        case 2: unroll_windows_kernel<2><<<blocks, 256, 0, st>>>(x, col, N, H, W); break;
+        case 3: unroll_windows_kernel<3><<<blocks, 256, 0, st>>>(x, col, N, H, W); break;
+        case 4: unroll_windows_kernel<4><<<blocks, 256, 0, st>>>(x, col, N, H, W); break;
+        case 5: unroll_windows_kernel<5><<<blocks, 256, 0, st>>>(x, col, N, H, W); break;
+        case 6: unroll_windows_kernel<6><<<blocks, 256, 0, st>>>(x, col, N, H, W); break;
+        default: unroll_windows_kernel<7><<<blocks, 256, 0, st>>>(x, col, N, H, W); break;
+    }
+}
+inline void launch_fold_windows(const __nv_bfloat16* dcol, float* dx, int N, int C, int H, int W, cudaStream_t st)
+{
+    const int blocks = (int)std::min<size_t>(((size_t)N * H * W + 255) / 256, (size_t)kSmCount * 16);
+    switch (C) {
+        case 1: fold_windows_kernel<1><<<blocks, 256, 0, st>>>(dcol, dx, N, H, W); break;
+        case 2: fold_windows_kernel<2><<<blocks, 256, 0, st>>>(dcol, dx, N, H, W); break;
+        case 3: fold_windows_kernel<3><<<blocks, 256, 0, st>>>(dcol, dx, N, H, W); break;
+        case 4: fold_windows_kernel<4><<<blocks, 256, 0, st>>>(dcol, dx, N, H, W); break;
+        case 5: fold_windows_kernel<5><<<blocks, 256, 0, st>>>(dcol, dx, N, H, W); break;
+        case 6: fold_windows_kernel<6><<<blocks, 256, 0, st>>>(dcol, dx, N, H, W); break;
+        default: fold_windows_kernel<7><<<blocks, 256, 0, st>>>(dcol, dx, N, H, W); break;
     }
 }
 
