@@ -261,3 +261,32 @@ def test_backward_split_is_refined_for_balance():
     # fewer stacks than blocks: one block per stack
     small = ftp.ftp_plan(layers, 1, 64, 16, 16, (2, 2), ((1, 1),), max_subtile=64, stationary=-1).subtiles(1, 0)
     assert small["blocks"] == small["rows"] * small["cols"]
+
+
+def test_bf16_plans_run_conv_layers_as_groups_of_their_own():
+    """bf16 path: by default every conv layer the banded tensor-core kernels can take (1x1 / 3x3 window; the first
+    layer as a 3x3 conv with few channels) is an executed group of its own (with its pool), reported as mode 2 with as
+    many partial sets as its filter gradient has pixel shares; `stationary = -1` keeps the fused stacks; a window
+    the kernels do not take stays fused."""
+    for name in ["C1", "C2", "C3"]:
+        wl = synth.workload(name)
+        plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=ftp.FTP_BF16_FP32ACC)
+        eg = plan.exec_groups()
+        assert _conv_counts(list(wl.layers), eg) == [1] * len(eg)
+        assert {g[0] for g in wl.groups} <= {g[0] for g in eg}
+        for gi in range(len(eg)):
+            mode, sets = plan.group_mode(gi)
+            assert mode == 2 and 1 <= sets <= 148
+        fused = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=ftp.FTP_BF16_FP32ACC, stationary=-1)
+        assert all(fused.group_mode(gi)[0] == 0 for gi in range(len(fused.exec_groups())))
+        assert plan.workspace_bytes < fused.workspace_bytes or name != "C3"     # no per-sub-tile delta blocks, fewer sets
+    # a 5x5 layer stays a fused stack; the layers around it do not
+    layers = (synth.conv(3, 16, 3), synth.conv(16, 16, 5), synth.conv(16, 32, 3))
+    plan = ftp.ftp_plan(layers, 2, 3, 32, 32, (2, 2), ((1, 3),), precision=ftp.FTP_BF16_FP32ACC)
+    modes = {g: plan.group_mode(i)[0] for i, g in enumerate(plan.exec_groups())}
+    assert modes[(1, 1)] == 2 and modes[(3, 3)] == 2 and modes[(2, 2)] == 0, modes
+    # a first layer with a 1x1 window reads the fp32 input: fused
+    layers = (synth.conv(3, 16, 1), synth.conv(16, 16, 3))
+    plan = ftp.ftp_plan(layers, 2, 3, 32, 32, (2, 2), ((1, 2),), precision=ftp.FTP_BF16_FP32ACC)
+    modes = [plan.group_mode(i)[0] for i in range(len(plan.exec_groups()))]
+    assert modes[0] == 0 and modes[-1] == 2, (plan.exec_groups(), modes)
