@@ -196,13 +196,16 @@ bool encode_rows_map(unsigned char out[128], const void* base, int N, int planes
 }
 
 // One launch of the banded convolution kernel: `in` planes (cin16 channels) -> `out` planes (cout16 channels).
+struct PrevLayer { const uint4* y; const unsigned long long* arg; float slope; };   // see TcConvRowsArgs::prev_y
+
 bool launch_tc_conv(ftp_plan* p, const TcConvPlan& c, int kind, int gi, const void* in, const __nv_bfloat16* w, const float* bias,
                     void* out, unsigned char* arg, int K, int cin16, int cout16, int cout, int H, int W, bool pool, float slope,
-                    int* error, cudaStream_t st)
+                    int* error, cudaStream_t st, const PrevLayer* prev = nullptr)
 {
     TcConvRowsArgs a{};
     if (!encode_rows_map(a.tmap_x, in, p->N, cin16 / 8, H, W, W, c.R + K - 1, c.Wp)) return false;
     a.w = w;
+    if (prev) { a.prev_y = prev->y; a.prev_arg = prev->arg; a.prev_slope = prev->slope; }
     a.bias = bias; a.out = static_cast<uint4*>(out); a.arg = reinterpret_cast<unsigned long long*>(arg);
     a.error = error;
     a.N = p->N; a.K = K; a.cin16 = cin16; a.cout16 = cout16; a.cout = cout; a.H = H; a.W = W; a.pool = pool ? 1 : 0;
@@ -463,7 +466,13 @@ bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& 
     // the layer's input as bf16 planes: the saved map, or (first layer) the window-unrolled network input of the forward pass
     void* xin = g.col_cin16 ? static_cast<void*>(ws_ptr(ws, p->ws.col_off)) : const_cast<void*>(a.map[0]);
     const int cin16 = g.col_cin16 ? g.col_cin16 : op.cin16;
-    uint4* dz = reinterpret_cast<uint4*>(ws_ptr(ws, p->ws.dz_off));
+    // dz planes: the two areas take turns; when the group above is a one-conv group too, its input-delta kernel has
+    // already written this group's dz (see below), otherwise delta_act_planes_kernel makes them from the stored delta
+    const int G = (int)p->groups.size();
+    uint4* dz = reinterpret_cast<uint4*>(ws_ptr(ws, p->ws.dz_off + (size_t)(gi & 1) * p->ws.dz_bytes));
+    uint4* dz_below = reinterpret_cast<uint4*>(ws_ptr(ws, p->ws.dz_off + (size_t)((gi + 1) & 1) * p->ws.dz_bytes));
+    const bool dz_ready = gi + 1 < G && p->groups[gi + 1].tfg.on;
+    const bool feeds_below = gi > 0 && p->groups[gi - 1].tfg.on;
     DeltaActPlanesArgs d{};
     d.dmap = a.dmap_out; d.dmap_planes = a.dmap_planes;
     d.y = static_cast<const uint4*>(a.map[1]);
@@ -473,9 +482,11 @@ bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& 
     d.pool = op.kind == kOpConvPool ? 1 : 0;
     d.slope = op.slope;
     const size_t total = (size_t)p->N * (op.cout16 / 8) * op.out_H * op.out_W;
-    { Timed tm(p, st, 6, gi);
-      delta_act_planes_kernel<<<(int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16), 256, 0, st>>>(d); }
-    if (!launched_ok()) return false;
+    if (!dz_ready) {
+        { Timed tm(p, st, 6, gi);
+          delta_act_planes_kernel<<<(int)std::min<size_t>((total + 255) / 256, (size_t)kSmCount * 16), 256, 0, st>>>(d); }
+        if (!launched_ok()) return false;
+    }
 
     TcFilterGradArgs f{};
     for (int cc = 0; cc < t.ncc; ++cc)          // one dz map per column chunk: its columns only, zeros behind them
@@ -497,9 +508,18 @@ bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& 
     // input delta: the convolution of dz with the rotated filters (dz planes in, delta planes out)
     if (!need_dx) return true;
     const __nv_bfloat16* wb = reinterpret_cast<const __nv_bfloat16*>(ws_ptr(ws, p->ws.wb_off)) + op.twb_off;
-    if (!g.col_cin16)
-        return launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, ws_ptr(ws, p->ws.dmap_off[gi]), nullptr, t.k, op.cout16, cin16, op.cin,
-                              op.in_H, op.in_W, false, 1.0f, a.error, st);
+    if (!g.col_cin16) {
+        if (!feeds_below)
+            return launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, ws_ptr(ws, p->ws.dmap_off[gi]), nullptr, t.k, op.cout16, cin16, op.cin,
+                                  op.in_H, op.in_W, false, 1.0f, a.error, st);
+        const OpDesc& below = p->groups[gi - 1].fwd_ops[0];       // its output map is this group's input map
+        PrevLayer pv{static_cast<const uint4*>(a.map[0]),
+                     below.kind == kOpConvPool ? reinterpret_cast<const unsigned long long*>(static_cast<unsigned char*>(ws) + p->ws.arg_off[below.out_map - 1])
+                                               : nullptr,
+                     below.slope};
+        return launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, dz_below, nullptr, t.k, op.cout16, cin16, op.cin,
+                              op.in_H, op.in_W, false, 1.0f, a.error, st, &pv);
+    }
     // first layer: the delta of the window-unrolled input (over the unrolled input itself, which nobody reads any more),
     // folded back into the caller's fp32 map
     if (!launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, xin, nullptr, 1, op.cout16, cin16, g.col_cin, op.in_H, op.in_W, false, 1.0f,

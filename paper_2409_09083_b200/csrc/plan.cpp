@@ -1087,6 +1087,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
     {
         size_t need[2] = {0, 0};
         for (int gi = 1; gi < n_exec; ++gi) {
+            if (p.groups[gi].tfg.on && p.groups[gi - 1].tfg.on) continue;   // bf16 one-conv groups hand over dz planes instead
             const MapShape& s = p.maps[p.groups[gi].first - 1];
             const size_t bytes = tcp ? (size_t)N * round_up(s.C, 16) * s.H * s.W * 2     // bf16 planes
                                      : (size_t)N * s.C * s.H * s.W * 4;
@@ -1108,16 +1109,21 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         ws.t_stage_off = take(2 * ws.t_stage_bytes);
         ws.x_stage_off = take(2 * ws.x_stage_bytes);
     }
-    size_t scratch = 0, dz = 0;
-    for (const GroupPlan& g : p.groups) {
+    // dz areas: fp32 one-conv groups take two equal areas in turn; bf16 one-conv groups use the first area for the
+    // groups with an even index and the second for the odd ones (a group's input-delta kernel writes the dz planes
+    // of the group below while it reads its own), each as large as its users need
+    size_t scratch = 0, dz[2] = {0, 0};
+    for (int gi = 0; gi < n_exec; ++gi) {
+        const GroupPlan& g = p.groups[gi];
         scratch = std::max(scratch, g.bwd.scratch_floats);
-        if (g.st.on && !g.st.thin) dz = std::max(dz, (size_t)N * g.fwd_ops[0].cout * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W);
-        if (g.tfg.on) dz = std::max(dz, (size_t)N * g.fwd_ops[0].cout16 * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W / 2);   // bf16
+        if (g.st.on && !g.st.thin)
+            dz[0] = dz[1] = std::max(dz[0], (size_t)N * g.fwd_ops[0].cout * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W * 4);
+        if (g.tfg.on) dz[gi & 1] = std::max(dz[gi & 1], (size_t)N * g.fwd_ops[0].cout16 * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W * 2);
     }
     ws.scratch_off = take(scratch * 4);
     if (!p.groups.empty() && p.groups[0].col_cin16) ws.col_off = take((size_t)N * p.groups[0].col_cin16 * H * W * 2);
-    ws.dz_bytes = align_up(dz * 4, 256);
-    ws.dz_off = take((tcp ? 1 : 2) * ws.dz_bytes);
+    ws.dz_bytes = align_up(dz[0], 256);             // = offset of the second area
+    ws.dz_off = take(ws.dz_bytes + align_up(dz[1], 256));
     ws.wf_off = take(p.wf_floats * (tcp ? 2 : 4));
     ws.wb_off = take(p.wb_floats * (tcp ? 2 : 4));
     ws.err_off = take(256);

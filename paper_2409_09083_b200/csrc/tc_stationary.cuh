@@ -356,12 +356,17 @@ struct TcConvRowsArgs {
     int x_plane, stage_bytes, stages;
     int items;                                // N * bands_img * slices
     int pool_planes;                          // pool: 8-channel planes the staging area holds (even)
+    // input delta only: when the layer below is a one-conv group too, the delta goes straight into ITS dz planes (`out`;
+    // at twice the resolution if it ends with a pool): prev_y = that layer's saved output (= this conv's output shape),
+    // prev_arg = its pool's arg-max bytes or null, prev_slope = its leaky slope.  prev_y null: plain delta planes.
+    const uint4* prev_y; const unsigned long long* prev_arg; float prev_slope;
     int nbuf;                                 // accumulator buffers (2: items of at most 256 columns alternate between the halves
                                               //   of the tensor memory, so the MMAs of one run while the other is read back)
 };
 
 constexpr int kTcConvMaxStages = 4;
-constexpr int kTcConvEpiWarps = 8;
+constexpr int kTcConvEpiWarps = 16;           // four per lane quarter of the tensor memory
+constexpr int kTcConvEpiThreads = kTcConvEpiWarps * 32;
 constexpr int kTcConvThreads = (kTcConvEpiWarps + kTcIssuers + 1) * 32;
 
 __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const __grid_constant__ TcConvRowsArgs A)
@@ -501,38 +506,74 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
     } else {
         // epilogue warps: lane quarter q = warp % 4 of every accumulator block; the two warps of a quarter take
         // alternate blocks
-        const int q = warp & 3, half = warp >> 2;
+        const int q = warp & 3, part = warp >> 2;                  // the warps of a quarter share its (block, 16 columns) units
+        constexpr int kParts = kTcConvEpiWarps / 4;
         const int oplanes = A.cout16 / 8;
         const float slope = A.slope;
         const int E = A.nblk * 128;                                   // entries per plane of the pooling layout
         uint4* S = reinterpret_cast<uint4*>(stages + (size_t)A.stages * A.stage_bytes);
-        const int et = threadIdx.x;                                   // 0 .. 255
+        const int et = threadIdx.x;                                   // 0 .. kTcConvEpiThreads - 1
         uint32_t k = 0;
         for (int it = blockIdx.x; it < A.items; it += gridDim.x, ++k) {
             const Item I = item_of(it);
-            asm volatile("bar.sync 1, 256;" ::: "memory");            // every warp is through with the bias of the item before
-            for (int c = et; c < A.Ns; c += 256) H->bias[c] = (A.bias && I.co0 + c < A.cout) ? __ldg(A.bias + I.co0 + c) : 0.f;
+            asm volatile("bar.sync 1, %0;" :: "n"(kTcConvEpiThreads) : "memory");            // every warp is through with the bias of the item before
+            for (int c = et; c < A.Ns; c += kTcConvEpiThreads) H->bias[c] = (A.bias && I.co0 + c < A.cout) ? __ldg(A.bias + I.co0 + c) : 0.f;
             if (et == 0) H->epi_stop = H->failed;
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (H->epi_stop) break;                                   // the same answer for all 256 threads: they leave together
+            asm volatile("bar.sync 1, %0;" :: "n"(kTcConvEpiThreads) : "memory");
+            if (H->epi_stop) break;                                   // the same answer for all epilogue threads: they leave together
             const uint32_t buf = k % (uint32_t)A.nbuf, use = k / (uint32_t)A.nbuf;
             const uint32_t tbuf = tmem + buf * 256u;
             wait(&H->done[buf], use & 1u);                            // (ran out: the item is written from whatever is there; the error word is set)
             fence_after_sync();
             if (!A.pool) {
-                for (int b = half; b < I.nblk; b += 2) {
+                const int nc = I.cols >> 4;
+                for (int u = part; u < I.nblk * nc; u += kParts) {
+                    const int b = u / nc, c0 = (u - b * nc) << 4;
                     const int p = b * 128 + q * 32 + lane;
                     const int r = p / A.Wp, c = p - r * A.Wp;
                     const bool valid = r < I.rows && c < I.cw;
                     uint4* o = A.out + (((size_t)I.n * oplanes + (I.co0 >> 3)) * A.H + I.y0 + r) * A.W + I.x0 + c;
-                    for (int c0 = 0; c0 < I.cols; c0 += 16) {
+                    {
+                        // (what the fused dz step reads is requested before the accumulators, so that the latencies overlap)
+                        const size_t g0 = (((size_t)I.n * oplanes + ((I.co0 + c0) >> 3)) * A.H + I.y0 + r) * A.W + I.x0 + c;
+                        const size_t gstep = (size_t)A.H * A.W;
+                        uint4 yq[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+                        unsigned long long amq[2] = {0ull, 0ull};
+                        if (A.prev_y && valid) {
+                            yq[0] = __ldg(A.prev_y + g0); yq[1] = __ldg(A.prev_y + g0 + gstep);
+                            if (A.prev_arg) { amq[0] = __ldg(A.prev_arg + g0); amq[1] = __ldg(A.prev_arg + g0 + gstep); }
+                        }
                         float v[16];
                         tmem_ld16(tbuf + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * A.Ns + c0), v);
 #pragma unroll
                         for (int j = 0; j < 16; ++j) { const float z = v[j] + H->bias[c0 + j]; v[j] = z > 0.f ? z : slope * z; }
-                        if (valid) {
+                        if (!valid) continue;
+                        if (!A.prev_y) {
                             o[(size_t)(c0 >> 3) * A.H * A.W] = tcd::pack8(v);
                             o[(size_t)((c0 >> 3) + 1) * A.H * A.W] = tcd::pack8(v + 8);
+                            continue;
+                        }
+                        // input delta straight into the dz planes of the layer below: rounded as a stored delta
+                        // would be, times the derivative of that layer's activation, through its pool's arg-max
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const size_t gi = g0 + h * gstep;
+                            float d[8], yv[8];
+                            tcd::unpack8(tcd::pack8(v + 8 * h), d);
+                            tcd::unpack8(yq[h], yv);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) d[j] *= yv[j] > 0.f ? 1.f : A.prev_slope;
+                            if (!A.prev_arg) { A.out[gi] = tcd::pack8(d); continue; }
+                            const unsigned long long am = amq[h];
+                            const int W2 = 2 * A.W;
+                            uint4* o2 = A.out + (((size_t)I.n * oplanes + ((I.co0 + c0) >> 3) + h) * (2 * A.H) + 2 * (I.y0 + r)) * W2 + 2 * (I.x0 + c);
+#pragma unroll
+                            for (int w = 0; w < 4; ++w) {
+                                float z[8];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) z[j] = (int)((am >> (j * 8)) & 3ull) == w ? d[j] : 0.f;
+                                o2[(w >> 1) * W2 + (w & 1)] = tcd::pack8(z);
+                            }
                         }
                     }
                 }
@@ -541,9 +582,11 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
                 for (int pl0 = 0; pl0 < (I.cols >> 3); pl0 += A.pool_planes) {
                     const int npl = min(A.pool_planes, (I.cols >> 3) - pl0);
                     // the band as it would be stored, planes pl0 .. pl0 + npl - 1
-                    for (int b = half; b < I.nblk; b += 2) {
+                    const int nc = npl >> 1;
+                    for (int u = part; u < I.nblk * nc; u += kParts) {
+                        const int b = u / nc, c0 = pl0 * 8 + ((u - b * nc) << 4);
                         const int p = b * 128 + q * 32 + lane;
-                        for (int c0 = pl0 * 8; c0 < (pl0 + npl) * 8; c0 += 16) {
+                        {
                             float v[16];
                             tmem_ld16(tbuf + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * A.Ns + c0), v);
 #pragma unroll
@@ -552,11 +595,11 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
                             S[(size_t)((c0 >> 3) - pl0 + 1) * E + p] = tcd::pack8(v + 8);
                         }
                     }
-                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    asm volatile("bar.sync 1, %0;" :: "n"(kTcConvEpiThreads) : "memory");
                     // one thread per pooled pixel and plane; the four window members are compared as stored, two
                     // channels (a bf16 pair) per instruction: a later member wins only if it is greater
                     const int npix = prs * pcs, total = npl * npix;
-                    for (int e = et; e < total; e += 256) {
+                    for (int e = et; e < total; e += kTcConvEpiThreads) {
                         const int pl = e / npix, pix = e - pl * npix, pr = pix / pcs, pc = pix - pr * pcs;
                         const uint4* s4 = S + (size_t)pl * E + (size_t)(2 * pr) * A.Wp + 2 * pc;
                         const uint4 m0 = s4[0], m1 = s4[1], m2 = s4[A.Wp], m3 = s4[A.Wp + 1];
@@ -582,7 +625,7 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
                         A.out[gi] = make_uint4(best[0], best[1], best[2], best[3]);
                         A.arg[gi] = am;
                     }
-                    asm volatile("bar.sync 1, 256;" ::: "memory");    // the staging area is free for the next planes
+                    asm volatile("bar.sync 1, %0;" :: "n"(kTcConvEpiThreads) : "memory");    // the staging area is free for the next planes
                 }
             }
             fence_before_sync();
