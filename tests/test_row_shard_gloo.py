@@ -176,3 +176,61 @@ def test_tables_partition_the_maps_and_name_the_owners():
                 assert got == set(range(lo, hi + 1))          # own rows + received rows = needed rows
             assert covered == list(range(rows[t["last"]]))    # owned output rows partition the map
         assert tables[0]["recv"] == [[] for _ in range(world)]
+
+
+# ---------------------------------------------------------------------------------------------
+# The same step as the library runs it on GPUs (`shard.RowShardedStep` over `shard.DistTransport`), here with two
+# and three gloo ranks on the CPU and the oracle's layer routines in the place of the CUDA library.
+# ---------------------------------------------------------------------------------------------
+class OracleGroup:
+    """Stand-in for shard.LibraryGroup: a requested group on a slab, computed by the oracle (fp64, CPU)."""
+
+    def __init__(self, glayers, N, c_in, hs, w_in, out_shape, device, **_):
+        self.glayers = list(glayers)
+
+    def forward(self, slab, pg):
+        self.maps, self.tape = orc.forward(self.glayers, slab.numpy(), pg.numpy())
+        return torch.from_numpy(self.maps[-1])
+
+    def backward(self, slab, dslab, pg, grad_out):
+        dxs, dpar, _ = orc.backward(self.glayers, self.maps, self.tape, pg.numpy(), dslab.numpy())
+        grad_out += torch.from_numpy(dpar)
+        return torch.from_numpy(dxs)
+
+    @staticmethod
+    def sgd(params, grad, lr):
+        params -= lr * grad
+
+
+def _shard_worker(rank, world, port, out_dir):
+    from paper_2409_09083_b200 import shard
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    wl = WL
+    x, params, target = synth.draw(wl, bias_std=0.3)
+    xd, pd, td = (torch.from_numpy(a.astype(np.float64)) for a in (x, params, target))
+    st = shard.RowShardedStep(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.groups, shard.DistTransport(dist), device="cpu",
+                              group_cls=OracleGroup, dtype=torch.float64)
+    loss = st.step(xd, td, pd, 0.05)
+    np.savez(os.path.join(out_dir, f"s{rank}.npz"), loss=loss, y_lo=st.y_lo, y=st.y_owned.numpy(), dx_lo=st.dx_lo,
+             dx=st.dx_needed.numpy(), grad=st.grad.numpy(), params=pd.numpy())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_row_sharded_step_class_over_gloo_matches_the_oracle(world, tmp_path):
+    mp.spawn(_shard_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    wl = WL
+    x, params, target = synth.draw(wl, bias_std=0.3)
+    ref = orc.step(list(wl.layers), x.astype(np.float64), params.astype(np.float64), 0.05, target=target.astype(np.float64))
+    outs = [np.load(os.path.join(str(tmp_path), f"s{r}.npz")) for r in range(world)]
+    y = np.zeros_like(ref["y"]); dx = np.zeros_like(ref["dx"])
+    for o in outs:
+        y[:, :, int(o["y_lo"]):int(o["y_lo"]) + o["y"].shape[2], :] = o["y"]
+        dx[:, :, int(o["dx_lo"]):int(o["dx_lo"]) + o["dx"].shape[2], :] += o["dx"]
+        assert float(o["loss"]) == pytest.approx(ref["loss"], rel=1e-12)
+        assert np.abs(o["grad"] - ref["dparams"]).max() <= 1e-12 * max(1.0, np.abs(ref["dparams"]).max())
+        assert np.abs(o["params"] - ref["new_params"]).max() <= 1e-12 * max(1.0, np.abs(ref["new_params"]).max())
+    assert np.abs(y - ref["y"]).max() <= 1e-12 * np.abs(ref["y"]).max()
+    assert np.abs(dx - ref["dx"]).max() <= 1e-12 * max(1.0, np.abs(ref["dx"]).max())
