@@ -130,13 +130,16 @@ typedef struct {
                            global memory as at any group boundary (the paper's weight-dominated layers, Section 6).
                            Default (0): groups whose conv has at least 32 input channels; 1: every such group
                            whatever its channel count; -1: never.
-                           bf16 path: a conv layer with a 1x1 or 3x3 window behind the first layer, on a map whose rows
-                           have at most 254 pixels, becomes an executed group of its own (with its pool).  Its forward
-                           pass stays a fused sub-tile kernel; its filter gradient is computed by a weight-stationary
-                           tensor-core kernel that keeps a slice of the gradient in tensor memory while the batch
-                           streams past, and the delta at its input by a convolution with the rotated filters that
-                           writes every cell once.  0 and 1: every such layer; -1: never (fused stacks only) */
-    int tc_tma;           /* bf16 path: how the tiles of maps saved as bf16 planes reach shared memory.  Default (0): tensor
+                           bf16 path: a conv layer with a 1x1 or 3x3 window on a map of at most 1008 columns (the first
+                           layer: a 3x3 window and at most 7 input channels) becomes an executed group of its own (with
+                           its pool).  Forward pass and input delta run as banded tensor-core convolutions (a band of
+                           rows x a slice of output channels stays in tensor memory while the input channels stream
+                           past; the delta is the convolution of dz with the rotated filters and writes every cell
+                           once), the filter gradient by a weight-stationary kernel that keeps a slice of the gradient
+                           in tensor memory while the batch streams past; the first layer runs as a 1x1 conv on a
+                           window-unrolled bf16 copy of the network input, with the same parameters.
+                           0 and 1: every such layer; -1: never (fused stacks only) */
+    int tc_tma;           /* bf16 path, fused sub-tile kernels: how the tiles of maps saved as bf16 planes reach shared memory.  Default (0): tensor
                            copies by the TMA engine (cp.async.bulk.tensor, one box per 8-channel plane, zeros outside the map;
                            the tensor maps cover the calling GPU's own memory only and no copy is multicast); -1: plain
                            loads by the threads */
@@ -154,8 +157,8 @@ int ftp_plan_create_opts(const ftp_layer* layers, int n_layers,
 int ftp_plan_exec_groups(const ftp_plan* plan, int* n_groups, ftp_group* groups_out, int capacity);
 
 /* How executed group `group` (0-based index into ftp_plan_exec_groups) runs: *stationary = 1 if it is a one-conv
- * group run by the weight-stationary kernels (see ftp_plan_opts.stationary), 2 (bf16 path) if only its filter
- * gradient is computed weight-stationary, 0 if as fused sub-tile stacks;
+ * group run by the weight-stationary kernels of the fp32 path (see ftp_plan_opts.stationary), 2 if by the banded
+ * tensor-core kernels of the bf16 path, 0 if as fused sub-tile stacks;
  * *partial_sets (may be NULL) = the partial gradient sets of the group that the cross-tile reduction sums
  * (Section 4.1).  FTP_ERR_ARG on a bad index or NULL. */
 int ftp_plan_group_mode(const ftp_plan* plan, int group, int* stationary, int* partial_sets);

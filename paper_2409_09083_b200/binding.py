@@ -237,9 +237,9 @@ class Plan:
         return [(g.first, g.last) for g in arr]
 
     def group_mode(self, group):
-        """(stationary, partial_sets) of executed group `group`: 1 if the weight-stationary kernels run it, 2 (bf16
-        path) if only its filter gradient is computed weight-stationary, 0 if it runs as fused sub-tile stacks; and
-        how many partial gradient sets the cross-tile reduction sums for it."""
+        """(stationary, partial_sets) of executed group `group`: 1 if the weight-stationary kernels of the fp32 path run
+        it, 2 if the banded tensor-core kernels of the bf16 path, 0 if it runs as fused sub-tile stacks; and how many
+        partial gradient sets the cross-tile reduction sums for it."""
         st, sets = _i(), _i()
         _check(_lib.ftp_plan_group_mode(self._h, group, ctypes.byref(st), ctypes.byref(sets)))
         return st.value, sets.value
