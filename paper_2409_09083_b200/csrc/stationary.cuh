@@ -557,17 +557,27 @@ __global__ void __launch_bounds__(kStThreads, 2) thin_bwd_kernel(const __grid_co
         // stage v and arg-max: one warp per output channel at a time, lanes along the 10 x 34 pooled pixels of the tile
         for (int co = warp; co < A.Cout; co += kStThreads / 32) {
             const size_t base = ((size_t)n * A.Cout + co) * pplane;
-            for (int e = lane; e < kThinPH * kThinPW; e += 32) {
+            // (all loads of a channel are issued before the first value is used: the loop is unrolled whole)
+            constexpr int kIt = (kThinPH * kThinPW + 31) / 32;
+            float dv[kIt], yv[kIt]; unsigned char av[kIt];
+#pragma unroll
+            for (int it = 0; it < kIt; ++it) {
+                const int e = lane + 32 * it;
                 const int ly = e / kThinPW, lx = e - ly * kThinPW;
                 const int py = py0 + ly - 1, px = px0 + lx - 1;
-                float v = 0.f; unsigned char a = 0;
-                if (py >= 0 && py < A.OH && px >= 0 && px < A.OW) {
+                dv[it] = 0.f; yv[it] = 0.f; av[it] = 0;
+                if (e < kThinPH * kThinPW && py >= 0 && py < A.OH && px >= 0 && px < A.OW) {
                     const size_t gi = base + (size_t)py * A.OW + px;
-                    v = __ldg(A.dyp + gi) * (__ldg(A.yp + gi) > 0.f ? 1.f : A.slope);
-                    a = A.arg[gi];
+                    dv[it] = __ldg(A.dyp + gi); yv[it] = __ldg(A.yp + gi); av[it] = __ldg(A.arg + gi);
                 }
-                sv[e * kThinVs + co] = v;
-                sa[e * kThinAs + co] = a;
+            }
+#pragma unroll
+            for (int it = 0; it < kIt; ++it) {
+                const int e = lane + 32 * it;
+                if (e < kThinPH * kThinPW) {
+                    sv[e * kThinVs + co] = dv[it] * (yv[it] > 0.f ? 1.f : A.slope);
+                    sa[e * kThinAs + co] = av[it];
+                }
             }
         }
         // stage the input patch
