@@ -372,6 +372,10 @@ SAFE = {
     "yolo8-small": (FWD["yolo8-small"], None),
     "yolo8-two-groups": (FWD["yolo8-two-groups"], None),
     "yolo16-small": (FWD["yolo16-small"], None),
+    # shapes that leave the banded kernels ragged everywhere: 3 and 2 column chunks (280 and 140 columns), channel
+    # counts that fill neither a 128-channel slice nor a chunk of input planes (200, 136, 48), a last band of a few rows
+    "ragged": (W("r", (conv(3, 24, 3), pool(), conv(24, 200, 3), conv(200, 136, 1), conv(136, 48, 3), pool()), 2, 3, 36, 280,
+                 (2, 2), ((1, 6),)), None),
     "C1": (synth.workload("C1"), None),                 # benchmark launch configurations, full batch
     "C2": (synth.workload("C2"), None),
     "C3": (synth.workload("C3"), (0, 15)),              # full batch on the GPU, loss delta on two images
