@@ -520,13 +520,13 @@ bool tc_filter_grad(ftp_plan* p, const GroupPlan& g, int gi, const TcGroupArgs& 
         return launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, dz_below, nullptr, t.k, op.cout16, cin16, op.cin,
                               op.in_H, op.in_W, false, 1.0f, a.error, st, &pv);
     }
-    // first layer: the delta of the window-unrolled input (over the unrolled input itself, which nobody reads any more),
-    // folded back into the caller's fp32 map
-    if (!launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, xin, nullptr, 1, op.cout16, cin16, g.col_cin, op.in_H, op.in_W, false, 1.0f,
+    // first layer: the delta of the window-unrolled input (in the dz area that is not in use, sized for it; the unrolled
+    // input stays as the forward pass left it), folded back into the caller's fp32 map
+    if (!launch_tc_conv(p, g.cd, 8, gi, dz, wb, nullptr, dz_below, nullptr, 1, op.cout16, cin16, g.col_cin, op.in_H, op.in_W, false, 1.0f,
                         a.error, st))
         return false;
     { Timed tm(p, st, 10, gi);
-      launch_fold_windows(static_cast<const __nv_bfloat16*>(xin), dx, p->N, op.cin, op.in_H, op.in_W, st); }
+      launch_fold_windows(reinterpret_cast<const __nv_bfloat16*>(dz_below), dx, p->N, op.cin, op.in_H, op.in_W, st); }
     return launched_ok();
 }
 

@@ -1119,6 +1119,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         if (g.st.on && !g.st.thin)
             dz[0] = dz[1] = std::max(dz[0], (size_t)N * g.fwd_ops[0].cout * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W * 4);
         if (g.tfg.on) dz[gi & 1] = std::max(dz[gi & 1], (size_t)N * g.fwd_ops[0].cout16 * g.fwd_ops[0].in_H * g.fwd_ops[0].in_W * 2);
+        if (gi == 0 && g.col_cin16) dz[1] = std::max(dz[1], (size_t)N * g.col_cin16 * H * W * 2);   // delta of the unrolled input
     }
     ws.scratch_off = take(scratch * 4);
     if (!p.groups.empty() && p.groups[0].col_cin16) ws.col_off = take((size_t)N * p.groups[0].col_cin16 * H * W * 2);

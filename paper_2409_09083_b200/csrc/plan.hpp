@@ -189,7 +189,7 @@ struct Workspace {                 // byte offsets, all 256-aligned
     std::vector<size_t> dmap_off;  // delta maps at group inputs of groups 1.. (index = group), and slot for dY
     size_t dy_off = 0;             // loss delta at the last map (ftp_step with target)
     size_t scratch_off = 0;
-    size_t col_off = 0;                // first layer of the bf16 path: the window-unrolled network input (bf16 planes), later its delta
+    size_t col_off = 0;                // first layer of the bf16 path: the window-unrolled network input (bf16 planes)
     size_t dz_off = 0, dz_bytes = 0;   // one-conv groups: two areas (taken in turn, the second dz_bytes behind the first) for the
                                        // delta in front of the activation at the conv's resolution
     size_t wf_off = 0, wb_off = 0; // packed filters

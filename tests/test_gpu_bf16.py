@@ -79,6 +79,32 @@ def backward_bf16(wl, x, params, dy, want_dx=True, **opts):
 DEEP = {"yolo8-small", "yolo8-two-groups", "yolo16-small"}
 
 
+def test_backward_can_be_repeated_after_one_forward():
+    """ftp_backward leaves what the forward pass saved untouched: a second call (other delta) after the same forward
+    pass gives what it gives after a forward pass of its own, bit for bit, on both routes."""
+    wl = FWD["yolo8-small"]
+    x, params, target = synth.draw(wl, bias_std=0.3)
+    x, params = bf16_grid(x), bf16_grid(params)
+    c, h, w = synth.map_shapes(wl.layers, wl.C, wl.H, wl.W)[-1]
+    rng = np.random.default_rng(5)
+    dy1, dy2 = (rng.standard_normal((wl.N, c, h, w)).astype(np.float32) for _ in range(2))
+    for st in (0, -1):
+        plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, precision=BF16, stationary=st)
+        ws = plan.new_workspace()
+        xd, pd = torch.from_numpy(x).cuda(), torch.from_numpy(params).cuda()
+        y = torch.empty((wl.N, c, h, w), dtype=torch.float32, device="cuda")
+        out = []
+        for fresh_forward, dy in ((True, dy1), (False, dy2), (True, dy2)):
+            if fresh_forward:
+                ftp.ftp_forward(plan, xd, pd, y, ws)
+            dx, dp_ = torch.empty_like(xd), torch.empty_like(pd)
+            ftp.ftp_backward(plan, xd, torch.from_numpy(dy).cuda(), pd, dx, dp_, ws)
+            out.append((dx.cpu().numpy(), dp_.cpu().numpy()))
+        plan.check(ws)
+        assert np.array_equal(out[1][0], out[2][0]) and np.array_equal(out[1][1], out[2][1]), st
+        assert not np.array_equal(out[0][1], out[1][1])
+
+
 def l2_err(a, o):
     a, o = np.asarray(a, dtype=np.float64), np.asarray(o, dtype=np.float64)
     return float(np.linalg.norm(a - o) / max(np.linalg.norm(o), 1e-300))
