@@ -948,19 +948,26 @@ __global__ void pack_filters_tc_kernel(const __grid_constant__ TcPackArgs A, con
         const int nch_f = (L.cin16 / 8 + L.kpc_f - 1) / L.kpc_f, nch_d = (L.cout16 / 8 + L.kpc_d - 1) / L.kpc_d;
         const long long per_f = (long long)((L.cout16 + L.ns_f - 1) / L.ns_f) * nch_f * KK * L.kpc_f * L.ns_f * 8;
         const long long per_d = (long long)((L.cin16 + L.ns_d - 1) / L.ns_d) * nch_d * KK * L.kpc_d * L.ns_d * 8;
-        for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < per_f + per_d; e += (long long)gridDim.x * blockDim.x) {
-            const bool fwd = e < per_f;
+        // one thread per 16-byte entry (8 contraction channels of one row): the position is worked out once per entry
+        const long long ent_f = per_f / 8, ent_d = per_d / 8;
+        for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < ent_f + ent_d; e += (long long)gridDim.x * blockDim.x) {
+            const bool fwd = e < ent_f;
             const int ns = fwd ? L.ns_f : L.ns_d, kpc = fwd ? L.kpc_f : L.kpc_d, nch = fwd ? nch_f : nch_d;
-            long long t = fwd ? e : e - per_f;
-            const int c8 = (int)(t % 8); t /= 8;
+            long long t = fwd ? e : e - ent_f;
             const int r = (int)(t % ns); t /= ns;
             const int j = (int)(t % kpc); t /= kpc;
             const int tap = (int)(t % KK); t /= KK;
             const int c = (int)(t % nch); const int sl = (int)(t / nch);
-            const int row = sl * ns + r, kch = (c * kpc + j) * 8 + c8;            // output row of the GEMM, contraction channel
-            const int co = fwd ? row : kch, ci = fwd ? kch : row;
-            const float v = (co < L.cout && ci < L.cin) ? params[L.p_off + ((long long)co * L.cin + ci) * KK + (fwd ? tap : KK - 1 - tap)] : 0.f;
-            if (fwd) wf[L.w_off + e] = __float2bfloat16(v); else wb[L.w_off + (e - per_f)] = __float2bfloat16(v);
+            const int row = sl * ns + r, k0 = (c * kpc + j) * 8;                  // output row of the GEMM, first contraction channel
+            const int ptap = fwd ? tap : KK - 1 - tap;
+            float v[8];
+#pragma unroll
+            for (int c8 = 0; c8 < 8; ++c8) {
+                const int co = fwd ? row : k0 + c8, ci = fwd ? k0 + c8 : row;
+                v[c8] = (co < L.cout && ci < L.cin) ? __ldg(params + L.p_off + ((long long)co * L.cin + ci) * KK + ptap) : 0.f;
+            }
+            uint4* dst = reinterpret_cast<uint4*>(fwd ? wf + L.w_off : wb + L.w_off) + (fwd ? e : e - ent_f);
+            *dst = tcd::pack8(v);
         }
         return;
     }
