@@ -1,6 +1,8 @@
-// bf16 path, one-conv groups: the filter gradient by a weight-stationary tensor-core kernel.
+// bf16 path, executed groups of one conv layer (with its pool): the filter gradient by a weight-stationary
+// tensor-core kernel, the forward pass and the input delta by a banded tensor-core convolution (further down),
+// and their helpers (dz planes, window unroll / fold for the first layer).
 //
-// In the fused tile-stack kernel every sub-tile adds its whole partial filter gradient (K*K*cout*cin fp32) to
+// Filter gradient.  In the fused tile-stack kernel every sub-tile adds its whole partial filter gradient (K*K*cout*cin fp32) to
 // the block's partial set, because tensor memory cannot keep the accumulators of a wide layer across sub-tiles.
 // For layers with hundreds of channels that flush costs several times the MMAs.  Here the roles are turned
 // round: a block owns a slice of the FILTER GRADIENT (64 or 128 output channels x up to 48 input channels x all
@@ -9,10 +11,11 @@
 // once.  The pixels are dealt out in `shares`; a share is one partial gradient set of Section 4.1, summed by
 // the same cross-tile reduction as the sets of the fused kernels.
 //
-// A band is R rows of one image at the conv's resolution.  The delta in front of the activation (dz, bf16
-// planes, written by delta_act_planes_kernel) and the layer's saved input map arrive by TMA tensor copies
-// into tiles of the same pitch Wp = W + K - 1: dz at columns 0 .. W-1 with zeros behind them (beyond the
-// tensor's edge), the input shifted by the padding.  With equal pitches one run of 16 consecutive tile entries
+// A band is R rows x Cw columns (Cw = W, or a column chunk of at most 126 columns of a wider map) of one image at
+// the conv's resolution.  The delta in front of the activation (dz, bf16 planes, written by the input-delta
+// kernel of the layer above or by delta_act_planes_kernel) and the layer's saved input map arrive by TMA tensor
+// copies into tiles of the same pitch Wp = Cw + K - 1: dz at columns 0 .. Cw-1 with zeros behind them (beyond
+// the edge of the chunk's tensor map), the input shifted by the padding.  With equal pitches one run of 16 consecutive tile entries
 // is a K step of both operands (MN-major, 8 pixels x 8 channels per core matrix), and window position (ky, kx)
 // only moves the start of the input operand by ky * Wp + kx entries.  Two stages: the copies of the next band
 // run behind the MMAs of the current one.
