@@ -105,11 +105,20 @@ __global__ void unroll_windows_kernel(const float* __restrict__ x, uint4* __rest
         const int px = (int)(e % W); size_t t = e / W;
         const int py = (int)(t % H); const int n = (int)(t / H);
         float v[planes * 8];
+        const float* ctr = x + (size_t)n * C * HW + (size_t)py * W + px;       // this pixel in channel 0
+        if (py > 0 && py < H - 1 && px > 0 && px < W - 1) {                    // the whole window lies inside the map
 #pragma unroll
-        for (int j = 0; j < planes * 8; ++j) {
-            const int ci = j / 9, tap = j - ci * 9, ky = tap / 3, kx = tap - ky * 3;
-            const int yy = py + ky - 1, xx = px + kx - 1;
-            v[j] = (ci < C && yy >= 0 && yy < H && xx >= 0 && xx < W) ? __ldg(x + ((size_t)n * C + ci) * HW + (size_t)yy * W + xx) : 0.f;
+            for (int j = 0; j < planes * 8; ++j) {
+                const int ci = j / 9, tap = j - ci * 9, ky = tap / 3, kx = tap - ky * 3;
+                v[j] = ci < C ? __ldg(ctr + (size_t)ci * HW + (ky - 1) * W + (kx - 1)) : 0.f;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < planes * 8; ++j) {
+                const int ci = j / 9, tap = j - ci * 9, ky = tap / 3, kx = tap - ky * 3;
+                const int yy = py + ky - 1, xx = px + kx - 1;
+                v[j] = (ci < C && yy >= 0 && yy < H && xx >= 0 && xx < W) ? __ldg(ctr + (size_t)ci * HW + (ky - 1) * W + (kx - 1)) : 0.f;
+            }
         }
 #pragma unroll
         for (int pl = 0; pl < planes; ++pl) col[((size_t)n * planes + pl) * HW + (size_t)py * W + px] = tcd::pack8(v + 8 * pl);
