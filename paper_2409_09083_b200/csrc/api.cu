@@ -44,7 +44,7 @@ int ensure_device(ftp_plan* p)
         cudaFuncSetAttribute(bwd_group_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(bwd_group_tc_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(filter_grad_tc_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcFgSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(conv_tc_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcFgSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(conv_tc_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcConvSmemBudget) != cudaSuccess ||
         !st_prepare_device())
         return FTP_ERR_CUDA;
     if (!p->grad_stream) {

@@ -676,9 +676,19 @@ TcConvPlan plan_tc_conv(int N, int H, int W, int K, int cin16, int cout16, bool 
     const size_t entries = std::max<size_t>((size_t)(c.R + K - 1) * c.Wp, (size_t)c.nblk * 128 + (size_t)(K - 1) * c.Wp + K);
     c.x_plane = (int)align_up(entries * 16, 128);
     c.stage_bytes = c.kpc * c.x_plane + (K == 1 ? c.kpc : 2 * K * K) * c.Ns * 16;
-    const size_t staging = pool ? kTcPoolStageBytes : 0;                                     // the band as stored, 16 channels or more at a time
-    c.stages = (int)std::min<size_t>(4, ((size_t)kTcFgSmemBudget - kTcFgHeader - staging) / c.stage_bytes);
-    c.pool_planes = pool ? (int)(kTcPoolStageBytes / ((size_t)c.nblk * 128 * 16)) / 2 * 2 : 0;
+    // fused pool: the band as stored goes through a staging area, all channels of the slice at once where that leaves
+    // three stages (two for short rings), else 16 channels or more at a time
+    const size_t room = (size_t)kTcConvSmemBudget - kTcFgHeader;
+    const size_t plane_pair = (size_t)c.nblk * 128 * 16 * 2, whole = (size_t)(c.Ns / 16) * plane_pair;
+    size_t staging = pool ? kTcPoolStageBytes : 0;
+    c.stages = (int)std::min<size_t>(4, (room - staging) / c.stage_bytes);
+    if (pool) {
+        const int keep = std::min(c.stages, 3);
+        if (room >= (size_t)keep * c.stage_bytes + whole) { c.stages = std::min<int>(c.stages, (int)((room - whole) / c.stage_bytes)); staging = whole; }
+        else staging = std::max<size_t>(staging, (room - (size_t)c.stages * c.stage_bytes) / plane_pair * plane_pair);
+        c.pool_planes = (int)(staging / plane_pair) * 2;
+        c.pool_stage_bytes = (int)staging;
+    }
     if (c.stages < 2 || (pool && c.pool_planes < 2)) return c;
     c.smem_bytes = kTcFgHeader + c.stages * c.stage_bytes + (int)staging;
     const long long items = (long long)N * c.bands_img * c.slices;

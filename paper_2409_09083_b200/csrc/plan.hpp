@@ -152,9 +152,11 @@ struct TcConvPlan {
     int items = 0;                          // N * bands_img * slices
     int blocks = 0;                         // persistent blocks: min(items, SMs)
     int pool_planes = 0;                    // fused pool: 8-channel planes the staging area holds
+    int pool_stage_bytes = 0;               //             and its size
     int nbuf = 1;                           // accumulator buffers (2 for slices of at most 64 channels)
 };
-constexpr int kTcPoolStageBytes = 32 * 1024;  // staging area of the fused pool in the banded convolution
+constexpr int kTcPoolStageBytes = 32 * 1024;  // least staging area of the fused pool in the banded convolution (more where it fits)
+constexpr int kTcConvSmemBudget = 224 * 1024; // banded convolution: header + stages + pool staging
 constexpr int kTcMaxColChunks = 8;            // a band spans at most 126 columns (a TMA box row of 128 pixels with the halo): wider maps are cut into chunks
 constexpr int kTcFgHeader = 1024;             // barriers, tensor-memory slot, a core matrix of ones
 constexpr int kTcFgSmemBudget = 200 * 1024;   // header + two stages
