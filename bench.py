@@ -77,7 +77,8 @@ def parse():
     ap.add_argument("--cost-model", type=int, default=0, choices=[-1, 0, 1],
                     help="planner's time model for cutting the requested groups: 0 planner default, 1 on, -1 off (fixed rule)")
     ap.add_argument("--stationary", type=int, default=0, choices=[-1, 0, 1],
-                    help="fp32 path: weight-stationary kernels for one-conv groups: 0 planner default, -1 never (fused stacks only)")
+                    help="one-conv groups on their own kernels (fp32: weight-stationary; bf16: banded tensor-core kernels): 0 planner default, "
+                         "-1 never (fused stacks only)")
     ap.add_argument("--strict-groups", action="store_true", help="execute the requested grouping profile as it is (no cuts)")
     ap.add_argument("--no-bf16", action="store_true", help="skip the second measurement on the bf16 tensor-core path")
     return ap.parse_args()
@@ -223,6 +224,10 @@ def run_ours(args):
                 into["bf16_tensor_core_path"] = {k: second[k] for k in ("value", "unit", "ms_per_step", "dtype", "roofline",
                                                                         "breakdown_ms_per_step", "gpu_launches", "e2e", "loss")}
                 into["bf16_tensor_core_path"]["executed_groups"] = second["config"]["executed_groups"]
+                try:        # the same step as fused sub-tile stacks only (what the one-conv kernels replace)
+                    into["bf16_tensor_core_path"]["fused_stacks_only"] = measure(ctx, name, "bf16", light=True, stationary=-1)
+                except Exception as e:                        # noqa: BLE001
+                    into["bf16_tensor_core_path"]["fused_stacks_only"] = {"unavailable": str(e)}
         with_bf16(head, line)
         if args.workload is None and world == 1:
             line["workloads"] = {}
