@@ -346,7 +346,7 @@ bool stationary_forward(ftp_plan* p, const GroupPlan& g, int gi, const float* x,
     a.N = p->N; a.Cin = op.cin; a.Cout = op.cout; a.CoutPad = op.cout_pad; a.H = op.in_H; a.W = op.in_W;
     a.slope = op.slope; a.act = 1; a.pool = g.st.pool;
     { Timed t(p, st, 1, gi);
-      st_launch_conv_rows(a, op.k, g.st.fwd_co_tile, g.st.fwd_blocks, st); }
+      st_launch_conv_rows(a, op.k, g.st.fwd_co_tile, g.st.fwd_threads, g.st.fwd_blocks, st); }
     return launched_ok();
 }
 
@@ -412,7 +412,7 @@ bool stationary_backward(ftp_plan* p, const GroupPlan& g, int gi, const float* x
         a.N = p->N; a.Cin = op.cout; a.Cout = op.cin; a.CoutPad = op.cin_pad; a.H = H; a.W = W;
         a.slope = 0.f; a.act = 0; a.pool = 0;
         { Timed t(p, st, 8, gi);
-          st_launch_conv_rows(a, op.k, g.st.dx_co_tile, g.st.dx_blocks, st); }
+          st_launch_conv_rows(a, op.k, g.st.dx_co_tile, g.st.dx_threads, g.st.dx_blocks, st); }
         if (!launched_ok()) return false;
     }
     return true;
@@ -812,10 +812,10 @@ int ftp_plan_subtiles(const ftp_plan* plan, int pass, int group, int* rows, int*
     const GroupPlan& gp = plan->groups[group];
     if (gp.st.on) {         // weight-stationary group: row-pair tiles of the whole batch x column tiles, 256-thread blocks
         const OpDesc& op = gp.fwd_ops[0];
-        const int per = pass ? kFgRowPairs : st_row_pairs(gp.st.fwd_co_tile);
+        const int per = pass ? kFgRowPairs : st_row_pairs(gp.st.fwd_co_tile, gp.st.fwd_threads);
         if (rows) *rows = (plan->N * ((op.in_H + 1) / 2) + per - 1) / per;
         if (cols) *cols = (op.in_W + kStCols - 1) / kStCols;
-        if (smem_bytes) *smem_bytes = pass ? st_filter_grad_smem_bytes(op.k) : st_conv_smem_bytes(op.k, gp.st.fwd_co_tile);
+        if (smem_bytes) *smem_bytes = pass ? st_filter_grad_smem_bytes(op.k) : st_conv_smem_bytes(op.k, gp.st.fwd_co_tile, gp.st.fwd_threads);
         if (blocks) *blocks = pass ? gp.st.fg_blocks : gp.st.fwd_blocks;
         return FTP_OK;
     }

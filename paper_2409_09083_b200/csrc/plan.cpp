@@ -584,10 +584,14 @@ void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     const int x_tiles = (W + kStCols - 1) / kStCols;
     // blocks of 64 output channels x 16 row pairs, or of 32 x 32 where that wastes fewer channels or rows, i.e. takes
     // fewer rounds of blocks (two blocks run per SM)
-    auto conv_blocks = [&](int cout, int ct) {
-        const int rpt = st_row_pairs(ct);
+    auto conv_blocks = [&](int cout, int ct, int threads = kStThreads) {
+        const int rpt = st_row_pairs(ct, threads);
         return (rp_total + rpt - 1) / rpt * x_tiles * ((cout + ct - 1) / ct);
     };
+    // Blocks of 128 threads (half the row pairs, four per SM) where whole blocks fill less than a round and a half of
+    // the 2 x 148 slots: the SMs that get one block more than the others then wait for half a block, not a whole one
+    // (measured on C1, batch 4: 15-20 % on such launches; with more rounds the shorter stages cost more than they save).
+    auto pick_threads = [&](long long blocks256) { return blocks256 <= 3LL * kSmCount ? 128 : kStThreads; };
     auto pick_tile = [&](int cout) {
         if (cout <= 32) return 32;
         const long long slots = 2LL * kSmCount;
@@ -597,7 +601,9 @@ void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
         return r32 < r64 ? 32 : 64;
     };
     const int fwd_ct = pick_tile(op.cout), dx_ct = pick_tile(op.cin);
-    const long long fwd_blocks = conv_blocks(op.cout, fwd_ct), dx_blocks = conv_blocks(op.cin, dx_ct);
+    const int fwd_thr = o.stationary == 1 ? kStThreads : pick_threads(conv_blocks(op.cout, fwd_ct));
+    const int dx_thr = o.stationary == 1 ? kStThreads : pick_threads(conv_blocks(op.cin, dx_ct));
+    const long long fwd_blocks = conv_blocks(op.cout, fwd_ct, fwd_thr), dx_blocks = conv_blocks(op.cin, dx_ct, dx_thr);
     // filter gradient: 3 x 3 in stages of 4 row pairs x 8 columns and 64 x 32 channel slices; 1 x 1 as a contraction over
     // stages of 32 flat pixels of an image and 64 x 128 channel slices
     const long long stages = op.k == 1 ? (long long)p.N * ((H * W + kFg1Px - 1) / kFg1Px)
@@ -608,6 +614,7 @@ void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     g.st.on = 1; g.st.k = op.k; g.st.pool = op.kind == kOpConvPool ? 1 : 0;
     g.st.fwd_blocks = (int)fwd_blocks; g.st.dx_blocks = (int)dx_blocks;
     g.st.fwd_co_tile = fwd_ct; g.st.dx_co_tile = dx_ct;
+    g.st.fwd_threads = fwd_thr; g.st.dx_threads = dx_thr;
     g.st.fg_stages = (int)stages;
     // one round of the blocks that run at once (2 per SM; 1 x 1: 3): the input-delta convolution on the other stream fills
     // what a round leaves idle, and every share costs a partial set that the reduction has to read; at least 4 stages a share

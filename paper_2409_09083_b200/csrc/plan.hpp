@@ -42,7 +42,7 @@ constexpr int kStThreads = 256;
 // convolution: 64 output channels x 16 row pairs per block (8 channels x 2 rows x 4 columns per thread), or 32 x 32 for layers
 // with at most 32 output channels
 // with at most 32 output channels or with so few blocks that the last round of 64-channel blocks would leave SMs idle
-constexpr int st_row_pairs(int co_tile) { return 1024 / co_tile; }
+constexpr int st_row_pairs(int co_tile, int threads = kStThreads) { return threads * 4 / co_tile; }
 constexpr int kStCols    = 8;             // columns per block, both kernels
 constexpr int kFgCo = 64, kFgCi = 32;     // filter gradient: (output, input) channel slice of a block (8 x 1 per thread)
 constexpr int kFgRowPairs = 4;            // filter gradient: row pairs per pixel stage
@@ -121,6 +121,7 @@ struct StatPlan {
     int k = 0, pool = 0;
     int fwd_blocks = 0, dx_blocks = 0;      // convolution launches: (row-pair tiles) x (column tiles) x (channel slices)
     int fwd_co_tile = 64, dx_co_tile = 64;  // output channels per block of the two convolutions (64 or 32)
+    int fwd_threads = kStThreads, dx_threads = kStThreads;   // threads per block (256, or 128 where whole blocks would leave SMs idle)
     int fg_stages = 0, fg_splits = 0;       // filter gradient: pixel stages over the batch, and the shares they are dealt out in
     int fg_blocks = 0;                      // (64 x 32 channel slices) x shares; a share is one partial gradient set
 };

@@ -10,27 +10,28 @@ namespace ftp {
 
 namespace {
 
-template <int K, int CO, int VEC>
+template <int K, int CO, int VEC, int T>
 void launch_conv(const ConvRowsArgs& a, int blocks, cudaStream_t st)
 {
-    conv_rows_kernel<K, CO, VEC><<<blocks, kStThreads, StGeom<K, CO>::smem_bytes, st>>>(a);
+    conv_rows_kernel<K, CO, VEC, T><<<blocks, T, StGeom<K, CO, T>::smem_bytes, st>>>(a);
 }
 
-template <int K, int CO>
+template <int K, int CO, int T>
 void launch_conv_vec(const ConvRowsArgs& a, int blocks, cudaStream_t st)
 {
-    if ((a.W & 3) == 0) launch_conv<K, CO, 4>(a, blocks, st);
-    else if ((a.W & 1) == 0) launch_conv<K, CO, 2>(a, blocks, st);
-    else launch_conv<K, CO, 1>(a, blocks, st);
+    if ((a.W & 3) == 0) launch_conv<K, CO, 4, T>(a, blocks, st);
+    else if ((a.W & 1) == 0) launch_conv<K, CO, 2, T>(a, blocks, st);
+    else launch_conv<K, CO, 1, T>(a, blocks, st);
 }
 
-template <int K, int CO>
-bool conv_attr()
+template <int K, int CO, int T>
+bool conv_attr_t()
 {
-    return cudaFuncSetAttribute(conv_rows_kernel<K, CO, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<K, CO>::smem_bytes) == cudaSuccess &&
-           cudaFuncSetAttribute(conv_rows_kernel<K, CO, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<K, CO>::smem_bytes) == cudaSuccess &&
-           cudaFuncSetAttribute(conv_rows_kernel<K, CO, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<K, CO>::smem_bytes) == cudaSuccess;
+    return cudaFuncSetAttribute(conv_rows_kernel<K, CO, 4, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<K, CO, T>::smem_bytes) == cudaSuccess &&
+           cudaFuncSetAttribute(conv_rows_kernel<K, CO, 2, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<K, CO, T>::smem_bytes) == cudaSuccess &&
+           cudaFuncSetAttribute(conv_rows_kernel<K, CO, 1, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, StGeom<K, CO, T>::smem_bytes) == cudaSuccess;
 }
+template <int K, int CO> bool conv_attr() { return conv_attr_t<K, CO, 256>() && conv_attr_t<K, CO, 128>(); }
 
 }  // namespace
 
@@ -45,22 +46,32 @@ bool st_prepare_device()
            cudaFuncSetAttribute(filter_grad_rows_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, FgGeom<3>::smem_bytes) == cudaSuccess;
 }
 
-size_t st_conv_smem_bytes(int k, int co_tile)
+size_t st_conv_smem_bytes(int k, int co_tile, int threads)
 {
+    if (threads == 128)
+        return k == 3 ? (co_tile == 64 ? StGeom<3, 64, 128>::smem_bytes : StGeom<3, 32, 128>::smem_bytes)
+                      : (co_tile == 64 ? StGeom<1, 64, 128>::smem_bytes : StGeom<1, 32, 128>::smem_bytes);
     return k == 3 ? (co_tile == 64 ? StGeom<3, 64>::smem_bytes : StGeom<3, 32>::smem_bytes)
                   : (co_tile == 64 ? StGeom<1, 64>::smem_bytes : StGeom<1, 32>::smem_bytes);
 }
 
 size_t st_filter_grad_smem_bytes(int k) { return k == 3 ? FgGeom<3>::smem_bytes : kF1SmemBytes; }
 
-void st_launch_conv_rows(ConvRowsArgs& a, int k, int co_tile, int blocks, void* stream)
+template <int T>
+void launch_conv_t(const ConvRowsArgs& a, int k, int co_tile, int blocks, cudaStream_t st)
+{
+    if (k == 3 && co_tile == 64) launch_conv_vec<3, 64, T>(a, blocks, st);
+    else if (k == 3) launch_conv_vec<3, 32, T>(a, blocks, st);
+    else if (co_tile == 64) launch_conv_vec<1, 64, T>(a, blocks, st);
+    else launch_conv_vec<1, 32, T>(a, blocks, st);
+}
+
+void st_launch_conv_rows(ConvRowsArgs& a, int k, int co_tile, int threads, int blocks, void* stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     a.rp_img = (a.H + 1) / 2; a.x_tiles = (a.W + kStCols - 1) / kStCols; a.co_tiles = (a.Cout + co_tile - 1) / co_tile;
-    if (k == 3 && co_tile == 64) launch_conv_vec<3, 64>(a, blocks, st);
-    else if (k == 3) launch_conv_vec<3, 32>(a, blocks, st);
-    else if (co_tile == 64) launch_conv_vec<1, 64>(a, blocks, st);
-    else launch_conv_vec<1, 32>(a, blocks, st);
+    if (threads == 128) launch_conv_t<128>(a, k, co_tile, blocks, st);
+    else launch_conv_t<256>(a, k, co_tile, blocks, st);
 }
 
 void st_launch_filter_grad_rows(FilterGradRowsArgs& a, int k, int blocks, void* stream)

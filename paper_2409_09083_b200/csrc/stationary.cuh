@@ -34,14 +34,16 @@ namespace ftp {
 // 3 and the right halo the first, otherwise unused, slot of the next row.  The stride between row
 // pairs is 8 or 24 modulo 32, so that the eight lanes of a quarter warp (two column quads of four row
 // pairs) read 4-wide without bank conflicts.
-template <int K, int CO> struct StGeom {
+// T = threads of a block: 256 (two blocks per SM), or 128 (four per SM, half the row pairs and half the channels per
+// stage each) for launches with so few blocks that whole blocks would leave SMs idle in the last round.
+template <int K, int CO, int T = kStThreads> struct StGeom {
     static constexpr int P = K / 2, RR = K + 1;
-    static constexpr int npg = kStThreads * 8 / CO;                  // pixel groups (2 rows x 4 columns) per block: 32 or 64
-    static constexpr int row_pairs = npg / 2;                        // row pairs per block: 16 or 32
+    static constexpr int npg = T * 8 / CO;                           // pixel groups (2 rows x 4 columns) per block: 32 or 64 (T = 256)
+    static constexpr int row_pairs = npg / 2;                        // row pairs per block: 16 or 32 (T = 256)
     static constexpr int pitch = kStCols + (K > 1 ? 4 : 0);
     static constexpr int rp_stride = K == 3 ? 56 : 24;
     static constexpr int ci_stride = row_pairs * rp_stride;
-    static constexpr int ci_chunk = (K == 3 ? 8 : 32) * CO / 64;     // input channels per stage
+    static constexpr int ci_chunk = (K == 3 ? 8 : 32) * CO / 64 * T / kStThreads;   // input channels per stage
     static constexpr int w_stage = ci_chunk * K * K * CO;            // floats
     static constexpr int in_stage = ci_chunk * ci_stride;
     static constexpr int smem_bytes = 2 * (w_stage + in_stage) * 4;
@@ -72,10 +74,10 @@ template <int N> __device__ __forceinline__ void st_wait() { asm volatile("cp.as
 // K = 1 or 3 (stride 1, padding K / 2); CO = 64 or 32 output channels per block (32 for layers with at most 32,
 // which then take twice the row pairs).  Thread tile: 8 output channels x (2 rows x 4 columns).
 // VEC = floats per copy of the input columns: 4 where the map's rows are 16-byte aligned (width a multiple of 4), else 2 or 1.
-template <int K, int CO, int VEC>
-__global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_constant__ ConvRowsArgs A)
+template <int K, int CO, int VEC, int T = kStThreads>
+__global__ void __launch_bounds__(T, 512 / T) conv_rows_kernel(const __grid_constant__ ConvRowsArgs A)
 {
-    using G = StGeom<K, CO>;
+    using G = StGeom<K, CO, T>;
     extern __shared__ __align__(16) float st_smem[];
     constexpr int KK = K * K, P = G::P, RR = G::RR;
     const int tid = threadIdx.x;
@@ -94,11 +96,11 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
     // block is (row pair, row, piece of the row).
     constexpr int vec = VEC;
     constexpr int per_row = kStCols / vec + 2 * P, nitems = G::row_pairs * RR * per_row;
-    constexpr int max_items = (nitems + kStThreads - 1) / kStThreads;
+    constexpr int max_items = (nitems + T - 1) / T;
     int it_s[max_items]; long long it_g[max_items]; unsigned it_ok = 0, it_halo = 0;
 #pragma unroll
     for (int e = 0; e < max_items; ++e) {
-        const int idx = tid + e * kStThreads;
+        const int idx = tid + e * T;
         it_s[e] = -1; it_g[e] = 0;
         if (idx < nitems) {
             const int piece = idx % per_row, t = idx / per_row, r = t % RR, rl = t / RR;
@@ -123,7 +125,7 @@ __global__ void __launch_bounds__(kStThreads, 2) conv_rows_kernel(const __grid_c
         float* di = si + (chunk & 1) * G::in_stage;
         // filters: a row of CO floats per (channel, tap)
         constexpr int q = CO / 4;
-        for (int i = tid; i < nci * KK * q; i += kStThreads) {
+        for (int i = tid; i < nci * KK * q; i += T) {
             const int row = i / q, j = i - row * q;
             const int co = co0 + 4 * j;
             st_cp_async16(dw + row * CO + 4 * j, A.w + ((size_t)ci0 * KK + row) * A.CoutPad + min(co, A.CoutPad - 4), co < A.CoutPad);

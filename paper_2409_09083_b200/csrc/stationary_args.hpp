@@ -48,12 +48,12 @@ struct ThinBwdArgs {
 
 // Launchers (stationary.cu); `stream` is a cudaStream_t.  They fill in the tiling fields of the arguments.
 bool st_prepare_device();                                                   // opt-in shared-memory sizes; once per device
-void st_launch_conv_rows(ConvRowsArgs& a, int k, int co_tile, int blocks, void* stream);
+void st_launch_conv_rows(ConvRowsArgs& a, int k, int co_tile, int threads, int blocks, void* stream);   // threads: 256 or 128
 void st_launch_filter_grad_rows(FilterGradRowsArgs& a, int k, int blocks, void* stream);
 void st_launch_delta_act(const float* dy, const float* y, const unsigned char* arg, float* dz, size_t count, int pooled_width,
                          float slope, int pool, void* stream);
 void st_launch_thin_bwd(const ThinBwdArgs& a, int blocks, void* stream);
-size_t st_conv_smem_bytes(int k, int co_tile);
+size_t st_conv_smem_bytes(int k, int co_tile, int threads);
 size_t st_filter_grad_smem_bytes(int k);
 
 }  // namespace ftp
