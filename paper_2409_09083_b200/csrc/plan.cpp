@@ -590,8 +590,11 @@ void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     };
     // Blocks of 128 threads (half the row pairs, four per SM) where whole blocks fill less than a round and a half of
     // the 2 x 148 slots: the SMs that get one block more than the others then wait for half a block, not a whole one
-    // (measured on C1, batch 4: 15-20 % on such launches; with more rounds the shorter stages cost more than they save).
-    auto pick_threads = [&](long long blocks256) { return blocks256 <= 3LL * kSmCount ? 128 : kStThreads; };
+    // (measured on C1, batch 4: 10-18 % on such launches; with more rounds, or with a contraction over 512 channels x 9
+    // window positions, where C3's 38 x 38 input deltas lost 10 %, the shorter stages cost more than the finer split saves).
+    auto pick_threads = [&](long long blocks256, int depth) {
+        return blocks256 <= 3LL * kSmCount && depth <= 2304 ? 128 : kStThreads;
+    };
     auto pick_tile = [&](int cout) {
         if (cout <= 32) return 32;
         const long long slots = 2LL * kSmCount;
@@ -601,8 +604,8 @@ void plan_stationary(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
         return r32 < r64 ? 32 : 64;
     };
     const int fwd_ct = pick_tile(op.cout), dx_ct = pick_tile(op.cin);
-    const int fwd_thr = o.stationary == 1 ? kStThreads : pick_threads(conv_blocks(op.cout, fwd_ct));
-    const int dx_thr = o.stationary == 1 ? kStThreads : pick_threads(conv_blocks(op.cin, dx_ct));
+    const int fwd_thr = o.stationary == 1 ? kStThreads : pick_threads(conv_blocks(op.cout, fwd_ct), op.cin * op.k * op.k);
+    const int dx_thr = o.stationary == 1 ? kStThreads : pick_threads(conv_blocks(op.cin, dx_ct), op.cout * op.k * op.k);
     const long long fwd_blocks = conv_blocks(op.cout, fwd_ct, fwd_thr), dx_blocks = conv_blocks(op.cin, dx_ct, dx_thr);
     // filter gradient: 3 x 3 in stages of 4 row pairs x 8 columns and 64 x 32 channel slices; 1 x 1 as a contraction over
     // stages of 32 flat pixels of an image and 64 x 128 channel slices
