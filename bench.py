@@ -45,8 +45,8 @@ KERNEL = {("fwd_group", "fp32"): "fwd_group_kernel / conv_rows_kernel", ("bwd_gr
           ("filter_grad_rows", "bf16"): "filter_grad_tc_rows_kernel", ("delta_conv_rows", "bf16"): "conv_tc_rows_kernel (input delta)"}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised
 # under profiles/ (static: null for every kernel / workload without a capture of the current code)
-NCU_TRAFFIC = {("C3", "fp32", "fwd_group"): 129.3e6, ("C3", "fp32", "filter_grad_rows"): 245.0e6,
-               ("C3", "fp32", "delta_conv_rows"): 160.4e6, ("C3", "fp32", "bwd_group"): 952.8e6,
+NCU_TRAFFIC = {("C3", "fp32", "fwd_group"): 128.4e6, ("C3", "fp32", "filter_grad_rows"): 245.8e6,
+               ("C3", "fp32", "delta_conv_rows"): 159.3e6, ("C3", "fp32", "bwd_group"): 950.4e6,
                ("C3", "bf16", "fwd_group"): 84.8e6, ("C3", "bf16", "filter_grad_rows"): 153.2e6, ("C3", "bf16", "delta_conv_rows"): 202.2e6}
 
 
