@@ -290,3 +290,21 @@ def test_bf16_plans_run_conv_layers_as_groups_of_their_own():
     plan = ftp.ftp_plan(layers, 2, 3, 32, 32, (2, 2), ((1, 2),), precision=ftp.FTP_BF16_FP32ACC)
     modes = [plan.group_mode(i)[0] for i in range(len(plan.exec_groups()))]
     assert modes[0] == 0 and modes[-1] == 2, (plan.exec_groups(), modes)
+
+
+def test_small_launches_of_the_row_convolution_use_half_size_blocks():
+    """fp32 one-conv groups: a convolution launch of at most a round and a half of whole (256-thread, 16 row pairs)
+    blocks is cut into 128-thread blocks of 8 row pairs (C1, batch 4, layer 5: 4 x 52 row pairs -> 26 tiles instead of
+    13); larger launches and `stationary = 1` keep whole blocks."""
+    wl = synth.workload("C1")
+    plan = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups)
+    gi = plan.exec_groups().index((5, 5))
+    st = plan.subtiles(0, gi)
+    assert st["rows"] == 26 and st["cols"] == 13 and st["blocks"] == 26 * 13 * 2 and st["smem_bytes"] == 32768
+    whole = ftp.ftp_plan(wl.layers, wl.N, wl.C, wl.H, wl.W, wl.grid, wl.groups, stationary=1)
+    st = whole.subtiles(0, whole.exec_groups().index((5, 5)))
+    assert st["rows"] == 13 and st["blocks"] == 13 * 13 * 2
+    big = synth.workload("C3")
+    plan = ftp.ftp_plan(big.layers, big.N, big.C, big.H, big.W, big.grid, big.groups)
+    st = plan.subtiles(0, plan.exec_groups().index((5, 5)))
+    assert st["rows"] == (16 * 76 + 15) // 16
