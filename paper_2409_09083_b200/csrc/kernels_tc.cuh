@@ -80,10 +80,10 @@ struct Pipe {
     int* error;
 };
 
-__device__ __forceinline__ bool wait_or_fail(Pipe& p, unsigned long long* bar, uint32_t parity)
+__device__ __forceinline__ bool wait_or_fail(Pipe& p, unsigned long long* bar, uint32_t parity, unsigned sleep_ns = 0)
 {
     if (p.h->failed) return false;
-    if (mbar_wait(smem_u32(bar), parity)) return true;
+    if (mbar_wait(smem_u32(bar), parity, kWaitLimitCycles, sleep_ns)) return true;
     p.h->failed = 1;
     if (p.error) atomicExch(p.error, 1);
     return false;
@@ -202,7 +202,7 @@ __device__ __forceinline__ void conv_mma(Pipe& p, uint32_t a_base, int a_Wp, uin
         }
         p.stages_done += nstages;
         __syncwarp();
-        wait_or_fail(p, &p.h->done, p.passes_done & 1);
+        wait_or_fail(p, &p.h->done, p.passes_done & 1, 128);   // every thread waits here: asleep between polls
         p.passes_done++;
         fence_after_sync();
         const int q = warp & 3;
@@ -433,7 +433,7 @@ __device__ __forceinline__ void filter_grad_mma(Pipe& p, uint32_t dz_run /*addre
             mma_commit(smem_u32(&p.h->done));
         }
         __syncwarp();
-        wait_or_fail(p, &p.h->done, p.passes_done & 1);
+        wait_or_fail(p, &p.h->done, p.passes_done & 1, 128);   // every thread waits here: asleep between polls
         p.passes_done++;
         fence_after_sync();
         // flush: lane quarter q holds rows 32q.. (M = 128) or rows 16q..16q+15 in its first 16 lanes (M = 64)

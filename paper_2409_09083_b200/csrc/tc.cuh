@@ -131,12 +131,16 @@ __device__ __forceinline__ bool mbar_try(uint32_t mbar, uint32_t parity)
 // Waits for the phase with the given parity to complete, for at most `limit_cycles` SM clock cycles
 // (default: about 2 s) and 2^26 polls; false = gave up.  Every wait of the tile kernels goes through
 // here, so a missing arrival ends the kernel with an error word instead of hanging it.
+// `sleep_ns` > 0: the warp sleeps that long between two polls.  Warps that wait for a whole phase of the kernel (the
+// epilogue warps for the MMAs of an item) would otherwise poll in a tight loop and take issue slots from the one
+// thread per warp that feeds the tensor core (measured: an MMA every 100 cycles instead of every 40-64).
 constexpr long long kWaitLimitCycles = 4000000000ll;
-__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, long long limit_cycles = kWaitLimitCycles)
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, long long limit_cycles = kWaitLimitCycles, unsigned sleep_ns = 0)
 {
     if (mbar_try(mbar, parity)) return true;
     const long long t0 = clock64();
     for (int it = 0; it < (1 << 26); ++it) {
+        if (sleep_ns) __nanosleep(sleep_ns);
         if (mbar_try(mbar, parity)) return true;
         if (clock64() - t0 > limit_cycles) break;
     }

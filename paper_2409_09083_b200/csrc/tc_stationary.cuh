@@ -230,9 +230,9 @@ __global__ void __launch_bounds__(kTcFgThreads, 1) filter_grad_tc_rows_kernel(co
     fence_after_sync();
     const uint32_t tmem = H->tmem_base;
 
-    auto wait = [&](unsigned long long* bar, uint32_t parity) {
+    auto wait = [&](unsigned long long* bar, uint32_t parity, unsigned sleep_ns = 0) {
         if (H->failed) return false;
-        if (mbar_wait(smem_u32(bar), parity)) return true;
+        if (mbar_wait(smem_u32(bar), parity, kWaitLimitCycles, sleep_ns)) return true;
         H->failed = 1;
         atomicExch(A.error, 1);
         return false;
@@ -296,7 +296,7 @@ __global__ void __launch_bounds__(kTcFgThreads, 1) filter_grad_tc_rows_kernel(co
         mma_commit(smem_u32(&H->done));
     }
     __syncwarp();
-    const bool have = nb > 0 && wait(&H->done, 0);
+    const bool have = nb > 0 && wait(&H->done, 0, 256);        // (asleep between polls: the issuers share the schedulers)
     if (!have && nb > 0) mbar_wait(smem_u32(&H->done), 0, 200000000ll);   // gave up: the MMAs under way still end first
     fence_after_sync();
 
@@ -417,9 +417,9 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
     fence_after_sync();
     const uint32_t tmem = H->tmem_base;
 
-    auto wait = [&](unsigned long long* bar, uint32_t parity) {
+    auto wait = [&](unsigned long long* bar, uint32_t parity, unsigned sleep_ns = 0) {
         if (H->failed) return false;
-        if (mbar_wait(smem_u32(bar), parity)) return true;
+        if (mbar_wait(smem_u32(bar), parity, kWaitLimitCycles, sleep_ns)) return true;
         H->failed = 1;
         atomicExch(A.error, 1);
         return false;
@@ -496,16 +496,27 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
                     // (the thread that issues is the bottleneck of a narrow MMA: descriptors advance by adds only)
                     for (int b = iw; b < I.nblk; b += kTcIssuers) {
                         const uint32_t tcol = tmem + buf * 256u + (uint32_t)(b * A.Ns);
-                        uint32_t a_row = desc_lo(xaddr + (uint32_t)b * 2048u, (uint32_t)A.x_plane), b_t = b_lo0;
-                        bool acc = c > 0;
-                        for (int ky = 0; ky < K; ++ky, a_row += (uint32_t)A.Wp) {
-                            uint32_t a_t = a_row;
-                            for (int kx = 0; kx < K; ++kx, ++a_t, b_t += w_tap16) {
-                                uint32_t a_lo = a_t, b_lo = b_t;
-                                for (int ks = 0; ks < nks; ++ks) {
-                                    mma_bf16(tcol, desc64(a_hi, a_lo), desc64(b_hi, b_lo), idesc, acc);
-                                    acc = true; a_lo += xstep; b_lo += wstep;
-                                }
+                        const uint32_t a0 = desc_lo(xaddr + (uint32_t)b * 2048u, (uint32_t)A.x_plane);
+                        if (K == 3) {
+                            // nine MMAs, one per window position (a chunk is one K step): the issuing thread runs a few dozen
+                            // instructions per MMA if it has to loop, and then it, not the tensor core, sets the pace
+                            // (measured: an MMA every 100 cycles with the loops, every 40-64 with straight-line code)
+                            const uint32_t wp = (uint32_t)A.Wp;
+                            mma_bf16(tcol, desc64(a_hi, a0), desc64(b_hi, b_lo0), idesc, c > 0);
+                            mma_bf16(tcol, desc64(a_hi, a0 + 1), desc64(b_hi, b_lo0 + w_tap16), idesc, true);
+                            mma_bf16(tcol, desc64(a_hi, a0 + 2), desc64(b_hi, b_lo0 + 2 * w_tap16), idesc, true);
+                            mma_bf16(tcol, desc64(a_hi, a0 + wp), desc64(b_hi, b_lo0 + 3 * w_tap16), idesc, true);
+                            mma_bf16(tcol, desc64(a_hi, a0 + wp + 1), desc64(b_hi, b_lo0 + 4 * w_tap16), idesc, true);
+                            mma_bf16(tcol, desc64(a_hi, a0 + wp + 2), desc64(b_hi, b_lo0 + 5 * w_tap16), idesc, true);
+                            mma_bf16(tcol, desc64(a_hi, a0 + 2 * wp), desc64(b_hi, b_lo0 + 6 * w_tap16), idesc, true);
+                            mma_bf16(tcol, desc64(a_hi, a0 + 2 * wp + 1), desc64(b_hi, b_lo0 + 7 * w_tap16), idesc, true);
+                            mma_bf16(tcol, desc64(a_hi, a0 + 2 * wp + 2), desc64(b_hi, b_lo0 + 8 * w_tap16), idesc, true);
+                        } else {
+                            uint32_t a_lo = a0, b_lo = b_lo0;
+                            bool acc = c > 0;
+                            for (int ks = 0; ks < nks; ++ks) {
+                                mma_bf16(tcol, desc64(a_hi, a_lo), desc64(b_hi, b_lo), idesc, acc);
+                                acc = true; a_lo += xstep; b_lo += wstep;
                             }
                         }
                     }
@@ -535,7 +546,8 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
             if (H->epi_stop) break;                                   // the same answer for all epilogue threads: they leave together
             const uint32_t buf = k % (uint32_t)A.nbuf, use = k / (uint32_t)A.nbuf;
             const uint32_t tbuf = tmem + buf * 256u;
-            wait(&H->done[buf], use & 1u);                            // (ran out: the item is written from whatever is there; the error word is set)
+            wait(&H->done[buf], use & 1u, 128);                       // asleep between polls; (ran out: the item is written from
+                                                                      // whatever is there; the error word is set)
             fence_after_sync();
             if (!A.pool) {
                 const int nc = I.cols >> 4;
