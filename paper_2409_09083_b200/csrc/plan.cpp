@@ -661,7 +661,20 @@ void tc_col_chunks(int W, int* ncc, int* Cw)
 // Launch shape of the banded convolution kernel for a conv with `cout16` output and `cin16` input channels (padded)
 // on N maps of H x W: bands as tall as the accumulators allow (512 columns = blocks of 128 entries x Ns channels),
 // among those the height with the fewest rounds of blocks over the SMs; as many stages as fit.
+TcConvPlan plan_tc_conv_kpc(int N, int H, int W, int K, int cin16, int cout16, bool pool, int kpc3);
+
 TcConvPlan plan_tc_conv(int N, int H, int W, int K, int cin16, int cout16, bool pool)
+{
+    // input channels per chunk: 3x3: 16, or 32 with slices of at most 64 channels where two stages of that size fit
+    // (their filters are small, and every chunk costs the issuers a wait, a fence and a commit); 1x1: up to 64
+    if (K == 3 && std::min(cout16, 128) <= 64 && cin16 >= 32) {
+        const TcConvPlan c = plan_tc_conv_kpc(N, H, W, K, cin16, cout16, pool, 4);
+        if (c.on) return c;
+    }
+    return plan_tc_conv_kpc(N, H, W, K, cin16, cout16, pool, 2);
+}
+
+TcConvPlan plan_tc_conv_kpc(int N, int H, int W, int K, int cin16, int cout16, bool pool, int kpc3)
 {
     TcConvPlan c;
     tc_col_chunks(W, &c.ncc, &c.Cw);
@@ -672,7 +685,7 @@ TcConvPlan plan_tc_conv(int N, int H, int W, int K, int cin16, int cout16, bool 
     // core idle while an item is read back); wider slices: one buffer of 512 columns (their filters are read per item)
     c.nbuf = c.Ns <= 64 ? 2 : 1;
     const int max_blk = std::min(8, kTcTmemCols / c.nbuf / c.Ns);
-    c.kpc = K == 1 ? std::min(cin16 / 8, 8) : 2;
+    c.kpc = K == 1 ? std::min(cin16 / 8, 8) : kpc3;
     const int step = pool ? 2 : 1;
     const int r_max = std::min((max_blk * 128) / c.Wp, H) / step * step;
     if (r_max < step) return c;
@@ -685,7 +698,7 @@ TcConvPlan plan_tc_conv(int N, int H, int W, int K, int cin16, int cout16, bool 
     }
     const size_t entries = std::max<size_t>((size_t)(c.R + K - 1) * c.Wp, (size_t)c.nblk * 128 + (size_t)(K - 1) * c.Wp + K);
     c.x_plane = (int)align_up(entries * 16, 128);
-    c.stage_bytes = c.kpc * c.x_plane + (K == 1 ? c.kpc : 2 * K * K) * c.Ns * 16;
+    c.stage_bytes = c.kpc * c.x_plane + K * K * c.kpc * c.Ns * 16;
     // fused pool: the band as stored goes through a staging area, all channels of the slice at once where that leaves
     // three stages (two for short rings), else 16 channels or more at a time
     const size_t room = (size_t)kTcConvSmemBudget - kTcFgHeader;

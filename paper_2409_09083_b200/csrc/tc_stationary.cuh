@@ -364,7 +364,7 @@ struct TcConvRowsArgs {
     int Ns, slices;                           // output channels per item, number of slices
     int R, Wp, bands_img, nblk;               // rows per band, tile pitch, bands per image, accumulator blocks of a full band
     int ncc, Cw;                              // column chunks per row band and their width (even with the pool; Wp = Cw + K - 1)
-    int kpc;                                  // 8-channel planes per chunk (2 for 3x3)
+    int kpc;                                  // 8-channel planes per chunk (3x3: 2, or 4 with narrow slices; 1x1: up to 8)
     int x_plane, stage_bytes, stages;
     int items;                                // N * bands_img * slices
     int pool_planes;                          // pool: 8-channel planes the staging area holds (even)
@@ -498,19 +498,22 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
                         const uint32_t tcol = tmem + buf * 256u + (uint32_t)(b * A.Ns);
                         const uint32_t a0 = desc_lo(xaddr + (uint32_t)b * 2048u, (uint32_t)A.x_plane);
                         if (K == 3) {
-                            // nine MMAs, one per window position (a chunk is one K step): the issuing thread runs a few dozen
+                            // nine MMAs per K step, one per window position, written out: the issuing thread runs a few dozen
                             // instructions per MMA if it has to loop, and then it, not the tensor core, sets the pace
                             // (measured: an MMA every 100 cycles with the loops, every 40-64 with straight-line code)
                             const uint32_t wp = (uint32_t)A.Wp;
-                            mma_bf16(tcol, desc64(a_hi, a0), desc64(b_hi, b_lo0), idesc, c > 0);
-                            mma_bf16(tcol, desc64(a_hi, a0 + 1), desc64(b_hi, b_lo0 + w_tap16), idesc, true);
-                            mma_bf16(tcol, desc64(a_hi, a0 + 2), desc64(b_hi, b_lo0 + 2 * w_tap16), idesc, true);
-                            mma_bf16(tcol, desc64(a_hi, a0 + wp), desc64(b_hi, b_lo0 + 3 * w_tap16), idesc, true);
-                            mma_bf16(tcol, desc64(a_hi, a0 + wp + 1), desc64(b_hi, b_lo0 + 4 * w_tap16), idesc, true);
-                            mma_bf16(tcol, desc64(a_hi, a0 + wp + 2), desc64(b_hi, b_lo0 + 5 * w_tap16), idesc, true);
-                            mma_bf16(tcol, desc64(a_hi, a0 + 2 * wp), desc64(b_hi, b_lo0 + 6 * w_tap16), idesc, true);
-                            mma_bf16(tcol, desc64(a_hi, a0 + 2 * wp + 1), desc64(b_hi, b_lo0 + 7 * w_tap16), idesc, true);
-                            mma_bf16(tcol, desc64(a_hi, a0 + 2 * wp + 2), desc64(b_hi, b_lo0 + 8 * w_tap16), idesc, true);
+                            uint32_t a = a0, w0 = b_lo0;
+                            for (int ks = 0; ks < nks; ++ks, a += xstep, w0 += wstep) {
+                                mma_bf16(tcol, desc64(a_hi, a), desc64(b_hi, w0), idesc, (c | ks) != 0);
+                                mma_bf16(tcol, desc64(a_hi, a + 1), desc64(b_hi, w0 + w_tap16), idesc, true);
+                                mma_bf16(tcol, desc64(a_hi, a + 2), desc64(b_hi, w0 + 2 * w_tap16), idesc, true);
+                                mma_bf16(tcol, desc64(a_hi, a + wp), desc64(b_hi, w0 + 3 * w_tap16), idesc, true);
+                                mma_bf16(tcol, desc64(a_hi, a + wp + 1), desc64(b_hi, w0 + 4 * w_tap16), idesc, true);
+                                mma_bf16(tcol, desc64(a_hi, a + wp + 2), desc64(b_hi, w0 + 5 * w_tap16), idesc, true);
+                                mma_bf16(tcol, desc64(a_hi, a + 2 * wp), desc64(b_hi, w0 + 6 * w_tap16), idesc, true);
+                                mma_bf16(tcol, desc64(a_hi, a + 2 * wp + 1), desc64(b_hi, w0 + 7 * w_tap16), idesc, true);
+                                mma_bf16(tcol, desc64(a_hi, a + 2 * wp + 2), desc64(b_hi, w0 + 8 * w_tap16), idesc, true);
+                            }
                         } else {
                             uint32_t a_lo = a0, b_lo = b_lo0;
                             bool acc = c > 0;
