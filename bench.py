@@ -87,7 +87,8 @@ def parse():
 def config_of(wl, extra=None):
     cfg = {"workload": f"{wl.name}: {len(wl.layers)}-layer YOLOv2-style stack, batch {wl.N}x{wl.C}x{wl.H}x{wl.W} fp32, "
                        f"tile grid {wl.grid[0]}x{wl.grid[1]}, requested groups {[list(g) for g in wl.groups]}, MSE loss, SGD lr {wl.lr}",
-           "global_batch": wl.N, "tile_grid": list(wl.grid), "groups": [list(g) for g in wl.groups]}
+           "global_batch": wl.N, "tile_grid": list(wl.grid), "groups": [list(g) for g in wl.groups],
+           "input_delta": True}
     cfg.update(extra or {})
     return cfg
 
