@@ -138,7 +138,10 @@ typedef struct {
                            once), the filter gradient by a weight-stationary kernel that keeps a slice of the gradient
                            in tensor memory while the batch streams past; the first layer runs as a 1x1 conv on a
                            window-unrolled bf16 copy of the network input, with the same parameters.
-                           0 and 1: every such layer; -1: never (fused stacks only) */
+                           0 and 1: every such layer; -1: never (fused stacks only).  Conv layers with more than 512
+                           input or output channels run this way only (the fused kernels keep all output channels of
+                           an op in the 512 tensor-memory columns): a bf16 plan that would put such a layer into a
+                           fused stack is refused with FTP_ERR_LAYERS */
     int tc_tma;           /* bf16 path, fused sub-tile kernels: how the tiles of maps saved as bf16 planes reach shared memory.  Default (0): tensor
                            copies by the TMA engine (cp.async.bulk.tensor, one box per 8-channel plane, zeros outside the map;
                            the tensor maps cover the calling GPU's own memory only and no copy is multicast); -1: plain

@@ -1081,7 +1081,7 @@ const char* ftp_strerror(int code)
     switch (code) {
     case FTP_OK: return "ok";
     case FTP_ERR_ARG: return "invalid argument (null pointer, bad size or index, unaligned workspace)";
-    case FTP_ERR_LAYERS: return "unsupported layer (conv: odd k<=7, stride 1, pad k/2; maxpool: 2x2/2 on even extents) or channel mismatch";
+    case FTP_ERR_LAYERS: return "unsupported layer (conv: odd k<=7, stride 1, pad k/2; maxpool: 2x2/2 on even extents; bf16 fused stacks: at most 512 channels) or channel mismatch";
     case FTP_ERR_GRID: return "tile grid has more tiles than pixels in a group's output map";
     case FTP_ERR_GROUPS: return "groups must be contiguous, cover layers 1..L, and hold at most 16 layers each";
     case FTP_ERR_WORKSPACE: return "no sub-tile of a group fits in shared memory; use smaller groups";

@@ -402,7 +402,8 @@ void pass_cost_terms(const ftp_plan& p, const GroupPlan& g, bool backward, bool 
                     }
                 } else if (!backward) {
                     const int nblocks = ((coh + 15) / 16) * ((cow + 7) / 8);
-                    const int rounds = (nblocks + tmem_cols / op.cout16 - 1) / (tmem_cols / op.cout16);
+                    const int at_once = std::max(1, tmem_cols / op.cout16);
+                    const int rounds = (nblocks + at_once - 1) / at_once;
                     const double per_block = (double)op.k * op.k * (op.cin16 / 16) *
                                              (mma_cycles(std::min(op.cout16, 256)) + mma_cycles(op.cout16 - 256));
                     f[0] += nblocks * per_block / 1e3;
@@ -419,7 +420,8 @@ void pass_cost_terms(const ftp_plan& p, const GroupPlan& g, bool backward, bool 
                     f[0] += (double)slices * nk * (units * (mma_cycles(std::min(ucols, 256)) + mma_cycles(ucols - 256)) + 45.0) / 1e3;
                     if (dx) {
                         const int nblocks = ((ih + 15) / 16) * ((iw + 7) / 8);
-                        const int rounds = (nblocks + tmem_cols / op.cin16 - 1) / (tmem_cols / op.cin16);
+                        const int at_once = std::max(1, tmem_cols / op.cin16);
+                        const int rounds = (nblocks + at_once - 1) / at_once;
                         f[1] += (double)nblocks * op.k * op.k * (op.cout16 / 16) *
                                 (mma_cycles(std::min(op.cin16, 256)) + mma_cycles(op.cin16 - 256)) / 1e3;
                         f[3] += rounds * w_mb;
@@ -741,6 +743,19 @@ void plan_tc_filter_grad(const ftp_plan& p, GroupPlan& g, const PlanOpts& o)
     t.Ms = op.cout16 <= 64 ? 64 : 128;
     t.slices = (op.cout16 + t.Ms - 1) / t.Ms;
     t.ncols = std::min(cin16, K == 1 ? 256 : 48);
+    if (K == 3 && cin16 > 32) {
+        // 48 or 32 input channels a block: the slowest block sets the time, i.e. rounds of blocks over the SMs x the pixels
+        // of a share x the cycles of an MMA that wide (32 + columns / 4: both operands come from shared memory).  32 wins
+        // where 48 leaves a ragged last slice as wide (64 = 48 + 16 against 32 + 32) or too few blocks for the SMs
+        // (512 -> 1024: 88 blocks against 128)
+        double best_cost = -1;
+        for (int nc : {48, 32}) {
+            const long long roles = (long long)t.slices * ((cin16 + nc - 1) / nc);
+            const long long shares = std::max<long long>(1, kSmCount / roles);
+            const double cost = (double)((roles * shares + kSmCount - 1) / kSmCount) / (double)shares * (32.0 + nc / 4.0);
+            if (best_cost < 0 || cost < best_cost) { best_cost = cost; t.ncols = nc; }
+        }
+    }
     t.nci = (cin16 + t.ncols - 1) / t.ncols;
     long long best = -1;
     for (int R = 1; R <= std::min(H, 64); ++R) {
@@ -910,6 +925,11 @@ int make_group(const ftp_plan& p, const LayerOffsets& lo, int first, int last, c
                            g.bwd.x.scratch_off[g.bwd.x.count];
     plan_stationary(p, g, o);
     plan_tc_filter_grad(p, g, o);
+    // bf16 path: the fused kernels keep all output channels of an op in the 512 tensor-memory columns; wider layers
+    // run on the banded kernels (a group of their own) or not at all
+    if (tcp && !g.tfg.on)
+        for (int i = 0; i < g.n_ops; ++i)
+            if (g.fwd_ops[i].cin > kTcTmemCols || g.fwd_ops[i].cout > kTcTmemCols) return FTP_ERR_LAYERS;
     if (g.st.on) {                                  // no sub-tile stacks, no halo recomputation
         g.macs_done = g.macs_untiled;
         if (redundancy) *redundancy = 1.0;
@@ -957,7 +977,6 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
             int cin_pad = (l.cin + kCoutTile - 1) / kCoutTile * kCoutTile;
             lo.wf_off[i] = wf; wf += (long long)l.cin * l.k * l.k * cout_pad;
             lo.wb_off[i] = wb; wb += (long long)l.cout * l.k * l.k * cin_pad;
-            if (tcp && (l.cin > kTcTmemCols || l.cout > kTcTmemCols)) return FTP_ERR_LAYERS;
             lo.twf_off[i] = lo.twb_off[i] = twf;        // both packed layouts hold k*k*cin16*cout16 elements; room for the
             twf += (long long)l.k * l.k * round_up(l.cin, 128) * round_up(l.cout, 128);   // banded kernels' padded slices
         } else if (l.kind == FTP_MAXPOOL) {
@@ -1008,7 +1027,7 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
         while (start <= last) {
             GroupPlan g;
             double red = 1.0;
-            int chosen = -1;
+            int chosen = -1, last_rc = FTP_OK;
             int hi = std::min(last, start + kMaxOps - 1);
             if (!opts.strict_groups && opts.max_group_convs > 0) {
                 int convs = 0, end = start - 1;
@@ -1038,9 +1057,10 @@ int build_plan(ftp_plan& p, const ftp_layer* layers, int n_layers, int N, int C,
                                                  p.layers[end].kind == FTP_MAXPOOL;
                         if (pass == 0 && splits_pair) continue;
                         int rc = make_group(p, lo, start, end, popts, g, &red);
+                        last_rc = rc;
                         if (rc == FTP_OK && (pass == 2 || red * 100.0 <= opts.max_redundancy_pct)) { chosen = end; break; }
                     }
-                if (chosen < 0) return FTP_ERR_WORKSPACE;
+                if (chosen < 0) return last_rc == FTP_ERR_LAYERS ? FTP_ERR_LAYERS : FTP_ERR_WORKSPACE;
             }
             cut.push_back(g);
             start = chosen + 1;

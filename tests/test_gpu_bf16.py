@@ -402,6 +402,10 @@ SAFE = {
     # counts that fill neither a 128-channel slice nor a chunk of input planes (200, 136, 48), a last band of a few rows
     "ragged": (W("r", (conv(3, 24, 3), pool(), conv(24, 200, 3), conv(200, 136, 1), conv(136, 48, 3), pool()), 2, 3, 36, 280,
                  (2, 2), ((1, 6),)), None),
+    # the shapes of the layers behind the 16-layer stack: 512 -> 1024 3x3 and 1024 -> 512 1x1 on a 10 x 14 map (more
+    # channels than the fused kernels hold: banded kernels only, 8 slices of output channels, 128 planes of input)
+    "wide-1024": (W("w", (conv(3, 16, 3), pool(), conv(16, 512, 1), pool(), conv(512, 1024, 3), conv(1024, 512, 1)), 2, 3, 40, 56,
+                    (2, 2), ((1, 2), (3, 4), (5, 5), (6, 6))), None),
     "C1": (synth.workload("C1"), None),                 # benchmark launch configurations, full batch
     "C2": (synth.workload("C2"), None),
     "C3": (synth.workload("C3"), (0, 15)),              # full batch on the GPU, loss delta on two images

@@ -70,6 +70,8 @@ def test_step_updates_parameters_like_the_oracle(name):
 
 Y8 = W("y8", tuple(synth.stack_yolo8()), 2, 3, 64, 96, (3, 3), ((1, 8),))
 Y16 = W("y16", tuple(synth.stack_yolo16()), 1, 3, 96, 160, (5, 5), ((1, 4), (5, 8), (9, 16)))
+WIDE = W("wide", (conv(3, 16, 3), pool(), conv(16, 512, 1), pool(), conv(512, 1024, 3), conv(1024, 512, 1)), 2, 3, 40, 56,
+         (2, 2), ((1, 2), (3, 4), (5, 5), (6, 6)))
 DYADIC = {
     "yolo8-one-group": (Y8, 3, {}),
     "yolo8-strict-one-group": (Y8, 3, dict(strict_groups=True)),
@@ -81,6 +83,10 @@ DYADIC = {
     "yolo8-1x1grid": (Y8.with_(grid=(1, 1), N=3), 3, {}),
     "yolo16-three-groups": (Y16, 2, {}),
     "yolo16-all-in-one": (Y16.with_(groups=((1, 16),), grid=(2, 3)), 2, {}),
+    # the shapes of the layers behind the 16-layer stack (512 -> 1024 3x3, 1024 -> 512 1x1 on a map of a few hundred
+    # pixels): filters of 19 MB against maps of 0.6 MB, one-conv groups and two of them fused
+    "wide-1024": (WIDE, 3, {}),
+    "wide-1024-fused-pair": (WIDE.with_(groups=((1, 4), (5, 6))), 3, dict(strict_groups=True)),
 }
 
 

@@ -5,6 +5,7 @@ import ctypes
 import os
 import re
 
+import numpy as np
 import pytest
 
 import paper_2409_09083_b200 as ftp
@@ -290,6 +291,30 @@ def test_bf16_plans_run_conv_layers_as_groups_of_their_own():
     plan = ftp.ftp_plan(layers, 2, 3, 32, 32, (2, 2), ((1, 2),), precision=ftp.FTP_BF16_FP32ACC)
     modes = [plan.group_mode(i)[0] for i in range(len(plan.exec_groups()))]
     assert modes[0] == 0 and modes[-1] == 2, (plan.exec_groups(), modes)
+
+
+def test_bf16_layers_wider_than_the_tensor_memory_run_banded_or_not_at_all():
+    """bf16 path: a conv layer with more than 512 input or output channels (the 512 -> 1024 -> 512 layers behind the
+    16-layer stack) is planned as a banded one-conv group; a plan that would put it into a fused stack (fused stacks
+    only, a strict profile that fuses it, a 5x5 window) is refused with the layer error, not planned into a kernel
+    that cannot hold it; the cost query of such a group answers; the fp32 path plans all of them."""
+    conv, pool = synth.conv, synth.pool
+    layers = (conv(3, 16, 3), pool(), conv(16, 512, 1), pool(), conv(512, 1024, 3), conv(1024, 512, 1))
+    shape = (2, 3, 40, 56, (2, 2))
+    bf16 = ftp.FTP_BF16_FP32ACC
+    plan = ftp.ftp_plan(layers, *shape, ((1, 6),), precision=bf16)
+    assert plan.exec_groups() == [(1, 2), (3, 4), (5, 5), (6, 6)]
+    assert [plan.group_mode(i)[0] for i in range(4)] == [2, 2, 2, 2]
+    for gi in range(4):
+        for pass_ in (0, 1):
+            terms, est = plan.cost(pass_, gi, True)
+            assert np.isfinite(est) and est > 0 and np.all(np.isfinite(terms))
+    assert _code(lambda: ftp.ftp_plan(layers, *shape, ((1, 6),), precision=bf16, stationary=-1)) == -2
+    assert _code(lambda: ftp.ftp_plan(layers, *shape, ((1, 4), (5, 6)), precision=bf16, strict_groups=True)) == -2
+    five = (conv(3, 16, 3), conv(16, 640, 5))
+    assert _code(lambda: ftp.ftp_plan(five, 1, 3, 16, 16, (2, 2), ((1, 2),), precision=bf16)) == -2
+    for kw in ({}, dict(stationary=-1), dict(strict_groups=True)):
+        ftp.ftp_plan(layers, *shape, ((1, 4), (5, 6)), **kw)
 
 
 def test_small_launches_of_the_row_convolution_use_half_size_blocks():
