@@ -553,53 +553,59 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
                                                                       // whatever is there; the error word is set)
             fence_after_sync();
             if (!A.pool) {
-                const int nc = I.cols >> 4;
-                for (int u = part; u < I.nblk * nc; u += kParts) {
-                    const int b = u / nc, c0 = (u - b * nc) << 4;
+                const int nc = I.cols >> 4, nunits = I.nblk * nc;
+                const size_t gstep = (size_t)A.H * A.W;
+                // where unit u (accumulator block b, channels c0 .. c0 + 15) of this thread lies in the output planes
+                auto place = [&](int u, int& b, int& c0, size_t& g0) {
+                    b = u / nc; c0 = (u - b * nc) << 4;
                     const int p = b * 128 + q * 32 + lane;
                     const int r = p / A.Wp, c = p - r * A.Wp;
-                    const bool valid = r < I.rows && c < I.cw;
-                    uint4* o = A.out + (((size_t)I.n * oplanes + (I.co0 >> 3)) * A.H + I.y0 + r) * A.W + I.x0 + c;
-                    {
-                        // (what the fused dz step reads is requested before the accumulators, so that the latencies overlap)
-                        const size_t g0 = (((size_t)I.n * oplanes + ((I.co0 + c0) >> 3)) * A.H + I.y0 + r) * A.W + I.x0 + c;
-                        const size_t gstep = (size_t)A.H * A.W;
-                        uint4 yq[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-                        unsigned long long amq[2] = {0ull, 0ull};
-                        if (A.prev_y && valid) {
-                            yq[0] = __ldg(A.prev_y + g0); yq[1] = __ldg(A.prev_y + g0 + gstep);
-                            if (A.prev_arg) { amq[0] = __ldg(A.prev_arg + g0); amq[1] = __ldg(A.prev_arg + g0 + gstep); }
-                        }
-                        float v[16];
-                        tmem_ld16(tbuf + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * A.Ns + c0), v);
+                    g0 = (((size_t)I.n * oplanes + ((I.co0 + c0) >> 3)) * A.H + I.y0 + r) * A.W + I.x0 + c;
+                    return r < I.rows && c < I.cw;
+                };
+                for (int u = part; u < nunits; u += kParts) {
+                    int b, c0; size_t g0;
+                    const bool valid = place(u, b, c0, g0);
+                    // what the fused dz step reads of the layer below is requested before the accumulators, so that the
+                    // latencies overlap (requested a whole unit ahead, even for the launches through a pool only, the
+                    // kernel was measured slower)
+                    uint4 yq[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+                    unsigned long long amq[2] = {0ull, 0ull};
+                    if (A.prev_y && valid) {
+                        yq[0] = __ldg(A.prev_y + g0); yq[1] = __ldg(A.prev_y + g0 + gstep);
+                        if (A.prev_arg) { amq[0] = __ldg(A.prev_arg + g0); amq[1] = __ldg(A.prev_arg + g0 + gstep); }
+                    }
+                    float v[16];
+                    tmem_ld16(tbuf + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * A.Ns + c0), v);
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) { const float z = v[j] + H->bias[c0 + j]; v[j] = z > 0.f ? z : slope * z; }
-                        if (!valid) continue;
-                        if (!A.prev_y) {
-                            o[(size_t)(c0 >> 3) * A.H * A.W] = tcd::pack8(v);
-                            o[(size_t)((c0 >> 3) + 1) * A.H * A.W] = tcd::pack8(v + 8);
-                            continue;
-                        }
+                    for (int j = 0; j < 16; ++j) { const float z = v[j] + H->bias[c0 + j]; v[j] = z > 0.f ? z : slope * z; }
+                    if (valid && !A.prev_y) {
+                        A.out[g0] = tcd::pack8(v);
+                        A.out[g0 + gstep] = tcd::pack8(v + 8);
+                    } else if (valid) {
                         // input delta straight into the dz planes of the layer below: rounded as a stored delta
                         // would be, times the derivative of that layer's activation, through its pool's arg-max
+                        const int p = b * 128 + q * 32 + lane;
+                        const int r = p / A.Wp, c = p - r * A.Wp;
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            const size_t gi = g0 + h * gstep;
                             float d[8], yv[8];
                             tcd::unpack8(tcd::pack8(v + 8 * h), d);
                             tcd::unpack8(yq[h], yv);
 #pragma unroll
                             for (int j = 0; j < 8; ++j) d[j] *= yv[j] > 0.f ? 1.f : A.prev_slope;
-                            if (!A.prev_arg) { A.out[gi] = tcd::pack8(d); continue; }
-                            const unsigned long long am = amq[h];
+                            const uint4 dq = tcd::pack8(d);
+                            if (!A.prev_arg) { A.out[g0 + h * gstep] = dq; continue; }
+                            // the four members of every channel's pool window: the delta where the arg-max byte names the
+                            // member, zero elsewhere (byte masks widened to the bf16 halves)
+                            const uint32_t alo = (uint32_t)amq[h] & 0x03030303u, ahi = (uint32_t)(amq[h] >> 32) & 0x03030303u;
                             const int W2 = 2 * A.W;
                             uint4* o2 = A.out + (((size_t)I.n * oplanes + ((I.co0 + c0) >> 3) + h) * (2 * A.H) + 2 * (I.y0 + r)) * W2 + 2 * (I.x0 + c);
 #pragma unroll
                             for (int w = 0; w < 4; ++w) {
-                                float z[8];
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) z[j] = (int)((am >> (j * 8)) & 3ull) == w ? d[j] : 0.f;
-                                o2[(w >> 1) * W2 + (w & 1)] = tcd::pack8(z);
+                                const uint32_t ml = __vcmpeq4(alo, (uint32_t)w * 0x01010101u), mh = __vcmpeq4(ahi, (uint32_t)w * 0x01010101u);
+                                o2[(w >> 1) * W2 + (w & 1)] = make_uint4(dq.x & __byte_perm(ml, 0u, 0x1100), dq.y & __byte_perm(ml, 0u, 0x3322),
+                                                                         dq.z & __byte_perm(mh, 0u, 0x1100), dq.w & __byte_perm(mh, 0u, 0x3322));
                             }
                         }
                     }
