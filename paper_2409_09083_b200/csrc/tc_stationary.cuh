@@ -392,7 +392,7 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
         unsigned long long drain;       // all MMAs of the block have completed
         uint32_t tmem_base;
         volatile int failed;
-        volatile int epi_stop;          // the epilogue warps' common view of `failed` (they meet at named barriers)
+        volatile int epi_stop[2];       // the epilogue warps' common view of `failed` (they meet at named barriers), items in turn
         float bias[128];
     };
     static_assert(sizeof(Hdr) <= kTcFgHeader, "header does not fit");
@@ -540,13 +540,21 @@ __global__ void __launch_bounds__(kTcConvThreads, 1) conv_tc_rows_kernel(const _
         uint4* S = reinterpret_cast<uint4*>(stages + (size_t)A.stages * A.stage_bytes);
         const int et = threadIdx.x;                                   // 0 .. kTcConvEpiThreads - 1
         uint32_t k = 0;
+        // one slice of output channels: its bias is fetched once, and an item costs the epilogue warps one barrier (the
+        // stop word of item k is written before that barrier and read behind it; its slot is written again two items
+        // on, behind the barrier of the item between, at which every thread has read it)
+        const bool one_slice = A.slices == 1;
+        if (one_slice)
+            for (int c = et; c < A.Ns; c += kTcConvEpiThreads) H->bias[c] = (A.bias && c < A.cout) ? __ldg(A.bias + c) : 0.f;
         for (int it = blockIdx.x; it < A.items; it += gridDim.x, ++k) {
             const Item I = item_of(it);
-            asm volatile("bar.sync 1, %0;" :: "n"(kTcConvEpiThreads) : "memory");            // every warp is through with the bias of the item before
-            for (int c = et; c < A.Ns; c += kTcConvEpiThreads) H->bias[c] = (A.bias && I.co0 + c < A.cout) ? __ldg(A.bias + I.co0 + c) : 0.f;
-            if (et == 0) H->epi_stop = H->failed;
+            if (!one_slice) {
+                asm volatile("bar.sync 1, %0;" :: "n"(kTcConvEpiThreads) : "memory");        // every warp is through with the bias of the item before
+                for (int c = et; c < A.Ns; c += kTcConvEpiThreads) H->bias[c] = (A.bias && I.co0 + c < A.cout) ? __ldg(A.bias + I.co0 + c) : 0.f;
+            }
+            if (et == 0) H->epi_stop[k & 1u] = H->failed;
             asm volatile("bar.sync 1, %0;" :: "n"(kTcConvEpiThreads) : "memory");
-            if (H->epi_stop) break;                                   // the same answer for all epilogue threads: they leave together
+            if (H->epi_stop[k & 1u]) break;                           // the same answer for all epilogue threads: they leave together
             const uint32_t buf = k % (uint32_t)A.nbuf, use = k / (uint32_t)A.nbuf;
             const uint32_t tbuf = tmem + buf * 256u;
             wait(&H->done[buf], use & 1u, 128);                       // asleep between polls; (ran out: the item is written from
