@@ -47,7 +47,7 @@ KERNEL = {("fwd_group", "fp32"): "fwd_group_kernel / conv_rows_kernel", ("bwd_gr
 # under profiles/ (static: null for every kernel / workload without a capture of the current code)
 NCU_TRAFFIC = {("C3", "fp32", "fwd_group"): 128.4e6, ("C3", "fp32", "filter_grad_rows"): 245.8e6,
                ("C3", "fp32", "delta_conv_rows"): 159.3e6, ("C3", "fp32", "bwd_group"): 950.4e6,
-               ("C3", "bf16", "fwd_group"): 84.7e6, ("C3", "bf16", "filter_grad_rows"): 153.1e6, ("C3", "bf16", "delta_conv_rows"): 201.6e6}
+               ("C3", "bf16", "fwd_group"): 84.7e6, ("C3", "bf16", "filter_grad_rows"): 153.2e6, ("C3", "bf16", "delta_conv_rows"): 201.5e6}
 
 
 def measured_bf16_peak():
